@@ -1,0 +1,170 @@
+/*
+ * gdn_tree.h -- C ABI of the B200 (sm_100a) library for rollback-free tree
+ * verification of Gated DeltaNet (GDN) layers in speculative decoding.
+ *
+ * The operations are those of Section 3.4 of "Trees from Marginals":
+ * every node of a draft tree is evaluated under the gated delta rule (Eq. 7)
+ * conditioned only on its ancestors, starting from the committed state S0,
+ * and the per-node outputs follow Eq. 8 ("verify", which never writes the
+ * state); once the accepted root path is known the state is advanced along
+ * that path in place ("commit", the delayed commit of Section 3.4 and the
+ * last sentence of Section 3.4.2).
+ *
+ * Conventions common to every entry point
+ *   - Pointers marked [device] are CUDA device pointers on the current
+ *     device, contiguous, row-major, 16-byte aligned; pointers marked [host]
+ *     are ordinary host pointers.  The caller owns every buffer.  The library
+ *     allocates no memory and keeps no state between calls.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*,
+ *     NULL = the legacy default stream).  The [device] entry points never
+ *     synchronise; the *_host entry points synchronise the stream before
+ *     returning.
+ *   - Return value: GDN_OK or a negative gdn_status decided on the host
+ *     before anything is launched (nothing is launched on error).
+ *     Data-dependent faults that only the device can see (a bad parent[],
+ *     a root path longer than max_depth, a path that is not a root chain)
+ *     are reported by writing a negative gdn_status into *status_dev with
+ *     an atomic compare-and-swap from 0; the affected tree then produces no
+ *     output (verify) or keeps its state unchanged (commit).  The library
+ *     never clears *status_dev: zero it before a sequence of calls and read
+ *     it after synchronising.  Kernels never trap and never wait unboundedly.
+ *   - Tensors (N = total_nodes = node_offsets[n_seq]):
+ *       S0 / S      [n_seq][h_v][d_v][d_k]  fp32   (Section 3.4.2: [H_v, d_v, d_k];
+ *                                                   element [c][r] is S_{r,c} of Eq. 7)
+ *       q, k        [N][h_qk][d_k]          in_dtype
+ *       v           [N][h_v][d_v]           in_dtype
+ *       g, beta     [N][h_v]                in_dtype   g = log(alpha) <= 0
+ *       o           [N][h_v][d_v]           out_dtype
+ *       parent      [N] int32   index local to the node's own tree, -1 = root,
+ *                               parent[i] < i (topological numbering, Section 3.4.1)
+ *       node_offsets[n_seq+1] int32, node_offsets[0] = 0 (ragged packing of trees)
+ *     Value head h uses key head h / (h_v / h_qk).  L2-normalising q and k
+ *     and the gate activations are the caller's business.
+ */
+#ifndef GDN_TREE_H_
+#define GDN_TREE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum gdn_dtype { GDN_F32 = 0, GDN_BF16 = 1 };
+
+enum gdn_status {
+    GDN_OK = 0,
+    GDN_ERR_NULL = -1,        /* a required pointer is NULL                                   */
+    GDN_ERR_SHAPE = -2,       /* a size is out of range or inconsistent                       */
+    GDN_ERR_DTYPE = -3,       /* unknown in_dtype / out_dtype                                 */
+    GDN_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned                             */
+    GDN_ERR_UNSUPPORTED = -5, /* valid request that this build cannot run                     */
+    GDN_ERR_CUDA = -6,        /* a CUDA runtime call failed (launch, copy, attribute)         */
+    GDN_ERR_TREE = -7,        /* parent[] / node_offsets[] do not describe a topological forest */
+    GDN_ERR_DEPTH = -8,       /* a root path has more than max_depth nodes                    */
+    GDN_ERR_PATH = -9,        /* accepted path is not a root chain of its tree, or too long   */
+    GDN_ERR_WORKSPACE = -10,  /* workspace pointer missing or smaller than required           */
+    GDN_ERR_TIMEOUT = -11     /* a bounded device-side wait expired                           */
+};
+
+#define GDN_MAX_HEAD_DIM 128   /* d_k, d_v <= 128                     */
+#define GDN_MAX_DEPTH_CAP 64   /* max_depth <= 64 nodes on a root path */
+#define GDN_MAX_TREE_NODES 4096
+
+/* Problem description shared by all entry points. */
+typedef struct gdn_shape {
+    int32_t n_seq;          /* B: number of trees / state slots (a sequence, or a (sequence, layer) pair) */
+    int32_t h_qk;           /* q/k heads                                                   */
+    int32_t h_v;            /* v heads, a multiple of h_qk                                  */
+    int32_t d_k;            /* key dim, multiple of 4, <= GDN_MAX_HEAD_DIM                  */
+    int32_t d_v;            /* value dim, <= GDN_MAX_HEAD_DIM                               */
+    int32_t in_dtype;       /* gdn_dtype of q, k, v, g, beta                                */
+    int32_t out_dtype;      /* gdn_dtype of o                                               */
+    int32_t max_depth;      /* bound on the nodes of a root path, 1..GDN_MAX_DEPTH_CAP;
+                               the paper's draft trees have at most 16 (Section 6)          */
+    int32_t total_nodes;    /* N = node_offsets[n_seq]                                      */
+    int32_t max_tree_nodes; /* upper bound on the size of any one tree, <= GDN_MAX_TREE_NODES */
+    float scale;            /* multiplies o; Eq. 8 uses 1/sqrt(d_k)                         */
+} gdn_shape_t;
+
+/* Text for a gdn_status value (static storage, never NULL). */
+const char *gdn_status_string(int status);
+
+/*
+ * Bytes of device scratch gdn_tree_verify needs for this shape (tree metadata
+ * of Section 3.4.2 -- per node its depth and ancestor list -- plus the cached
+ * solve result u~ [N][h_v][d_v] fp32, the quantity "u_j - w_j^T S0" that the
+ * substitution of Eq. 13 returns).  Returns 0 if the shape is invalid.
+ */
+size_t gdn_tree_workspace_bytes(const gdn_shape_t *shape);
+
+/*
+ * Pure host check of tree and path arrays (no CUDA call): parent[] in [-1, i),
+ * node_offsets monotone from 0 to total_nodes, every tree <= max_tree_nodes,
+ * every root path <= max_depth nodes, and (if path_h != NULL) every accepted
+ * path a chain from a root with path_offsets monotone from 0.
+ * All four arrays are [host].  path_h / path_offsets_h may both be NULL.
+ */
+int gdn_tree_validate_host(const gdn_shape_t *shape, const int32_t *parent_h,
+                           const int32_t *node_offsets_h, const int32_t *path_h,
+                           const int32_t *path_offsets_h);
+
+/*
+ * Tree verification (Section 3.4.1, Eq. 7-11): for every node i of every tree,
+ *   o_i = scale * q_i^T S_i,  S_i = Eq. 7 applied over the root path of i
+ * (root first, i last) starting from S0 -- evaluated in the triangular form of
+ * Eq. 9-11, so no per-node state is ever materialised and S0 is only read.
+ *   S0, q, k, v, g, beta, parent, node_offsets : [device], read-only
+ *   o            : [device], written for every node of every valid tree
+ *   workspace    : [device], >= gdn_tree_workspace_bytes(shape) bytes, 256-byte aligned;
+ *                  contents after the call: the tree metadata and u~ (reused by nothing else)
+ *   status_dev   : [device] one int32, see "Return value" above
+ */
+int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const void *q, const void *k,
+                    const void *v, const void *g, const void *beta, const int32_t *parent,
+                    const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
+                    int32_t *status_dev, void *cuda_stream);
+
+/*
+ * Commit (Section 3.4, "delay the state commit ... replay the selected path";
+ * Section 3.4.2, last sentence): for every tree b, S[b] <- Eq. 7 replayed over
+ * path[path_offsets[b] .. path_offsets[b+1]) (local node ids, root first),
+ * in place.  An empty path leaves S[b] untouched.
+ *   S            : [device] in: S0, out: S_new (the only state write of a decode step)
+ *   k, v, g, beta, node_offsets : [device] the same packed tensors verify read
+ *   parent       : [device] or NULL; when given, each path is checked to be a
+ *                  root chain (GDN_ERR_PATH in *status_dev, that tree's state unchanged)
+ *   path         : [device] int32 [path_offsets[n_seq]]
+ *   path_offsets : [device] int32 [n_seq+1], path_offsets[0] = 0, each length <= max_depth
+ */
+int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k, const void *v, const void *g,
+                    const void *beta, const int32_t *parent, const int32_t *node_offsets,
+                    const int32_t *path, const int32_t *path_offsets, int32_t *status_dev,
+                    void *cuda_stream);
+
+/*
+ * Host-buffer variants: same operations with every tensor in [host] memory
+ * (pinned memory makes the copies asynchronous).  Inputs are copied into
+ * `dev_arena` ([device], >= gdn_tree_host_arena_bytes(shape, total_path_len) bytes, 256-byte
+ * aligned), the kernels run, results are copied back and the stream is
+ * synchronised.  Returns the host-side status, or the device-side status if
+ * that is non-zero.  total_path_len = path_offsets[n_seq] (0 for verify).
+ */
+size_t gdn_tree_host_arena_bytes(const gdn_shape_t *shape, int32_t total_path_len);
+
+int gdn_tree_verify_host(const gdn_shape_t *shape, const float *S0_h, const void *q_h,
+                         const void *k_h, const void *v_h, const void *g_h, const void *beta_h,
+                         const int32_t *parent_h, const int32_t *node_offsets_h, void *o_h,
+                         void *dev_arena, size_t arena_bytes, void *cuda_stream);
+
+int gdn_tree_commit_host(const gdn_shape_t *shape, float *S_h, const void *k_h, const void *v_h,
+                         const void *g_h, const void *beta_h, const int32_t *parent_h,
+                         const int32_t *node_offsets_h, const int32_t *path_h,
+                         const int32_t *path_offsets_h, int32_t total_path_len, void *dev_arena,
+                         size_t arena_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GDN_TREE_H_ */

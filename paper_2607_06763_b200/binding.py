@@ -1,0 +1,156 @@
+"""ctypes binding of the C-ABI library declared in ``include/gdn_tree.h``.
+
+Argument marshalling only: every step of verify and commit runs in the CUDA kernels of ``libgdn_tree.so``.
+Tensor arguments may be torch tensors (their ``data_ptr()`` is passed), numpy arrays (host entry points) or raw
+integer addresses.  There is no fallback of any kind: if the library has not been built, ``load_library`` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_NAME = "libgdn_tree.so"
+_lib = None
+
+GDN_F32 = 0
+GDN_BF16 = 1
+DTYPE_CODES = {"f32": GDN_F32, "bf16": GDN_BF16}
+
+EXPORTS = (
+    "gdn_status_string",
+    "gdn_tree_workspace_bytes",
+    "gdn_tree_validate_host",
+    "gdn_tree_verify",
+    "gdn_tree_commit",
+    "gdn_tree_host_arena_bytes",
+    "gdn_tree_verify_host",
+    "gdn_tree_commit_host",
+)
+
+
+class GdnShape(ctypes.Structure):
+    """Mirror of ``gdn_shape_t``."""
+    _fields_ = [
+        ("n_seq", ctypes.c_int32),
+        ("h_qk", ctypes.c_int32),
+        ("h_v", ctypes.c_int32),
+        ("d_k", ctypes.c_int32),
+        ("d_v", ctypes.c_int32),
+        ("in_dtype", ctypes.c_int32),
+        ("out_dtype", ctypes.c_int32),
+        ("max_depth", ctypes.c_int32),
+        ("total_nodes", ctypes.c_int32),
+        ("max_tree_nodes", ctypes.c_int32),
+        ("scale", ctypes.c_float),
+    ]
+
+    @classmethod
+    def from_workload(cls, w, max_depth: int = 16, max_tree_nodes: int | None = None) -> "GdnShape":
+        """Shape of a ``synth.Workload``."""
+        import numpy as np
+        sizes = np.diff(w.node_offsets)
+        mt = int(sizes.max()) if len(sizes) else 1
+        return cls(w.n_seq, w.h_qk, w.h_v, w.d_k, w.d_v, DTYPE_CODES[w.in_dtype], DTYPE_CODES[w.out_dtype],
+                   max_depth, w.total_nodes, max(1, mt if max_tree_nodes is None else max_tree_nodes), w.scale)
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, _LIB_NAME)
+
+
+def load_library():
+    """Load ``libgdn_tree.so`` (built in-tree by ``paper_2607_06763_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: the CUDA library has not been built "
+                "(run `python -m paper_2607_06763_b200.build`); there is no CPU fallback")
+        lib = ctypes.CDLL(path)
+        vp, sp = ctypes.c_void_p, ctypes.POINTER(GdnShape)
+        lib.gdn_status_string.restype = ctypes.c_char_p
+        lib.gdn_status_string.argtypes = [ctypes.c_int]
+        lib.gdn_tree_workspace_bytes.restype = ctypes.c_size_t
+        lib.gdn_tree_workspace_bytes.argtypes = [sp]
+        lib.gdn_tree_validate_host.restype = ctypes.c_int
+        lib.gdn_tree_validate_host.argtypes = [sp, vp, vp, vp, vp]
+        lib.gdn_tree_verify.restype = ctypes.c_int
+        lib.gdn_tree_verify.argtypes = [sp] + [vp] * 10 + [ctypes.c_size_t, vp, vp]
+        lib.gdn_tree_commit.restype = ctypes.c_int
+        lib.gdn_tree_commit.argtypes = [sp] + [vp] * 11
+        lib.gdn_tree_host_arena_bytes.restype = ctypes.c_size_t
+        lib.gdn_tree_host_arena_bytes.argtypes = [sp, ctypes.c_int32]
+        lib.gdn_tree_verify_host.restype = ctypes.c_int
+        lib.gdn_tree_verify_host.argtypes = [sp] + [vp] * 10 + [ctypes.c_size_t, vp]
+        lib.gdn_tree_commit_host.restype = ctypes.c_int
+        lib.gdn_tree_commit_host.argtypes = [sp] + [vp] * 9 + [ctypes.c_int32, vp, ctypes.c_size_t, vp]
+        _lib = lib
+    return _lib
+
+
+def _ptr(x):
+    """Address of a torch tensor / numpy array / int / None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError(f"cannot take the address of {type(x)!r}")
+
+
+def _stream(stream):
+    if stream is None:
+        return None
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def gdn_status_string(status: int) -> str:
+    return load_library().gdn_status_string(int(status)).decode()
+
+
+def gdn_tree_workspace_bytes(shape: GdnShape) -> int:
+    return int(load_library().gdn_tree_workspace_bytes(ctypes.byref(shape)))
+
+
+def gdn_tree_validate_host(shape: GdnShape, parent, node_offsets, path=None, path_offsets=None) -> int:
+    return int(load_library().gdn_tree_validate_host(ctypes.byref(shape), _ptr(parent), _ptr(node_offsets),
+                                                      _ptr(path), _ptr(path_offsets)))
+
+
+def gdn_tree_verify(shape: GdnShape, S0, q, k, v, g, beta, parent, node_offsets, o, workspace, workspace_bytes,
+                    status_dev, stream=None) -> int:
+    return int(load_library().gdn_tree_verify(ctypes.byref(shape), _ptr(S0), _ptr(q), _ptr(k), _ptr(v), _ptr(g),
+                                               _ptr(beta), _ptr(parent), _ptr(node_offsets), _ptr(o),
+                                               _ptr(workspace), int(workspace_bytes), _ptr(status_dev),
+                                               _stream(stream)))
+
+
+def gdn_tree_commit(shape: GdnShape, S, k, v, g, beta, parent, node_offsets, path, path_offsets, status_dev,
+                    stream=None) -> int:
+    return int(load_library().gdn_tree_commit(ctypes.byref(shape), _ptr(S), _ptr(k), _ptr(v), _ptr(g), _ptr(beta),
+                                               _ptr(parent), _ptr(node_offsets), _ptr(path), _ptr(path_offsets),
+                                               _ptr(status_dev), _stream(stream)))
+
+
+def gdn_tree_host_arena_bytes(shape: GdnShape, total_path_len: int = 0) -> int:
+    return int(load_library().gdn_tree_host_arena_bytes(ctypes.byref(shape), int(total_path_len)))
+
+
+def gdn_tree_verify_host(shape: GdnShape, S0, q, k, v, g, beta, parent, node_offsets, o, dev_arena, arena_bytes,
+                         stream=None) -> int:
+    return int(load_library().gdn_tree_verify_host(ctypes.byref(shape), _ptr(S0), _ptr(q), _ptr(k), _ptr(v),
+                                                    _ptr(g), _ptr(beta), _ptr(parent), _ptr(node_offsets), _ptr(o),
+                                                    _ptr(dev_arena), int(arena_bytes), _stream(stream)))
+
+
+def gdn_tree_commit_host(shape: GdnShape, S, k, v, g, beta, parent, node_offsets, path, path_offsets,
+                         total_path_len, dev_arena, arena_bytes, stream=None) -> int:
+    return int(load_library().gdn_tree_commit_host(ctypes.byref(shape), _ptr(S), _ptr(k), _ptr(v), _ptr(g),
+                                                    _ptr(beta), _ptr(parent), _ptr(node_offsets), _ptr(path),
+                                                    _ptr(path_offsets), int(total_path_len), _ptr(dev_arena),
+                                                    int(arena_bytes), _stream(stream)))
