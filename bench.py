@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the GDN tree verify + commit hot path.
+
+One *step* = one verify (all nodes of all trees, all heads, all layer slots) followed by one commit of the accepted
+paths, through the C ABI.  The default workload is the stack configuration the headline target is quoted on: all GDN
+heads of a 48-layer stack (48 layer slots x 32 value heads, d_k = d_v = 128), one 64-node draft tree, batch 1, bf16
+inputs, fp32 state, everything in one launch per call.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+With N > 1 (under torchrun) every rank runs its own replica of the workload (the path has no exchange step: each
+(sequence, layer, head) is independent), timing is the max over ranks and the value is the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_06763_b200 import synth  # noqa: E402
+
+METRIC = "verified tree-nodes/sec per GDN layer"
+UNIT = "nodes/s"
+WORKLOADS = {"stack48_T64": 5, "layer_T64": 1, "stack48_T256": 2, "ragged32": 3, "chains64x16": 4}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.file = index, None, None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.file,
+                                         stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()   # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def algorithmic_bytes(w: synth.Workload):
+    """(verify bytes, commit bytes, step bytes).  Step bytes follow the headline definition: S0 read once + S_new
+    written once + q,k,v,g,beta read + o written.  Per launch: verify reads S0 and the node tensors and writes o;
+    commit reads and writes the state (its re-read of the accepted nodes' rows is not counted)."""
+    isz = 4 if w.in_dtype == synth.F32 else 2
+    osz = 4 if w.out_dtype == synth.F32 else 2
+    N = w.total_nodes
+    state = w.n_seq * w.h_v * w.d_v * w.d_k * 4
+    nodes_in = 2 * N * w.h_qk * w.d_k * isz + N * w.h_v * w.d_v * isz + 2 * N * w.h_v * isz
+    o = N * w.h_v * w.d_v * osz
+    return state + nodes_in + o, 2 * state, 2 * state + nodes_in + o
+
+
+def oracle_sample(w: synth.Workload, target_slots: int):
+    """Time the fp64 oracle on the first `target_slots` sequences (verify + commit)."""
+    from oracle import gdn_oracle as orc
+    n = max(1, min(target_slots, w.n_seq))
+    seqs = list(range(n))
+    lo, hi = 0, int(w.node_offsets[n])
+    args = dict(S0=w.S0[:n].astype(np.float64), q=synth.widen(w.q[lo:hi], w.in_dtype),
+                k=synth.widen(w.k[lo:hi], w.in_dtype), v=synth.widen(w.v[lo:hi], w.in_dtype),
+                g=synth.widen(w.g[lo:hi], w.in_dtype), beta=synth.widen(w.beta[lo:hi], w.in_dtype))
+    parent, offs = w.parent[lo:hi], w.node_offsets[: n + 1]
+    poffs = w.path_offsets[: n + 1]
+    path = w.path[: int(poffs[-1])]
+
+    def run():
+        t0 = time.perf_counter()
+        orc.verify(args["S0"], args["q"], args["k"], args["v"], args["g"], args["beta"], parent, offs, w.scale)
+        orc.commit(args["S0"], args["k"], args["v"], args["g"], args["beta"], parent, offs, path, poffs)
+        return time.perf_counter() - t0
+
+    return run, hi - lo, n, orc.threads(), seqs
+
+
+def run_reference(args, w: synth.Workload):
+    """--impl reference: the oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    run, nodes, n_slots, cores, _ = oracle_sample(w, args.oracle_slots)
+    for _ in range(args.warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = nodes / dt
+    sample = f"first {n_slots} of {w.n_seq} layer slots/sequences ({nodes} nodes) per step, verify + commit"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(w: synth.Workload, args):
+    sizes = np.diff(w.node_offsets)
+    return {"workload": args.workload, "name": w.name, "n_seq_or_layer_slots": w.n_seq, "h_qk": w.h_qk, "h_v": w.h_v,
+            "d_k": w.d_k, "d_v": w.d_v, "tree_nodes": int(sizes.max()), "total_nodes": w.total_nodes,
+            "in_dtype": w.in_dtype, "state_dtype": "f32", "out_dtype": w.out_dtype,
+            "accepted_path_len_mean": float(np.diff(w.path_offsets).mean()),
+            "l2_policy": "inputs rotate over buffer sets larger than L2 in total"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=6)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="stack48_T64", choices=sorted(WORKLOADS))
+    ap.add_argument("--sets", type=int, default=0, help="buffer sets to rotate over (0 = enough to exceed 2x L2)")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--oracle-slots", type=int, default=24, help="layer slots / sequences in the oracle's sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    w = synth.config(WORKLOADS[args.workload], 0)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2607_06763_b200 as gdn
+    from paper_2607_06763_b200.binding import to_device as to_dev
+
+    gdn.load_library()   # raises if the CUDA library is missing: there is no fallback
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    shape = gdn.GdnShape.from_workload(w)
+    vbytes, cbytes, sbytes = algorithmic_bytes(w)
+    n_sets = args.sets or max(2, int(np.ceil(2 * 126e6 / sbytes)) + 1)
+    n_sets = min(n_sets, 64)
+    sets = []
+    ws_bytes = gdn.gdn_tree_workspace_bytes(shape)
+    for i in range(n_sets):
+        wi = w   # same bytes in every set, distinct device buffers
+        d = {n: to_dev(getattr(wi, n)) for n in ("S0", "q", "k", "v", "g", "beta", "parent", "node_offsets",
+                                                    "path_offsets")}
+        d["path"] = to_dev(wi.path if wi.path.size else np.zeros(1, np.int32))
+        odt = torch.float32 if w.out_dtype == synth.F32 else torch.bfloat16
+        d["o"] = torch.empty((w.total_nodes, w.h_v, w.d_v), dtype=odt, device="cuda")
+        d["ws"] = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        sets.append(d)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(d):
+        rc = gdn.gdn_tree_verify(shape, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
+                                 d["node_offsets"], d["o"], d["ws"], ws_bytes, status, stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+        rc = gdn.gdn_tree_commit(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"], d["node_offsets"],
+                                 d["path"], d["path_offsets"], status, stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(sets[i % n_sets])
+    barrier()
+    assert int(status.item()) == 0, gdn.gdn_status_string(int(status.item()))
+
+    # ---- timed region: K steps, device timing with events on the launching stream
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        d = sets[(args.warmup + i) % n_sets]
+        ev[i][0].record()
+        rc = gdn.gdn_tree_verify(shape, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
+                                 d["node_offsets"], d["o"], d["ws"], ws_bytes, status, stream)
+        ev[i][1].record()
+        rc2 = gdn.gdn_tree_commit(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"], d["node_offsets"],
+                                  d["path"], d["path_offsets"], status, stream)
+        ev[i][2].record()
+        assert rc == 0 and rc2 == 0
+    t_end.record()
+    barrier()
+    total_ms = t_start.elapsed_time(t_end)
+    time.sleep(0.15)
+    clocks = sampler.stop()
+    assert int(status.item()) == 0, gdn.gdn_status_string(int(status.item()))
+    verify_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    commit_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    nodes_per_step = w.total_nodes * world
+    value = nodes_per_step / (ms_per_step * 1e-3)
+
+    # ---- end-to-end: host buffers through the *_host entry points (copies inside the timed region)
+    L = int(w.path_offsets[-1])
+    arena_bytes = gdn.gdn_tree_host_arena_bytes(shape, L)
+    arena = torch.empty(arena_bytes, dtype=torch.uint8, device="cuda")
+    pin = {n: torch.from_numpy(np.ascontiguousarray(getattr(w, n)).view(np.int16) if getattr(w, n).dtype == np.uint16
+                               else np.ascontiguousarray(getattr(w, n))).pin_memory()
+           for n in ("S0", "q", "k", "v", "g", "beta", "parent", "node_offsets", "path_offsets")}
+    pin["path"] = torch.from_numpy(w.path if w.path.size else np.zeros(1, np.int32)).pin_memory()
+    osz = 4 if w.out_dtype == synth.F32 else 2
+    o_pin = torch.empty(w.total_nodes * w.h_v * w.d_v * osz, dtype=torch.uint8).pin_memory()
+
+    def e2e_step():
+        rc = gdn.gdn_tree_verify_host(shape, pin["S0"], pin["q"], pin["k"], pin["v"], pin["g"], pin["beta"],
+                                      pin["parent"], pin["node_offsets"], o_pin, arena, arena_bytes, stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+        rc = gdn.gdn_tree_commit_host(shape, pin["S0"], pin["k"], pin["v"], pin["g"], pin["beta"], pin["parent"],
+                                      pin["node_offsets"], pin["path"], pin["path_offsets"], L, arena, arena_bytes,
+                                      stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+
+    isz = 4 if w.in_dtype == synth.F32 else 2
+    state_b = w.n_seq * w.h_v * w.d_v * w.d_k * 4
+    qk_b, v_b, gb_b = w.total_nodes * w.h_qk * w.d_k * isz, w.total_nodes * w.h_v * w.d_v * isz, w.total_nodes * w.h_v * isz
+    idx_b = 4 * (w.total_nodes + 2 * (w.n_seq + 1) + (w.n_seq + 1) + L)
+    h2d = (state_b + 2 * qk_b + v_b + 2 * gb_b) + (state_b + qk_b + v_b + 2 * gb_b) + idx_b
+    d2h = w.total_nodes * w.h_v * w.d_v * osz + state_b + 8
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / args.e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = nodes_per_step / e2e_s
+
+    out = None
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        v_med, c_med = statistics.median(verify_ms), statistics.median(commit_ms)
+        v_avg = sum(verify_ms) / len(verify_ms)
+        achieved = vbytes / (v_avg * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(w, args),
+            "verify_us": v_med * 1e3, "commit_us": c_med * 1e3, "verify_commit_us": ms_per_step * 1e3,
+            "step_bytes": sbytes,
+            "step_roofline": {"achieved_gbs": sbytes / (ms_per_step * 1e-3) / 1e9, "peak_gbs": peak,
+                              "frac_of_" + peak_src: sbytes / (ms_per_step * 1e-3) / 1e9 / peak,
+                              "frac_of_nominal_8000": sbytes / (ms_per_step * 1e-3) / 1e9 / 8000.0},
+            "roofline": {"kernel": "verify", "bound": "hbm", "achieved": achieved, "peak": peak,
+                         "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                         "bytes_per_launch": vbytes, "avg_launch_us": v_avg * 1e3},
+            "commit_roofline": {"bound": "hbm", "achieved": cbytes / (c_med * 1e-3) / 1e9, "peak": peak,
+                                "unit": "GB/s", "frac": cbytes / (c_med * 1e-3) / 1e9 / peak,
+                                "bytes_per_launch": cbytes},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_s * 1e3},
+            "gpu_launches": 3 * args.steps,
+            "clocks": clocks, "buffer_sets": n_sets,
+            "paper_context": {"fused_verify_us_T64_one_layer_B200": 27.8, "note": "Table 1, another build; context only"},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            run, nodes, n_slots, cores, _ = oracle_sample(w, args.oracle_slots)
+            dt = run()
+            out["cpu_baseline"] = {"value": nodes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                   "sample": f"first {n_slots} of {w.n_seq} layer slots/sequences ({nodes} nodes), "
+                                             f"verify + commit, one pass, {dt:.2f} s"}
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -90,6 +90,16 @@ def load_library():
     return _lib
 
 
+def to_device(a, device="cuda"):
+    """numpy array -> torch tensor on ``device``; ``uint16`` arrays are bf16 bit patterns and come back as bf16."""
+    import numpy as np
+    import torch
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).to(device)
+    return torch.from_numpy(a).to(device)
+
+
 def _ptr(x):
     """Address of a torch tensor / numpy array / int / None."""
     if x is None:

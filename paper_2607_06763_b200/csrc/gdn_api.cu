@@ -1,0 +1,291 @@
+// C-ABI entry points of libgdn_tree.so: argument validation, workspace carving, kernel launches,
+// and the host-buffer variants.  See include/gdn_tree.h for the contract of every function.
+#include <cstring>
+
+#include "gdn_internal.cuh"
+
+using namespace gdn;
+
+namespace {
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned256(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+inline size_t dtype_size(int dt) { return dt == GDN_BF16 ? 2 : 4; }
+
+int check_shape(const gdn_shape_t *s)
+{
+    if (!s) return GDN_ERR_NULL;
+    if (s->in_dtype != GDN_F32 && s->in_dtype != GDN_BF16) return GDN_ERR_DTYPE;
+    if (s->out_dtype != GDN_F32 && s->out_dtype != GDN_BF16) return GDN_ERR_DTYPE;
+    if (s->n_seq < 0 || s->h_qk < 1 || s->h_v < 1 || s->h_v % s->h_qk != 0) return GDN_ERR_SHAPE;
+    if (s->d_k < 4 || s->d_k > GDN_MAX_HEAD_DIM || s->d_k % 4 != 0) return GDN_ERR_SHAPE;
+    if (s->d_v < 1 || s->d_v > GDN_MAX_HEAD_DIM) return GDN_ERR_SHAPE;
+    if (s->max_depth < 1 || s->max_depth > GDN_MAX_DEPTH_CAP) return GDN_ERR_SHAPE;
+    if (s->total_nodes < 0 || s->max_tree_nodes < 1 || s->max_tree_nodes > GDN_MAX_TREE_NODES)
+        return GDN_ERR_SHAPE;
+    if ((long long)s->n_seq * s->h_v > 0x7fffffffLL) return GDN_ERR_SHAPE;
+    if (!(s->scale == s->scale)) return GDN_ERR_SHAPE;   // NaN
+    // rows of q/k/v must keep 16-byte alignment of the tensor bases meaningful for vector loads
+    if ((s->d_k * dtype_size(s->in_dtype)) % 8 != 0) return GDN_ERR_SHAPE;
+    return GDN_OK;
+}
+
+struct TensorBytes {
+    size_t state, qk, v, gb, o, parent, offsets;
+};
+
+TensorBytes tensor_bytes(const gdn_shape_t &s)
+{
+    const size_t N = (size_t)s.total_nodes, isz = dtype_size(s.in_dtype), osz = dtype_size(s.out_dtype);
+    TensorBytes t;
+    t.state = (size_t)s.n_seq * s.h_v * s.d_v * s.d_k * sizeof(float);
+    t.qk = N * s.h_qk * s.d_k * isz;
+    t.v = N * s.h_v * s.d_v * isz;
+    t.gb = N * s.h_v * isz;
+    t.o = N * s.h_v * s.d_v * osz;
+    t.parent = N * sizeof(int32_t);
+    t.offsets = ((size_t)s.n_seq + 1) * sizeof(int32_t);
+    return t;
+}
+
+// Bump allocator over the caller's device arena (host-buffer entry points).
+struct Arena {
+    char *base;
+    size_t off, cap;
+    void *take(size_t bytes)
+    {
+        void *p = base + off;
+        off = align256(off + bytes);
+        return off <= cap ? p : nullptr;
+    }
+};
+
+}  // namespace
+
+extern "C" const char *gdn_status_string(int status)
+{
+    switch (status) {
+    case GDN_OK: return "ok";
+    case GDN_ERR_NULL: return "a required pointer is NULL";
+    case GDN_ERR_SHAPE: return "a size is out of range or inconsistent";
+    case GDN_ERR_DTYPE: return "unknown dtype";
+    case GDN_ERR_ALIGN: return "a pointer is not aligned as required";
+    case GDN_ERR_UNSUPPORTED: return "request not supported by this build";
+    case GDN_ERR_CUDA: return "a CUDA runtime call failed";
+    case GDN_ERR_TREE: return "parent[]/node_offsets[] do not describe a topological forest";
+    case GDN_ERR_DEPTH: return "a root path has more than max_depth nodes";
+    case GDN_ERR_PATH: return "accepted path is not a root chain of its tree";
+    case GDN_ERR_WORKSPACE: return "workspace missing or too small";
+    case GDN_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+    }
+}
+
+extern "C" size_t gdn_tree_workspace_bytes(const gdn_shape_t *shape)
+{
+    if (check_shape(shape) != GDN_OK) return 0;
+    return workspace_layout(*shape).total;
+}
+
+extern "C" int gdn_tree_validate_host(const gdn_shape_t *shape, const int32_t *parent_h,
+                                      const int32_t *node_offsets_h, const int32_t *path_h,
+                                      const int32_t *path_offsets_h)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    if (!node_offsets_h || (!parent_h && shape->total_nodes > 0)) return GDN_ERR_NULL;
+    if ((path_h == nullptr) != (path_offsets_h == nullptr) && path_offsets_h == nullptr) return GDN_ERR_NULL;
+    const gdn_shape_t &s = *shape;
+    if (node_offsets_h[0] != 0 || node_offsets_h[s.n_seq] != s.total_nodes) return GDN_ERR_TREE;
+    for (int b = 0; b < s.n_seq; ++b) {
+        const int lo = node_offsets_h[b], T = node_offsets_h[b + 1] - lo;
+        if (T < 0 || T > s.max_tree_nodes) return GDN_ERR_TREE;
+    }
+    // depth of every node by one forward pass (parents come first)
+    int worst = GDN_OK;
+    for (int b = 0; b < s.n_seq && worst == GDN_OK; ++b) {
+        const int lo = node_offsets_h[b], T = node_offsets_h[b + 1] - lo;
+        for (int i = 0; i < T; ++i) {
+            const int p = parent_h[lo + i];
+            if (p < -1 || p >= i) return GDN_ERR_TREE;
+        }
+        for (int i = 0; i < T; ++i) {
+            int d = 0;
+            for (int cur = i; cur >= 0; cur = parent_h[lo + cur])
+                if (++d > s.max_depth) return GDN_ERR_DEPTH;
+        }
+    }
+    if (path_offsets_h) {
+        if (path_offsets_h[0] != 0) return GDN_ERR_PATH;
+        for (int b = 0; b < s.n_seq; ++b) {
+            const int lo = node_offsets_h[b], T = node_offsets_h[b + 1] - lo;
+            const int p0 = path_offsets_h[b], L = path_offsets_h[b + 1] - p0;
+            if (L < 0 || L > s.max_depth) return GDN_ERR_PATH;
+            if (L > 0 && !path_h) return GDN_ERR_NULL;
+            for (int t = 0; t < L; ++t) {
+                const int n = path_h[p0 + t];
+                if (n < 0 || n >= T) return GDN_ERR_PATH;
+                if (parent_h[lo + n] != (t ? path_h[p0 + t - 1] : -1)) return GDN_ERR_PATH;
+            }
+        }
+    }
+    return worst;
+}
+
+extern "C" int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const void *q, const void *k,
+                               const void *v, const void *g, const void *beta, const int32_t *parent,
+                               const int32_t *node_offsets, void *o, void *workspace,
+                               size_t workspace_bytes, int32_t *status_dev, void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
+    if (!S0 || !q || !k || !v || !g || !beta || !parent || !node_offsets || !o || !status_dev)
+        return GDN_ERR_NULL;
+    if (!workspace) return GDN_ERR_WORKSPACE;
+    if (!aligned16(S0) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) ||
+        !aligned16(beta) || !aligned16(o) || !aligned256(workspace) ||
+        (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(node_offsets) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    const WorkspaceLayout lay = workspace_layout(s);
+    if (workspace_bytes < lay.total) return GDN_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const PlanPtrs plan = plan_ptrs(workspace, lay);
+    if (launch_plan(s, parent, node_offsets, plan, status_dev, stream) != cudaSuccess) return GDN_ERR_CUDA;
+    if (launch_verify_generic(s, S0, q, k, v, g, beta, node_offsets, o, plan, stream) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
+extern "C" int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k, const void *v,
+                               const void *g, const void *beta, const int32_t *parent,
+                               const int32_t *node_offsets, const int32_t *path,
+                               const int32_t *path_offsets, int32_t *status_dev, void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0) return GDN_OK;
+    if (!S || !node_offsets || !path_offsets || !status_dev) return GDN_ERR_NULL;
+    if (s.total_nodes > 0 && (!k || !v || !g || !beta || !path)) return GDN_ERR_NULL;
+    if (!aligned16(S) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(node_offsets) & 3u) ||
+        (reinterpret_cast<uintptr_t>(path) & 3u) || (reinterpret_cast<uintptr_t>(path_offsets) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (launch_commit_generic(s, S, k, v, g, beta, parent, node_offsets, path, path_offsets, status_dev,
+                              stream) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
+extern "C" size_t gdn_tree_host_arena_bytes(const gdn_shape_t *shape, int32_t total_path_len)
+{
+    if (check_shape(shape) != GDN_OK || total_path_len < 0) return 0;
+    const TensorBytes t = tensor_bytes(*shape);
+    size_t n = 0;
+    n += align256(t.state) + 2 * align256(t.qk) + align256(t.v) + 2 * align256(t.gb) + align256(t.o);
+    n += align256(t.parent) + 2 * align256(t.offsets) + align256((size_t)total_path_len * sizeof(int32_t) + 4);
+    n += align256(sizeof(int32_t));            // status word
+    n += workspace_layout(*shape).total;       // verify workspace
+    return n + 256;
+}
+
+#define GDN_CUDA_TRY(expr)                         \
+    do {                                           \
+        if ((expr) != cudaSuccess) return GDN_ERR_CUDA; \
+    } while (0)
+
+extern "C" int gdn_tree_verify_host(const gdn_shape_t *shape, const float *S0_h, const void *q_h,
+                                    const void *k_h, const void *v_h, const void *g_h,
+                                    const void *beta_h, const int32_t *parent_h,
+                                    const int32_t *node_offsets_h, void *o_h, void *dev_arena,
+                                    size_t arena_bytes, void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
+    if (!S0_h || !q_h || !k_h || !v_h || !g_h || !beta_h || !parent_h || !node_offsets_h || !o_h)
+        return GDN_ERR_NULL;
+    if (!dev_arena || arena_bytes < gdn_tree_host_arena_bytes(shape, 0)) return GDN_ERR_WORKSPACE;
+    if (!aligned256(dev_arena)) return GDN_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const TensorBytes t = tensor_bytes(s);
+    Arena a{static_cast<char *>(dev_arena), 0, arena_bytes};
+    float *S0 = static_cast<float *>(a.take(t.state));
+    void *q = a.take(t.qk), *k = a.take(t.qk), *v = a.take(t.v), *g = a.take(t.gb), *beta = a.take(t.gb);
+    void *o = a.take(t.o);
+    int32_t *parent = static_cast<int32_t *>(a.take(t.parent));
+    int32_t *offs = static_cast<int32_t *>(a.take(t.offsets));
+    int32_t *status = static_cast<int32_t *>(a.take(sizeof(int32_t)));
+    const size_t ws_bytes = workspace_layout(s).total;
+    void *ws = a.take(ws_bytes);
+    if (!ws) return GDN_ERR_WORKSPACE;
+    GDN_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(S0, S0_h, t.state, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(q, q_h, t.qk, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(k, k_h, t.qk, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(v, v_h, t.v, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(g, g_h, t.gb, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(beta, beta_h, t.gb, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(parent, parent_h, t.parent, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(offs, node_offsets_h, t.offsets, cudaMemcpyHostToDevice, stream));
+    rc = gdn_tree_verify(shape, S0, q, k, v, g, beta, parent, offs, o, ws, ws_bytes, status, cuda_stream);
+    if (rc != GDN_OK) return rc;
+    int32_t status_h = 0;
+    GDN_CUDA_TRY(cudaMemcpyAsync(o_h, o, t.o, cudaMemcpyDeviceToHost, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(&status_h, status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    GDN_CUDA_TRY(cudaStreamSynchronize(stream));
+    return status_h;
+}
+
+extern "C" int gdn_tree_commit_host(const gdn_shape_t *shape, float *S_h, const void *k_h,
+                                    const void *v_h, const void *g_h, const void *beta_h,
+                                    const int32_t *parent_h, const int32_t *node_offsets_h,
+                                    const int32_t *path_h, const int32_t *path_offsets_h,
+                                    int32_t total_path_len, void *dev_arena, size_t arena_bytes,
+                                    void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || total_path_len == 0) return GDN_OK;
+    if (total_path_len < 0) return GDN_ERR_SHAPE;
+    if (!S_h || !k_h || !v_h || !g_h || !beta_h || !node_offsets_h || !path_h || !path_offsets_h)
+        return GDN_ERR_NULL;
+    if (!dev_arena || arena_bytes < gdn_tree_host_arena_bytes(shape, total_path_len)) return GDN_ERR_WORKSPACE;
+    if (!aligned256(dev_arena)) return GDN_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const TensorBytes t = tensor_bytes(s);
+    Arena a{static_cast<char *>(dev_arena), 0, arena_bytes};
+    float *S = static_cast<float *>(a.take(t.state));
+    void *k = a.take(t.qk), *v = a.take(t.v), *g = a.take(t.gb), *beta = a.take(t.gb);
+    int32_t *parent = parent_h ? static_cast<int32_t *>(a.take(t.parent)) : nullptr;
+    int32_t *offs = static_cast<int32_t *>(a.take(t.offsets));
+    int32_t *poffs = static_cast<int32_t *>(a.take(t.offsets));
+    const size_t path_bytes = (size_t)total_path_len * sizeof(int32_t);
+    int32_t *path = static_cast<int32_t *>(a.take(path_bytes));
+    int32_t *status = static_cast<int32_t *>(a.take(sizeof(int32_t)));
+    if (!status) return GDN_ERR_WORKSPACE;
+    GDN_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(S, S_h, t.state, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(k, k_h, t.qk, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(v, v_h, t.v, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(g, g_h, t.gb, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(beta, beta_h, t.gb, cudaMemcpyHostToDevice, stream));
+    if (parent) GDN_CUDA_TRY(cudaMemcpyAsync(parent, parent_h, t.parent, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(offs, node_offsets_h, t.offsets, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(poffs, path_offsets_h, t.offsets, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(path, path_h, path_bytes, cudaMemcpyHostToDevice, stream));
+    rc = gdn_tree_commit(shape, S, k, v, g, beta, parent, offs, path, poffs, status, cuda_stream);
+    if (rc != GDN_OK) return rc;
+    int32_t status_h = 0;
+    GDN_CUDA_TRY(cudaMemcpyAsync(S_h, S, t.state, cudaMemcpyDeviceToHost, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(&status_h, status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    GDN_CUDA_TRY(cudaStreamSynchronize(stream));
+    return status_h;
+}

@@ -1,0 +1,155 @@
+// Commit kernel: replay Eq. 7 along the accepted root path and write the state in place
+// (Section 3.4: the commit is delayed until the accepted branch is known and is "a short
+// recurrence"; Section 3.4.2: it is the only state write of a decode step).
+//
+// With S' = alpha S (decay first), Eq. 7 reads S <- S' - beta k (k^T S') + beta k v^T, i.e. per
+// value component c (one contiguous row of the [d_v][d_k] tile):
+//     s_c <- alpha s_c + k * beta (v_c - alpha (k . s_c)).
+// One CTA per (tree, value head); thread (c, s) owns 32 floats of row c (quarter s of the key
+// dimension, interleaved in 16-byte pieces so that the four lanes of a row read 64 contiguous
+// bytes) and k . s_c is reduced over the four lanes with warp shuffles.  The path nodes' k rows
+// are fetched once into shared memory; the state is read once and written once.
+#include "gdn_internal.cuh"
+
+namespace gdn {
+
+namespace {
+
+constexpr int CM_THREADS = 512;
+constexpr int CM_SPLIT = 4;
+constexpr int CM_DK = GDN_MAX_HEAD_DIM;
+constexpr int CM_REGS = CM_DK / CM_SPLIT;
+
+struct CommitParams {
+    int h_qk, h_v, d_k, d_v, max_depth;
+    float *S;
+    const void *k, *v, *g, *beta;
+    const int32_t *parent, *node_offsets, *path, *path_offsets;
+    int32_t *status_dev;
+};
+
+template <typename TIn>
+__global__ void __launch_bounds__(CM_THREADS, 1) commit_generic_kernel(const CommitParams p)
+{
+    extern __shared__ __align__(16) float cm_smem[];
+    float (*ks)[CM_DK] = reinterpret_cast<float (*)[CM_DK]>(cm_smem);   // [L][CM_DK]
+    float *alpha_s = cm_smem + (size_t)p.max_depth * CM_DK;             // [L]
+    float *beta_s = alpha_s + p.max_depth;                              // [L]
+    __shared__ int path_bad;
+
+    const int b = blockIdx.x / p.h_v, h = blockIdx.x % p.h_v;
+    const int base = p.node_offsets[b];
+    const int T = p.node_offsets[b + 1] - base;
+    const int p0 = p.path_offsets[b];
+    const int L = p.path_offsets[b + 1] - p0;
+    if (L == 0) return;   // nothing accepted from this tree: state untouched
+    const int tid = threadIdx.x;
+    const int d_k = p.d_k, d_v = p.d_v;
+
+    // The accepted path must be a chain from a root inside this tree.
+    if (tid == 0) {
+        int bad = (L < 0 || L > p.max_depth || T <= 0 || p0 < 0);
+        for (int t = 0; !bad && t < L; ++t) {
+            const int n = p.path[p0 + t];
+            if (n < 0 || n >= T) { bad = 1; break; }
+            if (p.parent) {
+                const int want = t ? p.path[p0 + t - 1] : -1;
+                if (p.parent[base + n] != want) bad = 1;
+            } else if (t && n <= p.path[p0 + t - 1]) {
+                bad = 1;   // without parent[] only the topological order can be checked
+            }
+        }
+        path_bad = bad;
+        if (bad) report_status(p.status_dev, GDN_ERR_PATH);
+    }
+    __syncthreads();
+    if (path_bad) return;
+
+    const int hk = h / (p.h_v / p.h_qk);
+    const int c = tid / CM_SPLIT, s = tid % CM_SPLIT;
+    const bool comp_on = c < d_v;
+    const TIn *k = static_cast<const TIn *>(p.k), *v = static_cast<const TIn *>(p.v);
+    const TIn *g = static_cast<const TIn *>(p.g), *beta = static_cast<const TIn *>(p.beta);
+
+    // k rows of the path (fp32, zero padded to CM_DK) and the per-step scalars
+    for (int idx = tid; idx < L * CM_DK; idx += CM_THREADS) {
+        const int t = idx / CM_DK, r = idx % CM_DK;
+        const size_t n = (size_t)base + p.path[p0 + t];
+        ks[t][r] = r < d_k ? load_as_float(k + (n * p.h_qk + hk) * d_k + r) : 0.f;
+    }
+    if (tid < L) {
+        const size_t n = (size_t)base + p.path[p0 + tid];
+        alpha_s[tid] = expf(load_as_float(g + n * p.h_v + h));
+        beta_s[tid] = load_as_float(beta + n * p.h_v + h);
+    }
+
+    float *row = p.S + ((size_t)(b * p.h_v + h) * d_v + (comp_on ? c : 0)) * d_k;
+    float sreg[CM_REGS];
+#pragma unroll
+    for (int j = 0; j < CM_REGS / 4; ++j) {
+        const int r = 16 * j + 4 * s;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (comp_on && r < d_k) x = *reinterpret_cast<const float4 *>(row + r);
+        sreg[4 * j + 0] = x.x; sreg[4 * j + 1] = x.y; sreg[4 * j + 2] = x.z; sreg[4 * j + 3] = x.w;
+    }
+    __syncthreads();
+
+    for (int t = 0; t < L; ++t) {
+        float kreg[CM_REGS];
+        float dot = 0.f;
+#pragma unroll
+        for (int j = 0; j < CM_REGS / 4; ++j) {
+            const float4 kx = *reinterpret_cast<const float4 *>(&ks[t][16 * j + 4 * s]);
+            kreg[4 * j + 0] = kx.x; kreg[4 * j + 1] = kx.y; kreg[4 * j + 2] = kx.z; kreg[4 * j + 3] = kx.w;
+        }
+#pragma unroll
+        for (int e = 0; e < CM_REGS; ++e) dot = fmaf(kreg[e], sreg[e], dot);
+        dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+        dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+        const size_t n = (size_t)base + p.path[p0 + t];
+        const float vc = comp_on ? load_as_float(v + (n * p.h_v + h) * d_v + c) : 0.f;
+        const float alpha = alpha_s[t];
+        const float w = beta_s[t] * (vc - alpha * dot);
+#pragma unroll
+        for (int e = 0; e < CM_REGS; ++e) sreg[e] = fmaf(kreg[e], w, alpha * sreg[e]);
+    }
+
+    if (comp_on) {
+#pragma unroll
+        for (int j = 0; j < CM_REGS / 4; ++j) {
+            const int r = 16 * j + 4 * s;
+            if (r < d_k)
+                *reinterpret_cast<float4 *>(row + r) =
+                    make_float4(sreg[4 * j + 0], sreg[4 * j + 1], sreg[4 * j + 2], sreg[4 * j + 3]);
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k, const void *v,
+                                  const void *g, const void *beta, const int32_t *parent,
+                                  const int32_t *node_offsets, const int32_t *path,
+                                  const int32_t *path_offsets, int32_t *status_dev, cudaStream_t stream)
+{
+    const int grid = s.n_seq * s.h_v;
+    if (grid == 0) return cudaSuccess;
+    CommitParams p{s.h_qk, s.h_v, s.d_k, s.d_v, s.max_depth, S, k, v, g, beta,
+                   parent, node_offsets, path, path_offsets, status_dev};
+    const size_t smem = sizeof(float) * ((size_t)s.max_depth * CM_DK + 2 * (size_t)s.max_depth);
+    cudaError_t e;
+    if (s.in_dtype == GDN_BF16) {
+        e = cudaFuncSetAttribute(commit_generic_kernel<__nv_bfloat16>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        commit_generic_kernel<__nv_bfloat16><<<grid, CM_THREADS, smem, stream>>>(p);
+    } else {
+        e = cudaFuncSetAttribute(commit_generic_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem);
+        if (e != cudaSuccess) return e;
+        commit_generic_kernel<float><<<grid, CM_THREADS, smem, stream>>>(p);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace gdn

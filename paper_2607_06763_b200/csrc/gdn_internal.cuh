@@ -1,0 +1,87 @@
+// Internal declarations shared by the translation units of libgdn_tree.so.
+// Nothing here is part of the public ABI (that is include/gdn_tree.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gdn_tree.h"
+
+namespace gdn {
+
+// Layout of the caller-provided verify workspace (all offsets 256-byte aligned).
+//   tree_ok  int32 [n_seq]                 1 = tree passed the metadata checks
+//   depth    uint8 [N]                     nodes on the root path of node n (root = 1)
+//   anc      uint16[N][max_depth]          local ids of the root path of n, root first, n itself last
+//   utilde   float [N][h_v][d_v]           solve result u~ (Eq. 10 with the W S0 term folded in)
+struct WorkspaceLayout {
+    size_t tree_ok, depth, anc, utilde, total;
+};
+
+inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
+{
+    WorkspaceLayout w;
+    size_t off = 0;
+    const size_t N = (size_t)s.total_nodes;
+    w.tree_ok = off;  off = align256(off + sizeof(int32_t) * (size_t)s.n_seq);
+    w.depth = off;    off = align256(off + N);
+    w.anc = off;      off = align256(off + sizeof(uint16_t) * N * (size_t)s.max_depth);
+    w.utilde = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
+    w.total = off;
+    return w;
+}
+
+struct PlanPtrs {
+    int32_t *tree_ok;
+    uint8_t *depth;
+    uint16_t *anc;
+    float *utilde;
+};
+
+inline PlanPtrs plan_ptrs(void *workspace, const WorkspaceLayout &w)
+{
+    char *b = static_cast<char *>(workspace);
+    return {reinterpret_cast<int32_t *>(b + w.tree_ok), reinterpret_cast<uint8_t *>(b + w.depth),
+            reinterpret_cast<uint16_t *>(b + w.anc), reinterpret_cast<float *>(b + w.utilde)};
+}
+
+// Host launchers (each returns the cudaError_t of its launch).
+cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32_t *node_offsets,
+                        const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream);
+
+cudaError_t launch_verify_generic(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
+                                  const void *v, const void *g, const void *beta,
+                                  const int32_t *node_offsets, void *o, const PlanPtrs &plan,
+                                  cudaStream_t stream);
+
+cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k, const void *v,
+                                  const void *g, const void *beta, const int32_t *parent,
+                                  const int32_t *node_offsets, const int32_t *path,
+                                  const int32_t *path_offsets, int32_t *status_dev, cudaStream_t stream);
+
+#ifdef __CUDACC__
+// First error wins; later ones are dropped.
+__device__ __forceinline__ void report_status(int32_t *status_dev, int code)
+{
+    if (status_dev) atomicCAS(status_dev, 0, code);
+}
+
+template <typename T> __device__ __forceinline__ float load_as_float(const T *p);
+template <> __device__ __forceinline__ float load_as_float<float>(const float *p) { return __ldg(p); }
+template <> __device__ __forceinline__ float load_as_float<__nv_bfloat16>(const __nv_bfloat16 *p)
+{
+    return __bfloat162float(__ldg(p));
+}
+
+template <typename T> __device__ __forceinline__ void store_from_float(T *p, float x);
+template <> __device__ __forceinline__ void store_from_float<float>(float *p, float x) { *p = x; }
+template <> __device__ __forceinline__ void store_from_float<__nv_bfloat16>(__nv_bfloat16 *p, float x)
+{
+    *p = __float2bfloat16_rn(x);
+}
+#endif
+
+}  // namespace gdn

@@ -1,0 +1,249 @@
+"""GPU parity: the CUDA library (through the C ABI) against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+
+from paper_2607_06763_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tl(cuda_device):
+    from tests import gdn_testlib
+    return gdn_testlib
+
+
+def _check_full(tl, w, what, max_depth=16):
+    """verify + commit on the GPU, whole-workload oracle comparison."""
+    dc = tl.DeviceCase(w, max_depth=max_depth)
+    S0_before = dc.S0.clone()
+    assert dc.verify() == 0
+    assert dc.device_status() == 0
+    assert bool((dc.S0 == S0_before).all()), "verify must leave the state bit-identical"
+    ref = tl.oracle_verify(w)
+    tl.assert_close_per_head(dc.o_host(), ref, w.node_offsets, what + " o", bf16_out=tl.is_bf16_out(w))
+    assert dc.commit() == 0
+    assert dc.device_status() == 0
+    tl.assert_state_close(dc.S0.cpu().numpy().astype(np.float64), tl.oracle_commit(w), what=what + " S_new")
+    return dc
+
+
+def _check_sampled(tl, w, seqs, what):
+    """verify + commit on the full workload; the oracle evaluates only the sampled sequences."""
+    dc = tl.DeviceCase(w)
+    assert dc.verify() == 0
+    assert dc.device_status() == 0
+    o = dc.o_host()
+    assert np.all(np.isfinite(o))
+    sub, nodes = tl.sub_workload(w, seqs)
+    tl.assert_close_per_head(o[nodes], tl.oracle_verify(sub), sub.node_offsets, what + " o",
+                             bf16_out=tl.is_bf16_out(w))
+    assert dc.commit() == 0
+    assert dc.device_status() == 0
+    S = dc.S0.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(S))
+    tl.assert_state_close(S[list(seqs)], tl.oracle_commit(sub), what=what + " S_new")
+    # sequences with an empty accepted path keep their state bit for bit
+    for b in range(w.n_seq):
+        if w.path_offsets[b + 1] == w.path_offsets[b]:
+            np.testing.assert_array_equal(S[b].astype(np.float32), w.S0[b])
+
+
+@pytest.mark.parametrize("rep", [0, 1, 2])
+def test_config0_tiny_fp32(tl, rep):
+    _check_full(tl, synth.config(0, rep), f"cfg0 rep{rep}")
+
+
+@pytest.mark.parametrize("rep", [0, 1, 2])
+@pytest.mark.parametrize("out_dtype", [synth.BF16, synth.F32])
+def test_config1_single_layer(tl, rep, out_dtype):
+    _check_full(tl, synth.config(1, rep, out_dtype=out_dtype), f"cfg1 rep{rep} {out_dtype}")
+
+
+def test_config5_stack48_T64_sampled(tl):
+    w = synth.config(5, 0)
+    _check_sampled(tl, w, [0, 17, 47], "cfg1x48")
+
+
+def test_config2_stack48_T256_sampled(tl):
+    w = synth.config(2, 0)
+    _check_sampled(tl, w, [3, 47], "cfg2")
+
+
+def test_config3_ragged_sampled(tl):
+    w = synth.config(3, 0)
+    sizes = np.diff(w.node_offsets)
+    seqs = sorted({0, int(np.argmin(sizes)), int(np.argmax(sizes)), 31})
+    _check_sampled(tl, w, seqs, "cfg3")
+
+
+def test_config4_chains_sampled(tl):
+    w = synth.config(4, 0)
+    L = np.diff(w.path_offsets)
+    seqs = sorted({0, int(np.argmin(L)), int(np.argmax(L)), 63})
+    _check_sampled(tl, w, seqs, "cfg4")
+
+
+# ------------------------------------------------------------------ edge shapes
+def _edge_trees():
+    rng = np.random.default_rng(7)
+    deep = synth.tree_chain(16)
+    return {
+        "single": [np.array([-1], np.int32)],
+        "star": [synth.tree_star(37)],
+        "chain16": [deep],
+        "forest": [np.array([-1, -1, 0, 1, 1, -1, 5, 2], np.int32)],
+        "ragged_tail": [synth.tree_geo(rng, 33), synth.tree_geo(rng, 1), synth.tree_geo(rng, 95),
+                        synth.tree_geo(rng, 130)],
+        "bestfirst": [synth.tree_bestfirst(rng, 64)],
+    }
+
+
+@pytest.mark.parametrize("name", ["single", "star", "chain16", "forest", "ragged_tail", "bestfirst"])
+@pytest.mark.parametrize("dims", [(2, 4, 128, 128, synth.BF16, synth.F32), (1, 1, 64, 64, synth.BF16, synth.BF16),
+                                  (2, 2, 32, 48, synth.F32, synth.F32), (1, 3, 20, 7, synth.F32, synth.BF16)])
+def test_edge_shapes(tl, name, dims):
+    h_qk, h_v, d_k, d_v, idt, odt = dims
+    w = synth.random_case(100 + len(name), _edge_trees()[name], h_qk, h_v, d_k, d_v, idt, odt, name=name)
+    _check_full(tl, w, f"{name} {dims}")
+
+
+def test_deep_chain_needs_larger_max_depth(tl):
+    w = synth.random_case(5, [synth.tree_chain(40)], 1, 2, 64, 64, synth.F32, synth.F32,
+                          paths=[np.arange(40, dtype=np.int32)])
+    _check_full(tl, w, "chain40", max_depth=40)
+    dc = tl.DeviceCase(w, max_depth=16)
+    sentinel = 123.0
+    dc.o.fill_(sentinel)
+    assert dc.verify() == 0
+    assert dc.device_status() == -8  # GDN_ERR_DEPTH
+    assert bool((dc.o == sentinel).all()), "a rejected tree must produce no output"
+
+
+def test_empty_inputs(tl):
+    import torch
+    import paper_2607_06763_b200 as gdn
+    w = synth.random_case(1, [np.array([-1], np.int32)], 1, 1, 32, 32)
+    dc = tl.DeviceCase(w)
+    dc.shape.n_seq = 0
+    dc.shape.total_nodes = 0
+    assert dc.verify() == 0 and dc.commit() == 0
+    # an all-empty accepted path set leaves every state untouched
+    w2 = synth.random_case(2, [synth.tree_chain(5), synth.tree_star(4)], 1, 2, 32, 32,
+                           paths=[np.zeros(0, np.int32), np.zeros(0, np.int32)])
+    dc2 = tl.DeviceCase(w2)
+    before = dc2.S0.clone()
+    assert dc2.commit() == 0 and dc2.device_status() == 0
+    assert bool((dc2.S0 == before).all())
+    assert gdn.gdn_status_string(0) == "ok"
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ invariants on GPU results
+def test_chain_equals_token_by_token_commit(tl):
+    """A chain's node t output equals a 1-node verify after committing the first t tokens one by one."""
+    T = 6
+    w = synth.random_case(9, [synth.tree_chain(T)], 2, 4, 128, 128, synth.BF16, synth.F32)
+    dc = tl.DeviceCase(w)
+    assert dc.verify() == 0 and dc.device_status() == 0
+    o_tree = dc.o_host()
+    S = w.S0.copy()
+    for t in range(T):
+        sl = slice(t, t + 1)
+        one = synth.Workload("one", 1, w.h_qk, w.h_v, w.d_k, w.d_v, w.in_dtype, w.out_dtype, w.scale, S.copy(), w.q[sl],
+                             w.k[sl], w.v[sl], w.g[sl], w.beta[sl], np.array([-1], np.int32),
+                             np.array([0, 1], np.int32), np.array([0], np.int32), np.array([0, 1], np.int32))
+        d1 = tl.DeviceCase(one)
+        assert d1.verify() == 0 and d1.commit() == 0 and d1.device_status() == 0
+        np.testing.assert_allclose(d1.o_host()[0], o_tree[t], rtol=2e-4, atol=2e-5)
+        S = d1.S0.cpu().numpy()
+
+
+def test_sibling_permutation_permutes_outputs(tl):
+    rng = np.random.default_rng(3)
+    t = synth.tree_geo(rng, 40)
+    w = synth.random_case(3, [t], 2, 4, 128, 128, synth.BF16, synth.F32)
+    # swap two sibling subtrees by a valid renumbering: reverse the order of nodes within each BFS level
+    d = synth.depths(t)
+    order = np.concatenate([np.nonzero(d == lev)[0][::-1] for lev in range(1, d.max() + 1)])
+    new_id = np.empty(len(t), np.int64)
+    new_id[order] = np.arange(len(t))
+    w2 = synth.random_case(3, [t], 2, 4, 128, 128, synth.BF16, synth.F32)
+    w2.parent = np.asarray([-1 if t[old] < 0 else new_id[t[old]] for old in order], dtype=np.int32)
+    for name in ("q", "k", "v", "g", "beta"):
+        setattr(w2, name, np.ascontiguousarray(getattr(w, name)[order]))
+    a, b = tl.DeviceCase(w), tl.DeviceCase(w2)
+    assert a.verify() == 0 and b.verify() == 0 and a.device_status() == 0 and b.device_status() == 0
+    np.testing.assert_allclose(b.o_host(), a.o_host()[order], rtol=1e-5, atol=1e-6)
+
+
+# ------------------------------------------------------------------ error reporting (host-made faults only)
+def test_device_side_rejections(tl):
+    w = synth.random_case(11, [synth.tree_chain(6), synth.tree_star(5)], 1, 2, 64, 64, synth.F32, synth.F32,
+                          paths=[np.array([0, 1, 2], np.int32), np.array([0, 3], np.int32)])
+    # (1) parent[] not topological in tree 0: tree 0 yields nothing, tree 1 is still verified
+    bad = synth.random_case(11, [synth.tree_chain(6), synth.tree_star(5)], 1, 2, 64, 64, synth.F32, synth.F32)
+    bad.parent = w.parent.copy()
+    bad.parent[2] = 4
+    dc = tl.DeviceCase(bad)
+    dc.o.fill_(77.0)
+    assert dc.verify() == 0
+    assert dc.device_status() == -7  # GDN_ERR_TREE
+    o = dc.o_host()
+    assert np.all(o[:6] == 77.0)
+    good = tl.oracle_verify(w)
+    tl.assert_close_per_head(o[6:], good[6:], np.array([0, 5]), "tree after a rejected one")
+    # (2) accepted path that is not a chain from a root: state unchanged, status set
+    wp = synth.random_case(11, [synth.tree_chain(6), synth.tree_star(5)], 1, 2, 64, 64, synth.F32, synth.F32,
+                           paths=[np.array([0, 2], np.int32), np.array([0, 3], np.int32)])
+    dp = tl.DeviceCase(wp)
+    before = dp.S0.clone()
+    assert dp.commit() == 0
+    assert dp.device_status() == -9  # GDN_ERR_PATH
+    assert bool((dp.S0[0] == before[0]).all()), "rejected path must leave the state untouched"
+    sub, _ = tl.sub_workload(wp, [1])
+    tl.assert_state_close(dp.S0[1:2].cpu().numpy().astype(np.float64), tl.oracle_commit(sub))
+
+
+def test_host_side_rejections(tl):
+    import paper_2607_06763_b200 as gdn
+    w = synth.random_case(12, [synth.tree_chain(4)], 1, 2, 64, 64)
+    dc = tl.DeviceCase(w)
+    args = (dc.S0, dc.q, dc.k, dc.v, dc.g, dc.beta, dc.parent, dc.node_offsets, dc.o, dc.ws, dc.ws_bytes, dc.status)
+    assert gdn.gdn_tree_verify(dc.shape, None, *args[1:]) == -1           # NULL
+    assert gdn.gdn_tree_verify(dc.shape, dc.S0.data_ptr() + 4, *args[1:]) == -4   # misaligned
+    assert gdn.gdn_tree_verify(dc.shape, *args[:9], dc.ws, dc.ws_bytes - 1, dc.status) == -10  # workspace too small
+    s = gdn.GdnShape.from_workload(w)
+    s.d_k = 130
+    assert gdn.gdn_tree_verify(s, *args) == -2
+    s = gdn.GdnShape.from_workload(w)
+    s.in_dtype = 9
+    assert gdn.gdn_tree_verify(s, *args) == -3
+    s = gdn.GdnShape.from_workload(w)
+    s.h_v = 3
+    s.h_qk = 2
+    assert gdn.gdn_tree_commit(s, dc.S0, dc.k, dc.v, dc.g, dc.beta, dc.parent, dc.node_offsets, dc.path,
+                               dc.path_offsets, dc.status) == -2
+    assert dc.device_status() == 0
+
+
+# ------------------------------------------------------------------ host-buffer entry points
+def test_host_buffer_entry_points(tl):
+    import torch
+    import paper_2607_06763_b200 as gdn
+    w = synth.config(1, 0)
+    shape = gdn.GdnShape.from_workload(w)
+    L = int(w.path_offsets[-1])
+    arena_bytes = gdn.gdn_tree_host_arena_bytes(shape, L)
+    arena = torch.empty(arena_bytes, dtype=torch.uint8, device="cuda")
+    o_h = np.zeros((w.total_nodes, w.h_v, w.d_v), dtype=np.uint16)
+    rc = gdn.gdn_tree_verify_host(shape, w.S0, w.q, w.k, w.v, w.g, w.beta, w.parent, w.node_offsets, o_h, arena,
+                                  arena_bytes)
+    assert rc == 0
+    tl.assert_close_per_head(synth.bf16_bits_to_f32(o_h).astype(np.float64), tl.oracle_verify(w), w.node_offsets,
+                             "verify_host o", bf16_out=True)
+    S_h = w.S0.copy()
+    rc = gdn.gdn_tree_commit_host(shape, S_h, w.k, w.v, w.g, w.beta, w.parent, w.node_offsets, w.path,
+                                  w.path_offsets, L, arena, arena_bytes)
+    assert rc == 0
+    tl.assert_state_close(S_h.astype(np.float64), tl.oracle_commit(w), what="commit_host S_new")
