@@ -9,7 +9,8 @@ from paper_2607_06763_b200 import synth
 # Tolerances.  The arithmetic is held to |gpu - ref| <= 1e-4*|ref| + 1e-4*rms(ref over the same tree and head)
 # for outputs and for the committed state.  A bf16 output additionally carries its own rounding: round-to-nearest
 # with an 8-bit significand is off by at most 2^-8*|ref|, so that much is added elementwise, and the norm-wise
-# relative error of a head (about 1.6e-3 for ideally rounded values) must stay below 2e-3.
+# relative error of a head (about 1.6e-3 for ideally rounded values, a statistical figure, hence only checked
+# where a head has at least 1024 output elements) must stay below 2e-3.
 TOL_F32 = 1e-4
 TOL_STATE = 1e-4
 BF16_HALF_ULP = 2.0 ** -8
@@ -103,7 +104,7 @@ def assert_close_per_head(got: np.ndarray, ref: np.ndarray, node_offsets, what: 
         bound = tol * np.abs(r) + tol * rms + (BF16_HALF_ULP * np.abs(r) if bf16_out else 0.0)
         ratio = np.abs(x - r) / np.maximum(bound, 1e-300)
         worst = max(worst, float(ratio.max()))
-        if bf16_out:
+        if bf16_out and r.shape[0] * r.shape[2] >= 1024:
             nw = np.sqrt(np.sum((x - r) ** 2, axis=(0, 2)) / np.maximum(np.sum(r * r, axis=(0, 2)), 1e-300))
             assert float(nw.max()) <= TOL_BF16_NORMWISE, f"{what}: norm-wise relative error {nw.max():.2e}"
     assert worst <= 1.0, f"{what}: worst error is {worst:.3f}x the allowed bound (tol {tol})"

@@ -182,7 +182,8 @@ def test_device_side_rejections(tl):
     w = synth.random_case(11, [synth.tree_chain(6), synth.tree_star(5)], 1, 2, 64, 64, synth.F32, synth.F32,
                           paths=[np.array([0, 1, 2], np.int32), np.array([0, 3], np.int32)])
     # (1) parent[] not topological in tree 0: tree 0 yields nothing, tree 1 is still verified
-    bad = synth.random_case(11, [synth.tree_chain(6), synth.tree_star(5)], 1, 2, 64, 64, synth.F32, synth.F32)
+    bad = synth.random_case(11, [synth.tree_chain(6), synth.tree_star(5)], 1, 2, 64, 64, synth.F32, synth.F32,
+                            paths=[np.array([0, 1, 2], np.int32), np.array([0, 3], np.int32)])  # same tensors as w
     bad.parent = w.parent.copy()
     bad.parent[2] = 4
     dc = tl.DeviceCase(bad)
