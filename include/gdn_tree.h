@@ -127,8 +127,9 @@ int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const void *q, co
                     int32_t *status_dev, void *cuda_stream);
 
 /*
- * Commit (Section 3.4, "delay the state commit ... replay the selected path";
- * Section 3.4.2, last sentence): for every tree b, S[b] <- Eq. 7 replayed over
+ * Commit (Section 3.4: the state write is postponed until the accepted branch is known and
+ * is then a short recurrence over that branch; Section 3.4.2, end: it is the only state
+ * write of a decode step): for every tree b, S[b] <- Eq. 7 replayed over
  * path[path_offsets[b] .. path_offsets[b+1]) (local node ids, root first),
  * in place.  An empty path leaves S[b] untouched.
  *   S            : [device] in: S0, out: S_new (the only state write of a decode step)
@@ -163,6 +164,32 @@ int gdn_tree_commit_host(const gdn_shape_t *shape, float *S_h, const void *k_h, 
                          const int32_t *node_offsets_h, const int32_t *path_h,
                          const int32_t *path_offsets_h, int32_t total_path_len, void *dev_arena,
                          size_t arena_bytes, void *cuda_stream);
+
+/*
+ * Tree verification without a caller-provided workspace, for callers that cannot allocate device
+ * memory at all (a server whose own pool owns every free byte, a latency-critical loop that must
+ * not hit cudaMalloc's device-wide synchronisation, a plug-in that is forbidden to allocate).
+ * The paper has no counterpart of this entry point; it is a packaging variant of gdn_tree_verify.
+ *
+ * Same arguments, results and error reporting as gdn_tree_verify, minus `workspace`: the scratch
+ * is a fixed array of GDN_STATIC_SCRATCH_BYTES inside the library image, resident on every GPU
+ * that loads the library until the process exits.  The call performs no cudaMalloc / cudaFree
+ * and calls no allocating routine.
+ *   - Limit: gdn_tree_workspace_bytes(shape) must not exceed GDN_STATIC_SCRATCH_BYTES (about
+ *     one layer of 32 value heads x 128 with a tree of up to ~250 nodes); larger problems get
+ *     GDN_ERR_WORKSPACE and nothing is launched.
+ *   - The first call on each device resolves the array's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in
+ *     it (verify rewrites every part it later reads, so nothing needs clearing).  Two calls
+ *     whose kernels overlap on the GPU -- different streams, or the same stream from two threads
+ *     without ordering -- race on it; serialise them.
+ */
+#define GDN_STATIC_SCRATCH_BYTES (4u << 20)
+int gdn_tree_verify_static(const gdn_shape_t *shape, const float *S0, const void *q, const void *k,
+                           const void *v, const void *g, const void *beta, const int32_t *parent,
+                           const int32_t *node_offsets, void *o, int32_t *status_dev,
+                           void *cuda_stream);
 
 #ifdef __cplusplus
 }

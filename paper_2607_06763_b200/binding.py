@@ -26,7 +26,10 @@ EXPORTS = (
     "gdn_tree_host_arena_bytes",
     "gdn_tree_verify_host",
     "gdn_tree_commit_host",
+    "gdn_tree_verify_static",
 )
+
+GDN_STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class GdnShape(ctypes.Structure):
@@ -86,6 +89,8 @@ def load_library():
         lib.gdn_tree_verify_host.argtypes = [sp] + [vp] * 10 + [ctypes.c_size_t, vp]
         lib.gdn_tree_commit_host.restype = ctypes.c_int
         lib.gdn_tree_commit_host.argtypes = [sp] + [vp] * 9 + [ctypes.c_int32, vp, ctypes.c_size_t, vp]
+        lib.gdn_tree_verify_static.restype = ctypes.c_int
+        lib.gdn_tree_verify_static.argtypes = [sp] + [vp] * 11
         _lib = lib
     return _lib
 
@@ -164,3 +169,12 @@ def gdn_tree_commit_host(shape: GdnShape, S, k, v, g, beta, parent, node_offsets
                                                     _ptr(beta), _ptr(parent), _ptr(node_offsets), _ptr(path),
                                                     _ptr(path_offsets), int(total_path_len), _ptr(dev_arena),
                                                     int(arena_bytes), _stream(stream)))
+
+
+def gdn_tree_verify_static(shape: GdnShape, S0, q, k, v, g, beta, parent, node_offsets, o, status_dev,
+                           stream=None) -> int:
+    """``gdn_tree_verify`` for callers that cannot allocate device memory: the scratch is a fixed array inside the
+    library (at most ``GDN_STATIC_SCRATCH_BYTES``), shared by all calls on a device, so overlapping calls race."""
+    return int(load_library().gdn_tree_verify_static(ctypes.byref(shape), _ptr(S0), _ptr(q), _ptr(k), _ptr(v),
+                                                      _ptr(g), _ptr(beta), _ptr(parent), _ptr(node_offsets),
+                                                      _ptr(o), _ptr(status_dev), _stream(stream)))
