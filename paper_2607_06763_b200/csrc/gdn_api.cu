@@ -154,8 +154,10 @@ extern "C" int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const PlanPtrs plan = plan_ptrs(workspace, lay);
     if (launch_plan(s, parent, node_offsets, plan, status_dev, stream) != cudaSuccess) return GDN_ERR_CUDA;
-    if (launch_verify_generic(s, S0, q, k, v, g, beta, node_offsets, o, plan, stream) != cudaSuccess)
-        return GDN_ERR_CUDA;
+    const cudaError_t e = verify_sm100_supported(s)
+                              ? launch_verify_sm100(s, S0, q, k, v, g, beta, node_offsets, o, plan, status_dev, stream)
+                              : launch_verify_generic(s, S0, q, k, v, g, beta, node_offsets, o, plan, stream);
+    if (e != cudaSuccess) return GDN_ERR_CUDA;
     return GDN_OK;
 }
 

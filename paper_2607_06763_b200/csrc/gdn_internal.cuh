@@ -57,6 +57,13 @@ cudaError_t launch_verify_generic(const gdn_shape_t &s, const float *S0, const v
                                   const int32_t *node_offsets, void *o, const PlanPtrs &plan,
                                   cudaStream_t stream);
 
+// Tensor-core fast path (d_k = d_v = 128, bf16 inputs, trees <= 64 nodes, root paths <= 16 nodes).
+bool verify_sm100_supported(const gdn_shape_t &s);
+cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
+                                const void *v, const void *g, const void *beta,
+                                const int32_t *node_offsets, void *o, const PlanPtrs &plan,
+                                int32_t *status_dev, cudaStream_t stream);
+
 cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k, const void *v,
                                   const void *g, const void *beta, const int32_t *parent,
                                   const int32_t *node_offsets, const int32_t *path,
