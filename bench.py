@@ -171,11 +171,13 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--oracle-slots", type=int, default=24, help="layer slots / sequences in the oracle's sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--layers", type=int, default=48, help="layer slots of the stack workloads (profiling: fewer)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
 
-    w = synth.config(WORKLOADS[args.workload], 0)
+    w = synth.config(WORKLOADS[args.workload], 0, n_layers=args.layers)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -290,14 +292,16 @@ def main():
     idx_b = 4 * (w.total_nodes + 2 * (w.n_seq + 1) + (w.n_seq + 1) + L)
     h2d = (state_b + 2 * qk_b + v_b + 2 * gb_b) + (state_b + qk_b + v_b + 2 * gb_b) + idx_b
     d2h = w.total_nodes * w.h_v * w.d_v * osz + state_b + 8
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.e2e_steps):
-        e2e_step()
-    barrier()
-    e2e_s = (time.perf_counter() - t0) / args.e2e_steps
+    e2e_s = float("nan")
+    if not args.no_e2e:
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        barrier()
+        e2e_s = (time.perf_counter() - t0) / args.e2e_steps
     if world > 1:
         t = torch.tensor([e2e_s], device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
