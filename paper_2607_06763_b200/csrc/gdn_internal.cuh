@@ -14,15 +14,11 @@ namespace gdn {
 //   tree_ok  int32 [n_seq]                 1 = tree passed the metadata checks
 //   depth    uint8 [N]                     nodes on the root path of node n (root = 1)
 //   anc      uint16[N][max_depth]          local ids of the root path of n, root first, n itself last
-// Depth-first tables, filled when max_depth <= 16 and the tree has <= 256 nodes (else unused).
-// "Position" = index of a node in the pre-order traversal of its tree (children by increasing id):
-//   order8   uint8 [N]                     node id at position r
-//   dpos8    uint8 [N]                     depth of the node at position r
-//   ancpos8  uint8 [N][16]                 positions of the root path of the node at position r,
-//                                          root first, the node itself last; unused entries 0xFF
+//   anc8     uint8 [N][16]                 the same list as bytes (filled when max_depth <= 16 and the
+//                                          tree has <= 256 nodes; unused entries are 0xFF)
 //   utilde   float [N][h_v][d_v]           solve result u~ (Eq. 10 with the W S0 term folded in)
 struct WorkspaceLayout {
-    size_t tree_ok, depth, anc, order8, dpos8, ancpos8, utilde, total;
+    size_t tree_ok, depth, anc, anc8, utilde, total;
 };
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
@@ -35,9 +31,7 @@ inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
     w.tree_ok = off;  off = align256(off + sizeof(int32_t) * (size_t)s.n_seq);
     w.depth = off;    off = align256(off + N);
     w.anc = off;      off = align256(off + sizeof(uint16_t) * N * (size_t)s.max_depth);
-    w.order8 = off;   off = align256(off + N);
-    w.dpos8 = off;    off = align256(off + N);
-    w.ancpos8 = off;  off = align256(off + 16 * N);
+    w.anc8 = off;     off = align256(off + 16 * N);
     w.utilde = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
     w.total = off;
     return w;
@@ -47,7 +41,7 @@ struct PlanPtrs {
     int32_t *tree_ok;
     uint8_t *depth;
     uint16_t *anc;
-    uint8_t *order8, *dpos8, *ancpos8;
+    uint8_t *anc8;
     float *utilde;
 };
 
@@ -55,8 +49,7 @@ inline PlanPtrs plan_ptrs(void *workspace, const WorkspaceLayout &w)
 {
     char *b = static_cast<char *>(workspace);
     return {reinterpret_cast<int32_t *>(b + w.tree_ok), reinterpret_cast<uint8_t *>(b + w.depth),
-            reinterpret_cast<uint16_t *>(b + w.anc), reinterpret_cast<uint8_t *>(b + w.order8),
-            reinterpret_cast<uint8_t *>(b + w.dpos8), reinterpret_cast<uint8_t *>(b + w.ancpos8),
+            reinterpret_cast<uint16_t *>(b + w.anc), reinterpret_cast<uint8_t *>(b + w.anc8),
             reinterpret_cast<float *>(b + w.utilde)};
 }
 

@@ -1,27 +1,26 @@
 // Tree-verify fast path for sm_100a: d_k = d_v = 128, bf16 inputs, trees of at most 64 nodes,
-// root paths of at most 16 nodes.  Same mathematics as the generic kernel (the triangular form of
-// Section 3.4.1 restricted to real ancestors, W S0 folded into the right-hand side as in
-// Section 3.4.2), but the dense part runs on the 5th-generation tensor cores:
+// root paths of at most 16 nodes.  It evaluates the triangular form of Section 3.4.1 (Eq. 9-11)
+// restricted to real ancestors, with the W S0 term folded into the right-hand side as in
+// Section 3.4.2, and turns all of the per-component work into two dense contractions on the
+// 5th-generation tensor cores (tcgen05.mma, bf16 operands, fp32 accumulators in tensor memory):
 //
-//   P  [d_v x 2T] = S0 [d_v x d_k] . [k_0;q_0;k_1;q_1;...]^T   (the S0 projections of Eq. 11 / Eq. 13: 86% of the FLOPs)
-//   Gr [2T x 2T]  = [k;q rows] . [k;q rows]^T                  (k_i.k_j and q_i.k_j of Eq. 9; the .q columns are unused)
+//   (1) P [d_v x 2T] = S0 [d_v x d_k] . [k_0;q_0;k_1;q_1;...]^T      the S0 projections of Eq. 11 / Eq. 13
+//       Gr [2T x 2T] = [k;q rows] . [k;q rows]^T                     k_i.k_j and q_i.k_j of Eq. 9
+//   (2) D [d_v x T]  = R^T [d_v x T] . Z^T [T x T]                   the whole masked solve + output
 //
-// Both are tcgen05.mma (kind::f16, bf16 operands, fp32 accumulators in tensor memory).  q and k
-// are bf16 already; the fp32 state is split on the fly into two bf16 terms S0 = hi + lo
-// (|S0 - hi - lo| <= 2^-16 |S0|), so P costs two accumulating MMA passes and keeps fp32-level
-// accuracy.  Operand orientation: d_v on the TMEM lanes, nodes on the TMEM columns -- a thread then
-// owns value component c and needs nothing from other components.
+// where r_j = beta_j (v_j - a_j S0^T k_j) is the folded right-hand side and row i of Z is
+// z_i^T = y_i^T (I + X_path(i))^-1: because the ancestors of a node form a chain, the inverse
+// restricted to one root path is a back-substitution with at most 16 unknowns that each node
+// can run on its own (one thread per node, no dependence between nodes).  Then
+//   o_i = scale (a_i S0^T q_i + sum_{j on the root path of i} Z_ij r_j),
+// which is Eq. 11 with U - W S0 eliminated; no per-component sequential substitution is left.
+// fp32 quantities that feed the tensor cores are split into two bf16 terms (x = hi + lo,
+// |x - hi - lo| <= 2^-16 |x|): S0 for (1), R and Z for (2), all four cross terms accumulated.
 //
-// Nodes are visited in depth-first (pre-order) order, prepared by the plan kernel.  In that order
-// the proper ancestors of the current node are exactly the current stack, so the solve results
-// u~ of the root path live in sixteen registers indexed by depth: the ancestor-masked forward
-// substitution (Eq. 10 / 13) and the output (Eq. 11) of a node are straight-line FMAs against
-// those registers, with the X / Y coefficients broadcast from shared memory, and u~ is never
-// stored.  Warps 0-3 take the first half of the traversal, warps 4-7 the second half (after
-// replaying the root path of their first node to rebuild its stack).
-//
-// One CTA per (tree, value head), 256 threads, about 106 KB of shared memory and 256 TMEM columns,
-// so two CTAs share an SM: while one streams its 64 KB state tile from HBM the other computes.
+// Operand orientation: d_v on the TMEM lanes, nodes on the TMEM columns, so every thread of a
+// warp owns one value component.  One CTA per (tree, value head), 256 threads, about 106 KB of
+// shared memory and 256 TMEM columns, so two CTAs share an SM: while one streams its 64 KB
+// state tile from HBM the other computes.
 #include "gdn_internal.cuh"
 
 namespace gdn {
@@ -32,26 +31,46 @@ constexpr int FV_THREADS = 256;
 constexpr int FV_D = 128;           // d_k = d_v
 constexpr int FV_T = 64;            // max nodes per tree
 constexpr int FV_MD = 16;           // max nodes on a root path
-constexpr int FV_TMEM_COLS = 256;   // P: columns [0,128) (2r: k_r, 2r+1: q_r), Gram: [128,256)
-constexpr int FV_GRAM_PITCH = 65;   // floats per Gram row in shared memory (odd: conflict-free column writes)
+constexpr int FV_TMEM_COLS = 256;   // P: columns [0,128) (2i: k_i, 2i+1: q_i); Gram: [128,256), later D: [128,192)
 
-// shared memory map (bytes from a 1024-byte aligned base); "r" is a depth-first position
-constexpr int SM_A_HI = 0;                       // [2][128 rows][128 B], 128B-swizzled, K-major
-constexpr int SM_A_LO = 32768;
-constexpr int SM_B_KQ = 65536;                   // row 2r = k of node r, row 2r+1 = q of node r
-constexpr int SM_GRAM = 0;                       // after the MMAs: fp32 [128][65] (columns = k_j) over A_HI/A_LO ...
-constexpr int SM_V = 34816;                      // ... and the tree's v rows, bf16 [64][128]
-constexpr int SM_X = 98304;                      // fp32 [64][16]: decay, then X coefficients
-constexpr int SM_Y = SM_X + 4096;                // fp32 [64][16]: gathered g, then Y coefficients
-constexpr int SM_ANCP = SM_Y + 4096;             // u8   [64][16]: positions of the root path
-constexpr int SM_AB = SM_ANCP + 1024;            // float2 [64]: (total decay a_r, beta_r)
-constexpr int SM_ORDER = SM_AB + 512;            // u8 [64] node id at position r
-constexpr int SM_DPOS = SM_ORDER + FV_T;         // u8 [64] depth at position r (0 beyond T)
-constexpr int SM_MBAR = SM_DPOS + FV_T;          // u64
+// shared memory map (bytes from a 1024-byte aligned base)
+constexpr int SM_A_HI = 0;                       // S0 hi: [2][128 rows][128 B], 128B-swizzled, K-major
+constexpr int SM_A_LO = 32768;                   // S0 lo
+constexpr int SM_B_KQ = 65536;                   // row 2i = k of node i, row 2i+1 = q of node i; same layout
+// after the first MMA group the operand tiles are dead and are reused:
+constexpr int SM_GRAM = 0;                       // fp32 [128][64], column j of row r stored at j ^ (r & 31)
+constexpr int SM_RT_HI = 0;                      // then R^T hi: [128 rows = components][64 nodes] bf16, swizzled
+constexpr int SM_RT_LO = 16384;                  //      R^T lo
+constexpr int SM_V = 32768;                      // v rows of the tree, bf16 [64][128]
+constexpr int SM_Z_HI = 49152;                   // Z hi: [64 rows = nodes i][64 nodes j] bf16, swizzled
+constexpr int SM_Z_LO = 57344;                   // Z lo
+constexpr int SM_X = 98304;                      // fp32 [64][16]  X(i, t-th path node)
+constexpr int SM_Y = SM_X + 4096;                // fp32 [64][16]  Y(i, t-th path node), node itself included
+constexpr int SM_ANC = SM_Y + 4096;              // u8   [64][16]  root-path node ids (0xFF = unused)
+constexpr int SM_GAB = SM_ANC + 1024;            // float4 [64]: (G_i = log a_i, a_i, beta_i, g_i)
+constexpr int SM_DEPTH = SM_GAB + 1024;          // u8 [64] (0 beyond T)
+constexpr int SM_MBAR = SM_DEPTH + FV_T;         // u64
 constexpr int SM_TMEM = SM_MBAR + 8;             // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
 constexpr int SM_BYTES = SM_FLAG + 4;
 constexpr int SM_ALLOC = SM_BYTES + 1024;        // slack for the 1024-byte alignment of the base
+
+// Development aid: with -DGDN_TRACE thread 0 of every CTA records clock64() at each phase boundary into a
+// buffer registered through gdn_trace_set_buffer(); normal builds compile none of it.
+#ifdef GDN_TRACE
+__device__ long long *g_trace_buf = nullptr;
+#define GDN_TRACE_MARK(k)                                                            \
+    do {                                                                             \
+        if (threadIdx.x == 0 && g_trace_buf) g_trace_buf[blockIdx.x * 16 + (k)] = clock64(); \
+    } while (0)
+#define GDN_TRACE_MARK_T(t, k)                                                       \
+    do {                                                                             \
+        if (threadIdx.x == (t) && g_trace_buf) g_trace_buf[blockIdx.x * 16 + (k)] = clock64(); \
+    } while (0)
+#else
+#define GDN_TRACE_MARK(k) do {} while (0)
+#define GDN_TRACE_MARK_T(t, k) do {} while (0)
+#endif
 
 struct VerifyFastParams {
     int h_qk, h_v;
@@ -61,7 +80,8 @@ struct VerifyFastParams {
     const int32_t *node_offsets;
     void *o;
     const int32_t *tree_ok;
-    const uint8_t *order8, *dpos8, *ancpos8;
+    const uint8_t *depth;
+    const uint8_t *anc8;
     int32_t *status_dev;
 };
 
@@ -166,40 +186,43 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo_elem, float hi_elem)
     return *reinterpret_cast<uint32_t *>(&t);
 }
 
-#define GDN_TMEM_LD2(taddr, r0, r1) \
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(taddr) : "memory")
+#define GDN_TMEM_LD32(taddr, r)                                                                              \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                  \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                  \
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"                 \
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),      \
+                   "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),  \
+                   "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),            \
+                   "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),            \
+                   "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])             \
+                 : "r"(taddr)                                                                                \
+                 : "memory")
 
-// ---------------------------------------------------------------------------------------- kernel
-// One node at depth D (D nodes on its root path).  st[a] holds u~ of the path node at depth a+1.
-//   u~ = rhs - sum_{a<D-1} X[a] st[a]                       (forward substitution, Eq. 10 / 13)
-//   ysum = sum_{a<D-1} Y[a] st[a] + Y[D-1] u~               (the Y term of Eq. 11)
-template <int D>
-__device__ __forceinline__ void node_step(float (&st)[FV_MD], const float *xr, const float *yr, float rhs,
-                                          float &ysum)
+// Byte offset of 16-byte piece `c16` (0..7) of row `r` in a one-atom-wide ([rows][128 B]) swizzled tile.
+__device__ __forceinline__ uint32_t sw128_row_offset(int r, int c16)
 {
-    float acc0 = 0.f, acc1 = 0.f, y0 = 0.f, y1 = 0.f, ylast = 0.f;
-#pragma unroll
-    for (int q4 = 0; q4 * 4 < D; ++q4) {
-        const float4 yv4 = *reinterpret_cast<const float4 *>(yr + q4 * 4);
-        float4 xv4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (q4 * 4 < D - 1) xv4 = *reinterpret_cast<const float4 *>(xr + q4 * 4);
-        const float xv[4] = {xv4.x, xv4.y, xv4.z, xv4.w}, yv[4] = {yv4.x, yv4.y, yv4.z, yv4.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int a = q4 * 4 + e;
-            if (a < D - 1) {
-                if (a & 1) { acc1 = fmaf(xv[e], st[a], acc1); y1 = fmaf(yv[e], st[a], y1); }
-                else       { acc0 = fmaf(xv[e], st[a], acc0); y0 = fmaf(yv[e], st[a], y0); }
-            } else if (a == D - 1) {
-                ylast = yv[e];
-            }
-        }
-    }
-    const float u = rhs - (acc0 + acc1);
-    st[D - 1] = u;
-    ysum = fmaf(ylast, u, y0 + y1);
+    return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c16 ^ (r & 7)) << 4));
 }
 
+// Bounded wait on an mbarrier phase; returns false if it expired.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    const long long t0 = clock64();
+    bool done = mbar_try_wait(bar, parity);
+    while (!done) {
+        if (clock64() - t0 > 400000000LL) break;   // ~0.2 s: far beyond any legitimate MMA latency
+        done = mbar_try_wait(bar, parity);
+    }
+    return done;
+}
+
+__device__ __forceinline__ void split_bf16(float x, float &hi, float &lo)
+{
+    hi = __bfloat162float(__float2bfloat16_rn(x));
+    lo = x - hi;
+}
+
+// ---------------------------------------------------------------------------------------- kernel
 template <typename TOut>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const VerifyFastParams p)
 {
@@ -214,10 +237,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     const uint32_t sbase = smem_u32(smem);
     float *xs = reinterpret_cast<float *>(smem + SM_X);
     float *ys = reinterpret_cast<float *>(smem + SM_Y);
-    float2 *ab_s = reinterpret_cast<float2 *>(smem + SM_AB);
-    uint8_t *ancp = smem + SM_ANCP;
-    uint8_t *order_s = smem + SM_ORDER;
-    uint8_t *dpos_s = smem + SM_DPOS;
+    float4 *gab = reinterpret_cast<float4 *>(smem + SM_GAB);
+    uint8_t *anc_s = smem + SM_ANC;
+    uint8_t *depth_s = smem + SM_DEPTH;
     float *gram = reinterpret_cast<float *>(smem + SM_GRAM);
     const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(smem + SM_V);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM_TMEM);
@@ -226,6 +248,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hk = h / (p.h_v / p.h_qk);
+    GDN_TRACE_MARK(0);
 
     // (1) state tile loads first (the longest latency of the prologue): a warp instruction covers
     // four rows; the eight lanes of a row each own one 16-byte bf16 piece of either K half.
@@ -243,38 +266,38 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             }
         }
     }
-
+    // (2) k and q rows -> B operand tile (rows beyond T are zero-filled)
+#pragma unroll
+    for (int it = 0; it < (128 * 16) / FV_THREADS; ++it) {
+        const int idx = it * FV_THREADS + tid;
+        const int r = idx >> 4, c16 = idx & 15;
+        const int node = r >> 1;
+        const bool valid = node < T;
+        const __nv_bfloat16 *src = ((r & 1) ? p.q : p.k) + ((size_t)(base + (valid ? node : 0)) * p.h_qk + hk) * FV_D + c16 * 8;
+        cp_async_16(sbase + SM_B_KQ + sw128_offset(r, c16), src, valid);
+    }
     if (warp == 0) tmem_alloc(sbase + SM_TMEM, FV_TMEM_COLS);
     if (tid == 32) {
         mbar_init(mbar, 1);
         *flag = 0;
     }
-    // (2) depth-first tables of this tree
+    // (3) per-node tables: depth, root-path ids, g, beta (zeros beyond T)
     if (tid < FV_T) {
-        int d = 0, node = 0;
+        int d = 0;
         uint4 row = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+        float gi = 0.f, be = 0.f;
         if (tid < T) {
-            node = p.order8[base + tid];
-            d = p.dpos8[base + tid];
-            row = __ldg(reinterpret_cast<const uint4 *>(p.ancpos8 + (size_t)(base + tid) * 16));
+            const int n = base + tid;
+            d = p.depth[n];
+            row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)n * 16));
+            gi = __bfloat162float(p.g[(size_t)n * p.h_v + h]);
+            be = __bfloat162float(p.beta[(size_t)n * p.h_v + h]);
         }
-        order_s[tid] = (uint8_t)node;
-        dpos_s[tid] = (uint8_t)d;
-        *reinterpret_cast<uint4 *>(ancp + tid * 16) = row;
+        depth_s[tid] = (uint8_t)d;
+        *reinterpret_cast<uint4 *>(anc_s + tid * 16) = row;
+        gab[tid] = make_float4(0.f, 0.f, be, gi);
     }
-    __syncthreads();
-
-    // (3) k and q rows in depth-first order -> B operand tile (rows beyond T are zero-filled)
-#pragma unroll
-    for (int it = 0; it < (128 * 16) / FV_THREADS; ++it) {
-        const int idx = it * FV_THREADS + tid;
-        const int r = idx >> 4, c16 = idx & 15;
-        const int pos = r >> 1;
-        const bool valid = pos < T;
-        const int node = valid ? order_s[pos] : 0;
-        const __nv_bfloat16 *src = ((r & 1) ? p.q : p.k) + ((size_t)(base + node) * p.h_qk + hk) * FV_D + c16 * 8;
-        cp_async_16(sbase + SM_B_KQ + sw128_offset(r, c16), src, valid);
-    }
+    GDN_TRACE_MARK(1);
 
     // (4) fp32 -> bf16 hi + lo, written as the A operand
 #pragma unroll
@@ -287,24 +310,27 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             uint32_t hi[4], lo[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float h0 = __bfloat162float(__float2bfloat16_rn(f[2 * e]));
-                const float h1 = __bfloat162float(__float2bfloat16_rn(f[2 * e + 1]));
+                float h0, l0, h1, l1;
+                split_bf16(f[2 * e], h0, l0);
+                split_bf16(f[2 * e + 1], h1, l1);
                 hi[e] = pack_bf16(h0, h1);
-                lo[e] = pack_bf16(f[2 * e] - h0, f[2 * e + 1] - h1);
+                lo[e] = pack_bf16(l0, l1);
             }
             const uint32_t off = sw128_offset(row, kh * 8 + l8);
             *reinterpret_cast<uint4 *>(smem + SM_A_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
             *reinterpret_cast<uint4 *>(smem + SM_A_LO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
     }
+    GDN_TRACE_MARK(2);
     cp_async_wait_all();
     fence_proxy_async();   // generic-proxy writes of the operands become visible to the tensor core
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    GDN_TRACE_MARK(3);
 
-    // (5) one thread issues the MMAs: P = S0.[k;q]^T (hi then lo), Gram = [k;q].[k;q]^T
+    // (5) one thread issues the first MMA group: P = S0.[k;q]^T (hi then lo), Gram = [k;q].[k;q]^T
     if (tid == 0) {
         const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
         const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
@@ -326,58 +352,34 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         }
         umma_commit(mbar);
     }
+    // (6) meanwhile: G_i = sum of g along the root path (root first), a_i = exp(G_i)
+    if (tid >= 64 && tid < 64 + FV_T) {
+        const int i = tid - 64;
+        const int d = depth_s[i];
+        float G = 0.f;
+        for (int t = 0; t < d; ++t) G += gab[anc_s[i * FV_MD + t]].w;
+        gab[i].x = G;
+        gab[i].y = d ? expf(G) : 0.f;
+    }
+    GDN_TRACE_MARK(4);
 
-    // (6) while the tensor core works: g of every path node, then the decay from each path
-    // position to the node as exp of a suffix sum (= a_i / a_j of Eq. 9 without cancellation)
-    for (int idx = tid; idx < FV_T * FV_MD; idx += FV_THREADS) {
-        const int r = idx >> 4, a = idx & 15;
-        float gv = 0.f;
-        if (a < dpos_s[r]) gv = __bfloat162float(p.g[(size_t)(base + order_s[ancp[idx]]) * p.h_v + h]);
-        ys[idx] = gv;
-    }
-    float beta_r = 0.f;
-    if (tid < T) beta_r = __bfloat162float(p.beta[(size_t)(base + order_s[tid]) * p.h_v + h]);
-    __syncthreads();
-    for (int idx = tid; idx < FV_T * FV_MD; idx += FV_THREADS) {
-        const int r = idx >> 4, a = idx & 15;
-        const int d = dpos_s[r];
-        if (a < d) {
-            float sfx = 0.f;
-            for (int u = a + 1; u < d; ++u) sfx += ys[r * FV_MD + u];
-            xs[idx] = expf(sfx);
-        }
-    }
-    if (tid < T) {
-        float tot = 0.f;
-        for (int u = 0; u < dpos_s[tid]; ++u) tot += ys[tid * FV_MD + u];
-        ab_s[tid] = make_float2(expf(tot), beta_r);
-    }
-
-    // (7) wait for the MMAs (bounded: on expiry flag the error and fall through to the clean-up)
-    {
-        const long long t0 = clock64();
-        bool done = mbar_try_wait(mbar, 0);
-        while (!done) {
-            if (clock64() - t0 > 400000000LL) break;   // ~0.2 s: far beyond any legitimate MMA latency
-            done = mbar_try_wait(mbar, 0);
-        }
-        if (!done) *flag = 1;
-    }
+    // (7) wait for the first MMA group (bounded: on expiry flag the error and fall through to the clean-up)
+    if (!mbar_wait_bounded(mbar, 0)) *flag = 1;
     tc_fence_after();
     __syncthreads();
-    const bool timed_out = *flag != 0;
+    bool ok = *flag == 0;
+    GDN_TRACE_MARK(5);
 
-    if (!timed_out) {
-        // (8) the operand tiles are free now: fetch the tree's v rows over them (depth-first order),
-        // and move the k-columns of the Gram block out of tensor memory
+    if (ok) {
+        // (8) the operand tiles are free now: fetch the tree's v rows over them and move the
+        // k-columns of the Gram block out of tensor memory
 #pragma unroll
         for (int it = 0; it < (FV_T * 16) / FV_THREADS; ++it) {
             const int idx = it * FV_THREADS + tid;
-            const int r = idx >> 4, c16 = idx & 15;
-            const bool valid = r < T;
-            const int node = valid ? order_s[r] : 0;
-            cp_async_16(sbase + SM_V + r * 256 + c16 * 16, p.v + ((size_t)(base + node) * p.h_v + h) * FV_D + c16 * 8,
-                        valid);
+            const int i = idx >> 4, c16 = idx & 15;
+            const bool valid = i < T;
+            cp_async_16(sbase + SM_V + i * 256 + c16 * 16,
+                        p.v + ((size_t)(base + (valid ? i : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
         }
         {
             const int row = (warp & 3) * 32 + lane;
@@ -385,86 +387,177 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 128 + half * 64;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
-                uint32_t r0[16], r1[16];
-                GDN_TMEM_LD16(taddr + part * 32, r0);
-                GDN_TMEM_LD16(taddr + part * 32 + 16, r1);
+                uint32_t rr[32];
+                GDN_TMEM_LD32(taddr + part * 32, rr);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    gram[row * FV_GRAM_PITCH + half * 32 + part * 16 + j] = __uint_as_float(r0[2 * j]);
-                    gram[row * FV_GRAM_PITCH + half * 32 + part * 16 + 8 + j] = __uint_as_float(r1[2 * j]);
+                for (int j = 0; j < 16; ++j) {
+                    const int col = half * 32 + part * 16 + j;
+                    gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(rr[2 * j]);
                 }
             }
         }
+        tc_fence_before();
         __syncthreads();
-        // (9) X and Y of Eq. 9 for real ancestors only
+        GDN_TRACE_MARK(6);
+        // (9) X and Y of Eq. 9 for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
         for (int idx = tid; idx < FV_T * FV_MD; idx += FV_THREADS) {
-            const int r = idx >> 4, a = idx & 15;
-            if (a < dpos_s[r]) {
-                const int j = ancp[idx];
-                const float dec = xs[idx];
-                ys[idx] = dec * gram[(2 * r + 1) * FV_GRAM_PITCH + j];
-                xs[idx] = ab_s[r].y * dec * gram[(2 * r) * FV_GRAM_PITCH + j];   // a = d-1 (self) is never read
+            const int i = idx >> 4, t = idx & 15;
+            const int d = depth_s[i];
+            float xv = 0.f, yv = 0.f;
+            if (t < d) {
+                const int j = anc_s[idx];
+                const float4 gi = gab[i];
+                const float dec = expf(gi.x - gab[j].x);
+                yv = dec * gram[(2 * i + 1) * 64 + (j ^ ((2 * i + 1) & 31))];
+                if (t < d - 1) xv = gi.z * dec * gram[(2 * i) * 64 + (j ^ ((2 * i) & 31))];
             }
+            xs[idx] = xv;
+            ys[idx] = yv;
         }
         cp_async_wait_all();
         __syncthreads();
+        GDN_TRACE_MARK(7);
 
-        // (10) depth-first sweep: thread c owns value component c; warps 0-3 take positions
-        // [0, r_mid), warps 4-7 rebuild the stack of r_mid's root path and take [r_mid, T)
-        {
-            const int c = tid & 127;
-            const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-            TOut *o = static_cast<TOut *>(p.o);
-            float st[FV_MD];
+        // (10a) warps 0-1, one thread per node: z^T = y^T (I + X_path)^-1 by back-substitution over the
+        // root path (column-oriented: once z_l is final, subtract z_l X(n_l, n_t) from every z_t, t < l),
+        // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path)
+        if (tid < FV_T) {
+            const int i = tid;
+            const int d = depth_s[i];
+            const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-            for (int a = 0; a < FV_MD; ++a) st[a] = 0.f;
-            const int r_mid = (T + 1) >> 1;
-            const bool second = warp >= 4;
-            const int n_pre = (second && r_mid < T) ? dpos_s[r_mid] - 1 : 0;
-            const int r_begin = second ? r_mid : 0, r_end = second ? T : r_mid;
-#pragma unroll 1
-            for (int it = -n_pre; it < r_end - r_begin; ++it) {
-                const bool store = it >= 0;
-                const int r = store ? r_begin + it : ancp[r_mid * FV_MD + (it + n_pre)];
-                uint32_t pk, pq;
-                GDN_TMEM_LD2(trow + 2 * r, pk, pq);
-                const float2 ab = ab_s[r];
-                const float v = __bfloat162float(vs[r * FV_D + c]);
-                const int d = dpos_s[r];
-                const float *xr = xs + r * FV_MD, *yr = ys + r * FV_MD;
-                tmem_wait_ld();
-                const float rhs = ab.y * (v - ab.x * __uint_as_float(pk));
-                float ysum = 0.f;
-                switch (d) {
-                case 1: node_step<1>(st, xr, yr, rhs, ysum); break;
-                case 2: node_step<2>(st, xr, yr, rhs, ysum); break;
-                case 3: node_step<3>(st, xr, yr, rhs, ysum); break;
-                case 4: node_step<4>(st, xr, yr, rhs, ysum); break;
-                case 5: node_step<5>(st, xr, yr, rhs, ysum); break;
-                case 6: node_step<6>(st, xr, yr, rhs, ysum); break;
-                case 7: node_step<7>(st, xr, yr, rhs, ysum); break;
-                case 8: node_step<8>(st, xr, yr, rhs, ysum); break;
-                case 9: node_step<9>(st, xr, yr, rhs, ysum); break;
-                case 10: node_step<10>(st, xr, yr, rhs, ysum); break;
-                case 11: node_step<11>(st, xr, yr, rhs, ysum); break;
-                case 12: node_step<12>(st, xr, yr, rhs, ysum); break;
-                case 13: node_step<13>(st, xr, yr, rhs, ysum); break;
-                case 14: node_step<14>(st, xr, yr, rhs, ysum); break;
-                case 15: node_step<15>(st, xr, yr, rhs, ysum); break;
-                case 16: node_step<16>(st, xr, yr, rhs, ysum); break;
-                default: break;
+            for (int c16 = 0; c16 < 8; ++c16) {
+                *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, c16)) = zero4;
+                *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, c16)) = zero4;
+            }
+            const uint4 row = *reinterpret_cast<const uint4 *>(anc_s + i * 16);
+            const uint32_t idw[4] = {row.x, row.y, row.z, row.w};
+            float z[FV_MD];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const float4 y4 = *reinterpret_cast<const float4 *>(ys + i * FV_MD + q4 * 4);
+                z[q4 * 4 + 0] = y4.x; z[q4 * 4 + 1] = y4.y; z[q4 * 4 + 2] = y4.z; z[q4 * 4 + 3] = y4.w;
+            }
+#pragma unroll
+            for (int l = FV_MD - 1; l >= 1; --l) {
+                if (l < d) {
+                    const int nl = (int)((idw[l >> 2] >> ((l & 3) * 8)) & 0xFFu);
+                    const float zl = z[l];
+#pragma unroll
+                    for (int q4 = 0; q4 * 4 < l; ++q4) {
+                        const float4 x4 = *reinterpret_cast<const float4 *>(xs + nl * FV_MD + q4 * 4);
+                        const float xv[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (q4 * 4 + e < l) z[q4 * 4 + e] = fmaf(-zl, xv[e], z[q4 * 4 + e]);
+                    }
                 }
-                if (store) {
-                    const float out = p.scale * fmaf(ab.x, __uint_as_float(pq), ysum);
-                    store_from_float(o + ((size_t)(base + order_s[r]) * p.h_v + h) * FV_D + c, out);
+            }
+#pragma unroll
+            for (int t = 0; t < FV_MD; ++t) {
+                if (t < d) {
+                    const int j = (int)((idw[t >> 2] >> ((t & 3) * 8)) & 0xFFu);
+                    float hi, lo;
+                    split_bf16(z[t], hi, lo);
+                    const uint32_t off = sw128_row_offset(i, j >> 3) + (j & 7) * 2;
+                    *reinterpret_cast<__nv_bfloat16 *>(smem + SM_Z_HI + off) = __float2bfloat16_rn(hi);
+                    *reinterpret_cast<__nv_bfloat16 *>(smem + SM_Z_LO + off) = __float2bfloat16_rn(lo);
                 }
             }
         }
-    } else if (tid == 0) {
-        report_status(p.status_dev, GDN_ERR_TIMEOUT);
-    }
+        // (10b) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
+        // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
+        {
+            const int c = (warp & 3) * 32 + lane;
+            const int half = warp >> 2;
+            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                uint32_t rr[32];
+                GDN_TMEM_LD32(taddr + part * 32, rr);   // columns 2j, 2j+1 for 16 nodes: p^k_j, p^q_j
+                tmem_wait_ld();
+#pragma unroll
+                for (int oct = 0; oct < 2; ++oct) {
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float rv[2];
+#pragma unroll
+                        for (int s2 = 0; s2 < 2; ++s2) {
+                            const int jj = oct * 8 + e * 2 + s2;
+                            const int j = half * 32 + part * 16 + jj;
+                            const float4 gj = gab[j];
+                            rv[s2] = gj.z * (__bfloat162float(vs[j * FV_D + c]) - gj.y * __uint_as_float(rr[2 * jj]));
+                        }
+                        float h0, l0, h1, l1;
+                        split_bf16(rv[0], h0, l0);
+                        split_bf16(rv[1], h1, l1);
+                        hi[e] = pack_bf16(h0, h1);
+                        lo[e] = pack_bf16(l0, l1);
+                    }
+                    const uint32_t off = sw128_row_offset(c, half * 4 + part * 2 + oct);
+                    *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4 *>(smem + SM_RT_LO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        GDN_TRACE_MARK(8);
 
+        // (11) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j], all four hi/lo cross terms
+        if (tid == 0) {
+            constexpr uint32_t id2 = idesc_bf16(128, 64);
+            const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
+            const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
+#pragma unroll
+            for (int combo = 0; combo < 4; ++combo) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16(tmem + 128, a2[combo & 1] + (uint64_t)(ks * 2), b2[combo >> 1] + (uint64_t)(ks * 2), id2,
+                              (combo | ks) != 0);
+            }
+            umma_commit(mbar);
+        }
+        if (!mbar_wait_bounded(mbar, 1)) {
+            *flag = 1;
+            ok = false;
+        }
+        tc_fence_after();
+        GDN_TRACE_MARK(9);
+
+        // (12) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i])
+        if (ok) {
+            const int c = (warp & 3) * 32 + lane;
+            const int half = warp >> 2;
+            const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+            TOut *o = static_cast<TOut *>(p.o);
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                const int i0 = half * 32 + part * 16;
+                if (i0 < T) {
+                    uint32_t pp[32], dd[16];
+                    GDN_TMEM_LD32(trow + 2 * i0, pp);
+                    GDN_TMEM_LD16(trow + 128 + i0, dd);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) {
+                        const int i = i0 + jj;
+                        if (i < T) {
+                            const float out = p.scale * fmaf(gab[i].y, __uint_as_float(pp[2 * jj + 1]), __uint_as_float(dd[jj]));
+                            store_from_float(o + ((size_t)(base + i) * p.h_v + h) * FV_D + c, out);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
+
+    GDN_TRACE_MARK(10);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
@@ -497,10 +590,17 @@ cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const voi
     VerifyFastParams p{s.h_qk, s.h_v, s.scale, S0,
                        static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k),
                        static_cast<const __nv_bfloat16 *>(v), static_cast<const __nv_bfloat16 *>(g),
-                       static_cast<const __nv_bfloat16 *>(beta), node_offsets, o, plan.tree_ok, plan.order8,
-                       plan.dpos8, plan.ancpos8, status_dev};
+                       static_cast<const __nv_bfloat16 *>(beta), node_offsets, o, plan.tree_ok, plan.depth,
+                       plan.anc8, status_dev};
     if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16>(s, p, stream);
     return launch_fast_typed<float>(s, p, stream);
 }
+
+#ifdef GDN_TRACE
+extern "C" int gdn_trace_set_buffer(long long *buf)
+{
+    return cudaMemcpyToSymbol(g_trace_buf, &buf, sizeof(buf)) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 }  // namespace gdn
