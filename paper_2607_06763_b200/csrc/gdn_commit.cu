@@ -8,7 +8,9 @@
 // One CTA per (tree, value head); thread (c, s) owns 32 floats of row c (quarter s of the key
 // dimension, interleaved in 16-byte pieces so that the four lanes of a row read 64 contiguous
 // bytes) and k . s_c is reduced over the four lanes with warp shuffles.  The path nodes' k rows
-// are fetched once into shared memory; the state is read once and written once.
+// are fetched once into shared memory; the state is read once and written once.  The state loads
+// are issued before anything else so that the path checks and the k-row staging run under their
+// latency, and the kernel keeps to 64 registers so that two CTAs (32 warps) share an SM.
 #include "gdn_internal.cuh"
 
 namespace gdn {
@@ -29,41 +31,25 @@ struct CommitParams {
 };
 
 template <typename TIn>
-__global__ void __launch_bounds__(CM_THREADS, 1) commit_generic_kernel(const CommitParams p)
+__global__ void __launch_bounds__(CM_THREADS, 2) commit_generic_kernel(const CommitParams p)
 {
     extern __shared__ __align__(16) float cm_smem[];
     float (*ks)[CM_DK] = reinterpret_cast<float (*)[CM_DK]>(cm_smem);   // [L][CM_DK]
     float *alpha_s = cm_smem + (size_t)p.max_depth * CM_DK;             // [L]
     float *beta_s = alpha_s + p.max_depth;                              // [L]
+    int *path_s = reinterpret_cast<int *>(beta_s + p.max_depth);        // [L] node ids
+    int *par_s = path_s + p.max_depth;                                  // [L] their parents
     __shared__ int path_bad;
 
     const int b = blockIdx.x / p.h_v, h = blockIdx.x % p.h_v;
-    const int base = p.node_offsets[b];
-    const int T = p.node_offsets[b + 1] - base;
     const int p0 = p.path_offsets[b];
     const int L = p.path_offsets[b + 1] - p0;
     if (L == 0) return;   // nothing accepted from this tree: state untouched
+    const int base = p.node_offsets[b];
+    const int T = p.node_offsets[b + 1] - base;
     const int tid = threadIdx.x;
     const int d_k = p.d_k, d_v = p.d_v;
-
-    // The accepted path must be a chain from a root inside this tree.
-    if (tid == 0) {
-        int bad = (L < 0 || L > p.max_depth || T <= 0 || p0 < 0);
-        for (int t = 0; !bad && t < L; ++t) {
-            const int n = p.path[p0 + t];
-            if (n < 0 || n >= T) { bad = 1; break; }
-            if (p.parent) {
-                const int want = t ? p.path[p0 + t - 1] : -1;
-                if (p.parent[base + n] != want) bad = 1;
-            } else if (t && n <= p.path[p0 + t - 1]) {
-                bad = 1;   // without parent[] only the topological order can be checked
-            }
-        }
-        path_bad = bad;
-        if (bad) report_status(p.status_dev, GDN_ERR_PATH);
-    }
-    __syncthreads();
-    if (path_bad) return;
+    const bool shape_ok = L > 0 && L <= p.max_depth && T > 0 && p0 >= 0;
 
     const int hk = h / (p.h_v / p.h_qk);
     const int c = tid / CM_SPLIT, s = tid % CM_SPLIT;
@@ -71,47 +57,77 @@ __global__ void __launch_bounds__(CM_THREADS, 1) commit_generic_kernel(const Com
     const TIn *k = static_cast<const TIn *>(p.k), *v = static_cast<const TIn *>(p.v);
     const TIn *g = static_cast<const TIn *>(p.g), *beta = static_cast<const TIn *>(p.beta);
 
-    // k rows of the path (fp32, zero padded to CM_DK) and the per-step scalars
-    for (int idx = tid; idx < L * CM_DK; idx += CM_THREADS) {
-        const int t = idx / CM_DK, r = idx % CM_DK;
-        const size_t n = (size_t)base + p.path[p0 + t];
-        ks[t][r] = r < d_k ? load_as_float(k + (n * p.h_qk + hk) * d_k + r) : 0.f;
-    }
-    if (tid < L) {
-        const size_t n = (size_t)base + p.path[p0 + tid];
-        alpha_s[tid] = expf(load_as_float(g + n * p.h_v + h));
-        beta_s[tid] = load_as_float(beta + n * p.h_v + h);
-    }
-
+    // The state slice goes first: its latency covers the path checks and the k-row staging below.
     float *row = p.S + ((size_t)(b * p.h_v + h) * d_v + (comp_on ? c : 0)) * d_k;
     float sreg[CM_REGS];
 #pragma unroll
     for (int j = 0; j < CM_REGS / 4; ++j) {
         const int r = 16 * j + 4 * s;
         float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (comp_on && r < d_k) x = *reinterpret_cast<const float4 *>(row + r);
+        if (shape_ok && comp_on && r < d_k) x = *reinterpret_cast<const float4 *>(row + r);
         sreg[4 * j + 0] = x.x; sreg[4 * j + 1] = x.y; sreg[4 * j + 2] = x.z; sreg[4 * j + 3] = x.w;
     }
+
+    // The accepted path must be a chain from a root inside this tree: every thread t < L fetches
+    // its entry (and that node's parent) in parallel, thread 0 then checks the chain.
+    if (shape_ok && tid < L) {
+        const int n = p.path[p0 + tid];
+        path_s[tid] = n;
+        par_s[tid] = (p.parent && n >= 0 && n < T) ? p.parent[base + n] : -2;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int bad = !shape_ok;
+        for (int t = 0; !bad && t < L; ++t) {
+            const int n = path_s[t];
+            if (n < 0 || n >= T) bad = 1;
+            else if (p.parent) bad = par_s[t] != (t ? path_s[t - 1] : -1);
+            else if (t && n <= path_s[t - 1]) bad = 1;   // without parent[] only the topological order can be checked
+        }
+        path_bad = bad;
+        if (bad) report_status(p.status_dev, GDN_ERR_PATH);
+    }
+    __syncthreads();
+    if (path_bad) return;
+
+    // k rows of the path (fp32, zero padded to CM_DK) and the per-step scalars
+    for (int idx = tid; idx < L * CM_DK; idx += CM_THREADS) {
+        const int t = idx / CM_DK, r = idx % CM_DK;
+        const size_t n = (size_t)base + path_s[t];
+        ks[t][r] = r < d_k ? load_as_float(k + (n * p.h_qk + hk) * d_k + r) : 0.f;
+    }
+    if (tid < L) {
+        const size_t n = (size_t)base + path_s[tid];
+        alpha_s[tid] = expf(load_as_float(g + n * p.h_v + h));
+        beta_s[tid] = load_as_float(beta + n * p.h_v + h);
+    }
+    float vc = comp_on ? load_as_float(v + (((size_t)base + path_s[0]) * p.h_v + h) * d_v + c) : 0.f;
     __syncthreads();
 
     for (int t = 0; t < L; ++t) {
-        float kreg[CM_REGS];
+        float vnext = 0.f;   // next step's v[c], fetched while this step computes
+        if (comp_on && t + 1 < L)
+            vnext = load_as_float(v + (((size_t)base + path_s[t + 1]) * p.h_v + h) * d_v + c);
         float dot = 0.f;
 #pragma unroll
         for (int j = 0; j < CM_REGS / 4; ++j) {
             const float4 kx = *reinterpret_cast<const float4 *>(&ks[t][16 * j + 4 * s]);
-            kreg[4 * j + 0] = kx.x; kreg[4 * j + 1] = kx.y; kreg[4 * j + 2] = kx.z; kreg[4 * j + 3] = kx.w;
+            dot = fmaf(kx.x, sreg[4 * j + 0], dot); dot = fmaf(kx.y, sreg[4 * j + 1], dot);
+            dot = fmaf(kx.z, sreg[4 * j + 2], dot); dot = fmaf(kx.w, sreg[4 * j + 3], dot);
         }
-#pragma unroll
-        for (int e = 0; e < CM_REGS; ++e) dot = fmaf(kreg[e], sreg[e], dot);
         dot += __shfl_xor_sync(0xffffffffu, dot, 1);
         dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-        const size_t n = (size_t)base + p.path[p0 + t];
-        const float vc = comp_on ? load_as_float(v + (n * p.h_v + h) * d_v + c) : 0.f;
         const float alpha = alpha_s[t];
         const float w = beta_s[t] * (vc - alpha * dot);
 #pragma unroll
-        for (int e = 0; e < CM_REGS; ++e) sreg[e] = fmaf(kreg[e], w, alpha * sreg[e]);
+        for (int j = 0; j < CM_REGS / 4; ++j) {
+            const float4 kx = *reinterpret_cast<const float4 *>(&ks[t][16 * j + 4 * s]);
+            sreg[4 * j + 0] = fmaf(kx.x, w, alpha * sreg[4 * j + 0]);
+            sreg[4 * j + 1] = fmaf(kx.y, w, alpha * sreg[4 * j + 1]);
+            sreg[4 * j + 2] = fmaf(kx.z, w, alpha * sreg[4 * j + 2]);
+            sreg[4 * j + 3] = fmaf(kx.w, w, alpha * sreg[4 * j + 3]);
+        }
+        vc = vnext;
     }
 
     if (comp_on) {
@@ -136,7 +152,7 @@ cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k,
     if (grid == 0) return cudaSuccess;
     CommitParams p{s.h_qk, s.h_v, s.d_k, s.d_v, s.max_depth, S, k, v, g, beta,
                    parent, node_offsets, path, path_offsets, status_dev};
-    const size_t smem = sizeof(float) * ((size_t)s.max_depth * CM_DK + 2 * (size_t)s.max_depth);
+    const size_t smem = sizeof(float) * ((size_t)s.max_depth * CM_DK + 4 * (size_t)s.max_depth);
     cudaError_t e;
     if (s.in_dtype == GDN_BF16) {
         e = cudaFuncSetAttribute(commit_generic_kernel<__nv_bfloat16>,

@@ -16,6 +16,8 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
             int32_t *__restrict__ tree_ok, uint8_t *__restrict__ depth, uint16_t *__restrict__ anc,
             uint8_t *__restrict__ anc8, int32_t *status_dev)
 {
+    // parent[] of this tree, staged once so that the root-path walks below run out of shared memory
+    __shared__ int32_t par_s[GDN_MAX_TREE_NODES];
     const int b = blockIdx.x;
     const int lo = node_offsets[b], hi = node_offsets[b + 1];
     const int T = hi - lo;
@@ -29,13 +31,15 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
         }
         return;
     }
+    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) par_s[i] = parent[lo + i];
+    __syncthreads();
     int err = 0;
     for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
         // first walk: count the nodes on the root path, checking parent[] as we go
         int d = 0, cur = i;
         while (cur >= 0) {
             if (++d > max_depth) { err = GDN_ERR_DEPTH; break; }
-            const int p = parent[lo + cur];
+            const int p = par_s[cur];
             if (p < -1 || p >= cur) { err = GDN_ERR_TREE; break; }
             cur = p;
         }
@@ -53,7 +57,7 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
             else if ((t >> 2) == 1) w1 = (w1 & keep) | put;
             else if ((t >> 2) == 2) w2 = (w2 & keep) | put;
             else if ((t >> 2) == 3) w3 = (w3 & keep) | put;
-            cur = parent[lo + cur];
+            cur = par_s[cur];
         }
         if (max_depth <= 16 && T <= 256)
             *reinterpret_cast<uint4 *>(anc8 + (size_t)(lo + i) * 16) = make_uint4(w0, w1, w2, w3);

@@ -74,6 +74,8 @@ __device__ long long *g_trace_buf = nullptr;
 
 struct VerifyFastParams {
     int h_qk, h_v;
+    int n_units;        // n_seq * h_v = gridDim.x
+    int prefetch_dist;  // a CTA warms L2 for unit blockIdx.x + prefetch_dist (about one wave ahead)
     float scale;
     const float *S0;
     const __nv_bfloat16 *q, *k, *v, *g, *beta;
@@ -95,6 +97,11 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool 
 {
     const int n = valid ? 16 : 0;   // src-size 0: nothing is read, the 16 bytes are zero-filled
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+// Ask L2 to fetch `bytes` (a multiple of 16) starting at `p`; nothing waits for it.
+__device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all()
 {
@@ -280,6 +287,30 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (tid == 32) {
         mbar_init(mbar, 1);
         *flag = 0;
+    }
+    // Warm L2 for the unit that a CTA will pick up about one wave from now, so that HBM keeps
+    // streaming while the resident CTAs are busy computing: its state tile and its q/k/v rows.
+    {
+        const int u2 = blockIdx.x + p.prefetch_dist;
+        if (u2 < p.n_units && tid >= 64) {
+            const int b2 = u2 / p.h_v, h2 = u2 % p.h_v;
+            const int t2 = tid - 64;   // 0..191
+            if (t2 < 4) {
+                prefetch_l2_bulk(p.S0 + (size_t)u2 * FV_D * FV_D + (size_t)t2 * 4096, 16384);
+            } else if (t2 < 4 + FV_T) {
+                const int base2 = p.node_offsets[b2];
+                const int T2 = min(p.node_offsets[b2 + 1] - base2, FV_T);
+                const int i = t2 - 4;
+                if (i < T2) {
+                    const int hk2 = h2 / (p.h_v / p.h_qk);
+                    prefetch_l2_bulk(p.v + ((size_t)(base2 + i) * p.h_v + h2) * FV_D, 256);
+                    if (h2 % (p.h_v / p.h_qk) == 0) {   // one value head per key head fetches q and k
+                        prefetch_l2_bulk(p.k + ((size_t)(base2 + i) * p.h_qk + hk2) * FV_D, 256);
+                        prefetch_l2_bulk(p.q + ((size_t)(base2 + i) * p.h_qk + hk2) * FV_D, 256);
+                    }
+                }
+            }
+        }
     }
     // (3) per-node tables: depth, root-path ids, g, beta (zeros beyond T)
     if (tid < FV_T) {
@@ -587,7 +618,9 @@ cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const voi
                                 int32_t *status_dev, cudaStream_t stream)
 {
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
-    VerifyFastParams p{s.h_qk, s.h_v, s.scale, S0,
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    VerifyFastParams p{s.h_qk, s.h_v, s.n_seq * s.h_v, 2 * sms, s.scale, S0,
                        static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k),
                        static_cast<const __nv_bfloat16 *>(v), static_cast<const __nv_bfloat16 *>(g),
                        static_cast<const __nv_bfloat16 *>(beta), node_offsets, o, plan.tree_ok, plan.depth,
