@@ -223,6 +223,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     return done;
 }
 
+// Two fp32 values -> packed bf16 pair of the leading parts and packed bf16 pair of the remainders.
+__device__ __forceinline__ void split_pack_bf16(float x0, float x1, uint32_t &hi, uint32_t &lo)
+{
+    hi = pack_bf16(x0, x1);
+    const float h0 = __uint_as_float(hi << 16), h1 = __uint_as_float(hi & 0xFFFF0000u);
+    lo = pack_bf16(x0 - h0, x1 - h1);
+}
 __device__ __forceinline__ void split_bf16(float x, float &hi, float &lo)
 {
     hi = __bfloat162float(__float2bfloat16_rn(x));
@@ -256,6 +263,16 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hk = h / (p.h_v / p.h_qk);
     GDN_TRACE_MARK(0);
+#ifdef GDN_TRACE
+    if (threadIdx.x == 0 && g_trace_buf) {
+        unsigned smid;
+        unsigned long long gt;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+        g_trace_buf[blockIdx.x * 16 + 14] = smid;
+        g_trace_buf[blockIdx.x * 16 + 15] = (long long)gt;
+    }
+#endif
 
     // (1) state tile loads first (the longest latency of the prologue): a warp instruction covers
     // four rows; the eight lanes of a row each own one 16-byte bf16 piece of either K half.
@@ -288,6 +305,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         mbar_init(mbar, 1);
         *flag = 0;
     }
+    // this tree's v rows are needed only after the first MMA group: pull them into L2 meanwhile
+    if (tid >= 192 && tid - 192 < T) prefetch_l2_bulk(p.v + ((size_t)(base + tid - 192) * p.h_v + h) * FV_D, 256);
     // Warm L2 for the unit that a CTA will pick up about one wave from now, so that HBM keeps
     // streaming while the resident CTAs are busy computing: its state tile and its q/k/v rows.
     {
@@ -340,13 +359,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             const float f[8] = {u.x, u.y, u.z, u.w, w.x, w.y, w.z, w.w};
             uint32_t hi[4], lo[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float h0, l0, h1, l1;
-                split_bf16(f[2 * e], h0, l0);
-                split_bf16(f[2 * e + 1], h1, l1);
-                hi[e] = pack_bf16(h0, h1);
-                lo[e] = pack_bf16(l0, l1);
-            }
+            for (int e = 0; e < 4; ++e) split_pack_bf16(f[2 * e], f[2 * e + 1], hi[e], lo[e]);
             const uint32_t off = sw128_offset(row, kh * 8 + l8);
             *reinterpret_cast<uint4 *>(smem + SM_A_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
             *reinterpret_cast<uint4 *>(smem + SM_A_LO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
@@ -394,10 +407,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     }
     GDN_TRACE_MARK(4);
 
-    // (7) wait for the first MMA group (bounded: on expiry flag the error and fall through to the clean-up)
-    if (!mbar_wait_bounded(mbar, 0)) *flag = 1;
-    tc_fence_after();
+    // (7) wait for the first MMA group: one thread polls the mbarrier (bounded: on expiry it flags the
+    // error and everybody falls through to the clean-up), the others sleep in the CTA barrier
+    if (tid == 0 && !mbar_wait_bounded(mbar, 0)) *flag = 1;
     __syncthreads();
+    tc_fence_after();
     bool ok = *flag == 0;
     GDN_TRACE_MARK(5);
 
@@ -416,16 +430,15 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             const int row = (warp & 3) * 32 + lane;
             const int half = warp >> 2;   // TMEM columns 128 + 64*half .. : k_j for j = 32*half ..
             const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 128 + half * 64;
+            uint32_t ra[32], rb[32];
+            GDN_TMEM_LD32(taddr, ra);
+            GDN_TMEM_LD32(taddr + 32, rb);
+            tmem_wait_ld();
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                uint32_t rr[32];
-                GDN_TMEM_LD32(taddr + part * 32, rr);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int col = half * 32 + part * 16 + j;
-                    gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(rr[2 * j]);
-                }
+            for (int j = 0; j < 16; ++j) {
+                const int col = half * 32 + j;
+                gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[2 * j]);
+                gram[row * 64 + ((col + 16) ^ (row & 31))] = __uint_as_float(rb[2 * j]);
             }
         }
         tc_fence_before();
@@ -450,47 +463,45 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         __syncthreads();
         GDN_TRACE_MARK(7);
 
-        // (10a) warps 0-1, one thread per node: z^T = y^T (I + X_path)^-1 by back-substitution over the
-        // root path (column-oriented: once z_l is final, subtract z_l X(n_l, n_t) from every z_t, t < l),
-        // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path)
-        if (tid < FV_T) {
-            const int i = tid;
+        // (10a) z^T = y^T (I + X_path)^-1 by back-substitution over the root path (column-oriented: once
+        // z_l is final, subtract z_l X(n_l, n_t) from every z_t, t < l).  Four threads per node, thread s of
+        // the quad owning path positions 4s..4s+3; the result is scattered into the dense bf16 hi/lo tiles
+        // Z[i][j] (zero off the root path).
+        {
+            const int i = tid >> 2, sq = tid & 3;
             const int d = depth_s[i];
+            const int dmax = __reduce_max_sync(0xffffffffu, d);
             const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-            for (int c16 = 0; c16 < 8; ++c16) {
-                *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, c16)) = zero4;
-                *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, c16)) = zero4;
-            }
+            *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, 2 * sq)) = zero4;
+            *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, 2 * sq + 1)) = zero4;
+            *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, 2 * sq)) = zero4;
+            *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, 2 * sq + 1)) = zero4;
             const uint4 row = *reinterpret_cast<const uint4 *>(anc_s + i * 16);
             const uint32_t idw[4] = {row.x, row.y, row.z, row.w};
-            float z[FV_MD];
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                const float4 y4 = *reinterpret_cast<const float4 *>(ys + i * FV_MD + q4 * 4);
-                z[q4 * 4 + 0] = y4.x; z[q4 * 4 + 1] = y4.y; z[q4 * 4 + 2] = y4.z; z[q4 * 4 + 3] = y4.w;
-            }
+            const float4 y4 = *reinterpret_cast<const float4 *>(ys + i * FV_MD + sq * 4);
+            float z[4] = {y4.x, y4.y, y4.z, y4.w};
 #pragma unroll
             for (int l = FV_MD - 1; l >= 1; --l) {
-                if (l < d) {
-                    const int nl = (int)((idw[l >> 2] >> ((l & 3) * 8)) & 0xFFu);
-                    const float zl = z[l];
-#pragma unroll
-                    for (int q4 = 0; q4 * 4 < l; ++q4) {
-                        const float4 x4 = *reinterpret_cast<const float4 *>(xs + nl * FV_MD + q4 * 4);
+                if (l < dmax) {   // warp-uniform
+                    const float zl = __shfl_sync(0xffffffffu, z[l & 3], (lane & ~3) | (l >> 2));
+                    if (l < d && sq * 4 < l) {
+                        const int nl = (int)((idw[l >> 2] >> ((l & 3) * 8)) & 0xFFu);
+                        const float4 x4 = *reinterpret_cast<const float4 *>(xs + nl * FV_MD + sq * 4);
                         const float xv[4] = {x4.x, x4.y, x4.z, x4.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
-                            if (q4 * 4 + e < l) z[q4 * 4 + e] = fmaf(-zl, xv[e], z[q4 * 4 + e]);
+                            if (sq * 4 + e < l) z[e] = fmaf(-zl, xv[e], z[e]);
                     }
                 }
             }
+            __syncwarp();   // the quad's zero fill precedes the scattered stores below
 #pragma unroll
-            for (int t = 0; t < FV_MD; ++t) {
+            for (int e = 0; e < 4; ++e) {
+                const int t = sq * 4 + e;
                 if (t < d) {
-                    const int j = (int)((idw[t >> 2] >> ((t & 3) * 8)) & 0xFFu);
+                    const int j = (int)((idw[sq] >> (e * 8)) & 0xFFu);
                     float hi, lo;
-                    split_bf16(z[t], hi, lo);
+                    split_bf16(z[e], hi, lo);
                     const uint32_t off = sw128_row_offset(i, j >> 3) + (j & 7) * 2;
                     *reinterpret_cast<__nv_bfloat16 *>(smem + SM_Z_HI + off) = __float2bfloat16_rn(hi);
                     *reinterpret_cast<__nv_bfloat16 *>(smem + SM_Z_LO + off) = __float2bfloat16_rn(lo);
@@ -503,11 +514,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             const int c = (warp & 3) * 32 + lane;
             const int half = warp >> 2;
             const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
+            uint32_t rr[2][32];
+            GDN_TMEM_LD32(taddr, rr[0]);        // columns 2j, 2j+1 for 16 nodes: p^k_j, p^q_j
+            GDN_TMEM_LD32(taddr + 32, rr[1]);   // the next 16 nodes
+            tmem_wait_ld();
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
-                uint32_t rr[32];
-                GDN_TMEM_LD32(taddr + part * 32, rr);   // columns 2j, 2j+1 for 16 nodes: p^k_j, p^q_j
-                tmem_wait_ld();
 #pragma unroll
                 for (int oct = 0; oct < 2; ++oct) {
                     uint32_t hi[4], lo[4];
@@ -519,13 +531,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
                             const int jj = oct * 8 + e * 2 + s2;
                             const int j = half * 32 + part * 16 + jj;
                             const float4 gj = gab[j];
-                            rv[s2] = gj.z * (__bfloat162float(vs[j * FV_D + c]) - gj.y * __uint_as_float(rr[2 * jj]));
+                            rv[s2] = gj.z * (__bfloat162float(vs[j * FV_D + c]) - gj.y * __uint_as_float(rr[part][2 * jj]));
                         }
-                        float h0, l0, h1, l1;
-                        split_bf16(rv[0], h0, l0);
-                        split_bf16(rv[1], h1, l1);
-                        hi[e] = pack_bf16(h0, h1);
-                        lo[e] = pack_bf16(l0, l1);
+                        split_pack_bf16(rv[0], rv[1], hi[e], lo[e]);
                     }
                     const uint32_t off = sw128_row_offset(c, half * 4 + part * 2 + oct);
                     *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -553,42 +561,57 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             }
             umma_commit(mbar);
         }
-        if (!mbar_wait_bounded(mbar, 1)) {
-            *flag = 1;
-            ok = false;
-        }
+        if (tid == 0 && !mbar_wait_bounded(mbar, 1)) *flag = 1;
+        __syncthreads();
         tc_fence_after();
+        ok = *flag == 0;
         GDN_TRACE_MARK(9);
 
-        // (12) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i])
+        // (12) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i]), staged through shared memory (over the
+        // dead R^T tiles) so that global memory sees 16-byte stores of whole rows
         if (ok) {
             const int c = (warp & 3) * 32 + lane;
             const int half = warp >> 2;
             const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-            TOut *o = static_cast<TOut *>(p.o);
+            TOut *o_s = reinterpret_cast<TOut *>(smem + SM_RT_HI);   // [64][128] TOut: 16 or 32 KB
+            uint32_t pp[2][32], dd[2][16];
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
-                const int i0 = half * 32 + part * 16;
-                if (i0 < T) {
-                    uint32_t pp[32], dd[16];
-                    GDN_TMEM_LD32(trow + 2 * i0, pp);
-                    GDN_TMEM_LD16(trow + 128 + i0, dd);
-                    tmem_wait_ld();
+                GDN_TMEM_LD32(trow + 2 * (half * 32 + part * 16), pp[part]);
+                GDN_TMEM_LD16(trow + 128 + half * 32 + part * 16, dd[part]);
+            }
+            tmem_wait_ld();
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) {
-                        const int i = i0 + jj;
-                        if (i < T) {
-                            const float out = p.scale * fmaf(gab[i].y, __uint_as_float(pp[2 * jj + 1]), __uint_as_float(dd[jj]));
-                            store_from_float(o + ((size_t)(base + i) * p.h_v + h) * FV_D + c, out);
-                        }
-                    }
+            for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) {
+                    const int i = half * 32 + part * 16 + jj;
+                    const float out = p.scale * fmaf(gab[i].y, __uint_as_float(pp[part][2 * jj + 1]), __uint_as_float(dd[part][jj]));
+                    store_from_float(o_s + i * FV_D + c, out);
                 }
+            }
+        }
+        __syncthreads();
+        if (*flag == 0) {
+            constexpr int ROW_CHUNKS = FV_D * (int)sizeof(TOut) / 16;   // 16-byte pieces per output row
+            uint8_t *o = static_cast<uint8_t *>(p.o);
+            for (int idx = tid; idx < T * ROW_CHUNKS; idx += FV_THREADS) {
+                const int i = idx / ROW_CHUNKS, ck = idx % ROW_CHUNKS;
+                const uint4 val = *reinterpret_cast<const uint4 *>(smem + SM_RT_HI + (size_t)i * FV_D * sizeof(TOut) + ck * 16);
+                *reinterpret_cast<uint4 *>(o + (((size_t)(base + i) * p.h_v + h) * FV_D) * sizeof(TOut) + ck * 16) = val;
             }
         }
     }
     if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
 
     GDN_TRACE_MARK(10);
+#ifdef GDN_TRACE
+    if (threadIdx.x == 0 && g_trace_buf) {
+        unsigned long long gt;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+        g_trace_buf[blockIdx.x * 16 + 13] = (long long)gt;
+    }
+#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
