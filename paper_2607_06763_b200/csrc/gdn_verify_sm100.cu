@@ -445,19 +445,30 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         __syncthreads();
         GDN_TRACE_MARK(6);
         // (9) X and Y of Eq. 9 for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
-        for (int idx = tid; idx < FV_T * FV_MD; idx += FV_THREADS) {
-            const int i = idx >> 4, t = idx & 15;
-            const int d = depth_s[i];
-            float xv = 0.f, yv = 0.f;
-            if (t < d) {
-                const int j = anc_s[idx];
+        {
+            float gdiff[4], gk[4], gq[4], bi[4];
+            bool on[4], onx[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = u * FV_THREADS + tid;
+                const int i = idx >> 4, t = idx & 15;
+                const int d = depth_s[i];
+                on[u] = t < d;
+                onx[u] = t < d - 1;
+                const int j = on[u] ? anc_s[idx] : 0;
                 const float4 gi = gab[i];
-                const float dec = expf(gi.x - gab[j].x);
-                yv = dec * gram[(2 * i + 1) * 64 + (j ^ ((2 * i + 1) & 31))];
-                if (t < d - 1) xv = gi.z * dec * gram[(2 * i) * 64 + (j ^ ((2 * i) & 31))];
+                gdiff[u] = gi.x - gab[j].x;
+                bi[u] = gi.z;
+                gq[u] = gram[(2 * i + 1) * 64 + (j ^ ((2 * i + 1) & 31))];
+                gk[u] = gram[(2 * i) * 64 + (j ^ ((2 * i) & 31))];
             }
-            xs[idx] = xv;
-            ys[idx] = yv;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = u * FV_THREADS + tid;
+                const float dec = expf(gdiff[u]);
+                ys[idx] = on[u] ? dec * gq[u] : 0.f;
+                xs[idx] = onx[u] ? bi[u] * dec * gk[u] : 0.f;
+            }
         }
         cp_async_wait_all();
         __syncthreads();
@@ -514,30 +525,32 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             const int c = (warp & 3) * 32 + lane;
             const int half = warp >> 2;
             const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
-            uint32_t rr[2][32];
-            GDN_TMEM_LD32(taddr, rr[0]);        // columns 2j, 2j+1 for 16 nodes: p^k_j, p^q_j
-            GDN_TMEM_LD32(taddr + 32, rr[1]);   // the next 16 nodes
-            tmem_wait_ld();
-#pragma unroll
+#pragma unroll 1
             for (int part = 0; part < 2; ++part) {
+                const int j0 = half * 32 + part * 16;
+                uint32_t rr[32];
+                GDN_TMEM_LD32(taddr + part * 32, rr);   // columns 2j, 2j+1 for 16 nodes: p^k_j, p^q_j
+                float vv[16], aj[16], bj[16];
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) {
+                    vv[jj] = __bfloat162float(vs[(j0 + jj) * FV_D + c]);
+                    const float4 gj = gab[j0 + jj];
+                    aj[jj] = gj.y;
+                    bj[jj] = gj.z;
+                }
+                tmem_wait_ld();
+                uint32_t hi[8], lo[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float r0 = bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[4 * e]));
+                    const float r1 = bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[4 * e + 2]));
+                    split_pack_bf16(r0, r1, hi[e], lo[e]);
+                }
 #pragma unroll
                 for (int oct = 0; oct < 2; ++oct) {
-                    uint32_t hi[4], lo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        float rv[2];
-#pragma unroll
-                        for (int s2 = 0; s2 < 2; ++s2) {
-                            const int jj = oct * 8 + e * 2 + s2;
-                            const int j = half * 32 + part * 16 + jj;
-                            const float4 gj = gab[j];
-                            rv[s2] = gj.z * (__bfloat162float(vs[j * FV_D + c]) - gj.y * __uint_as_float(rr[part][2 * jj]));
-                        }
-                        split_pack_bf16(rv[0], rv[1], hi[e], lo[e]);
-                    }
                     const uint32_t off = sw128_row_offset(c, half * 4 + part * 2 + oct);
-                    *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<uint4 *>(smem + SM_RT_LO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = make_uint4(hi[4 * oct], hi[4 * oct + 1], hi[4 * oct + 2], hi[4 * oct + 3]);
+                    *reinterpret_cast<uint4 *>(smem + SM_RT_LO + off) = make_uint4(lo[4 * oct], lo[4 * oct + 1], lo[4 * oct + 2], lo[4 * oct + 3]);
                 }
             }
         }
@@ -547,13 +560,13 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         tc_fence_after();
         GDN_TRACE_MARK(8);
 
-        // (11) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j], all four hi/lo cross terms
+        // (11) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
         if (tid == 0) {
             constexpr uint32_t id2 = idesc_bf16(128, 64);
             const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
             const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
 #pragma unroll
-            for (int combo = 0; combo < 4; ++combo) {
+            for (int combo = 0; combo < 3; ++combo) {   // hi.hi, lo.hi, hi.lo; lo.lo is below 2^-18 of the result
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
                     umma_bf16(tmem + 128, a2[combo & 1] + (uint64_t)(ks * 2), b2[combo >> 1] + (uint64_t)(ks * 2), id2,
@@ -574,20 +587,20 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             const int half = warp >> 2;
             const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
             TOut *o_s = reinterpret_cast<TOut *>(smem + SM_RT_HI);   // [64][128] TOut: 16 or 32 KB
-            uint32_t pp[2][32], dd[2][16];
-#pragma unroll
+#pragma unroll 1
             for (int part = 0; part < 2; ++part) {
-                GDN_TMEM_LD32(trow + 2 * (half * 32 + part * 16), pp[part]);
-                GDN_TMEM_LD16(trow + 128 + half * 32 + part * 16, dd[part]);
-            }
-            tmem_wait_ld();
+                const int i0 = half * 32 + part * 16;
+                uint32_t pp[32], dd[16];
+                GDN_TMEM_LD32(trow + 2 * i0, pp);
+                GDN_TMEM_LD16(trow + 128 + i0, dd);
+                float ai[16];
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
+                for (int jj = 0; jj < 16; ++jj) ai[jj] = gab[i0 + jj].y;
+                tmem_wait_ld();
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) {
-                    const int i = half * 32 + part * 16 + jj;
-                    const float out = p.scale * fmaf(gab[i].y, __uint_as_float(pp[part][2 * jj + 1]), __uint_as_float(dd[part][jj]));
-                    store_from_float(o_s + i * FV_D + c, out);
+                    const float out = p.scale * fmaf(ai[jj], __uint_as_float(pp[2 * jj + 1]), __uint_as_float(dd[jj]));
+                    store_from_float(o_s + (i0 + jj) * FV_D + c, out);
                 }
             }
         }
