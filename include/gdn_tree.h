@@ -145,6 +145,33 @@ int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k, const voi
                     void *cuda_stream);
 
 /*
+ * Commit of the previous decode step fused with the verification of the next one.  Section 3.4
+ * postpones the state commit to the next decoding iteration, when the accepted branch is known;
+ * this entry point does both halves of that iteration in one pass over the state:
+ *     S[b] <- Eq. 7 replayed over the accepted path of the PREVIOUS tree of b   (as gdn_tree_commit)
+ *     o    <- verification of the NEW tree of b against that advanced state     (as gdn_tree_verify)
+ * so every state tile is read from memory once and written once per step.  The results are those
+ * of gdn_tree_commit followed by gdn_tree_verify (same tolerances; on the tensor-core path it is
+ * one kernel, otherwise the two kernels are launched back to back).
+ *   shape        : describes the NEW tree (total_nodes, max_tree_nodes) and the common head shapes
+ *   S            : [device] in: committed state before the previous step, out: state after it
+ *   k_prev, v_prev, g_prev, beta_prev, parent_prev (may be NULL), node_offsets_prev :
+ *                  [device] the previous step's packed tensors (in_dtype), as given to its verify
+ *   path, path_offsets : [device] accepted paths in the previous trees, as for gdn_tree_commit
+ *   q, k, v, g, beta, parent, node_offsets, o, workspace, workspace_bytes, status_dev :
+ *                  the new tree, exactly as for gdn_tree_verify
+ * A rejected path (GDN_ERR_PATH) leaves that state unchanged and the new tree is verified
+ * against the unchanged state.
+ */
+int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
+                           const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                           const int32_t *node_offsets_prev, const int32_t *path,
+                           const int32_t *path_offsets, const void *q, const void *k, const void *v,
+                           const void *g, const void *beta, const int32_t *parent,
+                           const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
+                           int32_t *status_dev, void *cuda_stream);
+
+/*
  * Host-buffer variants: same operations with every tensor in [host] memory
  * (pinned memory makes the copies asynchronous).  Inputs are copied into
  * `dev_arena` ([device], >= gdn_tree_host_arena_bytes(shape, total_path_len) bytes, 256-byte

@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     gdn_status_string,
     gdn_tree_commit,
     gdn_tree_commit_host,
+    gdn_tree_commit_verify,
     gdn_tree_host_arena_bytes,
     gdn_tree_validate_host,
     gdn_tree_verify,

@@ -27,6 +27,7 @@ EXPORTS = (
     "gdn_tree_verify_host",
     "gdn_tree_commit_host",
     "gdn_tree_verify_static",
+    "gdn_tree_commit_verify",
 )
 
 GDN_STATIC_SCRATCH_BYTES = 4 << 20
@@ -89,6 +90,8 @@ def load_library():
         lib.gdn_tree_verify_host.argtypes = [sp] + [vp] * 10 + [ctypes.c_size_t, vp]
         lib.gdn_tree_commit_host.restype = ctypes.c_int
         lib.gdn_tree_commit_host.argtypes = [sp] + [vp] * 9 + [ctypes.c_int32, vp, ctypes.c_size_t, vp]
+        lib.gdn_tree_commit_verify.restype = ctypes.c_int
+        lib.gdn_tree_commit_verify.argtypes = [sp] + [vp] * 18 + [ctypes.c_size_t, vp, vp]
         lib.gdn_tree_verify_static.restype = ctypes.c_int
         lib.gdn_tree_verify_static.argtypes = [sp] + [vp] * 11
         _lib = lib
@@ -178,3 +181,14 @@ def gdn_tree_verify_static(shape: GdnShape, S0, q, k, v, g, beta, parent, node_o
     return int(load_library().gdn_tree_verify_static(ctypes.byref(shape), _ptr(S0), _ptr(q), _ptr(k), _ptr(v),
                                                       _ptr(g), _ptr(beta), _ptr(parent), _ptr(node_offsets),
                                                       _ptr(o), _ptr(status_dev), _stream(stream)))
+
+
+def gdn_tree_commit_verify(shape: GdnShape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev,
+                           path, path_offsets, q, k, v, g, beta, parent, node_offsets, o, workspace,
+                           workspace_bytes, status_dev, stream=None) -> int:
+    """Commit of the previous step's accepted paths fused with the verification of the new trees."""
+    return int(load_library().gdn_tree_commit_verify(
+        ctypes.byref(shape), _ptr(S), _ptr(k_prev), _ptr(v_prev), _ptr(g_prev), _ptr(beta_prev), _ptr(parent_prev),
+        _ptr(node_offsets_prev), _ptr(path), _ptr(path_offsets), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta),
+        _ptr(parent), _ptr(node_offsets), _ptr(o), _ptr(workspace), int(workspace_bytes), _ptr(status_dev),
+        _stream(stream)))

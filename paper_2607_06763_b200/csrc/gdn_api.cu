@@ -184,6 +184,50 @@ extern "C" int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k
     return GDN_OK;
 }
 
+extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
+                                      const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                      const int32_t *node_offsets_prev, const int32_t *path,
+                                      const int32_t *path_offsets, const void *q, const void *k, const void *v,
+                                      const void *g, const void *beta, const int32_t *parent,
+                                      const int32_t *node_offsets, void *o, void *workspace,
+                                      size_t workspace_bytes, int32_t *status_dev, void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0) return GDN_OK;
+    if (!S || !node_offsets_prev || !path_offsets || !status_dev) return GDN_ERR_NULL;
+    if (!verify_sm100_supported(s) || s.total_nodes == 0) {
+        // general shapes: the two kernels back to back on the stream (the shape's node counts are
+        // not used by commit, so the new tree's shape serves for the previous tree as well)
+        rc = gdn_tree_commit(shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
+                             path_offsets, status_dev, cuda_stream);
+        if (rc != GDN_OK) return rc;
+        return gdn_tree_verify(shape, S, q, k, v, g, beta, parent, node_offsets, o, workspace, workspace_bytes,
+                               status_dev, cuda_stream);
+    }
+    if (!k_prev || !v_prev || !g_prev || !beta_prev || !path) return GDN_ERR_NULL;
+    if (!q || !k || !v || !g || !beta || !parent || !node_offsets || !o) return GDN_ERR_NULL;
+    if (!workspace) return GDN_ERR_WORKSPACE;
+    if (!aligned16(S) || !aligned16(k_prev) || !aligned16(v_prev) || !aligned16(g_prev) || !aligned16(beta_prev) ||
+        !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) || !aligned16(o) ||
+        !aligned256(workspace) || (reinterpret_cast<uintptr_t>(parent_prev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(node_offsets_prev) & 3u) || (reinterpret_cast<uintptr_t>(path) & 3u) ||
+        (reinterpret_cast<uintptr_t>(path_offsets) & 3u) || (reinterpret_cast<uintptr_t>(parent) & 3u) ||
+        (reinterpret_cast<uintptr_t>(node_offsets) & 3u) || (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    const WorkspaceLayout lay = workspace_layout(s);
+    if (workspace_bytes < lay.total) return GDN_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const PlanPtrs plan = plan_ptrs(workspace, lay);
+    if (launch_plan(s, parent, node_offsets, plan, status_dev, stream) != cudaSuccess) return GDN_ERR_CUDA;
+    if (launch_commit_verify_sm100(s, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
+                                   path_offsets, q, k, v, g, beta, node_offsets, o, plan, status_dev,
+                                   stream) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
 extern "C" size_t gdn_tree_host_arena_bytes(const gdn_shape_t *shape, int32_t total_path_len)
 {
     if (check_shape(shape) != GDN_OK || total_path_len < 0) return 0;

@@ -69,6 +69,16 @@ cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const voi
                                 const int32_t *node_offsets, void *o, const PlanPtrs &plan,
                                 int32_t *status_dev, cudaStream_t stream);
 
+// Same kernel with the commit of the previous step's accepted paths fused in front of the verify:
+// the state tile is read once, advanced along the path (Eq. 7), written back, and the new tree is
+// verified against the advanced state.
+cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const void *k_prev, const void *v_prev,
+                                       const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                       const int32_t *node_offsets_prev, const int32_t *path,
+                                       const int32_t *path_offsets, const void *q, const void *k, const void *v,
+                                       const void *g, const void *beta, const int32_t *node_offsets, void *o,
+                                       const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream);
+
 cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k, const void *v,
                                   const void *g, const void *beta, const int32_t *parent,
                                   const int32_t *node_offsets, const int32_t *path,

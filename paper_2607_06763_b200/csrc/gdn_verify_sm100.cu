@@ -49,7 +49,10 @@ constexpr int SM_Y = SM_X + 4096;                // fp32 [64][16]  Y(i, t-th pat
 constexpr int SM_ANC = SM_Y + 4096;              // u8   [64][16]  root-path node ids (0xFF = unused)
 constexpr int SM_GAB = SM_ANC + 1024;            // float4 [64]: (G_i = log a_i, a_i, beta_i, g_i)
 constexpr int SM_DEPTH = SM_GAB + 1024;          // u8 [64] (0 beyond T)
-constexpr int SM_MBAR = SM_DEPTH + FV_T;         // u64
+constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit: int [16] node ids, int [16] parents, float2 [16] (alpha, beta)
+constexpr int SM_PK = SM_X;                      // fused commit: k rows of the accepted path, bf16 [16][128] (before X is needed)
+constexpr int SM_PV = SM_Y;                      // fused commit: v rows of the accepted path, bf16 [16][128]
+constexpr int SM_MBAR = SM_PATH + 256;           // u64
 constexpr int SM_TMEM = SM_MBAR + 8;             // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
 constexpr int SM_BYTES = SM_FLAG + 4;
@@ -85,6 +88,10 @@ struct VerifyFastParams {
     const uint8_t *depth;
     const uint8_t *anc8;
     int32_t *status_dev;
+    // fused commit of the previous step's accepted paths (only read by the FUSED instantiation)
+    float *S_rw;                                       // same tensor as S0, written in place
+    const __nv_bfloat16 *pk, *pv, *pg, *pbeta;         // the previous tree's k, v, g, beta
+    const int32_t *pparent, *pnode_offsets, *path, *path_offsets;
 };
 
 // ---------------------------------------------------------------------------------------- PTX
@@ -237,7 +244,7 @@ __device__ __forceinline__ void split_bf16(float x, float &hi, float &lo)
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <typename TOut>
+template <typename TOut, bool FUSED>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const VerifyFastParams p)
 {
     extern __shared__ uint8_t fv_smem_raw[];
@@ -348,6 +355,114 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         gab[tid] = make_float4(0.f, 0.f, be, gi);
     }
     GDN_TRACE_MARK(1);
+
+    // (3') fused commit: replay Eq. 7 along the previous step's accepted path on the state tile while it
+    // sits in registers, write it back, and let everything below verify the new tree against it.
+    // Per row c (one value component): s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that
+    // share a row reduce k.s_c with three shuffles.
+    if constexpr (FUSED) {
+        int *path_s = reinterpret_cast<int *>(smem + SM_PATH);
+        int *par_s = path_s + FV_MD;
+        float2 *ab_path = reinterpret_cast<float2 *>(smem + SM_PATH + 128);
+        const int pp0 = p.path_offsets[b];
+        const int L = p.path_offsets[b + 1] - pp0;
+        if (L != 0) {   // uniform over the CTA; an empty path leaves the state alone
+            const int pbase = p.pnode_offsets[b];
+            const int pT = p.pnode_offsets[b + 1] - pbase;
+            const bool shape_ok = L > 0 && L <= FV_MD && pT > 0 && pp0 >= 0;
+            if (shape_ok && tid < L) {
+                const int n = p.path[pp0 + tid];
+                path_s[tid] = n;
+                par_s[tid] = (p.pparent && n >= 0 && n < pT) ? p.pparent[pbase + n] : -2;
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int bad = !shape_ok;
+                for (int t = 0; !bad && t < L; ++t) {
+                    const int n = path_s[t];
+                    if (n < 0 || n >= pT) bad = 1;
+                    else if (p.pparent) bad = par_s[t] != (t ? path_s[t - 1] : -1);
+                    else if (t && n <= path_s[t - 1]) bad = 1;
+                }
+                if (bad) {
+                    report_status(p.status_dev, GDN_ERR_PATH);
+                    path_s[0] = -1;   // tells everybody to skip the replay: this state stays as it was
+                }
+            }
+            __syncthreads();
+            if (path_s[0] >= 0) {
+                // k and v rows of the path (bf16, 256 B each) and the per-step scalars
+                for (int idx = tid; idx < L * 32; idx += FV_THREADS) {
+                    const int t = idx >> 5, c16 = idx & 15;
+                    const size_t n = (size_t)pbase + path_s[t];
+                    if (idx & 16)
+                        cp_async_16(sbase + SM_PV + t * 256 + c16 * 16, p.pv + (n * p.h_v + h) * FV_D + c16 * 8, true);
+                    else
+                        cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + hk) * FV_D + c16 * 8, true);
+                }
+                if (tid < L) {
+                    const size_t n = (size_t)pbase + path_s[tid];
+                    ab_path[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + h])),
+                                               __bfloat162float(p.pbeta[n * p.h_v + h]));
+                }
+                cp_async_wait_all();   // also completes this thread's share of the k/q tile (harmless)
+                __syncthreads();
+                const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
+                const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
+#pragma unroll 1
+                for (int t = 0; t < L; ++t) {
+                    // this thread's sixteen key positions: 64*kh + 8*l8 + e
+                    float kf[16];
+#pragma unroll
+                    for (int kh = 0; kh < 2; ++kh) {
+                        const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
+                        const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            kf[kh * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
+                            kf[kh * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
+                        }
+                    }
+                    const float2 ab = ab_path[t];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = warp * 16 + i * 4 + r4;
+                        float xs16[16];
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            xs16[q4 * 4 + 0] = x[i][q4].x; xs16[q4 * 4 + 1] = x[i][q4].y;
+                            xs16[q4 * 4 + 2] = x[i][q4].z; xs16[q4 * 4 + 3] = x[i][q4].w;
+                        }
+                        float dot = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) dot = fmaf(kf[e], xs16[e], dot);
+                        dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                        dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                        dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                        const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
+                        const float w = ab.y * (vc - ab.x * dot);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) xs16[e] = fmaf(kf[e], w, ab.x * xs16[e]);
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4)
+                            x[i][q4] = make_float4(xs16[q4 * 4 + 0], xs16[q4 * 4 + 1], xs16[q4 * 4 + 2], xs16[q4 * 4 + 3]);
+                    }
+                }
+                // the committed state: the only state write of the step
+                float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float4 *dst = reinterpret_cast<float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+#pragma unroll
+                    for (int kh = 0; kh < 2; ++kh) {
+                        dst[kh * 16 + l8 * 2 + 0] = x[i][kh * 2 + 0];
+                        dst[kh * 16 + l8 * 2 + 1] = x[i][kh * 2 + 1];
+                    }
+                }
+            }
+            __syncthreads();   // the path rows share their shared memory with the X / Y tables
+        }
+    }
 
     // (4) fp32 -> bf16 hi + lo, written as the A operand
 #pragma unroll
@@ -630,14 +745,31 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
 }
 
-template <typename TOut>
+template <typename TOut, bool FUSED>
 cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, cudaStream_t stream)
 {
-    cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          SM_ALLOC);
     if (e != cudaSuccess) return e;
-    verify_sm100_kernel<TOut><<<s.n_seq * s.h_v, FV_THREADS, SM_ALLOC, stream>>>(p);
+    verify_sm100_kernel<TOut, FUSED><<<s.n_seq * s.h_v, FV_THREADS, SM_ALLOC, stream>>>(p);
     return cudaGetLastError();
+}
+
+VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *q, const void *k, const void *v,
+                             const void *g, const void *beta, const int32_t *node_offsets, void *o,
+                             const PlanPtrs &plan, int32_t *status_dev)
+{
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    VerifyFastParams p{};
+    p.h_qk = s.h_qk; p.h_v = s.h_v; p.n_units = s.n_seq * s.h_v; p.prefetch_dist = 2 * sms; p.scale = s.scale;
+    p.S0 = S0;
+    p.q = static_cast<const __nv_bfloat16 *>(q); p.k = static_cast<const __nv_bfloat16 *>(k);
+    p.v = static_cast<const __nv_bfloat16 *>(v); p.g = static_cast<const __nv_bfloat16 *>(g);
+    p.beta = static_cast<const __nv_bfloat16 *>(beta);
+    p.node_offsets = node_offsets; p.o = o;
+    p.tree_ok = plan.tree_ok; p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
+    return p;
 }
 
 }  // namespace
@@ -654,15 +786,26 @@ cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const voi
                                 int32_t *status_dev, cudaStream_t stream)
 {
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    VerifyFastParams p{s.h_qk, s.h_v, s.n_seq * s.h_v, 2 * sms, s.scale, S0,
-                       static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k),
-                       static_cast<const __nv_bfloat16 *>(v), static_cast<const __nv_bfloat16 *>(g),
-                       static_cast<const __nv_bfloat16 *>(beta), node_offsets, o, plan.tree_ok, plan.depth,
-                       plan.anc8, status_dev};
-    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16>(s, p, stream);
-    return launch_fast_typed<float>(s, p, stream);
+    const VerifyFastParams p = make_params(s, S0, q, k, v, g, beta, node_offsets, o, plan, status_dev);
+    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false>(s, p, stream);
+    return launch_fast_typed<float, false>(s, p, stream);
+}
+
+cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const void *k_prev, const void *v_prev,
+                                       const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                       const int32_t *node_offsets_prev, const int32_t *path,
+                                       const int32_t *path_offsets, const void *q, const void *k, const void *v,
+                                       const void *g, const void *beta, const int32_t *node_offsets, void *o,
+                                       const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream)
+{
+    if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
+    VerifyFastParams p = make_params(s, S, q, k, v, g, beta, node_offsets, o, plan, status_dev);
+    p.S_rw = S;
+    p.pk = static_cast<const __nv_bfloat16 *>(k_prev); p.pv = static_cast<const __nv_bfloat16 *>(v_prev);
+    p.pg = static_cast<const __nv_bfloat16 *>(g_prev); p.pbeta = static_cast<const __nv_bfloat16 *>(beta_prev);
+    p.pparent = parent_prev; p.pnode_offsets = node_offsets_prev; p.path = path; p.path_offsets = path_offsets;
+    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, true>(s, p, stream);
+    return launch_fast_typed<float, true>(s, p, stream);
 }
 
 #ifdef GDN_TRACE

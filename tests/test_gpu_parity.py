@@ -248,3 +248,86 @@ def test_host_buffer_entry_points(tl):
                                   w.path_offsets, L, arena, arena_bytes)
     assert rc == 0
     tl.assert_state_close(S_h.astype(np.float64), tl.oracle_commit(w), what="commit_host S_new")
+
+
+# ------------------------------------------------------------------ fused commit + verify
+def _fused_case(tl, prev, new, what):
+    """commit(prev.path) + verify(new tree) in one call against: oracle commit, then oracle verify on that state."""
+    import paper_2607_06763_b200 as gdn
+    assert prev.n_seq == new.n_seq
+    dp, dn = tl.DeviceCase(prev), tl.DeviceCase(new)
+    S = dp.S0.clone()
+    rc = gdn.gdn_tree_commit_verify(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path,
+                                    dp.path_offsets, dn.q, dn.k, dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets,
+                                    dn.o, dn.ws, dn.ws_bytes, dn.status)
+    assert rc == 0, gdn.gdn_status_string(rc)
+    assert dn.device_status() == 0
+    S_ref = tl.oracle_commit(prev)
+    tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what=what + " S_new")
+    from oracle import gdn_oracle as orc
+    o_ref = orc.verify(S_ref, new.f64("q"), new.f64("k"), new.f64("v"), new.f64("g"), new.f64("beta"), new.parent,
+                       new.node_offsets, new.scale)
+    tl.assert_close_per_head(dn.o_host(), o_ref, new.node_offsets, what + " o", bf16_out=tl.is_bf16_out(new))
+    for b in range(prev.n_seq):   # empty accepted paths leave their states bit-identical
+        if prev.path_offsets[b + 1] == prev.path_offsets[b]:
+            assert bool((S[b] == dp.S0[b]).all())
+
+
+@pytest.mark.parametrize("out_dtype", [synth.BF16, synth.F32])
+def test_fused_commit_verify_tensor_core_path(tl, out_dtype):
+    rng = np.random.default_rng(21)
+    prev_trees = [synth.tree_geo(rng, 64), synth.tree_chain(16), synth.tree_geo(rng, 40), synth.tree_star(9)]
+    paths = [synth.longest_path(prev_trees[0]), np.arange(16, dtype=np.int32), np.zeros(0, np.int32),
+             np.array([0, 5], np.int32)]
+    prev = synth.random_case(31, prev_trees, 2, 4, 128, 128, synth.BF16, out_dtype, paths=paths, name="prev")
+    new_trees = [synth.tree_geo(rng, 64), synth.tree_geo(rng, 17), synth.tree_chain(16), synth.tree_geo(rng, 33)]
+    new = synth.random_case(32, new_trees, 2, 4, 128, 128, synth.BF16, out_dtype, name="new")
+    _fused_case(tl, prev, new, f"fused {out_dtype}")
+
+
+def test_fused_commit_verify_general_shapes_and_rejected_path(tl):
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(22)
+    prev = synth.random_case(33, [synth.tree_geo(rng, 20), synth.tree_chain(7)], 1, 2, 64, 48, synth.F32, synth.F32)
+    new = synth.random_case(34, [synth.tree_geo(rng, 90), synth.tree_geo(rng, 5)], 1, 2, 64, 48, synth.F32, synth.F32)
+    _fused_case(tl, prev, new, "fused generic")
+    # tensor-core path, one accepted path that is not a chain: that state stays, its tree is verified on it
+    prev_trees = [synth.tree_chain(6), synth.tree_chain(6)]
+    bad = synth.random_case(35, prev_trees, 1, 2, 128, 128, synth.BF16, synth.F32,
+                            paths=[np.array([0, 2], np.int32), np.array([0, 1, 2], np.int32)])
+    new2 = synth.random_case(36, [synth.tree_star(8), synth.tree_star(8)], 1, 2, 128, 128, synth.BF16, synth.F32)
+    dp, dn = tl.DeviceCase(bad), tl.DeviceCase(new2)
+    S = dp.S0.clone()
+    rc = gdn.gdn_tree_commit_verify(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path,
+                                    dp.path_offsets, dn.q, dn.k, dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets,
+                                    dn.o, dn.ws, dn.ws_bytes, dn.status)
+    assert rc == 0 and dn.device_status() == -9
+    assert bool((S[0] == dp.S0[0]).all()), "a rejected path must leave its state untouched"
+    good = synth.random_case(35, prev_trees, 1, 2, 128, 128, synth.BF16, synth.F32,
+                             paths=[np.zeros(0, np.int32), np.array([0, 1, 2], np.int32)])
+    S_ref = tl.oracle_commit(good)
+    tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what="fused, rejected path")
+    from oracle import gdn_oracle as orc
+    o_ref = orc.verify(S_ref, new2.f64("q"), new2.f64("k"), new2.f64("v"), new2.f64("g"), new2.f64("beta"),
+                       new2.parent, new2.node_offsets, new2.scale)
+    tl.assert_close_per_head(dn.o_host(), o_ref, new2.node_offsets, "fused, rejected path o")
+
+
+def test_fused_commit_verify_full_stack_sampled(tl):
+    import paper_2607_06763_b200 as gdn
+    prev, new = synth.config(5, 0), synth.config(5, 1)
+    dp, dn = tl.DeviceCase(prev), tl.DeviceCase(new)
+    S = dp.S0.clone()
+    rc = gdn.gdn_tree_commit_verify(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path,
+                                    dp.path_offsets, dn.q, dn.k, dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets,
+                                    dn.o, dn.ws, dn.ws_bytes, dn.status)
+    assert rc == 0 and dn.device_status() == 0
+    seqs = [0, 23, 47]
+    psub, _ = tl.sub_workload(prev, seqs)
+    nsub, nodes = tl.sub_workload(new, seqs)
+    S_ref = tl.oracle_commit(psub)
+    tl.assert_state_close(S.cpu().numpy().astype(np.float64)[seqs], S_ref, what="fused 1x48 S_new")
+    from oracle import gdn_oracle as orc
+    o_ref = orc.verify(S_ref, nsub.f64("q"), nsub.f64("k"), nsub.f64("v"), nsub.f64("g"), nsub.f64("beta"),
+                       nsub.parent, nsub.node_offsets, nsub.scale)
+    tl.assert_close_per_head(dn.o_host()[nodes], o_ref, nsub.node_offsets, "fused 1x48 o", bf16_out=True)
