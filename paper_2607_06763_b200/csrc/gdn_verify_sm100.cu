@@ -50,10 +50,10 @@ constexpr int SM_ANC = SM_Y + 4096;              // u8   [64][16]  root-path nod
 constexpr int SM_GAB = SM_ANC + 1024;            // float4 [64]: (G_i = log a_i, a_i, beta_i, g_i)
 constexpr int SM_DEPTH = SM_GAB + 1024;          // u8 [64] (0 beyond T)
 constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit: int [16] node ids, int [16] parents, float2 [16] (alpha, beta)
-constexpr int SM_PK = SM_X;                      // fused commit: k rows of the accepted path, bf16 [16][128] (before X is needed)
-constexpr int SM_PV = SM_Y;                      // fused commit: v rows of the accepted path, bf16 [16][128]
-constexpr int SM_MBAR = SM_PATH + 256;           // u64
-constexpr int SM_TMEM = SM_MBAR + 8;             // u32
+constexpr int SM_PK = 32768;                     // fused commit: k rows of the accepted path, bf16 [16][128], parked in the
+constexpr int SM_PV = 36864;                     // state-operand area until the replay is over; v rows likewise
+constexpr int SM_MBAR = SM_PATH + 256;           // 3 x u64: Gram done, P done, D done
+constexpr int SM_TMEM = SM_MBAR + 24;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
 constexpr int SM_BYTES = SM_FLAG + 4;
 constexpr int SM_ALLOC = SM_BYTES + 1024;        // slack for the 1024-byte alignment of the base
@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(smem + SM_V);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM_TMEM);
     volatile uint32_t *flag = reinterpret_cast<volatile uint32_t *>(smem + SM_FLAG);
-    const uint32_t mbar = sbase + SM_MBAR;
+    const uint32_t mbar_g = sbase + SM_MBAR, mbar_p = mbar_g + 8, mbar_d = mbar_g + 16;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hk = h / (p.h_v / p.h_qk);
@@ -280,6 +280,31 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         g_trace_buf[blockIdx.x * 16 + 15] = (long long)gt;
     }
 #endif
+
+    // L2 warming for the unit that a CTA will pick up about one wave from now, issued in slices at
+    // phase boundaries (one thread, a few instructions each) so that HBM keeps streaming while the resident
+    // CTAs compute, instead of all demand loads of a wave hitting it at once.
+    const int u_next = blockIdx.x + p.prefetch_dist;
+    auto warm_l2_state = [&](int slice) {   // slice 0..3 of the next unit's 64 KB state tile
+        if (tid == 96 && u_next < p.n_units)
+            prefetch_l2_bulk(p.S0 + (size_t)u_next * FV_D * FV_D + (size_t)slice * 4096, 16384);
+    };
+    auto warm_l2_rows = [&]() {             // the next unit's q/k/v rows
+        if (u_next < p.n_units && tid >= 128 && tid < 128 + FV_T) {
+            const int b2 = u_next / p.h_v, h2 = u_next % p.h_v;
+            const int base2 = p.node_offsets[b2];
+            const int T2 = min(p.node_offsets[b2 + 1] - base2, FV_T);
+            const int i = tid - 128;
+            if (i < T2) {
+                const int hk2 = h2 / (p.h_v / p.h_qk);
+                prefetch_l2_bulk(p.v + ((size_t)(base2 + i) * p.h_v + h2) * FV_D, 256);
+                if (h2 % (p.h_v / p.h_qk) == 0) {   // one value head per key head fetches q and k
+                    prefetch_l2_bulk(p.k + ((size_t)(base2 + i) * p.h_qk + hk2) * FV_D, 256);
+                    prefetch_l2_bulk(p.q + ((size_t)(base2 + i) * p.h_qk + hk2) * FV_D, 256);
+                }
+            }
+        }
+    };
 
     // (1) state tile loads first (the longest latency of the prologue): a warp instruction covers
     // four rows; the eight lanes of a row each own one 16-byte bf16 piece of either K half.
@@ -309,35 +334,13 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     }
     if (warp == 0) tmem_alloc(sbase + SM_TMEM, FV_TMEM_COLS);
     if (tid == 32) {
-        mbar_init(mbar, 1);
+        mbar_init(mbar_g, 1);
+        mbar_init(mbar_p, 1);
+        mbar_init(mbar_d, 1);
         *flag = 0;
     }
     // this tree's v rows are needed only after the first MMA group: pull them into L2 meanwhile
     if (tid >= 192 && tid - 192 < T) prefetch_l2_bulk(p.v + ((size_t)(base + tid - 192) * p.h_v + h) * FV_D, 256);
-    // Warm L2 for the unit that a CTA will pick up about one wave from now, so that HBM keeps
-    // streaming while the resident CTAs are busy computing: its state tile and its q/k/v rows.
-    {
-        const int u2 = blockIdx.x + p.prefetch_dist;
-        if (u2 < p.n_units && tid >= 64) {
-            const int b2 = u2 / p.h_v, h2 = u2 % p.h_v;
-            const int t2 = tid - 64;   // 0..191
-            if (t2 < 4) {
-                prefetch_l2_bulk(p.S0 + (size_t)u2 * FV_D * FV_D + (size_t)t2 * 4096, 16384);
-            } else if (t2 < 4 + FV_T) {
-                const int base2 = p.node_offsets[b2];
-                const int T2 = min(p.node_offsets[b2 + 1] - base2, FV_T);
-                const int i = t2 - 4;
-                if (i < T2) {
-                    const int hk2 = h2 / (p.h_v / p.h_qk);
-                    prefetch_l2_bulk(p.v + ((size_t)(base2 + i) * p.h_v + h2) * FV_D, 256);
-                    if (h2 % (p.h_v / p.h_qk) == 0) {   // one value head per key head fetches q and k
-                        prefetch_l2_bulk(p.k + ((size_t)(base2 + i) * p.h_qk + hk2) * FV_D, 256);
-                        prefetch_l2_bulk(p.q + ((size_t)(base2 + i) * p.h_qk + hk2) * FV_D, 256);
-                    }
-                }
-            }
-        }
-    }
     // (3) per-node tables: depth, root-path ids, g, beta (zeros beyond T)
     if (tid < FV_T) {
         int d = 0;
@@ -354,164 +357,65 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         *reinterpret_cast<uint4 *>(anc_s + tid * 16) = row;
         gab[tid] = make_float4(0.f, 0.f, be, gi);
     }
+    // fused commit, step 1: this tree's accepted path of the previous step (ids and their parents)
+    int *path_s = reinterpret_cast<int *>(smem + SM_PATH);
+    int *par_s = path_s + FV_MD;
+    float2 *ab_path = reinterpret_cast<float2 *>(smem + SM_PATH + 128);
+    int path_len = 0, pbase = 0, pT = 0;
+    bool path_shape_ok = true;
+    if constexpr (FUSED) {
+        const int pp0 = p.path_offsets[b];
+        path_len = p.path_offsets[b + 1] - pp0;   // uniform over the CTA; 0 leaves the state alone
+        if (path_len != 0) {
+            pbase = p.pnode_offsets[b];
+            pT = p.pnode_offsets[b + 1] - pbase;
+            path_shape_ok = path_len > 0 && path_len <= FV_MD && pT > 0 && pp0 >= 0;
+            if (path_shape_ok && tid >= 128 && tid - 128 < path_len) {
+                const int n = p.path[pp0 + tid - 128];
+                path_s[tid - 128] = n;
+                par_s[tid - 128] = (p.pparent && n >= 0 && n < pT) ? p.pparent[pbase + n] : -2;
+            }
+        }
+    }
     GDN_TRACE_MARK(1);
 
-    // (3') fused commit: replay Eq. 7 along the previous step's accepted path on the state tile while it
-    // sits in registers, write it back, and let everything below verify the new tree against it.
-    // Per row c (one value component): s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that
-    // share a row reduce k.s_c with three shuffles.
-    if constexpr (FUSED) {
-        int *path_s = reinterpret_cast<int *>(smem + SM_PATH);
-        int *par_s = path_s + FV_MD;
-        float2 *ab_path = reinterpret_cast<float2 *>(smem + SM_PATH + 128);
-        const int pp0 = p.path_offsets[b];
-        const int L = p.path_offsets[b + 1] - pp0;
-        if (L != 0) {   // uniform over the CTA; an empty path leaves the state alone
-            const int pbase = p.pnode_offsets[b];
-            const int pT = p.pnode_offsets[b + 1] - pbase;
-            const bool shape_ok = L > 0 && L <= FV_MD && pT > 0 && pp0 >= 0;
-            if (shape_ok && tid < L) {
-                const int n = p.path[pp0 + tid];
-                path_s[tid] = n;
-                par_s[tid] = (p.pparent && n >= 0 && n < pT) ? p.pparent[pbase + n] : -2;
-            }
-            __syncthreads();
-            if (tid == 0) {
-                int bad = !shape_ok;
-                for (int t = 0; !bad && t < L; ++t) {
-                    const int n = path_s[t];
-                    if (n < 0 || n >= pT) bad = 1;
-                    else if (p.pparent) bad = par_s[t] != (t ? path_s[t - 1] : -1);
-                    else if (t && n <= path_s[t - 1]) bad = 1;
-                }
-                if (bad) {
-                    report_status(p.status_dev, GDN_ERR_PATH);
-                    path_s[0] = -1;   // tells everybody to skip the replay: this state stays as it was
-                }
-            }
-            __syncthreads();
-            if (path_s[0] >= 0) {
-                // k and v rows of the path (bf16, 256 B each) and the per-step scalars
-                for (int idx = tid; idx < L * 32; idx += FV_THREADS) {
-                    const int t = idx >> 5, c16 = idx & 15;
-                    const size_t n = (size_t)pbase + path_s[t];
-                    if (idx & 16)
-                        cp_async_16(sbase + SM_PV + t * 256 + c16 * 16, p.pv + (n * p.h_v + h) * FV_D + c16 * 8, true);
-                    else
-                        cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + hk) * FV_D + c16 * 8, true);
-                }
-                if (tid < L) {
-                    const size_t n = (size_t)pbase + path_s[tid];
-                    ab_path[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + h])),
-                                               __bfloat162float(p.pbeta[n * p.h_v + h]));
-                }
-                cp_async_wait_all();   // also completes this thread's share of the k/q tile (harmless)
-                __syncthreads();
-                const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
-                const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
-#pragma unroll 1
-                for (int t = 0; t < L; ++t) {
-                    // this thread's sixteen key positions: 64*kh + 8*l8 + e
-                    float kf[16];
-#pragma unroll
-                    for (int kh = 0; kh < 2; ++kh) {
-                        const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
-                        const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            kf[kh * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
-                            kf[kh * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
-                        }
-                    }
-                    const float2 ab = ab_path[t];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int row = warp * 16 + i * 4 + r4;
-                        float xs16[16];
-#pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {
-                            xs16[q4 * 4 + 0] = x[i][q4].x; xs16[q4 * 4 + 1] = x[i][q4].y;
-                            xs16[q4 * 4 + 2] = x[i][q4].z; xs16[q4 * 4 + 3] = x[i][q4].w;
-                        }
-                        float dot = 0.f;
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) dot = fmaf(kf[e], xs16[e], dot);
-                        dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-                        dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-                        dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-                        const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
-                        const float w = ab.y * (vc - ab.x * dot);
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) xs16[e] = fmaf(kf[e], w, ab.x * xs16[e]);
-#pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4)
-                            x[i][q4] = make_float4(xs16[q4 * 4 + 0], xs16[q4 * 4 + 1], xs16[q4 * 4 + 2], xs16[q4 * 4 + 3]);
-                    }
-                }
-                // the committed state: the only state write of the step
-                float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float4 *dst = reinterpret_cast<float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
-#pragma unroll
-                    for (int kh = 0; kh < 2; ++kh) {
-                        dst[kh * 16 + l8 * 2 + 0] = x[i][kh * 2 + 0];
-                        dst[kh * 16 + l8 * 2 + 1] = x[i][kh * 2 + 1];
-                    }
-                }
-            }
-            __syncthreads();   // the path rows share their shared memory with the X / Y tables
-        }
-    }
-
-    // (4) fp32 -> bf16 hi + lo, written as the A operand
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int row = warp * 16 + i * 4 + r4;
-#pragma unroll
-        for (int kh = 0; kh < 2; ++kh) {
-            const float4 u = x[i][kh * 2 + 0], w = x[i][kh * 2 + 1];
-            const float f[8] = {u.x, u.y, u.z, u.w, w.x, w.y, w.z, w.w};
-            uint32_t hi[4], lo[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) split_pack_bf16(f[2 * e], f[2 * e + 1], hi[e], lo[e]);
-            const uint32_t off = sw128_offset(row, kh * 8 + l8);
-            *reinterpret_cast<uint4 *>(smem + SM_A_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4 *>(smem + SM_A_LO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        }
-    }
-    GDN_TRACE_MARK(2);
     cp_async_wait_all();
-    fence_proxy_async();   // generic-proxy writes of the operands become visible to the tensor core
+    fence_proxy_async();   // the k/q tile (cp.async) becomes visible to the tensor core
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    GDN_TRACE_MARK(3);
+    GDN_TRACE_MARK(2);
 
-    // (5) one thread issues the first MMA group: P = S0.[k;q]^T (hi then lo), Gram = [k;q].[k;q]^T
+    // (4) Everything that depends only on q, k, g, beta runs now, under the latency of the state loads:
+    // Gram = [k;q].[k;q]^T on the tensor core, G_i / a_i tables, then X and Y of Eq. 9.
     if (tid == 0) {
-        const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
         const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
         constexpr uint32_t id = idesc_bf16(128, 128);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-            umma_bf16(tmem, a_hi + adv, b_kq + adv, id, ks > 0);
-        }
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-            umma_bf16(tmem, a_lo + adv, b_kq + adv, id, 1);
-        }
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
             umma_bf16(tmem + 128, b_kq + adv, b_kq + adv, id, ks > 0);
         }
-        umma_commit(mbar);
+        umma_commit(mbar_g);
     }
-    // (6) meanwhile: G_i = sum of g along the root path (root first), a_i = exp(G_i)
+    if constexpr (FUSED) {
+        // step 2: the path must be a chain from a root inside the previous tree
+        if (tid == 160 && path_len != 0) {
+            int bad = !path_shape_ok;
+            for (int t = 0; !bad && t < path_len; ++t) {
+                const int n = path_s[t];
+                if (n < 0 || n >= pT) bad = 1;
+                else if (p.pparent) bad = par_s[t] != (t ? path_s[t - 1] : -1);
+                else if (t && n <= path_s[t - 1]) bad = 1;
+            }
+            if (bad) {
+                report_status(p.status_dev, GDN_ERR_PATH);
+                path_s[0] = -1;   // tells everybody to skip the replay: this state stays as it was
+            }
+        }
+    }
+    // G_i = sum of g along the root path (root first), a_i = exp(G_i)
     if (tid >= 64 && tid < 64 + FV_T) {
         const int i = tid - 64;
         const int d = depth_s[i];
@@ -520,46 +424,54 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         gab[i].x = G;
         gab[i].y = d ? expf(G) : 0.f;
     }
-    GDN_TRACE_MARK(4);
-
-    // (7) wait for the first MMA group: one thread polls the mbarrier (bounded: on expiry it flags the
-    // error and everybody falls through to the clean-up), the others sleep in the CTA barrier
-    if (tid == 0 && !mbar_wait_bounded(mbar, 0)) *flag = 1;
+    // one thread polls the mbarrier (bounded: on expiry it flags the error and everybody falls through to
+    // the clean-up), the others sleep in the CTA barrier
+    if (tid == 0 && !mbar_wait_bounded(mbar_g, 0)) *flag = 1;
     __syncthreads();
     tc_fence_after();
-    bool ok = *flag == 0;
-    GDN_TRACE_MARK(5);
-
-    if (ok) {
-        // (8) the operand tiles are free now: fetch the tree's v rows over them and move the
-        // k-columns of the Gram block out of tensor memory
-#pragma unroll
-        for (int it = 0; it < (FV_T * 16) / FV_THREADS; ++it) {
-            const int idx = it * FV_THREADS + tid;
-            const int i = idx >> 4, c16 = idx & 15;
-            const bool valid = i < T;
-            cp_async_16(sbase + SM_V + i * 256 + c16 * 16,
-                        p.v + ((size_t)(base + (valid ? i : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
+    GDN_TRACE_MARK(3);
+    warm_l2_state(0);
+    if constexpr (FUSED) {
+        // step 3: k and v rows of the path (bf16, 256 B each) and the per-step scalars
+        if (path_len > 0 && path_s[0] >= 0) {
+            for (int idx = tid; idx < path_len * 32; idx += FV_THREADS) {
+                const int t = idx >> 5, c16 = idx & 15;
+                const size_t n = (size_t)pbase + path_s[t];
+                if (idx & 16)
+                    cp_async_16(sbase + SM_PV + t * 256 + c16 * 16, p.pv + (n * p.h_v + h) * FV_D + c16 * 8, true);
+                else
+                    cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + hk) * FV_D + c16 * 8, true);
+            }
+            if (tid < path_len) {
+                const size_t n = (size_t)pbase + path_s[tid];
+                ab_path[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + h])),
+                                           __bfloat162float(p.pbeta[n * p.h_v + h]));
+            }
         }
+    }
+    if (*flag == 0) {
+        // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
         {
             const int row = (warp & 3) * 32 + lane;
             const int half = warp >> 2;   // TMEM columns 128 + 64*half .. : k_j for j = 32*half ..
             const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 128 + half * 64;
-            uint32_t ra[32], rb[32];
-            GDN_TMEM_LD32(taddr, ra);
-            GDN_TMEM_LD32(taddr + 32, rb);
-            tmem_wait_ld();
+#pragma unroll 1
+            for (int part = 0; part < 2; ++part) {
+                uint32_t ra[32];
+                GDN_TMEM_LD32(taddr + part * 32, ra);
+                tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int col = half * 32 + j;
-                gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[2 * j]);
-                gram[row * 64 + ((col + 16) ^ (row & 31))] = __uint_as_float(rb[2 * j]);
+                for (int j = 0; j < 16; ++j) {
+                    const int col = half * 32 + part * 16 + j;
+                    gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[2 * j]);
+                }
             }
         }
         tc_fence_before();
         __syncthreads();
-        GDN_TRACE_MARK(6);
-        // (9) X and Y of Eq. 9 for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
+        GDN_TRACE_MARK(4);
+        warm_l2_state(1);
+        // X and Y for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
         {
             float gdiff[4], gk[4], gq[4], bi[4];
             bool on[4], onx[4];
@@ -585,41 +497,164 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
                 xs[idx] = onx[u] ? bi[u] * dec * gk[u] : 0.f;
             }
         }
-        cp_async_wait_all();
-        __syncthreads();
-        GDN_TRACE_MARK(7);
+    }
+    cp_async_wait_all();
+    __syncthreads();   // X and Y complete; the Gram copy is dead and its area can take the state operand
+    GDN_TRACE_MARK(5);
 
-        // (10a) z^T = y^T (I + X_path)^-1 by back-substitution over the root path (column-oriented: once
-        // z_l is final, subtract z_l X(n_l, n_t) from every z_t, t < l).  Four threads per node, thread s of
-        // the quad owning path positions 4s..4s+3; the result is scattered into the dense bf16 hi/lo tiles
-        // Z[i][j] (zero off the root path).
+    // (3') fused commit: replay Eq. 7 along the previous step's accepted path on the state tile while it
+    // sits in registers, write it back, and let everything below verify the new tree against it.
+    // Per row c (one value component): s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that
+    // share a row reduce k.s_c with three shuffles.  The path's k/v rows were fetched above.
+    if constexpr (FUSED) {
+        if (path_len > 0 && path_s[0] >= 0) {
+            const int L = path_len;
+        const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
+        const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
+#pragma unroll 1
+        for (int t = 0; t < L; ++t) {
+            // this thread's sixteen key positions: 64*kh + 8*l8 + e
+            float kf[16];
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
+                const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    kf[kh * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
+                    kf[kh * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
+                }
+            }
+            const float2 ab = ab_path[t];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = warp * 16 + i * 4 + r4;
+                float xs16[16];
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    xs16[q4 * 4 + 0] = x[i][q4].x; xs16[q4 * 4 + 1] = x[i][q4].y;
+                    xs16[q4 * 4 + 2] = x[i][q4].z; xs16[q4 * 4 + 3] = x[i][q4].w;
+                }
+                float dot = 0.f;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) dot = fmaf(kf[e], xs16[e], dot);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
+                const float w = ab.y * (vc - ab.x * dot);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) xs16[e] = fmaf(kf[e], w, ab.x * xs16[e]);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    x[i][q4] = make_float4(xs16[q4 * 4 + 0], xs16[q4 * 4 + 1], xs16[q4 * 4 + 2], xs16[q4 * 4 + 3]);
+            }
+        }
+        // the committed state: the only state write of the step
+        float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 *dst = reinterpret_cast<float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                dst[kh * 16 + l8 * 2 + 0] = x[i][kh * 2 + 0];
+                dst[kh * 16 + l8 * 2 + 1] = x[i][kh * 2 + 1];
+            }
+        }
+        }
+        __syncthreads();   // the path rows sit where the state operand is about to be written
+    }
+
+    // (4) fp32 -> bf16 hi + lo, written as the A operand
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = warp * 16 + i * 4 + r4;
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh) {
+            const float4 u = x[i][kh * 2 + 0], w = x[i][kh * 2 + 1];
+            const float f[8] = {u.x, u.y, u.z, u.w, w.x, w.y, w.z, w.w};
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) split_pack_bf16(f[2 * e], f[2 * e + 1], hi[e], lo[e]);
+            const uint32_t off = sw128_offset(row, kh * 8 + l8);
+            *reinterpret_cast<uint4 *>(smem + SM_A_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4 *>(smem + SM_A_LO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+    }
+    fence_proxy_async();   // generic-proxy writes of the operand become visible to the tensor core
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    GDN_TRACE_MARK(6);
+    warm_l2_state(2);
+
+    // (5) P = S0.[k;q]^T (hi then lo) on the tensor core; meanwhile the back-substitution below
+    if (tid == 0) {
+        const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
+        const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
+        constexpr uint32_t id = idesc_bf16(128, 128);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+            umma_bf16(tmem, a_hi + adv, b_kq + adv, id, ks > 0);
+        }
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+            umma_bf16(tmem, a_lo + adv, b_kq + adv, id, 1);
+        }
+        umma_commit(mbar_p);
+    }
+    // (6) z^T = y^T (I + X_path)^-1 by back-substitution over the root path (column-oriented: once z_l is
+    // final, subtract z_l X(n_l, n_t) from every z_t, t < l).  Four threads per node, thread sq of the quad
+    // owning path positions 4 sq .. 4 sq + 3; z stays in registers until the k/q tile can be overwritten.
+    const int zi = tid >> 2, sq = tid & 3;
+        const int d = depth_s[zi];
+        const int dmax = __reduce_max_sync(0xffffffffu, d);
+        const uint4 row = *reinterpret_cast<const uint4 *>(anc_s + zi * 16);
+        const uint32_t idw[4] = {row.x, row.y, row.z, row.w};
+        const float4 y4 = *reinterpret_cast<const float4 *>(ys + zi * FV_MD + sq * 4);
+        float z[4] = {y4.x, y4.y, y4.z, y4.w};
+#pragma unroll
+        for (int l = FV_MD - 1; l >= 1; --l) {
+            if (l < dmax) {   // warp-uniform
+                const float zl = __shfl_sync(0xffffffffu, z[l & 3], (lane & ~3) | (l >> 2));
+                if (l < d && sq * 4 < l) {
+                    const int nl = (int)((idw[l >> 2] >> ((l & 3) * 8)) & 0xFFu);
+                    const float4 x4 = *reinterpret_cast<const float4 *>(xs + nl * FV_MD + sq * 4);
+                    const float xv[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (sq * 4 + e < l) z[e] = fmaf(-zl, xv[e], z[e]);
+                }
+            }
+        }
+    GDN_TRACE_MARK(7);
+    if (tid == 0 && !mbar_wait_bounded(mbar_p, 0)) *flag = 1;
+    __syncthreads();
+    tc_fence_after();
+    bool ok = *flag == 0;
+    GDN_TRACE_MARK(8);
+    warm_l2_state(3);
+
+    if (ok) {
+        // (7) both operand tiles are dead now: the tree's v rows go over the state operand, and z is
+        // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path) over the k/q tile
+#pragma unroll
+        for (int it = 0; it < (FV_T * 16) / FV_THREADS; ++it) {
+            const int idx = it * FV_THREADS + tid;
+            const int i = idx >> 4, c16 = idx & 15;
+            const bool valid = i < T;
+            cp_async_16(sbase + SM_V + i * 256 + c16 * 16,
+                        p.v + ((size_t)(base + (valid ? i : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
+        }
         {
-            const int i = tid >> 2, sq = tid & 3;
-            const int d = depth_s[i];
-            const int dmax = __reduce_max_sync(0xffffffffu, d);
+            const int i = zi;
             const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
             *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, 2 * sq)) = zero4;
             *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, 2 * sq + 1)) = zero4;
             *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, 2 * sq)) = zero4;
             *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, 2 * sq + 1)) = zero4;
-            const uint4 row = *reinterpret_cast<const uint4 *>(anc_s + i * 16);
-            const uint32_t idw[4] = {row.x, row.y, row.z, row.w};
-            const float4 y4 = *reinterpret_cast<const float4 *>(ys + i * FV_MD + sq * 4);
-            float z[4] = {y4.x, y4.y, y4.z, y4.w};
-#pragma unroll
-            for (int l = FV_MD - 1; l >= 1; --l) {
-                if (l < dmax) {   // warp-uniform
-                    const float zl = __shfl_sync(0xffffffffu, z[l & 3], (lane & ~3) | (l >> 2));
-                    if (l < d && sq * 4 < l) {
-                        const int nl = (int)((idw[l >> 2] >> ((l & 3) * 8)) & 0xFFu);
-                        const float4 x4 = *reinterpret_cast<const float4 *>(xs + nl * FV_MD + sq * 4);
-                        const float xv[4] = {x4.x, x4.y, x4.z, x4.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            if (sq * 4 + e < l) z[e] = fmaf(-zl, xv[e], z[e]);
-                    }
-                }
-            }
             __syncwarp();   // the quad's zero fill precedes the scattered stores below
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -634,7 +669,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
                 }
             }
         }
-        // (10b) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
+        cp_async_wait_all();
+        __syncthreads();
+        GDN_TRACE_MARK(9);
+
+        // (8) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
         // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
         {
             const int c = (warp & 3) * 32 + lane;
@@ -673,9 +712,10 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        GDN_TRACE_MARK(8);
+        GDN_TRACE_MARK(10);
+        warm_l2_rows();
 
-        // (11) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
+        // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
         if (tid == 0) {
             constexpr uint32_t id2 = idesc_bf16(128, 64);
             const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
@@ -687,15 +727,15 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
                     umma_bf16(tmem + 128, a2[combo & 1] + (uint64_t)(ks * 2), b2[combo >> 1] + (uint64_t)(ks * 2), id2,
                               (combo | ks) != 0);
             }
-            umma_commit(mbar);
+            umma_commit(mbar_d);
         }
-        if (tid == 0 && !mbar_wait_bounded(mbar, 1)) *flag = 1;
+        if (tid == 0 && !mbar_wait_bounded(mbar_d, 0)) *flag = 1;
         __syncthreads();
         tc_fence_after();
         ok = *flag == 0;
-        GDN_TRACE_MARK(9);
+        GDN_TRACE_MARK(11);
 
-        // (12) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i]), staged through shared memory (over the
+        // (10) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i]), staged through shared memory (over the
         // dead R^T tiles) so that global memory sees 16-byte stores of whole rows
         if (ok) {
             const int c = (warp & 3) * 32 + lane;
@@ -732,7 +772,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     }
     if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
 
-    GDN_TRACE_MARK(10);
+    GDN_TRACE_MARK(12);
 #ifdef GDN_TRACE
     if (threadIdx.x == 0 && g_trace_buf) {
         unsigned long long gt;
