@@ -197,7 +197,7 @@ extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const 
     const gdn_shape_t &s = *shape;
     if (s.n_seq == 0) return GDN_OK;
     if (!S || !node_offsets_prev || !path_offsets || !status_dev) return GDN_ERR_NULL;
-    if (!verify_sm100_supported(s) || s.total_nodes == 0) {
+    if (!verify_sm100_single_group(s) || s.total_nodes == 0) {
         // general shapes: the two kernels back to back on the stream (the shape's node counts are
         // not used by commit, so the new tree's shape serves for the previous tree as well)
         rc = gdn_tree_commit(shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,

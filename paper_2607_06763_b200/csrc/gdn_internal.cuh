@@ -16,10 +16,22 @@ namespace gdn {
 //   anc      uint16[N][max_depth]          local ids of the root path of n, root first, n itself last
 //   anc8     uint8 [N][16]                 the same list as bytes (filled when max_depth <= 16 and the
 //                                          tree has <= 256 nodes; unused entries are 0xFF)
+// Grouped verification of trees with more than 64 nodes (filled when max_depth <= 16 and the tree has at
+// most GDN_GROUPED_MAX_NODES nodes).  "Position" = index in the depth-first pre-order of the tree (children
+// by increasing id).  The positions are cut into groups of GDN_GROUP_NODES; a group together with the proper
+// ancestors of its first node (at most 15, all outside the group) is closed under "ancestor of", so it can
+// be verified as a tree of at most 63 nodes: virtual index = depth-1 for those ancestors, n_prefix + offset
+// in the group for the group's own nodes.
+//   dfs_node  uint16[N]                    node id at position r
+//   dfs_depth uint8 [N]                    depth of that node
+//   dfs_anc8  uint8 [N][16]                its root path in virtual indices of its group (0xFF = unused)
 //   utilde   float [N][h_v][d_v]           solve result u~ (Eq. 10 with the W S0 term folded in)
 struct WorkspaceLayout {
-    size_t tree_ok, depth, anc, anc8, utilde, total;
+    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, utilde, total;
 };
+
+constexpr int GDN_GROUP_NODES = 48;           // own nodes of a group
+constexpr int GDN_GROUPED_MAX_NODES = 1024;   // largest tree the grouped tensor-core path takes
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -32,6 +44,9 @@ inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
     w.depth = off;    off = align256(off + N);
     w.anc = off;      off = align256(off + sizeof(uint16_t) * N * (size_t)s.max_depth);
     w.anc8 = off;     off = align256(off + 16 * N);
+    w.dfs_node = off; off = align256(off + 2 * N);
+    w.dfs_depth = off; off = align256(off + N);
+    w.dfs_anc8 = off; off = align256(off + 16 * N);
     w.utilde = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
     w.total = off;
     return w;
@@ -42,6 +57,8 @@ struct PlanPtrs {
     uint8_t *depth;
     uint16_t *anc;
     uint8_t *anc8;
+    uint16_t *dfs_node;
+    uint8_t *dfs_depth, *dfs_anc8;
     float *utilde;
 };
 
@@ -50,7 +67,8 @@ inline PlanPtrs plan_ptrs(void *workspace, const WorkspaceLayout &w)
     char *b = static_cast<char *>(workspace);
     return {reinterpret_cast<int32_t *>(b + w.tree_ok), reinterpret_cast<uint8_t *>(b + w.depth),
             reinterpret_cast<uint16_t *>(b + w.anc), reinterpret_cast<uint8_t *>(b + w.anc8),
-            reinterpret_cast<float *>(b + w.utilde)};
+            reinterpret_cast<uint16_t *>(b + w.dfs_node), reinterpret_cast<uint8_t *>(b + w.dfs_depth),
+            reinterpret_cast<uint8_t *>(b + w.dfs_anc8), reinterpret_cast<float *>(b + w.utilde)};
 }
 
 // Host launchers (each returns the cudaError_t of its launch).
@@ -64,6 +82,7 @@ cudaError_t launch_verify_generic(const gdn_shape_t &s, const float *S0, const v
 
 // Tensor-core fast path (d_k = d_v = 128, bf16 inputs, trees <= 64 nodes, root paths <= 16 nodes).
 bool verify_sm100_supported(const gdn_shape_t &s);
+bool verify_sm100_single_group(const gdn_shape_t &s);   // every tree fits one CTA (<= 64 nodes): fusable with commit
 cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
                                 const void *v, const void *g, const void *beta,
                                 const int32_t *node_offsets, void *o, const PlanPtrs &plan,

@@ -2,6 +2,9 @@
 // the list of nodes on its root path.  The ancestor sets of Section 3.4.2 are kept as explicit
 // root-first lists rather than bitmasks: with at most max_depth (16 in the paper) nodes per path a
 // list is smaller than a T-bit mask for T > 256 and lets the solve visit only real ancestors.
+// Trees of more than 64 nodes additionally get a depth-first numbering cut into groups that are
+// closed under "ancestor of" once the first node's root path is added (see gdn_internal.cuh); the
+// tensor-core verify kernel takes one such group at a time.
 #include "gdn_internal.cuh"
 
 namespace gdn {
@@ -14,8 +17,13 @@ __global__ void __launch_bounds__(PLAN_THREADS)
 plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
             const int32_t *__restrict__ parent, const int32_t *__restrict__ node_offsets,
             int32_t *__restrict__ tree_ok, uint8_t *__restrict__ depth, uint16_t *__restrict__ anc,
-            uint8_t *__restrict__ anc8, int32_t *status_dev)
+            uint8_t *__restrict__ anc8, uint16_t *__restrict__ dfs_node, uint8_t *__restrict__ dfs_depth,
+            uint8_t *__restrict__ dfs_anc8, int32_t *status_dev)
 {
+    __shared__ int size_s[GDN_GROUPED_MAX_NODES];        // subtree sizes
+    __shared__ uint16_t left_s[GDN_GROUPED_MAX_NODES];   // nodes in the subtrees of earlier siblings
+    __shared__ uint16_t pos_s[GDN_GROUPED_MAX_NODES];    // pre-order position of node i
+    __shared__ uint8_t dfirst_s[GDN_GROUPED_MAX_NODES / GDN_GROUP_NODES + 1];   // depth of each group's first node
     // parent[] of this tree, staged once so that the root-path walks below run out of shared memory
     __shared__ int32_t par_s[GDN_MAX_TREE_NODES];
     const int b = blockIdx.x;
@@ -31,7 +39,11 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
         }
         return;
     }
-    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) par_s[i] = parent[lo + i];
+    const bool grouped = max_depth <= 16 && T > 64 && T <= GDN_GROUPED_MAX_NODES;
+    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
+        par_s[i] = parent[lo + i];
+        if (grouped) size_s[i] = 1;
+    }
     __syncthreads();
     int err = 0;
     for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
@@ -58,6 +70,7 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
             else if ((t >> 2) == 2) w2 = (w2 & keep) | put;
             else if ((t >> 2) == 3) w3 = (w3 & keep) | put;
             cur = par_s[cur];
+            if (grouped && cur >= 0) atomicAdd(&size_s[cur], 1);   // node i lies in the subtree of each proper ancestor
         }
         if (max_depth <= 16 && T <= 256)
             *reinterpret_cast<uint4 *>(anc8 + (size_t)(lo + i) * 16) = make_uint4(w0, w1, w2, w3);
@@ -65,6 +78,46 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     const int any_err = __syncthreads_or(err != 0);
     if (err) report_status(status_dev, err);
     if (threadIdx.x == 0) tree_ok[b] = any_err ? 0 : 1;
+    if (any_err || !grouped) return;
+
+    // Pre-order position = (#proper ancestors) + sum over the root path of the sizes of the subtrees
+    // hanging off earlier siblings (roots count as siblings of one another; siblings by increasing id).
+    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
+        const int p = par_s[i];
+        int acc = 0;
+        for (int j = p + 1; j < i; ++j)
+            if (par_s[j] == p) acc += size_s[j];
+        left_s[i] = (uint16_t)acc;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
+        const uint16_t *row = anc + (size_t)(lo + i) * max_depth;
+        const int d = depth[lo + i];
+        int pos = d - 1;
+        for (int t = 0; t < d; ++t) pos += left_s[row[t]];
+        pos_s[i] = (uint16_t)pos;
+        dfs_node[lo + pos] = (uint16_t)i;
+        dfs_depth[lo + pos] = (uint8_t)d;
+        if (pos % GDN_GROUP_NODES == 0) dfirst_s[pos / GDN_GROUP_NODES] = (uint8_t)d;
+    }
+    __syncthreads();
+    // Root path of every node in the virtual indices of its group: an ancestor before the group's first
+    // position is an ancestor of the group's first node and gets index depth-1; one inside the group gets
+    // n_prefix + its offset in the group, n_prefix = depth(first node) - 1.
+    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
+        const uint16_t *row = anc + (size_t)(lo + i) * max_depth;
+        const int d = depth[lo + i];
+        const int pos = pos_s[i];
+        const int g0 = pos / GDN_GROUP_NODES * GDN_GROUP_NODES;
+        const int n_prefix = dfirst_s[pos / GDN_GROUP_NODES] - 1;
+        uint32_t w[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+        for (int t = 0; t < d; ++t) {
+            const int pa = pos_s[row[t]];
+            const uint32_t v = pa < g0 ? (uint32_t)t : (uint32_t)(n_prefix + pa - g0);
+            w[t >> 2] = (w[t >> 2] & ~(0xFFu << ((t & 3) * 8))) | (v << ((t & 3) * 8));
+        }
+        *reinterpret_cast<uint4 *>(dfs_anc8 + (size_t)(lo + pos) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
 }
 
 }  // namespace
@@ -75,7 +128,7 @@ cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32
     if (s.n_seq == 0) return cudaSuccess;
     plan_kernel<<<s.n_seq, PLAN_THREADS, 0, stream>>>(s.n_seq, s.total_nodes, s.max_tree_nodes,
                                                       s.max_depth, parent, node_offsets, plan.tree_ok,
-                                                      plan.depth, plan.anc, plan.anc8, status_dev);
+                                                      plan.depth, plan.anc, plan.anc8, plan.dfs_node, plan.dfs_depth, plan.dfs_anc8, status_dev);
     return cudaGetLastError();
 }
 

@@ -1,5 +1,5 @@
-// Tree-verify fast path for sm_100a: d_k = d_v = 128, bf16 inputs, trees of at most 64 nodes,
-// root paths of at most 16 nodes.  It evaluates the triangular form of Section 3.4.1 (Eq. 9-11)
+// Tree-verify fast path for sm_100a: d_k = d_v = 128, bf16 inputs, root paths of at most 16 nodes,
+// trees of at most 64 nodes per CTA (larger trees are cut into ancestor-closed groups, one CTA each).  It evaluates the triangular form of Section 3.4.1 (Eq. 9-11)
 // restricted to real ancestors, with the W S0 term folded into the right-hand side as in
 // Section 3.4.2, and turns all of the per-component work into two dense contractions on the
 // 5th-generation tensor cores (tcgen05.mma, bf16 operands, fp32 accumulators in tensor memory):
@@ -52,7 +52,8 @@ constexpr int SM_DEPTH = SM_GAB + 1024;          // u8 [64] (0 beyond T)
 constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit: int [16] node ids, int [16] parents, float2 [16] (alpha, beta)
 constexpr int SM_PK = 32768;                     // fused commit: k rows of the accepted path, bf16 [16][128], parked in the
 constexpr int SM_PV = 36864;                     // state-operand area until the replay is over; v rows likewise
-constexpr int SM_MBAR = SM_PATH + 256;           // 3 x u64: Gram done, P done, D done
+constexpr int SM_VNODE = SM_PATH + 256;          // grouped mode: u16 [64] node id of virtual index u
+constexpr int SM_MBAR = SM_VNODE + 128;          // 3 x u64: Gram done, P done, D done
 constexpr int SM_TMEM = SM_MBAR + 24;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
 constexpr int SM_BYTES = SM_FLAG + 4;
@@ -88,6 +89,10 @@ struct VerifyFastParams {
     const uint8_t *depth;
     const uint8_t *anc8;
     int32_t *status_dev;
+    // grouped verification of trees with more than 64 nodes (only read by the GROUPED instantiation)
+    int groups_per_tree, anc_stride;                   // CTAs per (tree, head); entries per row of anc16
+    const uint16_t *anc16, *dfs_node;
+    const uint8_t *dfs_depth, *dfs_anc8;
     // fused commit of the previous step's accepted paths (only read by the FUSED instantiation)
     float *S_rw;                                       // same tensor as S0, written in place
     const __nv_bfloat16 *pk, *pv, *pg, *pbeta;         // the previous tree's k, v, g, beta
@@ -244,15 +249,30 @@ __device__ __forceinline__ void split_bf16(float x, float &hi, float &lo)
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <typename TOut, bool FUSED>
+template <typename TOut, bool FUSED, bool GROUPED>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const VerifyFastParams p)
 {
     extern __shared__ uint8_t fv_smem_raw[];
-    const int b = blockIdx.x / p.h_v, h = blockIdx.x % p.h_v;
+    static_assert(!(FUSED && GROUPED), "the fused commit needs one CTA per state tile");
+    // GROUPED: the CTA takes group `grp` of tree b (see gdn_internal.cuh): T is then the size of the
+    // virtual tree (n_prefix ancestors of the group's first node + the group's own nodes), and virtual
+    // index u maps to node vnode[u].  Trees of at most 64 nodes are their own single group, identity map.
+    const int h = blockIdx.x % p.h_v;
+    const int b = GROUPED ? (blockIdx.x / p.h_v) / p.groups_per_tree : blockIdx.x / p.h_v;
+    const int grp = GROUPED ? (blockIdx.x / p.h_v) % p.groups_per_tree : 0;
     if (!p.tree_ok[b]) return;
     const int base = p.node_offsets[b];
-    const int T = p.node_offsets[b + 1] - base;
-    if (T <= 0 || T > FV_T) return;   // larger trees never reach this kernel (host-side dispatch)
+    const int T_tree = p.node_offsets[b + 1] - base;
+    if (T_tree <= 0) return;
+    if (!GROUPED && T_tree > FV_T) return;   // larger trees never reach that instantiation (host-side dispatch)
+    const bool ident = !GROUPED || T_tree <= FV_T;
+    const int g0 = grp * GDN_GROUP_NODES;
+    if (GROUPED && (ident ? grp > 0 : g0 >= T_tree)) return;   // no such group in this tree
+    int n_prefix = 0, T = T_tree;
+    if (GROUPED && !ident) {
+        n_prefix = p.dfs_depth[base + g0] - 1;
+        T = n_prefix + min(GDN_GROUP_NODES, T_tree - g0);
+    }
 
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fv_smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
@@ -269,6 +289,23 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hk = h / (p.h_v / p.h_qk);
+    uint16_t *vnode_s = reinterpret_cast<uint16_t *>(smem + SM_VNODE);
+    if constexpr (GROUPED) {
+        if (tid < FV_T) {
+            int node = tid;
+            if (!ident && tid < T) {
+                if (tid < n_prefix) {
+                    const int first = p.dfs_node[base + g0];
+                    node = p.anc16[(size_t)(base + first) * p.anc_stride + tid];
+                } else {
+                    node = p.dfs_node[base + g0 + tid - n_prefix];
+                }
+            }
+            vnode_s[tid] = (uint16_t)node;
+        }
+        __syncthreads();
+    }
+    auto node_of = [&](int u) -> int { return GROUPED ? (int)vnode_s[u] : u; };
     GDN_TRACE_MARK(0);
 #ifdef GDN_TRACE
     if (threadIdx.x == 0 && g_trace_buf) {
@@ -286,11 +323,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     // CTAs compute, instead of all demand loads of a wave hitting it at once.
     const int u_next = blockIdx.x + p.prefetch_dist;
     auto warm_l2_state = [&](int slice) {   // slice 0..3 of the next unit's 64 KB state tile
-        if (tid == 96 && u_next < p.n_units)
+        if (!GROUPED && tid == 96 && u_next < p.n_units)
             prefetch_l2_bulk(p.S0 + (size_t)u_next * FV_D * FV_D + (size_t)slice * 4096, 16384);
     };
     auto warm_l2_rows = [&]() {             // the next unit's q/k/v rows
-        if (u_next < p.n_units && tid >= 128 && tid < 128 + FV_T) {
+        if (!GROUPED && u_next < p.n_units && tid >= 128 && tid < 128 + FV_T) {
             const int b2 = u_next / p.h_v, h2 = u_next % p.h_v;
             const int base2 = p.node_offsets[b2];
             const int T2 = min(p.node_offsets[b2 + 1] - base2, FV_T);
@@ -329,7 +366,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         const int r = idx >> 4, c16 = idx & 15;
         const int node = r >> 1;
         const bool valid = node < T;
-        const __nv_bfloat16 *src = ((r & 1) ? p.q : p.k) + ((size_t)(base + (valid ? node : 0)) * p.h_qk + hk) * FV_D + c16 * 8;
+        const __nv_bfloat16 *src = ((r & 1) ? p.q : p.k) + ((size_t)(base + (valid ? node_of(node) : 0)) * p.h_qk + hk) * FV_D + c16 * 8;
         cp_async_16(sbase + SM_B_KQ + sw128_offset(r, c16), src, valid);
     }
     if (warp == 0) tmem_alloc(sbase + SM_TMEM, FV_TMEM_COLS);
@@ -347,9 +384,25 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         uint4 row = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
         float gi = 0.f, be = 0.f;
         if (tid < T) {
-            const int n = base + tid;
-            d = p.depth[n];
-            row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)n * 16));
+            const int n = base + node_of(tid);
+            if (ident) {
+                d = p.depth[n];
+                row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)n * 16));
+            } else if (tid < n_prefix) {   // an ancestor of the group's first node: its path is 0..tid
+                d = tid + 1;
+                const uint32_t all[4] = {0x03020100u, 0x07060504u, 0x0B0A0908u, 0x0F0E0D0Cu};
+                uint32_t w[4];
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int keep = d - 4 * q4;   // bytes of this word that are on the path
+                    w[q4] = keep >= 4 ? all[q4] : keep <= 0 ? 0xFFFFFFFFu : (all[q4] | (0xFFFFFFFFu << (8 * keep)));
+                }
+                row = make_uint4(w[0], w[1], w[2], w[3]);
+            } else {
+                const int r = base + g0 + tid - n_prefix;
+                d = p.dfs_depth[r];
+                row = __ldg(reinterpret_cast<const uint4 *>(p.dfs_anc8 + (size_t)r * 16));
+            }
             gi = __bfloat162float(p.g[(size_t)n * p.h_v + h]);
             be = __bfloat162float(p.beta[(size_t)n * p.h_v + h]);
         }
@@ -646,7 +699,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             const int i = idx >> 4, c16 = idx & 15;
             const bool valid = i < T;
             cp_async_16(sbase + SM_V + i * 256 + c16 * 16,
-                        p.v + ((size_t)(base + (valid ? i : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
+                        p.v + ((size_t)(base + (valid ? node_of(i) : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
         }
         {
             const int i = zi;
@@ -766,7 +819,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
             for (int idx = tid; idx < T * ROW_CHUNKS; idx += FV_THREADS) {
                 const int i = idx / ROW_CHUNKS, ck = idx % ROW_CHUNKS;
                 const uint4 val = *reinterpret_cast<const uint4 *>(smem + SM_RT_HI + (size_t)i * FV_D * sizeof(TOut) + ck * 16);
-                *reinterpret_cast<uint4 *>(o + (((size_t)(base + i) * p.h_v + h) * FV_D) * sizeof(TOut) + ck * 16) = val;
+                if (i >= n_prefix)   // the ancestors in front of a group belong to other groups' outputs
+                    *reinterpret_cast<uint4 *>(o + (((size_t)(base + node_of(i)) * p.h_v + h) * FV_D) * sizeof(TOut) + ck * 16) = val;
             }
         }
     }
@@ -785,13 +839,14 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
 }
 
-template <typename TOut, bool FUSED>
+template <typename TOut, bool FUSED, bool GROUPED>
 cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, cudaStream_t stream)
 {
-    cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         SM_ALLOC);
+    cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut, FUSED, GROUPED>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
     if (e != cudaSuccess) return e;
-    verify_sm100_kernel<TOut, FUSED><<<s.n_seq * s.h_v, FV_THREADS, SM_ALLOC, stream>>>(p);
+    const int grid = s.n_seq * s.h_v * (GROUPED ? p.groups_per_tree : 1);
+    verify_sm100_kernel<TOut, FUSED, GROUPED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -809,6 +864,9 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     p.beta = static_cast<const __nv_bfloat16 *>(beta);
     p.node_offsets = node_offsets; p.o = o;
     p.tree_ok = plan.tree_ok; p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
+    p.groups_per_tree = (s.max_tree_nodes + GDN_GROUP_NODES - 1) / GDN_GROUP_NODES;
+    p.anc_stride = s.max_depth;
+    p.anc16 = plan.anc; p.dfs_node = plan.dfs_node; p.dfs_depth = plan.dfs_depth; p.dfs_anc8 = plan.dfs_anc8;
     return p;
 }
 
@@ -816,9 +874,11 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
 
 bool verify_sm100_supported(const gdn_shape_t &s)
 {
-    return s.d_k == FV_D && s.d_v == FV_D && s.in_dtype == GDN_BF16 && s.max_tree_nodes <= FV_T &&
+    return s.d_k == FV_D && s.d_v == FV_D && s.in_dtype == GDN_BF16 && s.max_tree_nodes <= GDN_GROUPED_MAX_NODES &&
            s.max_depth <= FV_MD;
 }
+
+bool verify_sm100_single_group(const gdn_shape_t &s) { return verify_sm100_supported(s) && s.max_tree_nodes <= FV_T; }
 
 cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
                                 const void *v, const void *g, const void *beta,
@@ -827,8 +887,12 @@ cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const voi
 {
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
     const VerifyFastParams p = make_params(s, S0, q, k, v, g, beta, node_offsets, o, plan, status_dev);
-    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false>(s, p, stream);
-    return launch_fast_typed<float, false>(s, p, stream);
+    if (s.max_tree_nodes > FV_T) {
+        if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false, true>(s, p, stream);
+        return launch_fast_typed<float, false, true>(s, p, stream);
+    }
+    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false, false>(s, p, stream);
+    return launch_fast_typed<float, false, false>(s, p, stream);
 }
 
 cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const void *k_prev, const void *v_prev,
@@ -844,8 +908,8 @@ cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const voi
     p.pk = static_cast<const __nv_bfloat16 *>(k_prev); p.pv = static_cast<const __nv_bfloat16 *>(v_prev);
     p.pg = static_cast<const __nv_bfloat16 *>(g_prev); p.pbeta = static_cast<const __nv_bfloat16 *>(beta_prev);
     p.pparent = parent_prev; p.pnode_offsets = node_offsets_prev; p.path = path; p.path_offsets = path_offsets;
-    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, true>(s, p, stream);
-    return launch_fast_typed<float, true>(s, p, stream);
+    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, true, false>(s, p, stream);
+    return launch_fast_typed<float, true, false>(s, p, stream);
 }
 
 #ifdef GDN_TRACE

@@ -331,3 +331,29 @@ def test_fused_commit_verify_full_stack_sampled(tl):
     o_ref = orc.verify(S_ref, nsub.f64("q"), nsub.f64("k"), nsub.f64("v"), nsub.f64("g"), nsub.f64("beta"),
                        nsub.parent, nsub.node_offsets, nsub.scale)
     tl.assert_close_per_head(dn.o_host()[nodes], o_ref, nsub.node_offsets, "fused 1x48 o", bf16_out=True)
+
+
+# ------------------------------------------------------------------ trees larger than one CTA tile (grouped path)
+@pytest.mark.parametrize("case", ["t65", "t1000_bestfirst", "forest200", "deep_narrow", "mixed_batch"])
+def test_large_trees_grouped_tensor_core_path(tl, case):
+    rng = np.random.default_rng(77)
+    if case == "t65":
+        trees = [synth.tree_geo(rng, 65)]
+    elif case == "t1000_bestfirst":
+        trees = [synth.tree_bestfirst(rng, 1000, width=8)]
+    elif case == "forest200":
+        a, b2 = synth.tree_geo(rng, 120), synth.tree_geo(rng, 80)
+        trees = [np.concatenate([a, np.where(b2 < 0, -1, b2 + 120)]).astype(np.int32)]
+    elif case == "deep_narrow":   # many chains of 16 hanging off one root: every group starts deep in the tree
+        par = [-1]
+        for c in range(20):
+            prev = 0
+            for _ in range(15):
+                par.append(prev)
+                prev = len(par) - 1
+        trees = [np.asarray(par, np.int32)]
+    else:
+        trees = [synth.tree_geo(rng, 30), synth.tree_geo(rng, 257), synth.tree_chain(16), synth.tree_geo(rng, 64),
+                 synth.tree_geo(rng, 129)]
+    w = synth.random_case(500 + len(case), trees, 2, 4, 128, 128, synth.BF16, synth.F32, name=case)
+    _check_full(tl, w, case)
