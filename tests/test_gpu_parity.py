@@ -357,3 +357,13 @@ def test_large_trees_grouped_tensor_core_path(tl, case):
                  synth.tree_geo(rng, 129)]
     w = synth.random_case(500 + len(case), trees, 2, 4, 128, 128, synth.BF16, synth.F32, name=case)
     _check_full(tl, w, case)
+
+
+def test_fused_commit_with_extreme_decay_takes_the_plain_replay(tl):
+    """A path whose cumulative decay underflows (g very negative) must still commit correctly: S -> k w terms only."""
+    trees = [synth.tree_chain(12), synth.tree_chain(12)]
+    paths = [np.arange(12, dtype=np.int32), np.arange(5, dtype=np.int32)]
+    prev = synth.random_case(41, trees, 1, 2, 128, 128, synth.BF16, synth.F32, paths=paths, name="prev")
+    prev.g = synth.store(np.full(prev.g.shape, -9.0, np.float32), synth.BF16)   # alpha = e^-9 per step, A_12 ~ 1e-47
+    new = synth.random_case(42, [synth.tree_star(5), synth.tree_star(5)], 1, 2, 128, 128, synth.BF16, synth.F32)
+    _fused_case(tl, prev, new, "fused extreme decay")
