@@ -49,10 +49,10 @@ constexpr int SM_Y = SM_X + 4096;                // fp32 [64][16]  Y(i, t-th pat
 constexpr int SM_ANC = SM_Y + 4096;              // u8   [64][16]  root-path node ids (0xFF = unused)
 constexpr int SM_GAB = SM_ANC + 1024;            // float4 [64]: (G_i = log a_i, a_i, beta_i, g_i)
 constexpr int SM_DEPTH = SM_GAB + 1024;          // u8 [64] (0 beyond T)
-constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit: int [16] node ids, int [16] parents, float2 [16] (A_t, beta_t), float [16] alpha_t
+constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit: int [16] node ids, int [16] parents, float2 [16] (alpha, beta)
 constexpr int SM_PK = 32768;                     // fused commit: k rows of the accepted path, bf16 [16][128], parked in the
 constexpr int SM_PV = 36864;                     // state-operand area until the replay is over; v rows likewise
-constexpr int SM_VNODE = SM_PATH + 384;          // grouped mode: u16 [64] node id of virtual index u
+constexpr int SM_VNODE = SM_PATH + 256;          // grouped mode: u16 [64] node id of virtual index u
 constexpr int SM_MBAR = SM_VNODE + 128;          // 3 x u64: Gram done, P done, D done
 constexpr int SM_TMEM = SM_MBAR + 24;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
@@ -414,7 +414,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     int *path_s = reinterpret_cast<int *>(smem + SM_PATH);
     int *par_s = path_s + FV_MD;
     float2 *ab_path = reinterpret_cast<float2 *>(smem + SM_PATH + 128);
-    float *alpha_path = reinterpret_cast<float *>(smem + SM_PATH + 256);
     int path_len = 0, pbase = 0, pT = 0;
     bool path_shape_ok = true;
     if constexpr (FUSED) {
@@ -496,13 +495,10 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
                 else
                     cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + hk) * FV_D + c16 * 8, true);
             }
-            if (tid < path_len) {   // (A_t, beta_t): cumulative decay up to and including step t
-                float gsum = 0.f;
-                for (int t = 0; t <= tid; ++t)
-                    gsum += __bfloat162float(p.pg[((size_t)pbase + path_s[t]) * p.h_v + h]);
+            if (tid < path_len) {
                 const size_t n = (size_t)pbase + path_s[tid];
-                ab_path[tid] = make_float2(expf(gsum), __bfloat162float(p.pbeta[n * p.h_v + h]));
-                alpha_path[tid] = expf(__bfloat162float(p.pg[n * p.h_v + h]));
+                ab_path[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + h])),
+                                           __bfloat162float(p.pbeta[n * p.h_v + h]));
             }
         }
     }
@@ -566,80 +562,58 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if constexpr (FUSED) {
         if (path_len > 0 && path_s[0] >= 0) {
             const int L = path_len;
-            const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
-            const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
-            // Scaled form: with A_t = alpha_1..alpha_t and x~ = x / A_t the step is one packed FMA per pair,
-            //   x~ += k (beta_t (v - A_t k.x~) / A_t),
-            // and x = A_L x~ at the end.  It is used unless the path decays below 2^-80 (then 1/A_t could
-            // overflow and the plain form alpha x + k w is taken instead).
-            const bool scaled = ab_path[L - 1].x > 8.3e-25f;   // .x holds the cumulative decay A_t, .y beta_t
+        const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
+        const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
 #pragma unroll 1
-            for (int t = 0; t < L; ++t) {
-                // this thread's sixteen key positions, 64*kh + 8*l8 + e, as packed pairs
-                float2 kf2[8];
+        for (int t = 0; t < L; ++t) {
+            // this thread's sixteen key positions: 64*kh + 8*l8 + e
+            float kf[16];
 #pragma unroll
-                for (int kh = 0; kh < 2; ++kh) {
-                    const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
-                    const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
+            for (int kh = 0; kh < 2; ++kh) {
+                const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
+                const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        kf2[kh * 4 + e] = make_float2(__uint_as_float(w4[e] << 16), __uint_as_float(w4[e] & 0xFFFF0000u));
-                }
-                const float2 ab = ab_path[t];
-                const float alpha = alpha_path[t];            // only the plain form needs it
-                const float inv_a = scaled ? 1.f / ab.x : 0.f;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = warp * 16 + i * 4 + r4;
-                    float2 x2[8];
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        x2[2 * q4] = make_float2(x[i][q4].x, x[i][q4].y);
-                        x2[2 * q4 + 1] = make_float2(x[i][q4].z, x[i][q4].w);
-                    }
-                    float2 acc = make_float2(0.f, 0.f);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc = __ffma2_rn(kf2[e], x2[e], acc);
-                    float dot = acc.x + acc.y;
-                    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-                    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-                    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-                    const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
-                    if (scaled) {
-                        const float w = ab.y * (vc - ab.x * dot) * inv_a;
-                        const float2 w2 = make_float2(w, w);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) x2[e] = __ffma2_rn(kf2[e], w2, x2[e]);
-                    } else {
-                        const float w = ab.y * (vc - alpha * dot);
-                        const float2 w2 = make_float2(w, w), al2 = make_float2(alpha, alpha), z2 = make_float2(0.f, 0.f);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) x2[e] = __ffma2_rn(kf2[e], w2, __ffma2_rn(x2[e], al2, z2));
-                    }
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4)
-                        x[i][q4] = make_float4(x2[2 * q4].x, x2[2 * q4].y, x2[2 * q4 + 1].x, x2[2 * q4 + 1].y);
+                for (int e = 0; e < 4; ++e) {
+                    kf[kh * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
+                    kf[kh * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
                 }
             }
-            if (scaled) {
-                const float aL = ab_path[L - 1].x;
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4)
-                        x[i][q4] = make_float4(aL * x[i][q4].x, aL * x[i][q4].y, aL * x[i][q4].z, aL * x[i][q4].w);
-            }
-            // the committed state: the only state write of the step
-            float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
+            const float2 ab = ab_path[t];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                float4 *dst = reinterpret_cast<float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+                const int row = warp * 16 + i * 4 + r4;
+                float xs16[16];
 #pragma unroll
-                for (int kh = 0; kh < 2; ++kh) {
-                    dst[kh * 16 + l8 * 2 + 0] = x[i][kh * 2 + 0];
-                    dst[kh * 16 + l8 * 2 + 1] = x[i][kh * 2 + 1];
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    xs16[q4 * 4 + 0] = x[i][q4].x; xs16[q4 * 4 + 1] = x[i][q4].y;
+                    xs16[q4 * 4 + 2] = x[i][q4].z; xs16[q4 * 4 + 3] = x[i][q4].w;
                 }
+                float dot = 0.f;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) dot = fmaf(kf[e], xs16[e], dot);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
+                const float w = ab.y * (vc - ab.x * dot);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) xs16[e] = fmaf(kf[e], w, ab.x * xs16[e]);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    x[i][q4] = make_float4(xs16[q4 * 4 + 0], xs16[q4 * 4 + 1], xs16[q4 * 4 + 2], xs16[q4 * 4 + 3]);
             }
+        }
+        // the committed state: the only state write of the step
+        float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 *dst = reinterpret_cast<float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                dst[kh * 16 + l8 * 2 + 0] = x[i][kh * 2 + 0];
+                dst[kh * 16 + l8 * 2 + 1] = x[i][kh * 2 + 1];
+            }
+        }
         }
         __syncthreads();   // the path rows sit where the state operand is about to be written
     }
