@@ -42,6 +42,15 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def ncu_traffic(args, w, fused):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu capture
+    (profiles/verify_sm100_fused_stack24_T64.md: 85.4 MB for 24 layer slots), scaled by layer slots; only
+    quoted for the workload and mode that capture covers."""
+    if args.workload == "stack48_T64" and fused:
+        return 85.4e6 / 24.0 * w.n_seq
+    return None
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -169,7 +178,7 @@ def main():
     ap.add_argument("--workload", default="stack48_T64", choices=sorted(WORKLOADS))
     ap.add_argument("--sets", type=int, default=0, help="buffer sets to rotate over (0 = enough to exceed 2x L2)")
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--oracle-slots", type=int, default=24, help="layer slots / sequences in the oracle's sample")
+    ap.add_argument("--oracle-slots", type=int, default=48, help="layer slots / sequences in the oracle's sample")
     ap.add_argument("--mode", default="fused", choices=["fused", "separate"],
                     help="fused: one gdn_tree_commit_verify call per step; separate: gdn_tree_verify + gdn_tree_commit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -347,7 +356,8 @@ def main():
                               "frac_of_nominal_8000": sbytes / (ms_per_step * 1e-3) / 1e9 / 8000.0},
             "roofline": {"kernel": "verify_sm100_kernel<fused commit>" if fused else "verify_sm100_kernel",
                          "bound": "hbm", "achieved": achieved, "peak": peak,
-                         "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                         "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": ncu_traffic(args, w, fused),
                          "bytes_per_launch": dom_bytes,
                          "avg_launch_us": v_avg * 1e3,
                          "note": "launch time includes the ~5 us tree-metadata kernel that precedes it in the call"},
