@@ -53,7 +53,9 @@ constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit: int [16] node 
 constexpr int SM_PK = 32768;                     // fused commit: k rows of the accepted path, bf16 [16][128], parked in the
 constexpr int SM_PV = 36864;                     // state-operand area until the replay is over; v rows likewise
 constexpr int SM_VNODE = SM_PATH + 256;          // grouped mode: u16 [64] node id of virtual index u
-constexpr int SM_MBAR = SM_VNODE + 128;          // 3 x u64: Gram done, P done, D done
+constexpr int SM_TABLE2 = SM_VNODE + 128;        // persistent kernel: second copy of ANC / GAB / DEPTH (2112 B)
+constexpr int SM_TABLE_STRIDE = SM_TABLE2 - SM_ANC;   // table buffer tb lives SM_TABLE_STRIDE * tb further on
+constexpr int SM_MBAR = SM_TABLE2 + 2176;        // 3 x u64: Gram done, P done, D done
 constexpr int SM_TMEM = SM_MBAR + 24;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
 constexpr int SM_BYTES = SM_FLAG + 4;
@@ -67,18 +69,24 @@ __device__ long long *g_trace_buf = nullptr;
     do {                                                                             \
         if (threadIdx.x == 0 && g_trace_buf) g_trace_buf[blockIdx.x * 16 + (k)] = clock64(); \
     } while (0)
+#define GDN_TRACE_MARK_U(u, k)                                                       \
+    do {                                                                             \
+        if (threadIdx.x == 0 && g_trace_buf) g_trace_buf[(u) * 16 + (k)] = clock64(); \
+    } while (0)
 #define GDN_TRACE_MARK_T(t, k)                                                       \
     do {                                                                             \
         if (threadIdx.x == (t) && g_trace_buf) g_trace_buf[blockIdx.x * 16 + (k)] = clock64(); \
     } while (0)
 #else
 #define GDN_TRACE_MARK(k) do {} while (0)
+#define GDN_TRACE_MARK_U(u, k) do {} while (0)
 #define GDN_TRACE_MARK_T(t, k) do {} while (0)
 #endif
 
 struct VerifyFastParams {
     int h_qk, h_v;
-    int n_units;        // n_seq * h_v = gridDim.x
+    int skew_ns;        // persistent kernel: start delay of the second half of the grid
+    int n_units;        // n_seq * h_v
     int prefetch_dist;  // a CTA warms L2 for unit blockIdx.x + prefetch_dist (about one wave ahead)
     float scale;
     const float *S0;
@@ -115,6 +123,8 @@ __device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes)
 {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_group1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all()
 {
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
@@ -839,14 +849,609 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
 }
 
+// Persistent form of the kernel above for trees that fit one CTA: a CTA keeps its tensor memory and walks over
+// the units blockIdx.x, blockIdx.x + gridDim.x, ...  While it finishes one unit (R, second GEMM, outputs) the
+// next unit's k/q tile streams into the freed operand tile and its per-node tables into the other table buffer,
+// so that a unit starts on the tensor core at once; the state tile is asked for at the top of the unit and is
+// only needed after the Gram / coefficient phases.
+template <typename TOut, bool FUSED>
+__global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const VerifyFastParams p)
+{
+    extern __shared__ uint8_t fv_smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fv_smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    float *xs = reinterpret_cast<float *>(smem + SM_X);
+    float *ys = reinterpret_cast<float *>(smem + SM_Y);
+    float *gram = reinterpret_cast<float *>(smem + SM_GRAM);
+    const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(smem + SM_V);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM_TMEM);
+    volatile uint32_t *flag = reinterpret_cast<volatile uint32_t *>(smem + SM_FLAG);
+    const uint32_t mbar_g = sbase + SM_MBAR, mbar_p = mbar_g + 8, mbar_d = mbar_g + 16;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r4 = lane >> 3, l8 = lane & 7;
+
+    if (warp == 0) tmem_alloc(sbase + SM_TMEM, FV_TMEM_COLS);
+    if (tid == 32) {
+        mbar_init(mbar_g, 1);
+        mbar_init(mbar_p, 1);
+        mbar_init(mbar_d, 1);
+        *flag = 0;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    // unit -> (tree, head, first node, size); a unit whose tree was rejected or is empty is skipped
+    auto decode = [&](int u, int &ub, int &uh, int &uhk, int &ubase, int &uT) -> bool {
+        if (u >= p.n_units) return false;
+        ub = u / p.h_v;
+        uh = u % p.h_v;
+        uhk = uh / (p.h_v / p.h_qk);
+        ubase = p.node_offsets[ub];
+        uT = p.node_offsets[ub + 1] - ubase;
+        return p.tree_ok[ub] && uT > 0 && uT <= FV_T;
+    };
+    // k and q rows -> B operand tile (rows beyond T are zero-filled)
+    auto issue_kq = [&](int ub, int uhk, int ubase, int uT) {
+        (void)ub;
+#pragma unroll
+        for (int it2 = 0; it2 < (128 * 16) / FV_THREADS; ++it2) {
+            const int idx = it2 * FV_THREADS + tid;
+            const int r = idx >> 4, c16 = idx & 15;
+            const int node = r >> 1;
+            const bool valid = node < uT;
+            const __nv_bfloat16 *src = ((r & 1) ? p.q : p.k) + ((size_t)(ubase + (valid ? node : 0)) * p.h_qk + uhk) * FV_D + c16 * 8;
+            cp_async_16(sbase + SM_B_KQ + sw128_offset(r, c16), src, valid);
+        }
+    };
+    // per-node tables: depth, root-path ids, g, beta (zeros beyond T), into table buffer `tb`
+    auto load_tables = [&](int ub, int uh, int ubase, int uT, int tb) {
+        (void)ub;
+        if (tid < FV_T) {
+            int d = 0;
+            uint4 row = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+            float gi = 0.f, be = 0.f;
+            if (tid < uT) {
+                const int n = ubase + tid;
+                d = p.depth[n];
+                row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)n * 16));
+                gi = __bfloat162float(p.g[(size_t)n * p.h_v + uh]);
+                be = __bfloat162float(p.beta[(size_t)n * p.h_v + uh]);
+            }
+            (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[tid] = (uint8_t)d;
+            *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + tid * 16) = row;
+            reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[tid] = make_float4(0.f, 0.f, be, gi);
+        }
+    };
+
+    int b = 0, h = 0, hk = 0, base = 0, T = 0;
+    {
+        const bool ok0 = decode(blockIdx.x, b, h, hk, base, T);
+        if (ok0) {
+            issue_kq(b, hk, base, T);
+            load_tables(b, h, base, T, 0);
+        }
+        cp_async_commit();
+    }
+    // The two CTAs of an SM would otherwise march in step (same phases at the same time, nothing to overlap):
+    // the second half of the grid starts a little later.
+    if (blockIdx.x >= (gridDim.x + 1) / 2 && p.skew_ns > 0) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < (long long)p.skew_ns * 2) __nanosleep(200);
+    }
+
+#pragma unroll 1
+    for (int unit = blockIdx.x, iter = 0; unit < p.n_units; unit += gridDim.x, ++iter) {
+    const bool unit_ok = decode(unit, b, h, hk, base, T);
+    const uint32_t par = (uint32_t)(iter & 1);
+    int nb = 0, nh = 0, nhk = 0, nbase = 0, nT = 0;
+    const bool next_ok = decode(unit + gridDim.x, nb, nh, nhk, nbase, nT);
+    float4 *gab = reinterpret_cast<float4 *>(smem + SM_GAB + (iter & 1) * SM_TABLE_STRIDE);
+    uint8_t *anc_s = smem + SM_ANC + (iter & 1) * SM_TABLE_STRIDE;
+    uint8_t *depth_s = smem + SM_DEPTH + (iter & 1) * SM_TABLE_STRIDE;
+    if (!unit_ok) {   // nothing to compute here: only keep the pipeline fed
+        cp_async_wait_all();
+        __syncthreads();
+        if (next_ok) {
+            issue_kq(nb, nhk, nbase, nT);
+            load_tables(nb, nh, nbase, nT, (iter + 1) & 1);
+        }
+        cp_async_commit();
+        continue;
+    }
+    GDN_TRACE_MARK_U(unit, 0);
+#ifdef GDN_TRACE
+    if (threadIdx.x == 0 && g_trace_buf) {
+        unsigned smid;
+        unsigned long long gt;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+        g_trace_buf[unit * 16 + 14] = smid;
+        g_trace_buf[unit * 16 + 15] = (long long)gt;
+    }
+#endif
+    // L2 warming for this CTA's next unit, in slices at phase boundaries
+    const int u_next = unit + gridDim.x;
+    auto warm_l2_state = [&](int slice) {
+        if (tid == 96 && u_next < p.n_units)
+            prefetch_l2_bulk(p.S0 + (size_t)u_next * FV_D * FV_D + (size_t)slice * 4096, 16384);
+    };
+    auto warm_l2_rows = [&]() {
+        if (next_ok && tid >= 128 && tid < 128 + FV_T && tid - 128 < nT)
+            prefetch_l2_bulk(p.v + ((size_t)(nbase + tid - 128) * p.h_v + nh) * FV_D, 256);
+    };
+
+    // (1) state tile loads: a warp instruction covers four rows; the eight lanes of a row each own one
+    // 16-byte bf16 piece of either K half.  Needed only after the Gram / coefficient phases.
+    float4 x[4][4];   // [row i][kh*2 + half]
+    {
+        const float *S = p.S0 + (size_t)(b * p.h_v + h) * FV_D * FV_D;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 *src = reinterpret_cast<const float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                x[i][kh * 2 + 0] = __ldg(src + kh * 16 + l8 * 2 + 0);
+                x[i][kh * 2 + 1] = __ldg(src + kh * 16 + l8 * 2 + 1);
+            }
+        }
+    }
+    // fused commit, step 1: this tree's accepted path of the previous step (ids and their parents)
+    int *path_s = reinterpret_cast<int *>(smem + SM_PATH);
+    int *par_s = path_s + FV_MD;
+    float2 *ab_path = reinterpret_cast<float2 *>(smem + SM_PATH + 128);
+    int path_len = 0, pbase = 0, pT = 0;
+    bool path_shape_ok = true;
+    if constexpr (FUSED) {
+        const int pp0 = p.path_offsets[b];
+        path_len = p.path_offsets[b + 1] - pp0;   // uniform over the CTA; 0 leaves the state alone
+        if (path_len != 0) {
+            pbase = p.pnode_offsets[b];
+            pT = p.pnode_offsets[b + 1] - pbase;
+            path_shape_ok = path_len > 0 && path_len <= FV_MD && pT > 0 && pp0 >= 0;
+            if (path_shape_ok && tid >= 128 && tid - 128 < path_len) {
+                const int n = p.path[pp0 + tid - 128];
+                path_s[tid - 128] = n;
+                par_s[tid - 128] = (p.pparent && n >= 0 && n < pT) ? p.pparent[pbase + n] : -2;
+            }
+        }
+    }
+    GDN_TRACE_MARK_U(unit, 1);
+
+    cp_async_wait_all();
+    fence_proxy_async();   // the k/q tile (cp.async) becomes visible to the tensor core
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    GDN_TRACE_MARK_U(unit, 2);
+
+    // (4) Everything that depends only on q, k, g, beta runs now, under the latency of the state loads:
+    // Gram = [k;q].[k;q]^T on the tensor core, G_i / a_i tables, then X and Y of Eq. 9.
+    if (tid == 0) {
+        const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
+        constexpr uint32_t id = idesc_bf16(128, 128);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+            umma_bf16(tmem + 128, b_kq + adv, b_kq + adv, id, ks > 0);
+        }
+        umma_commit(mbar_g);
+    }
+    if constexpr (FUSED) {
+        // step 2: the path must be a chain from a root inside the previous tree
+        if (tid == 160 && path_len != 0) {
+            int bad = !path_shape_ok;
+            for (int t = 0; !bad && t < path_len; ++t) {
+                const int n = path_s[t];
+                if (n < 0 || n >= pT) bad = 1;
+                else if (p.pparent) bad = par_s[t] != (t ? path_s[t - 1] : -1);
+                else if (t && n <= path_s[t - 1]) bad = 1;
+            }
+            if (bad) {
+                report_status(p.status_dev, GDN_ERR_PATH);
+                path_s[0] = -1;   // tells everybody to skip the replay: this state stays as it was
+            }
+        }
+    }
+    // G_i = sum of g along the root path (root first), a_i = exp(G_i)
+    if (tid >= 64 && tid < 64 + FV_T) {
+        const int i = tid - 64;
+        const int d = depth_s[i];
+        float G = 0.f;
+        for (int t = 0; t < d; ++t) G += gab[anc_s[i * FV_MD + t]].w;
+        gab[i].x = G;
+        gab[i].y = d ? expf(G) : 0.f;
+    }
+    // one thread polls the mbarrier (bounded: on expiry it flags the error and everybody falls through to
+    // the clean-up), the others sleep in the CTA barrier
+    if (tid == 0 && !mbar_wait_bounded(mbar_g, par)) *flag = 1;
+    __syncthreads();
+    tc_fence_after();
+    GDN_TRACE_MARK_U(unit, 3);
+    warm_l2_state(0);
+    if constexpr (FUSED) {
+        // step 3: k and v rows of the path (bf16, 256 B each) and the per-step scalars
+        if (path_len > 0 && path_s[0] >= 0) {
+            for (int idx = tid; idx < path_len * 32; idx += FV_THREADS) {
+                const int t = idx >> 5, c16 = idx & 15;
+                const size_t n = (size_t)pbase + path_s[t];
+                if (idx & 16)
+                    cp_async_16(sbase + SM_PV + t * 256 + c16 * 16, p.pv + (n * p.h_v + h) * FV_D + c16 * 8, true);
+                else
+                    cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + hk) * FV_D + c16 * 8, true);
+            }
+            if (tid < path_len) {
+                const size_t n = (size_t)pbase + path_s[tid];
+                ab_path[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + h])),
+                                           __bfloat162float(p.pbeta[n * p.h_v + h]));
+            }
+        }
+    }
+    if (*flag == 0) {
+        // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
+        {
+            const int row = (warp & 3) * 32 + lane;
+            const int half = warp >> 2;   // TMEM columns 128 + 64*half .. : k_j for j = 32*half ..
+            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 128 + half * 64;
+#pragma unroll 1
+            for (int part = 0; part < 2; ++part) {
+                uint32_t ra[32];
+                GDN_TMEM_LD32(taddr + part * 32, ra);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int col = half * 32 + part * 16 + j;
+                    gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[2 * j]);
+                }
+            }
+        }
+        tc_fence_before();
+        __syncthreads();
+        GDN_TRACE_MARK_U(unit, 4);
+        warm_l2_state(1);
+        // X and Y for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
+        {
+            float gdiff[4], gk[4], gq[4], bi[4];
+            bool on[4], onx[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = u * FV_THREADS + tid;
+                const int i = idx >> 4, t = idx & 15;
+                const int d = depth_s[i];
+                on[u] = t < d;
+                onx[u] = t < d - 1;
+                const int j = on[u] ? anc_s[idx] : 0;
+                const float4 gi = gab[i];
+                gdiff[u] = gi.x - gab[j].x;
+                bi[u] = gi.z;
+                gq[u] = gram[(2 * i + 1) * 64 + (j ^ ((2 * i + 1) & 31))];
+                gk[u] = gram[(2 * i) * 64 + (j ^ ((2 * i) & 31))];
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int idx = u * FV_THREADS + tid;
+                const float dec = expf(gdiff[u]);
+                ys[idx] = on[u] ? dec * gq[u] : 0.f;
+                xs[idx] = onx[u] ? bi[u] * dec * gk[u] : 0.f;
+            }
+        }
+    }
+    cp_async_wait_all();
+    __syncthreads();   // X and Y complete; the Gram copy is dead and its area can take the state operand
+    GDN_TRACE_MARK_U(unit, 5);
+
+    // (3') fused commit: replay Eq. 7 along the previous step's accepted path on the state tile while it
+    // sits in registers, write it back, and let everything below verify the new tree against it.
+    // Per row c (one value component): s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that
+    // share a row reduce k.s_c with three shuffles.  The path's k/v rows were fetched above.
+    if constexpr (FUSED) {
+        if (path_len > 0 && path_s[0] >= 0) {
+            const int L = path_len;
+        const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
+        const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
+#pragma unroll 1
+        for (int t = 0; t < L; ++t) {
+            // this thread's sixteen key positions: 64*kh + 8*l8 + e
+            float kf[16];
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
+                const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    kf[kh * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
+                    kf[kh * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
+                }
+            }
+            const float2 ab = ab_path[t];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = warp * 16 + i * 4 + r4;
+                float xs16[16];
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    xs16[q4 * 4 + 0] = x[i][q4].x; xs16[q4 * 4 + 1] = x[i][q4].y;
+                    xs16[q4 * 4 + 2] = x[i][q4].z; xs16[q4 * 4 + 3] = x[i][q4].w;
+                }
+                float dot = 0.f;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) dot = fmaf(kf[e], xs16[e], dot);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
+                const float w = ab.y * (vc - ab.x * dot);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) xs16[e] = fmaf(kf[e], w, ab.x * xs16[e]);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    x[i][q4] = make_float4(xs16[q4 * 4 + 0], xs16[q4 * 4 + 1], xs16[q4 * 4 + 2], xs16[q4 * 4 + 3]);
+            }
+        }
+        // the committed state: the only state write of the step
+        float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 *dst = reinterpret_cast<float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                dst[kh * 16 + l8 * 2 + 0] = x[i][kh * 2 + 0];
+                dst[kh * 16 + l8 * 2 + 1] = x[i][kh * 2 + 1];
+            }
+        }
+        }
+        __syncthreads();   // the path rows sit where the state operand is about to be written
+    }
+
+    // (4) fp32 -> bf16 hi + lo, written as the A operand
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = warp * 16 + i * 4 + r4;
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh) {
+            const float4 u = x[i][kh * 2 + 0], w = x[i][kh * 2 + 1];
+            const float f[8] = {u.x, u.y, u.z, u.w, w.x, w.y, w.z, w.w};
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) split_pack_bf16(f[2 * e], f[2 * e + 1], hi[e], lo[e]);
+            const uint32_t off = sw128_offset(row, kh * 8 + l8);
+            *reinterpret_cast<uint4 *>(smem + SM_A_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4 *>(smem + SM_A_LO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+    }
+    fence_proxy_async();   // generic-proxy writes of the operand become visible to the tensor core
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    GDN_TRACE_MARK_U(unit, 6);
+    warm_l2_state(2);
+
+    // (5) P = S0.[k;q]^T (hi then lo) on the tensor core; meanwhile the back-substitution below
+    if (tid == 0) {
+        const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
+        const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
+        constexpr uint32_t id = idesc_bf16(128, 128);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+            umma_bf16(tmem, a_hi + adv, b_kq + adv, id, ks > 0);
+        }
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+            umma_bf16(tmem, a_lo + adv, b_kq + adv, id, 1);
+        }
+        umma_commit(mbar_p);
+    }
+    // (6) z^T = y^T (I + X_path)^-1 by back-substitution over the root path (column-oriented: once z_l is
+    // final, subtract z_l X(n_l, n_t) from every z_t, t < l).  Four threads per node, thread sq of the quad
+    // owning path positions 4 sq .. 4 sq + 3; z stays in registers until the k/q tile can be overwritten.
+    const int zi = tid >> 2, sq = tid & 3;
+        const int d = depth_s[zi];
+        const int dmax = __reduce_max_sync(0xffffffffu, d);
+        const uint4 row = *reinterpret_cast<const uint4 *>(anc_s + zi * 16);
+        const uint32_t idw[4] = {row.x, row.y, row.z, row.w};
+        const float4 y4 = *reinterpret_cast<const float4 *>(ys + zi * FV_MD + sq * 4);
+        float z[4] = {y4.x, y4.y, y4.z, y4.w};
+#pragma unroll
+        for (int l = FV_MD - 1; l >= 1; --l) {
+            if (l < dmax) {   // warp-uniform
+                const float zl = __shfl_sync(0xffffffffu, z[l & 3], (lane & ~3) | (l >> 2));
+                if (l < d && sq * 4 < l) {
+                    const int nl = (int)((idw[l >> 2] >> ((l & 3) * 8)) & 0xFFu);
+                    const float4 x4 = *reinterpret_cast<const float4 *>(xs + nl * FV_MD + sq * 4);
+                    const float xv[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (sq * 4 + e < l) z[e] = fmaf(-zl, xv[e], z[e]);
+                }
+            }
+        }
+    GDN_TRACE_MARK_U(unit, 7);
+    if (tid == 0 && !mbar_wait_bounded(mbar_p, par)) *flag = 1;
+    __syncthreads();
+    tc_fence_after();
+    bool ok = *flag == 0;
+    GDN_TRACE_MARK_U(unit, 8);
+    warm_l2_state(3);
+
+    if (ok) {
+        // (7) both operand tiles are dead now: the tree's v rows go over the state operand, and z is
+        // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path) over the k/q tile
+#pragma unroll
+        for (int it = 0; it < (FV_T * 16) / FV_THREADS; ++it) {
+            const int idx = it * FV_THREADS + tid;
+            const int i = idx >> 4, c16 = idx & 15;
+            const bool valid = i < T;
+            cp_async_16(sbase + SM_V + i * 256 + c16 * 16,
+                        p.v + ((size_t)(base + (valid ? i : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
+        }
+        cp_async_commit();
+        // the k/q tile is dead: start on the next unit of this CTA (its k/q tile, its tables), to be
+        // consumed after the loop comes round
+        if (next_ok) {
+            issue_kq(nb, nhk, nbase, nT);
+            load_tables(nb, nh, nbase, nT, (iter + 1) & 1);
+        }
+        cp_async_commit();
+        {
+            const int i = zi;
+            const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, 2 * sq)) = zero4;
+            *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, 2 * sq + 1)) = zero4;
+            *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, 2 * sq)) = zero4;
+            *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, 2 * sq + 1)) = zero4;
+            __syncwarp();   // the quad's zero fill precedes the scattered stores below
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int t = sq * 4 + e;
+                if (t < d) {
+                    const int j = (int)((idw[sq] >> (e * 8)) & 0xFFu);
+                    float hi, lo;
+                    split_bf16(z[e], hi, lo);
+                    const uint32_t off = sw128_row_offset(i, j >> 3) + (j & 7) * 2;
+                    *reinterpret_cast<__nv_bfloat16 *>(smem + SM_Z_HI + off) = __float2bfloat16_rn(hi);
+                    *reinterpret_cast<__nv_bfloat16 *>(smem + SM_Z_LO + off) = __float2bfloat16_rn(lo);
+                }
+            }
+        }
+        cp_async_wait_group1();   // the v rows have landed; the next unit's tile may still be in flight
+        __syncthreads();
+        GDN_TRACE_MARK_U(unit, 9);
+
+        // (8) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
+        // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
+        {
+            const int c = (warp & 3) * 32 + lane;
+            const int half = warp >> 2;
+            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
+#pragma unroll 1
+            for (int part = 0; part < 2; ++part) {
+                const int j0 = half * 32 + part * 16;
+                uint32_t rr[32];
+                GDN_TMEM_LD32(taddr + part * 32, rr);   // columns 2j, 2j+1 for 16 nodes: p^k_j, p^q_j
+                float vv[16], aj[16], bj[16];
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) {
+                    vv[jj] = __bfloat162float(vs[(j0 + jj) * FV_D + c]);
+                    const float4 gj = gab[j0 + jj];
+                    aj[jj] = gj.y;
+                    bj[jj] = gj.z;
+                }
+                tmem_wait_ld();
+                uint32_t hi[8], lo[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float r0 = bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[4 * e]));
+                    const float r1 = bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[4 * e + 2]));
+                    split_pack_bf16(r0, r1, hi[e], lo[e]);
+                }
+#pragma unroll
+                for (int oct = 0; oct < 2; ++oct) {
+                    const uint32_t off = sw128_row_offset(c, half * 4 + part * 2 + oct);
+                    *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = make_uint4(hi[4 * oct], hi[4 * oct + 1], hi[4 * oct + 2], hi[4 * oct + 3]);
+                    *reinterpret_cast<uint4 *>(smem + SM_RT_LO + off) = make_uint4(lo[4 * oct], lo[4 * oct + 1], lo[4 * oct + 2], lo[4 * oct + 3]);
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        GDN_TRACE_MARK_U(unit, 10);
+        warm_l2_rows();
+
+        // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
+        if (tid == 0) {
+            constexpr uint32_t id2 = idesc_bf16(128, 64);
+            const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
+            const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
+#pragma unroll
+            for (int combo = 0; combo < 3; ++combo) {   // hi.hi, lo.hi, hi.lo; lo.lo is below 2^-18 of the result
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16(tmem + 128, a2[combo & 1] + (uint64_t)(ks * 2), b2[combo >> 1] + (uint64_t)(ks * 2), id2,
+                              (combo | ks) != 0);
+            }
+            umma_commit(mbar_d);
+        }
+        if (tid == 0 && !mbar_wait_bounded(mbar_d, par)) *flag = 1;
+        __syncthreads();
+        tc_fence_after();
+        ok = *flag == 0;
+        GDN_TRACE_MARK_U(unit, 11);
+
+        // (10) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i]), staged through shared memory (over the
+        // dead R^T tiles) so that global memory sees 16-byte stores of whole rows
+        if (ok) {
+            const int c = (warp & 3) * 32 + lane;
+            const int half = warp >> 2;
+            const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+            TOut *o_s = reinterpret_cast<TOut *>(smem + SM_RT_HI);   // [64][128] TOut: 16 or 32 KB
+#pragma unroll 1
+            for (int part = 0; part < 2; ++part) {
+                const int i0 = half * 32 + part * 16;
+                uint32_t pp[32], dd[16];
+                GDN_TMEM_LD32(trow + 2 * i0, pp);
+                GDN_TMEM_LD16(trow + 128 + i0, dd);
+                float ai[16];
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) ai[jj] = gab[i0 + jj].y;
+                tmem_wait_ld();
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) {
+                    const float out = p.scale * fmaf(ai[jj], __uint_as_float(pp[2 * jj + 1]), __uint_as_float(dd[jj]));
+                    store_from_float(o_s + (i0 + jj) * FV_D + c, out);
+                }
+            }
+        }
+        __syncthreads();
+        if (*flag == 0) {
+            constexpr int ROW_CHUNKS = FV_D * (int)sizeof(TOut) / 16;   // 16-byte pieces per output row
+            uint8_t *o = static_cast<uint8_t *>(p.o);
+            for (int idx = tid; idx < T * ROW_CHUNKS; idx += FV_THREADS) {
+                const int i = idx / ROW_CHUNKS, ck = idx % ROW_CHUNKS;
+                const uint4 val = *reinterpret_cast<const uint4 *>(smem + SM_RT_HI + (size_t)i * FV_D * sizeof(TOut) + ck * 16);
+                *reinterpret_cast<uint4 *>(o + (((size_t)(base + i) * p.h_v + h) * FV_D) * sizeof(TOut) + ck * 16) = val;
+            }
+        }
+    }
+    GDN_TRACE_MARK_U(unit, 12);
+#ifdef GDN_TRACE
+    if (threadIdx.x == 0 && g_trace_buf) {
+        unsigned long long gt;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+        g_trace_buf[unit * 16 + 13] = (long long)gt;
+    }
+#endif
+    if (*flag != 0) break;   // a bounded wait expired: stop, report, release
+    }   // unit loop
+
+    if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
+    cp_async_wait_all();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
+}
+
 template <typename TOut, bool FUSED, bool GROUPED>
 cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, cudaStream_t stream)
 {
-    cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut, FUSED, GROUPED>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
-    if (e != cudaSuccess) return e;
-    const int grid = s.n_seq * s.h_v * (GROUPED ? p.groups_per_tree : 1);
-    verify_sm100_kernel<TOut, FUSED, GROUPED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
+    if constexpr (GROUPED) {
+        cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut, FUSED, GROUPED>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
+        if (e != cudaSuccess) return e;
+        const int grid = s.n_seq * s.h_v * p.groups_per_tree;
+        verify_sm100_kernel<TOut, FUSED, GROUPED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
+    } else {
+        // trees that fit one CTA: persistent CTAs, two per SM, pipelined across units
+        cudaError_t e = cudaFuncSetAttribute(verify_sm100_persistent_kernel<TOut, FUSED>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
+        if (e != cudaSuccess) return e;
+        const int grid = p.n_units < p.prefetch_dist ? p.n_units : p.prefetch_dist;
+        verify_sm100_persistent_kernel<TOut, FUSED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
+    }
     return cudaGetLastError();
 }
 
@@ -858,6 +1463,7 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     VerifyFastParams p{};
     p.h_qk = s.h_qk; p.h_v = s.h_v; p.n_units = s.n_seq * s.h_v; p.prefetch_dist = 2 * sms; p.scale = s.scale;
+    p.skew_ns = 3000;
     p.S0 = S0;
     p.q = static_cast<const __nv_bfloat16 *>(q); p.k = static_cast<const __nv_bfloat16 *>(k);
     p.v = static_cast<const __nv_bfloat16 *>(v); p.g = static_cast<const __nv_bfloat16 *>(g);
