@@ -259,11 +259,10 @@ __device__ __forceinline__ void split_bf16(float x, float &hi, float &lo)
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <typename TOut, bool FUSED, bool GROUPED>
+template <typename TOut, bool GROUPED>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const VerifyFastParams p)
 {
     extern __shared__ uint8_t fv_smem_raw[];
-    static_assert(!(FUSED && GROUPED), "the fused commit needs one CTA per state tile");
     // GROUPED: the CTA takes group `grp` of tree b (see gdn_internal.cuh): T is then the size of the
     // virtual tree (n_prefix ancestors of the group's first node + the group's own nodes), and virtual
     // index u maps to node vnode[u].  Trees of at most 64 nodes are their own single group, identity map.
@@ -420,26 +419,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         *reinterpret_cast<uint4 *>(anc_s + tid * 16) = row;
         gab[tid] = make_float4(0.f, 0.f, be, gi);
     }
-    // fused commit, step 1: this tree's accepted path of the previous step (ids and their parents)
-    int *path_s = reinterpret_cast<int *>(smem + SM_PATH);
-    int *par_s = path_s + FV_MD;
-    float2 *ab_path = reinterpret_cast<float2 *>(smem + SM_PATH + 128);
-    int path_len = 0, pbase = 0, pT = 0;
-    bool path_shape_ok = true;
-    if constexpr (FUSED) {
-        const int pp0 = p.path_offsets[b];
-        path_len = p.path_offsets[b + 1] - pp0;   // uniform over the CTA; 0 leaves the state alone
-        if (path_len != 0) {
-            pbase = p.pnode_offsets[b];
-            pT = p.pnode_offsets[b + 1] - pbase;
-            path_shape_ok = path_len > 0 && path_len <= FV_MD && pT > 0 && pp0 >= 0;
-            if (path_shape_ok && tid >= 128 && tid - 128 < path_len) {
-                const int n = p.path[pp0 + tid - 128];
-                path_s[tid - 128] = n;
-                par_s[tid - 128] = (p.pparent && n >= 0 && n < pT) ? p.pparent[pbase + n] : -2;
-            }
-        }
-    }
     GDN_TRACE_MARK(1);
 
     cp_async_wait_all();
@@ -462,22 +441,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         }
         umma_commit(mbar_g);
     }
-    if constexpr (FUSED) {
-        // step 2: the path must be a chain from a root inside the previous tree
-        if (tid == 160 && path_len != 0) {
-            int bad = !path_shape_ok;
-            for (int t = 0; !bad && t < path_len; ++t) {
-                const int n = path_s[t];
-                if (n < 0 || n >= pT) bad = 1;
-                else if (p.pparent) bad = par_s[t] != (t ? path_s[t - 1] : -1);
-                else if (t && n <= path_s[t - 1]) bad = 1;
-            }
-            if (bad) {
-                report_status(p.status_dev, GDN_ERR_PATH);
-                path_s[0] = -1;   // tells everybody to skip the replay: this state stays as it was
-            }
-        }
-    }
     // G_i = sum of g along the root path (root first), a_i = exp(G_i)
     if (tid >= 64 && tid < 64 + FV_T) {
         const int i = tid - 64;
@@ -494,24 +457,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     tc_fence_after();
     GDN_TRACE_MARK(3);
     warm_l2_state(0);
-    if constexpr (FUSED) {
-        // step 3: k and v rows of the path (bf16, 256 B each) and the per-step scalars
-        if (path_len > 0 && path_s[0] >= 0) {
-            for (int idx = tid; idx < path_len * 32; idx += FV_THREADS) {
-                const int t = idx >> 5, c16 = idx & 15;
-                const size_t n = (size_t)pbase + path_s[t];
-                if (idx & 16)
-                    cp_async_16(sbase + SM_PV + t * 256 + c16 * 16, p.pv + (n * p.h_v + h) * FV_D + c16 * 8, true);
-                else
-                    cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + hk) * FV_D + c16 * 8, true);
-            }
-            if (tid < path_len) {
-                const size_t n = (size_t)pbase + path_s[tid];
-                ab_path[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + h])),
-                                           __bfloat162float(p.pbeta[n * p.h_v + h]));
-            }
-        }
-    }
     if (*flag == 0) {
         // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
         {
@@ -565,68 +510,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     __syncthreads();   // X and Y complete; the Gram copy is dead and its area can take the state operand
     GDN_TRACE_MARK(5);
 
-    // (3') fused commit: replay Eq. 7 along the previous step's accepted path on the state tile while it
-    // sits in registers, write it back, and let everything below verify the new tree against it.
-    // Per row c (one value component): s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that
-    // share a row reduce k.s_c with three shuffles.  The path's k/v rows were fetched above.
-    if constexpr (FUSED) {
-        if (path_len > 0 && path_s[0] >= 0) {
-            const int L = path_len;
-        const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
-        const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
-#pragma unroll 1
-        for (int t = 0; t < L; ++t) {
-            // this thread's sixteen key positions: 64*kh + 8*l8 + e
-            float kf[16];
-#pragma unroll
-            for (int kh = 0; kh < 2; ++kh) {
-                const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
-                const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    kf[kh * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
-                    kf[kh * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
-                }
-            }
-            const float2 ab = ab_path[t];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = warp * 16 + i * 4 + r4;
-                float xs16[16];
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    xs16[q4 * 4 + 0] = x[i][q4].x; xs16[q4 * 4 + 1] = x[i][q4].y;
-                    xs16[q4 * 4 + 2] = x[i][q4].z; xs16[q4 * 4 + 3] = x[i][q4].w;
-                }
-                float dot = 0.f;
-#pragma unroll
-                for (int e = 0; e < 16; ++e) dot = fmaf(kf[e], xs16[e], dot);
-                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-                const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
-                const float w = ab.y * (vc - ab.x * dot);
-#pragma unroll
-                for (int e = 0; e < 16; ++e) xs16[e] = fmaf(kf[e], w, ab.x * xs16[e]);
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4)
-                    x[i][q4] = make_float4(xs16[q4 * 4 + 0], xs16[q4 * 4 + 1], xs16[q4 * 4 + 2], xs16[q4 * 4 + 3]);
-            }
-        }
-        // the committed state: the only state write of the step
-        float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float4 *dst = reinterpret_cast<float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
-#pragma unroll
-            for (int kh = 0; kh < 2; ++kh) {
-                dst[kh * 16 + l8 * 2 + 0] = x[i][kh * 2 + 0];
-                dst[kh * 16 + l8 * 2 + 1] = x[i][kh * 2 + 1];
-            }
-        }
-        }
-        __syncthreads();   // the path rows sit where the state operand is about to be written
-    }
 
     // (4) fp32 -> bf16 hi + lo, written as the A operand
 #pragma unroll
@@ -849,7 +732,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
 }
 
-// Persistent form of the kernel above for trees that fit one CTA: a CTA keeps its tensor memory and walks over
+// Persistent form of the kernel above for trees that fit one CTA, with the optional fused commit
+// (FUSED: Eq. 7 replayed along the previous step's accepted path on the state tile while it sits in
+// registers -- per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c), the eight lanes that share a row
+// reducing k.s_c with three shuffles -- written back as the only state write of the step, and the new tree
+// verified against it): a CTA keeps its tensor memory and walks over
 // the units blockIdx.x, blockIdx.x + gridDim.x, ...  While it finishes one unit (R, second GEMM, outputs) the
 // next unit's k/q tile streams into the freed operand tile and its per-node tables into the other table buffer,
 // so that a unit starts on the tensor core at once; the state tile is asked for at the top of the unit and is
@@ -1439,11 +1326,11 @@ template <typename TOut, bool FUSED, bool GROUPED>
 cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, cudaStream_t stream)
 {
     if constexpr (GROUPED) {
-        cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut, FUSED, GROUPED>,
+        cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut, GROUPED>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
         if (e != cudaSuccess) return e;
         const int grid = s.n_seq * s.h_v * p.groups_per_tree;
-        verify_sm100_kernel<TOut, FUSED, GROUPED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
+        verify_sm100_kernel<TOut, GROUPED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
     } else {
         // trees that fit one CTA: persistent CTAs, two per SM, pipelined across units
         cudaError_t e = cudaFuncSetAttribute(verify_sm100_persistent_kernel<TOut, FUSED>,
