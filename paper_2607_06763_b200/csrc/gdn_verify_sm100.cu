@@ -1052,28 +1052,35 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
             const float2 ab = ab_path[t];
+            // the four rows of this thread advance together: four independent FMA chains, then their
+            // shuffle reductions back to back, then the four updates
+            float dot[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    d0 = fmaf(kf[q4 * 4 + 0], x[i][q4].x, d0); d1 = fmaf(kf[q4 * 4 + 1], x[i][q4].y, d1);
+                    d0 = fmaf(kf[q4 * 4 + 2], x[i][q4].z, d0); d1 = fmaf(kf[q4 * 4 + 3], x[i][q4].w, d1);
+                }
+                dot[i] = d0 + d1;
+            }
+#pragma unroll
+            for (int m = 1; m < 8; m <<= 1)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) dot[i] += __shfl_xor_sync(0xffffffffu, dot[i], m);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int row = warp * 16 + i * 4 + r4;
-                float xs16[16];
+                const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
+                const float w = ab.y * (vc - ab.x * dot[i]);
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
-                    xs16[q4 * 4 + 0] = x[i][q4].x; xs16[q4 * 4 + 1] = x[i][q4].y;
-                    xs16[q4 * 4 + 2] = x[i][q4].z; xs16[q4 * 4 + 3] = x[i][q4].w;
+                    x[i][q4].x = fmaf(kf[q4 * 4 + 0], w, ab.x * x[i][q4].x);
+                    x[i][q4].y = fmaf(kf[q4 * 4 + 1], w, ab.x * x[i][q4].y);
+                    x[i][q4].z = fmaf(kf[q4 * 4 + 2], w, ab.x * x[i][q4].z);
+                    x[i][q4].w = fmaf(kf[q4 * 4 + 3], w, ab.x * x[i][q4].w);
                 }
-                float dot = 0.f;
-#pragma unroll
-                for (int e = 0; e < 16; ++e) dot = fmaf(kf[e], xs16[e], dot);
-                dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-                dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-                dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-                const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
-                const float w = ab.y * (vc - ab.x * dot);
-#pragma unroll
-                for (int e = 0; e < 16; ++e) xs16[e] = fmaf(kf[e], w, ab.x * xs16[e]);
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4)
-                    x[i][q4] = make_float4(xs16[q4 * 4 + 0], xs16[q4 * 4 + 1], xs16[q4 * 4 + 2], xs16[q4 * 4 + 3]);
             }
         }
         // the committed state: the only state write of the step
