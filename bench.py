@@ -284,13 +284,9 @@ def main():
     assert int(status.item()) == 0, gdn.gdn_status_string(int(status.item()))
     verify_ms = [e[0].elapsed_time(e[1]) for e in ev]
     commit_ms = [e[1].elapsed_time(e[2]) for e in ev]
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
+    from paper_2607_06763_b200 import multi
+    value, ms_per_step = multi.aggregate_throughput(w.total_nodes, total_ms / args.steps, "cuda")
     nodes_per_step = w.total_nodes * world
-    value = nodes_per_step / (ms_per_step * 1e-3)
 
     # ---- end-to-end: host buffers through the *_host entry points (copies inside the timed region)
     L = int(w.path_offsets[-1])
@@ -328,10 +324,7 @@ def main():
             e2e_step()
         barrier()
         e2e_s = (time.perf_counter() - t0) / args.e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = multi.reduce_max(e2e_s, "cuda") if e2e_s == e2e_s else e2e_s
     e2e_value = nodes_per_step / e2e_s
 
     out = None
