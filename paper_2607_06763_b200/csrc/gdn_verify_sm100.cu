@@ -733,6 +733,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 }
 
 // Persistent form of the kernel above for trees that fit one CTA, with the optional fused commit
+// In this kernel the k/q tile holds the k rows first and the q rows second (rows i and 64 + i), so P has
+// p^k in columns 0..63 and p^q in columns 64..127, and the Gram block needs only N = 64.
 // (FUSED: Eq. 7 replayed along the previous step's accepted path on the state tile while it sits in
 // registers -- per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c), the eight lanes that share a row
 // reducing k.s_c with three shuffles -- written back as the only state write of the step, and the new tree
@@ -786,9 +788,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         for (int it2 = 0; it2 < (128 * 16) / FV_THREADS; ++it2) {
             const int idx = it2 * FV_THREADS + tid;
             const int r = idx >> 4, c16 = idx & 15;
-            const int node = r >> 1;
+            const int node = r & 63;   // rows 0..63: k of node r, rows 64..127: q of node r - 64
             const bool valid = node < uT;
-            const __nv_bfloat16 *src = ((r & 1) ? p.q : p.k) + ((size_t)(ubase + (valid ? node : 0)) * p.h_qk + uhk) * FV_D + c16 * 8;
+            const __nv_bfloat16 *src = (r >= 64 ? p.q : p.k) + ((size_t)(ubase + (valid ? node : 0)) * p.h_qk + uhk) * FV_D + c16 * 8;
             cp_async_16(sbase + SM_B_KQ + sw128_offset(r, c16), src, valid);
         }
     };
@@ -914,10 +916,10 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     GDN_TRACE_MARK_U(unit, 2);
 
     // (4) Everything that depends only on q, k, g, beta runs now, under the latency of the state loads:
-    // Gram = [k;q].[k;q]^T on the tensor core, G_i / a_i tables, then X and Y of Eq. 9.
+    // Gram = [k;q].k^T on the tensor core, G_i / a_i tables, then X and Y of Eq. 9.
     if (tid == 0) {
         const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
-        constexpr uint32_t id = idesc_bf16(128, 128);
+        constexpr uint32_t id = idesc_bf16(128, 64);   // B = the 64 k rows
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
@@ -979,18 +981,15 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
         {
             const int row = (warp & 3) * 32 + lane;
-            const int half = warp >> 2;   // TMEM columns 128 + 64*half .. : k_j for j = 32*half ..
-            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 128 + half * 64;
-#pragma unroll 1
-            for (int part = 0; part < 2; ++part) {
-                uint32_t ra[32];
-                GDN_TMEM_LD32(taddr + part * 32, ra);
-                tmem_wait_ld();
+            const int half = warp >> 2;   // TMEM columns 128 + 32*half .. : k_j for j = 32*half ..
+            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 128 + half * 32;
+            uint32_t ra[32];
+            GDN_TMEM_LD32(taddr, ra);
+            tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int col = half * 32 + part * 16 + j;
-                    gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[2 * j]);
-                }
+            for (int j = 0; j < 32; ++j) {
+                const int col = half * 32 + j;
+                gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[j]);
             }
         }
         tc_fence_before();
@@ -1012,8 +1011,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 const float4 gi = gab[i];
                 gdiff[u] = gi.x - gab[j].x;
                 bi[u] = gi.z;
-                gq[u] = gram[(2 * i + 1) * 64 + (j ^ ((2 * i + 1) & 31))];
-                gk[u] = gram[(2 * i) * 64 + (j ^ ((2 * i) & 31))];
+                gq[u] = gram[(64 + i) * 64 + (j ^ (i & 31))];   // row 64 + i: q_i
+                gk[u] = gram[i * 64 + (j ^ (i & 31))];          // row i: k_i
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -1219,12 +1218,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         {
             const int c = (warp & 3) * 32 + lane;
             const int half = warp >> 2;
-            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
+            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 #pragma unroll 1
             for (int part = 0; part < 2; ++part) {
                 const int j0 = half * 32 + part * 16;
-                uint32_t rr[32];
-                GDN_TMEM_LD32(taddr + part * 32, rr);   // columns 2j, 2j+1 for 16 nodes: p^k_j, p^q_j
+                uint32_t rr[16];
+                GDN_TMEM_LD16(taddr + j0, rr);   // columns j0 .. j0+15: p^k of 16 nodes
                 float vv[16], aj[16], bj[16];
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) {
@@ -1237,8 +1236,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float r0 = bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[4 * e]));
-                    const float r1 = bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[4 * e + 2]));
+                    const float r0 = bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[2 * e]));
+                    const float r1 = bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[2 * e + 1]));
                     split_pack_bf16(r0, r1, hi[e], lo[e]);
                 }
 #pragma unroll
@@ -1286,8 +1285,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 #pragma unroll 1
             for (int part = 0; part < 2; ++part) {
                 const int i0 = half * 32 + part * 16;
-                uint32_t pp[32], dd[16];
-                GDN_TMEM_LD32(trow + 2 * i0, pp);
+                uint32_t pp[16], dd[16];
+                GDN_TMEM_LD16(trow + 64 + i0, pp);    // p^q of 16 nodes
                 GDN_TMEM_LD16(trow + 128 + i0, dd);
                 float ai[16];
 #pragma unroll
@@ -1295,7 +1294,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 tmem_wait_ld();
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) {
-                    const float out = p.scale * fmaf(ai[jj], __uint_as_float(pp[2 * jj + 1]), __uint_as_float(dd[jj]));
+                    const float out = p.scale * fmaf(ai[jj], __uint_as_float(pp[jj]), __uint_as_float(dd[jj]));
                     store_from_float(o_s + (i0 + jj) * FV_D + c, out);
                 }
             }
