@@ -21,6 +21,8 @@
 // warp owns one value component.  One CTA per (tree, value head), 256 threads, about 106 KB of
 // shared memory and 256 TMEM columns, so two CTAs share an SM: while one streams its 64 KB
 // state tile from HBM the other computes.
+#include <cuda.h>   // CUtensorMap and the cuTensorMapEncodeTiled prototype (resolved at run time, no libcuda link)
+
 #include "gdn_internal.cuh"
 
 namespace gdn {
@@ -55,8 +57,8 @@ constexpr int SM_PV = 36864;                     // state-operand area until the
 constexpr int SM_VNODE = SM_PATH + 256;          // grouped mode: u16 [64] node id of virtual index u
 constexpr int SM_TABLE2 = SM_VNODE + 128;        // persistent kernel: second copy of ANC / GAB / DEPTH (2112 B)
 constexpr int SM_TABLE_STRIDE = SM_TABLE2 - SM_ANC;   // table buffer tb lives SM_TABLE_STRIDE * tb further on
-constexpr int SM_MBAR = SM_TABLE2 + 2176;        // 3 x u64: Gram done, P done, D done
-constexpr int SM_TMEM = SM_MBAR + 24;            // u32
+constexpr int SM_MBAR = SM_TABLE2 + 2176;        // 5 x u64: Gram done, P done, D done, k/q tile landed, v tile landed
+constexpr int SM_TMEM = SM_MBAR + 40;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
 constexpr int SM_BYTES = SM_FLAG + 4;
 constexpr int SM_ALLOC = SM_BYTES + 1024;        // slack for the 1024-byte alignment of the base
@@ -84,6 +86,10 @@ __device__ long long *g_trace_buf = nullptr;
 #endif
 
 struct VerifyFastParams {
+    // TMA descriptors of the packed k, q, v tensors viewed as [N][heads][128] bf16 (persistent kernel only)
+    alignas(64) CUtensorMap tm_k;
+    alignas(64) CUtensorMap tm_q;
+    alignas(64) CUtensorMap tm_v;
     int h_qk, h_v;
     int skew_ns;        // persistent kernel: start delay of the second half of the grid
     int n_units;        // n_seq * h_v
@@ -122,6 +128,17 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool 
 __device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes)
 {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+// TMA: one thread announces the bytes a barrier has to see, then issues tiled loads that complete on it.
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar)
+                 : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_group1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
@@ -744,7 +761,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 // so that a unit starts on the tensor core at once; the state tile is asked for at the top of the unit and is
 // only needed after the Gram / coefficient phases.
 template <typename TOut, bool FUSED>
-__global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const VerifyFastParams p)
+__global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const __grid_constant__ VerifyFastParams p)
 {
     extern __shared__ uint8_t fv_smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fv_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -756,6 +773,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM_TMEM);
     volatile uint32_t *flag = reinterpret_cast<volatile uint32_t *>(smem + SM_FLAG);
     const uint32_t mbar_g = sbase + SM_MBAR, mbar_p = mbar_g + 8, mbar_d = mbar_g + 16;
+    const uint32_t mbar_kq = mbar_g + 24, mbar_v = mbar_g + 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r4 = lane >> 3, l8 = lane & 7;
 
@@ -764,6 +782,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         mbar_init(mbar_g, 1);
         mbar_init(mbar_p, 1);
         mbar_init(mbar_d, 1);
+        mbar_init(mbar_kq, 1);
+        mbar_init(mbar_v, 1);
         *flag = 0;
     }
     tc_fence_before();
@@ -781,17 +801,18 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         uT = p.node_offsets[ub + 1] - ubase;
         return p.tree_ok[ub] && uT > 0 && uT <= FV_T;
     };
-    // k and q rows -> B operand tile (rows beyond T are zero-filled)
+    // k and q rows -> B operand tile by TMA: four 64-row x 64-column boxes (k and q, either K half), 128-byte
+    // swizzled, completing on mbar_kq.  A box always spans 64 nodes: rows beyond the tree belong to the next tree
+    // (or are zero past the end of the tensor); every use of them is masked further down.
     auto issue_kq = [&](int ub, int uhk, int ubase, int uT) {
-        (void)ub;
+        (void)ub; (void)uT;
+        if (tid == 0) {
+            mbar_expect_tx(mbar_kq, 32768);
 #pragma unroll
-        for (int it2 = 0; it2 < (128 * 16) / FV_THREADS; ++it2) {
-            const int idx = it2 * FV_THREADS + tid;
-            const int r = idx >> 4, c16 = idx & 15;
-            const int node = r & 63;   // rows 0..63: k of node r, rows 64..127: q of node r - 64
-            const bool valid = node < uT;
-            const __nv_bfloat16 *src = (r >= 64 ? p.q : p.k) + ((size_t)(ubase + (valid ? node : 0)) * p.h_qk + uhk) * FV_D + c16 * 8;
-            cp_async_16(sbase + SM_B_KQ + sw128_offset(r, c16), src, valid);
+            for (int kh = 0; kh < 2; ++kh) {
+                tma_load_3d(sbase + SM_B_KQ + kh * 16384, &p.tm_k, kh * 64, uhk, ubase, mbar_kq);
+                tma_load_3d(sbase + SM_B_KQ + kh * 16384 + 8192, &p.tm_q, kh * 64, uhk, ubase, mbar_kq);
+            }
         }
     };
     // per-node tables: depth, root-path ids, g, beta (zeros beyond T), into table buffer `tb`
@@ -830,10 +851,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         while (clock64() - t0 < (long long)p.skew_ns * 2) __nanosleep(200);
     }
 
+    int done_units = 0;
 #pragma unroll 1
     for (int unit = blockIdx.x, iter = 0; unit < p.n_units; unit += gridDim.x, ++iter) {
     const bool unit_ok = decode(unit, b, h, hk, base, T);
-    const uint32_t par = (uint32_t)(iter & 1);
+    const uint32_t par = (uint32_t)(done_units & 1);   // every barrier completes once per processed unit
     int nb = 0, nh = 0, nhk = 0, nbase = 0, nT = 0;
     const bool next_ok = decode(unit + gridDim.x, nb, nh, nhk, nbase, nT);
     float4 *gab = reinterpret_cast<float4 *>(smem + SM_GAB + (iter & 1) * SM_TABLE_STRIDE);
@@ -865,10 +887,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     auto warm_l2_state = [&](int slice) {
         if (tid == 96 && u_next < p.n_units)
             prefetch_l2_bulk(p.S0 + (size_t)u_next * FV_D * FV_D + (size_t)slice * 4096, 16384);
-    };
-    auto warm_l2_rows = [&]() {
-        if (next_ok && tid >= 128 && tid < 128 + FV_T && tid - 128 < nT)
-            prefetch_l2_bulk(p.v + ((size_t)(nbase + tid - 128) * p.h_v + nh) * FV_D, 256);
     };
 
     // (1) state tile loads: a warp instruction covers four rows; the eight lanes of a row each own one
@@ -908,8 +926,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     }
     GDN_TRACE_MARK_U(unit, 1);
 
-    cp_async_wait_all();
-    fence_proxy_async();   // the k/q tile (cp.async) becomes visible to the tensor core
+    if (tid == 0 && !mbar_wait_bounded(mbar_kq, par)) *flag = 1;   // this unit's k/q tile has landed
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1172,22 +1189,16 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (ok) {
         // (7) both operand tiles are dead now: the tree's v rows go over the state operand, and z is
         // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path) over the k/q tile
-#pragma unroll
-        for (int it = 0; it < (FV_T * 16) / FV_THREADS; ++it) {
-            const int idx = it * FV_THREADS + tid;
-            const int i = idx >> 4, c16 = idx & 15;
-            const bool valid = i < T;
-            cp_async_16(sbase + SM_V + i * 256 + c16 * 16,
-                        p.v + ((size_t)(base + (valid ? i : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
+        if (tid == 0) {
+            mbar_expect_tx(mbar_v, FV_T * FV_D * 2);
+            tma_load_3d(sbase + SM_V, &p.tm_v, 0, h, base, mbar_v);
         }
-        cp_async_commit();
         // the k/q tile is dead: start on the next unit of this CTA (its k/q tile, its tables), to be
         // consumed after the loop comes round
         if (next_ok) {
             issue_kq(nb, nhk, nbase, nT);
             load_tables(nb, nh, nbase, nT, (iter + 1) & 1);
         }
-        cp_async_commit();
         {
             const int i = zi;
             const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
@@ -1209,7 +1220,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
-        cp_async_wait_group1();   // the v rows have landed; the next unit's tile may still be in flight
+        if (tid == 0 && !mbar_wait_bounded(mbar_v, par)) *flag = 1;   // the v rows have landed
         __syncthreads();
         GDN_TRACE_MARK_U(unit, 9);
 
@@ -1236,8 +1247,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float r0 = bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[2 * e]));
-                    const float r1 = bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[2 * e + 1]));
+                    // nodes beyond the tree hold another tree's rows: their r is forced to an exact zero
+                    const float r0 = j0 + 2 * e < T ? bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[2 * e])) : 0.f;
+                    const float r1 = j0 + 2 * e + 1 < T
+                                         ? bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[2 * e + 1]))
+                                         : 0.f;
                     split_pack_bf16(r0, r1, hi[e], lo[e]);
                 }
 #pragma unroll
@@ -1253,7 +1267,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         __syncthreads();
         tc_fence_after();
         GDN_TRACE_MARK_U(unit, 10);
-        warm_l2_rows();
 
         // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
         if (tid == 0) {
@@ -1318,6 +1331,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         g_trace_buf[unit * 16 + 13] = (long long)gt;
     }
 #endif
+    ++done_units;
     if (*flag != 0) break;   // a bounded wait expired: stop, report, release
     }   // unit loop
 
@@ -1326,6 +1340,37 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
+}
+
+// Tiled TMA descriptor of a packed row tensor [n_rows][heads][128] bf16: boxes of `box_cols` x 1 head x 64 rows.
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return static_cast<EncodeTiledFn>(nullptr);
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+bool make_row_tensor_map(CUtensorMap *tm, const void *ptr, int n_rows, int heads, int box_cols, bool swizzle128)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)FV_D, (cuuint64_t)heads, (cuuint64_t)n_rows};
+    const cuuint64_t strides[2] = {(cuuint64_t)FV_D * 2, (cuuint64_t)heads * FV_D * 2};   // bytes, dims 1 and 2
+    const cuuint32_t box[3] = {(cuuint32_t)box_cols, 1u, (cuuint32_t)FV_T};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <typename TOut, bool FUSED, bool GROUPED>
@@ -1339,11 +1384,16 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
         verify_sm100_kernel<TOut, GROUPED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
     } else {
         // trees that fit one CTA: persistent CTAs, two per SM, pipelined across units
+        VerifyFastParams pt = p;
+        if (!make_row_tensor_map(&pt.tm_k, p.k, s.total_nodes, s.h_qk, 64, true) ||
+            !make_row_tensor_map(&pt.tm_q, p.q, s.total_nodes, s.h_qk, 64, true) ||
+            !make_row_tensor_map(&pt.tm_v, p.v, s.total_nodes, s.h_v, FV_D, false))
+            return cudaErrorNotSupported;
         cudaError_t e = cudaFuncSetAttribute(verify_sm100_persistent_kernel<TOut, FUSED>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
         if (e != cudaSuccess) return e;
         const int grid = p.n_units < p.prefetch_dist ? p.n_units : p.prefetch_dist;
-        verify_sm100_persistent_kernel<TOut, FUSED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
+        verify_sm100_persistent_kernel<TOut, FUSED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(pt);
     }
     return cudaGetLastError();
 }

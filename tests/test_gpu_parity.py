@@ -367,3 +367,27 @@ def test_fused_commit_with_extreme_decay_takes_the_plain_replay(tl):
     prev.g = synth.store(np.full(prev.g.shape, -9.0, np.float32), synth.BF16)   # alpha = e^-9 per step, A_12 ~ 1e-47
     new = synth.random_case(42, [synth.tree_star(5), synth.tree_star(5)], 1, 2, 128, 128, synth.BF16, synth.F32)
     _fused_case(tl, prev, new, "fused extreme decay")
+
+
+def test_rows_of_a_neighbouring_tree_never_leak(tl):
+    """The tensor-core path stages 64-row boxes, so a short tree's tile also holds rows of the next tree.  Poison
+    that neighbour with NaNs: the short tree's outputs and committed state must be unaffected."""
+    trees = [synth.tree_chain(10), synth.tree_star(12)]
+    w = synth.random_case(61, trees, 2, 4, 128, 128, synth.BF16, synth.F32,
+                          paths=[np.arange(4, dtype=np.int32), np.zeros(0, np.int32)])
+    clean = tl.oracle_verify(w)
+    nan16 = np.uint16(0x7FC0)
+    for name in ("q", "k", "v", "g", "beta"):
+        getattr(w, name)[10:] = nan16          # every row of the second tree
+    dc = tl.DeviceCase(w)
+    assert dc.verify() == 0 and dc.device_status() == 0
+    o = dc.o.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(o[:10]))
+    tl.assert_close_per_head(o[:10], clean[:10], np.array([0, 10]), "short tree next to a poisoned one")
+    assert dc.commit() == 0 and dc.device_status() == 0
+    assert bool(torch_isfinite(dc.S0[0]))
+
+
+def torch_isfinite(t):
+    import torch
+    return torch.isfinite(t).all()
