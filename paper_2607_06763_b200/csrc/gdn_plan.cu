@@ -26,6 +26,9 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     __shared__ uint8_t dfirst_s[GDN_GROUPED_MAX_NODES / GDN_GROUP_NODES + 1];   // depth of each group's first node
     // parent[] of this tree, staged once so that the root-path walks below run out of shared memory
     __shared__ int32_t par_s[GDN_MAX_TREE_NODES];
+    // The kernel behind this one may be launched early (programmatic stream serialization); it waits for
+    // this grid to finish before it reads anything written here.
+    asm volatile("griddepcontrol.launch_dependents;");
     const int b = blockIdx.x;
     const int lo = node_offsets[b], hi = node_offsets[b + 1];
     const int T = hi - lo;

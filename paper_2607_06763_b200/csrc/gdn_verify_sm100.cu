@@ -141,7 +141,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
                  : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_group1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+// 32-byte global accesses (one instruction per eight floats: half the load/store instructions of float4).
+__device__ __forceinline__ void ldg_v8(const float *p, float4 &a, float4 &b)
+{
+    asm volatile("ld.global.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w), "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w)
+                 : "l"(p)
+                 : "memory");
+}
+__device__ __forceinline__ void stg_v8(float *p, const float4 &a, const float4 &b)
+{
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(p), "f"(a.x), "f"(a.y), "f"(a.z), "f"(a.w), "f"(b.x), "f"(b.y), "f"(b.z), "f"(b.w)
+                 : "memory");
+}
 __device__ __forceinline__ void cp_async_wait_all()
 {
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
@@ -790,6 +803,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // Launched with programmatic stream serialization: everything above overlaps the tail of the kernel
+    // in front (the tree-metadata kernel); nothing below may run before that kernel's writes are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // unit -> (tree, head, first node, size); a unit whose tree was rejected or is empty is skipped
     auto decode = [&](int u, int &ub, int &uh, int &uhk, int &ubase, int &uT) -> bool {
@@ -896,12 +912,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         const float *S = p.S0 + (size_t)(b * p.h_v + h) * FV_D * FV_D;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float4 *src = reinterpret_cast<const float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+            const float *src = S + (size_t)(warp * 16 + i * 4 + r4) * FV_D + l8 * 8;
 #pragma unroll
-            for (int kh = 0; kh < 2; ++kh) {
-                x[i][kh * 2 + 0] = __ldg(src + kh * 16 + l8 * 2 + 0);
-                x[i][kh * 2 + 1] = __ldg(src + kh * 16 + l8 * 2 + 1);
-            }
+            for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
         }
     }
     // fused commit, step 1: this tree's accepted path of the previous step (ids and their parents)
@@ -1103,12 +1116,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            float4 *dst = reinterpret_cast<float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+            float *dst = S + (size_t)(warp * 16 + i * 4 + r4) * FV_D + l8 * 8;
 #pragma unroll
-            for (int kh = 0; kh < 2; ++kh) {
-                dst[kh * 16 + l8 * 2 + 0] = x[i][kh * 2 + 0];
-                dst[kh * 16 + l8 * 2 + 1] = x[i][kh * 2 + 1];
-            }
+            for (int kh = 0; kh < 2; ++kh) stg_v8(dst + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
         }
         }
         __syncthreads();   // the path rows sit where the state operand is about to be written
@@ -1393,7 +1403,17 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
         if (e != cudaSuccess) return e;
         const int grid = p.n_units < p.prefetch_dist ? p.n_units : p.prefetch_dist;
-        verify_sm100_persistent_kernel<TOut, FUSED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(pt);
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(FV_THREADS);
+        cfg.dynamicSmemBytes = SM_ALLOC;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, verify_sm100_persistent_kernel<TOut, FUSED>, pt);
     }
     return cudaGetLastError();
 }
