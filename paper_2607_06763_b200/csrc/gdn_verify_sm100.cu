@@ -140,7 +140,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
                  ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 // 32-byte global accesses (one instruction per eight floats: half the load/store instructions of float4).
 __device__ __forceinline__ void ldg_v8(const float *p, float4 &a, float4 &b)
 {
@@ -851,26 +850,52 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
     };
 
-    int b = 0, h = 0, hk = 0, base = 0, T = 0;
-    {
-        const bool ok0 = decode(blockIdx.x, b, h, hk, base, T);
-        if (ok0) {
-            issue_kq(b, hk, base, T);
-            load_tables(b, h, base, T, 0);
+    // G_i = sum of g along the root path (root first), a_i = exp(G_i), for the tables in buffer `tb`
+    auto path_decay = [&](int tb) {
+        if (tid >= 64 && tid < 64 + FV_T) {
+            float4 *gab_t = reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE);
+            const uint8_t *anc_t = smem + SM_ANC + tb * SM_TABLE_STRIDE;
+            const int i = tid - 64;
+            const int d = (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[i];
+            float G = 0.f;
+            for (int t = 0; t < d; ++t) G += gab_t[anc_t[i * FV_MD + t]].w;
+            gab_t[i].x = G;
+            gab_t[i].y = d ? expf(G) : 0.f;
         }
-        cp_async_commit();
+    };
+    // Gram = [k;q].k^T of the tile in the k/q operand area, into TMEM columns 192..255, which nothing else uses:
+    // issued by one thread as soon as the tile has landed, one unit ahead of its use.
+    auto issue_gram = [&](uint32_t kq_parity) {
+        if (tid == 0) {
+            if (!mbar_wait_bounded(mbar_kq, kq_parity)) *flag = 1;
+            tc_fence_after();
+            const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
+            constexpr uint32_t id = idesc_bf16(128, 64);   // B = the 64 k rows
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+                umma_bf16(tmem + 192, b_kq + adv, b_kq + adv, id, ks > 0);
+            }
+            umma_commit(mbar_g);
+        }
+    };
+
+    int b = 0, h = 0, hk = 0, base = 0, T = 0;
+    bool cur_ok = decode(blockIdx.x, b, h, hk, base, T);
+    if (cur_ok) {
+        issue_kq(b, hk, base, T);
+        load_tables(b, h, base, T, 0);
     }
-    // The two CTAs of an SM would otherwise march in step (same phases at the same time, nothing to overlap):
-    // the second half of the grid starts a little later.
-    if (blockIdx.x >= (gridDim.x + 1) / 2 && p.skew_ns > 0) {
-        const long long t0 = clock64();
-        while (clock64() - t0 < (long long)p.skew_ns * 2) __nanosleep(200);
+    __syncthreads();
+    if (cur_ok) {
+        path_decay(0);
+        issue_gram(0);
     }
 
     int done_units = 0;
 #pragma unroll 1
     for (int unit = blockIdx.x, iter = 0; unit < p.n_units; unit += gridDim.x, ++iter) {
-    const bool unit_ok = decode(unit, b, h, hk, base, T);
+    const bool unit_ok = cur_ok;
     const uint32_t par = (uint32_t)(done_units & 1);   // every barrier completes once per processed unit
     int nb = 0, nh = 0, nhk = 0, nbase = 0, nT = 0;
     const bool next_ok = decode(unit + gridDim.x, nb, nh, nhk, nbase, nT);
@@ -878,13 +903,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     uint8_t *anc_s = smem + SM_ANC + (iter & 1) * SM_TABLE_STRIDE;
     uint8_t *depth_s = smem + SM_DEPTH + (iter & 1) * SM_TABLE_STRIDE;
     if (!unit_ok) {   // nothing to compute here: only keep the pipeline fed
-        cp_async_wait_all();
         __syncthreads();
         if (next_ok) {
             issue_kq(nb, nhk, nbase, nT);
             load_tables(nb, nh, nbase, nT, (iter + 1) & 1);
         }
-        cp_async_commit();
+        __syncthreads();
+        if (next_ok) {
+            path_decay((iter + 1) & 1);
+            issue_gram(par);   // no unit was processed in between: the tile's barrier phase is this one
+        }
+        b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
         continue;
     }
     GDN_TRACE_MARK_U(unit, 0);
@@ -939,24 +968,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     }
     GDN_TRACE_MARK_U(unit, 1);
 
-    if (tid == 0 && !mbar_wait_bounded(mbar_kq, par)) *flag = 1;   // this unit's k/q tile has landed
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+    __syncthreads();   // the path entries fetched above are visible to the thread that checks them
     GDN_TRACE_MARK_U(unit, 2);
 
-    // (4) Everything that depends only on q, k, g, beta runs now, under the latency of the state loads:
-    // Gram = [k;q].k^T on the tensor core, G_i / a_i tables, then X and Y of Eq. 9.
-    if (tid == 0) {
-        const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
-        constexpr uint32_t id = idesc_bf16(128, 64);   // B = the 64 k rows
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-            umma_bf16(tmem + 128, b_kq + adv, b_kq + adv, id, ks > 0);
-        }
-        umma_commit(mbar_g);
-    }
     if constexpr (FUSED) {
         // step 2: the path must be a chain from a root inside the previous tree
         if (tid == 160 && path_len != 0) {
@@ -973,20 +987,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
     }
-    // G_i = sum of g along the root path (root first), a_i = exp(G_i)
-    if (tid >= 64 && tid < 64 + FV_T) {
-        const int i = tid - 64;
-        const int d = depth_s[i];
-        float G = 0.f;
-        for (int t = 0; t < d; ++t) G += gab[anc_s[i * FV_MD + t]].w;
-        gab[i].x = G;
-        gab[i].y = d ? expf(G) : 0.f;
-    }
-    // one thread polls the mbarrier (bounded: on expiry it flags the error and everybody falls through to
-    // the clean-up), the others sleep in the CTA barrier
-    if (tid == 0 && !mbar_wait_bounded(mbar_g, par)) *flag = 1;
-    __syncthreads();
+    // Everything that depends only on q, k, g, beta runs now, under the latency of the state loads.  The Gram
+    // block of this unit was issued one unit ahead; every thread waits for it on its own (bounded: on expiry it
+    // flags the error and everybody falls through to the clean-up).
+    if (!mbar_wait_bounded(mbar_g, par)) *flag = 1;
     tc_fence_after();
+    __syncthreads();
     GDN_TRACE_MARK_U(unit, 3);
     warm_l2_state(0);
     if constexpr (FUSED) {
@@ -1011,8 +1017,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
         {
             const int row = (warp & 3) * 32 + lane;
-            const int half = warp >> 2;   // TMEM columns 128 + 32*half .. : k_j for j = 32*half ..
-            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 128 + half * 32;
+            const int half = warp >> 2;   // TMEM columns 192 + 32*half .. : k_j for j = 32*half ..
+            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 192 + half * 32;
             uint32_t ra[32];
             GDN_TMEM_LD32(taddr, ra);
             tmem_wait_ld();
@@ -1277,6 +1283,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         __syncthreads();
         tc_fence_after();
         GDN_TRACE_MARK_U(unit, 10);
+        if (next_ok) path_decay((iter + 1) & 1);   // the next unit's decay tables, while the tensor core works
 
         // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
         if (tid == 0) {
@@ -1343,6 +1350,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 #endif
     ++done_units;
     if (*flag != 0) break;   // a bounded wait expired: stop, report, release
+    if (next_ok) issue_gram((uint32_t)(done_units & 1));   // the next unit's Gram block, as soon as its tile is there
+    b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
     }   // unit loop
 
     if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
