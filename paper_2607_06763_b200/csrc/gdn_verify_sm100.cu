@@ -51,10 +51,11 @@ constexpr int SM_Y = SM_X + 4096;                // fp32 [64][16]  Y(i, t-th pat
 constexpr int SM_ANC = SM_Y + 4096;              // u8   [64][16]  root-path node ids (0xFF = unused)
 constexpr int SM_GAB = SM_ANC + 1024;            // float4 [64]: (G_i = log a_i, a_i, beta_i, g_i)
 constexpr int SM_DEPTH = SM_GAB + 1024;          // u8 [64] (0 beyond T)
-constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit: int [16] node ids, int [16] parents, float2 [16] (alpha, beta)
+constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit, two slots of 256 B: int [16] path node ids, int length (0 = no
+                                                 // replay), int first node of the tree; at +128 float2 [16] (alpha, beta)
 constexpr int SM_PK = 32768;                     // fused commit: k rows of the accepted path, bf16 [16][128], parked in the
 constexpr int SM_PV = 36864;                     // state-operand area until the replay is over; v rows likewise
-constexpr int SM_VNODE = SM_PATH + 256;          // grouped mode: u16 [64] node id of virtual index u
+constexpr int SM_VNODE = SM_PATH + 512;          // grouped mode: u16 [64] node id of virtual index u
 constexpr int SM_TABLE2 = SM_VNODE + 128;        // persistent kernel: second copy of ANC / GAB / DEPTH (2112 B)
 constexpr int SM_TABLE_STRIDE = SM_TABLE2 - SM_ANC;   // table buffer tb lives SM_TABLE_STRIDE * tb further on
 constexpr int SM_MBAR = SM_TABLE2 + 2176;        // 5 x u64: Gram done, P done, D done, k/q tile landed, v tile landed
@@ -260,6 +261,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo_elem, float hi_elem)
 __device__ __forceinline__ uint32_t sw128_row_offset(int r, int c16)
 {
     return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c16 ^ (r & 7)) << 4));
+}
+
+// One lane of a converged warp (the branch around it stays warp-uniform, so that descriptors can live in
+// uniform registers).
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 
 // Bounded wait on an mbarrier phase; returns false if it expired.
@@ -801,7 +811,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
+    const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // warp-uniform by construction
     // Launched with programmatic stream serialization: everything above overlaps the tail of the kernel
     // in front (the tree-metadata kernel); nothing below may run before that kernel's writes are visible.
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -821,7 +831,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // (or are zero past the end of the tensor); every use of them is masked further down.
     auto issue_kq = [&](int ub, int uhk, int ubase, int uT) {
         (void)ub; (void)uT;
-        if (tid == 0) {
+        if (warp == 0 && elect_one()) {
             mbar_expect_tx(mbar_kq, 32768);
 #pragma unroll
             for (int kh = 0; kh < 2; ++kh) {
@@ -850,15 +860,82 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
     };
 
+    // Fused commit: the accepted path of tree `ub` in the previous step goes to path slot `ps`.  One warp
+    // fetches it (lane t: entry t and that node's parent) and checks with shuffles that it is a chain from a
+    // root inside the previous tree; a bad path is reported and its length stored as 0, so that this state
+    // stays as it was.  Readable by the other warps after the next CTA barrier.
+    auto fetch_path = [&](int ub, int ps) {
+        if constexpr (FUSED) {
+            if (warp == 4) {
+                int *slot = reinterpret_cast<int *>(smem + SM_PATH + ps * 256);
+                const int pp0 = p.path_offsets[ub];
+                int len = p.path_offsets[ub + 1] - pp0;   // 0 leaves the state alone
+                int pb = 0;
+                if (len != 0) {
+                    pb = p.pnode_offsets[ub];
+                    const int pT = p.pnode_offsets[ub + 1] - pb;
+                    const bool shape_ok = len > 0 && len <= FV_MD && pT > 0 && pp0 >= 0;
+                    const bool mine = shape_ok && lane < len;
+                    int n = -1, parent_n = -2;
+                    if (mine) {
+                        n = p.path[pp0 + lane];
+                        if (p.pparent && n >= 0 && n < pT) parent_n = p.pparent[pb + n];
+                        slot[lane] = n;
+                    }
+                    const int n_up = __shfl_up_sync(0xffffffffu, n, 1);
+                    bool bad = false;
+                    if (mine) {
+                        if (n < 0 || n >= pT) bad = true;
+                        else if (p.pparent) bad = parent_n != (lane ? n_up : -1);
+                        else if (lane && n <= n_up) bad = true;   // without parent[] only the topological order can be checked
+                    }
+                    if (__any_sync(0xffffffffu, bad) || !shape_ok) {
+                        if (lane == 0) report_status(p.status_dev, GDN_ERR_PATH);
+                        len = 0;
+                    }
+                }
+                if (lane == 0) {
+                    slot[16] = len;
+                    slot[17] = pb;
+                }
+            }
+        }
+    };
+    // k and v rows of that path (bf16, 256 B each) into their parking area and the per-step scalars into the
+    // slot: issued by everybody once the slot is readable and the parking area is free
+    auto fetch_path_rows = [&](int uh, int uhk, int ps, bool scalars) {
+        if constexpr (FUSED) {
+            const int *slot = reinterpret_cast<const int *>(smem + SM_PATH + ps * 256);
+            float2 *ab = reinterpret_cast<float2 *>(smem + SM_PATH + ps * 256 + 128);
+            const int len = slot[16], pb = slot[17];
+            for (int idx = tid; idx < len * 32; idx += FV_THREADS) {
+                const int t = idx >> 5, c16 = idx & 15;
+                const size_t n = (size_t)pb + slot[t];
+                if (idx & 16)
+                    cp_async_16(sbase + SM_PV + t * 256 + c16 * 16, p.pv + (n * p.h_v + uh) * FV_D + c16 * 8, true);
+                else
+                    cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + uhk) * FV_D + c16 * 8, true);
+            }
+            if (scalars && tid < len) {
+                const size_t n = (size_t)pb + slot[tid];
+                ab[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + uh])),
+                                      __bfloat162float(p.pbeta[n * p.h_v + uh]));
+            }
+        }
+    };
     // G_i = sum of g along the root path (root first), a_i = exp(G_i), for the tables in buffer `tb`
-    auto path_decay = [&](int tb) {
-        if (tid >= 64 && tid < 64 + FV_T) {
-            float4 *gab_t = reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE);
-            const uint8_t *anc_t = smem + SM_ANC + tb * SM_TABLE_STRIDE;
-            const int i = tid - 64;
-            const int d = (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[i];
-            float G = 0.f;
-            for (int t = 0; t < d; ++t) G += gab_t[anc_t[i * FV_MD + t]].w;
+    auto path_decay = [&](int tb) {   // four threads per node, four path positions each
+        float4 *gab_t = reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE);
+        const int i = tid >> 2, s4 = tid & 3;
+        const int d = (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[i];
+        const uint32_t ids = *reinterpret_cast<const uint32_t *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + i * FV_MD + s4 * 4);
+        float G = 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (s4 * 4 + e < d) G += gab_t[(ids >> (8 * e)) & 0xFFu].w;
+        G += __shfl_xor_sync(0xffffffffu, G, 1);
+        G += __shfl_xor_sync(0xffffffffu, G, 2);
+        if (s4 == 0) {
             gab_t[i].x = G;
             gab_t[i].y = d ? expf(G) : 0.f;
         }
@@ -866,7 +943,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // Gram = [k;q].k^T of the tile in the k/q operand area, into TMEM columns 192..255, which nothing else uses:
     // issued by one thread as soon as the tile has landed, one unit ahead of its use.
     auto issue_gram = [&](uint32_t kq_parity) {
-        if (tid == 0) {
+        if (warp == 0 && elect_one()) {
             if (!mbar_wait_bounded(mbar_kq, kq_parity)) *flag = 1;
             tc_fence_after();
             const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
@@ -885,10 +962,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (cur_ok) {
         issue_kq(b, hk, base, T);
         load_tables(b, h, base, T, 0);
+        fetch_path(b, 0);
     }
     __syncthreads();
     if (cur_ok) {
         path_decay(0);
+        fetch_path_rows(h, hk, 0, true);
         issue_gram(0);
     }
 
@@ -907,10 +986,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if (next_ok) {
             issue_kq(nb, nhk, nbase, nT);
             load_tables(nb, nh, nbase, nT, (iter + 1) & 1);
+            fetch_path(nb, (iter + 1) & 1);
         }
         __syncthreads();
         if (next_ok) {
             path_decay((iter + 1) & 1);
+            fetch_path_rows(nh, nhk, (iter + 1) & 1, true);
             issue_gram(par);   // no unit was processed in between: the tile's barrier phase is this one
         }
         b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
@@ -946,73 +1027,24 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
         }
     }
-    // fused commit, step 1: this tree's accepted path of the previous step (ids and their parents)
-    int *path_s = reinterpret_cast<int *>(smem + SM_PATH);
-    int *par_s = path_s + FV_MD;
-    float2 *ab_path = reinterpret_cast<float2 *>(smem + SM_PATH + 128);
-    int path_len = 0, pbase = 0, pT = 0;
-    bool path_shape_ok = true;
-    if constexpr (FUSED) {
-        const int pp0 = p.path_offsets[b];
-        path_len = p.path_offsets[b + 1] - pp0;   // uniform over the CTA; 0 leaves the state alone
-        if (path_len != 0) {
-            pbase = p.pnode_offsets[b];
-            pT = p.pnode_offsets[b + 1] - pbase;
-            path_shape_ok = path_len > 0 && path_len <= FV_MD && pT > 0 && pp0 >= 0;
-            if (path_shape_ok && tid >= 128 && tid - 128 < path_len) {
-                const int n = p.path[pp0 + tid - 128];
-                path_s[tid - 128] = n;
-                par_s[tid - 128] = (p.pparent && n >= 0 && n < pT) ? p.pparent[pbase + n] : -2;
-            }
-        }
-    }
+    // this tree's v rows are wanted in shared memory only after the first MMA group: ask L2 for them now
+    if (tid >= 192 && tid - 192 < T)
+        prefetch_l2_bulk(p.v + ((size_t)(base + tid - 192) * p.h_v + h) * FV_D, FV_D * 2);
+    // fused commit: this tree's accepted path of the previous step was fetched one unit ahead
+    const float2 *ab_path = reinterpret_cast<const float2 *>(smem + SM_PATH + (iter & 1) * 256 + 128);
+    int path_len = 0;
+    if constexpr (FUSED) path_len = reinterpret_cast<const int *>(smem + SM_PATH + (iter & 1) * 256)[16];
     GDN_TRACE_MARK_U(unit, 1);
 
-    __syncthreads();   // the path entries fetched above are visible to the thread that checks them
-    GDN_TRACE_MARK_U(unit, 2);
-
-    if constexpr (FUSED) {
-        // step 2: the path must be a chain from a root inside the previous tree
-        if (tid == 160 && path_len != 0) {
-            int bad = !path_shape_ok;
-            for (int t = 0; !bad && t < path_len; ++t) {
-                const int n = path_s[t];
-                if (n < 0 || n >= pT) bad = 1;
-                else if (p.pparent) bad = par_s[t] != (t ? path_s[t - 1] : -1);
-                else if (t && n <= path_s[t - 1]) bad = 1;
-            }
-            if (bad) {
-                report_status(p.status_dev, GDN_ERR_PATH);
-                path_s[0] = -1;   // tells everybody to skip the replay: this state stays as it was
-            }
-        }
-    }
     // Everything that depends only on q, k, g, beta runs now, under the latency of the state loads.  The Gram
     // block of this unit was issued one unit ahead; every thread waits for it on its own (bounded: on expiry it
     // flags the error and everybody falls through to the clean-up).
     if (!mbar_wait_bounded(mbar_g, par)) *flag = 1;
+    GDN_TRACE_MARK_U(unit, 2);
     tc_fence_after();
     __syncthreads();
     GDN_TRACE_MARK_U(unit, 3);
     warm_l2_state(0);
-    if constexpr (FUSED) {
-        // step 3: k and v rows of the path (bf16, 256 B each) and the per-step scalars
-        if (path_len > 0 && path_s[0] >= 0) {
-            for (int idx = tid; idx < path_len * 32; idx += FV_THREADS) {
-                const int t = idx >> 5, c16 = idx & 15;
-                const size_t n = (size_t)pbase + path_s[t];
-                if (idx & 16)
-                    cp_async_16(sbase + SM_PV + t * 256 + c16 * 16, p.pv + (n * p.h_v + h) * FV_D + c16 * 8, true);
-                else
-                    cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + hk) * FV_D + c16 * 8, true);
-            }
-            if (tid < path_len) {
-                const size_t n = (size_t)pbase + path_s[tid];
-                ab_path[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + h])),
-                                           __bfloat162float(p.pbeta[n * p.h_v + h]));
-            }
-        }
-    }
     if (*flag == 0) {
         // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
         {
@@ -1068,7 +1100,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // Per row c (one value component): s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that
     // share a row reduce k.s_c with three shuffles.  The path's k/v rows were fetched above.
     if constexpr (FUSED) {
-        if (path_len > 0 && path_s[0] >= 0) {
+        if (path_len > 0) {
             const int L = path_len;
         const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
         const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
@@ -1152,9 +1184,35 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     tc_fence_after();
     GDN_TRACE_MARK_U(unit, 6);
     warm_l2_state(2);
+    // The next unit's tables and accepted path are fetched in stages, each load issued one phase before its
+    // value is used, so that no global-memory latency is paid in front of a barrier.
+    // stage 1: table entries of node `tid` and the path bounds (registers only)
+    int t_depth = 0;
+    uint4 t_row = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+    unsigned short t_g = 0, t_be = 0;
+    int q_pp0 = 0, q_len = 0, q_pb = 0, q_pT = 0, q_n = -1, q_par = -2;
+    unsigned short q_g = 0, q_be = 0;
+    bool q_shape_ok = false, q_mine = false;
+    if (next_ok) {
+        if (tid < nT) {
+            const int n = nbase + tid;
+            t_depth = p.depth[n];
+            t_row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)n * 16));
+            t_g = __ldg(reinterpret_cast<const unsigned short *>(p.g) + (size_t)n * p.h_v + nh);
+            t_be = __ldg(reinterpret_cast<const unsigned short *>(p.beta) + (size_t)n * p.h_v + nh);
+        }
+        if constexpr (FUSED) {
+            if (warp == 4) {
+                q_pp0 = p.path_offsets[nb];
+                q_len = p.path_offsets[nb + 1];
+                q_pb = p.pnode_offsets[nb];
+                q_pT = p.pnode_offsets[nb + 1];
+            }
+        }
+    }
 
     // (5) P = S0.[k;q]^T (hi then lo) on the tensor core; meanwhile the back-substitution below
-    if (tid == 0) {
+    if (warp == 0 && elect_one()) {
         const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
         const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
         constexpr uint32_t id = idesc_bf16(128, 128);
@@ -1195,6 +1253,16 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
     GDN_TRACE_MARK_U(unit, 7);
+    // stage 2: the path entries
+    if constexpr (FUSED) {
+        if (next_ok && warp == 4) {
+            q_len -= q_pp0;
+            q_pT -= q_pb;
+            q_shape_ok = q_len > 0 && q_len <= FV_MD && q_pT > 0 && q_pp0 >= 0;
+            q_mine = q_shape_ok && lane < q_len;
+            if (q_mine) q_n = p.path[q_pp0 + lane];
+        }
+    }
     if (tid == 0 && !mbar_wait_bounded(mbar_p, par)) *flag = 1;
     __syncthreads();
     tc_fence_after();
@@ -1205,7 +1273,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (ok) {
         // (7) both operand tiles are dead now: the tree's v rows go over the state operand, and z is
         // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path) over the k/q tile
-        if (tid == 0) {
+        if (warp == 0 && elect_one()) {
             mbar_expect_tx(mbar_v, FV_T * FV_D * 2);
             tma_load_3d(sbase + SM_V, &p.tm_v, 0, h, base, mbar_v);
         }
@@ -1213,7 +1281,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         // consumed after the loop comes round
         if (next_ok) {
             issue_kq(nb, nhk, nbase, nT);
-            load_tables(nb, nh, nbase, nT, (iter + 1) & 1);
+            // stage 3: the table entries go to the other table buffer; the parents of the path entries are asked for
+            if (tid < FV_T) {
+                const int tb = (iter + 1) & 1;
+                (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[tid] = (uint8_t)t_depth;
+                *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + tid * 16) = t_row;
+                reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[tid] =
+                    make_float4(0.f, 0.f, __uint_as_float((uint32_t)t_be << 16), __uint_as_float((uint32_t)t_g << 16));
+            }
+            if constexpr (FUSED) {
+                if (warp == 4 && q_mine && p.pparent && q_n >= 0 && q_n < q_pT) q_par = p.pparent[q_pb + q_n];
+            }
         }
         {
             const int i = zi;
@@ -1239,6 +1317,34 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if (tid == 0 && !mbar_wait_bounded(mbar_v, par)) *flag = 1;   // the v rows have landed
         __syncthreads();
         GDN_TRACE_MARK_U(unit, 9);
+        // stage 4: the path is checked (a chain from a root inside the previous tree) and published; the
+        // per-step scalars of its nodes are asked for
+        if constexpr (FUSED) {
+            if (next_ok && warp == 4) {
+                int *slot = reinterpret_cast<int *>(smem + SM_PATH + ((iter + 1) & 1) * 256);
+                const int n_up = __shfl_up_sync(0xffffffffu, q_n, 1);
+                bool bad = false;
+                if (q_mine) {
+                    slot[lane] = q_n;
+                    if (q_n < 0 || q_n >= q_pT) bad = true;
+                    else if (p.pparent) bad = q_par != (lane ? n_up : -1);
+                    else if (lane && q_n <= n_up) bad = true;
+                }
+                if (q_len != 0 && (__any_sync(0xffffffffu, bad) || !q_shape_ok)) {
+                    if (lane == 0) report_status(p.status_dev, GDN_ERR_PATH);
+                    q_len = 0;
+                }
+                if (lane == 0) {
+                    slot[16] = q_len;
+                    slot[17] = q_pb;
+                }
+                if (lane < q_len) {
+                    const size_t n = (size_t)q_pb + q_n;
+                    q_g = __ldg(reinterpret_cast<const unsigned short *>(p.pg) + n * p.h_v + nh);
+                    q_be = __ldg(reinterpret_cast<const unsigned short *>(p.pbeta) + n * p.h_v + nh);
+                }
+            }
+        }
 
         // (8) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
         // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
@@ -1283,10 +1389,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         __syncthreads();
         tc_fence_after();
         GDN_TRACE_MARK_U(unit, 10);
-        if (next_ok) path_decay((iter + 1) & 1);   // the next unit's decay tables, while the tensor core works
 
         // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
-        if (tid == 0) {
+        if (warp == 0 && elect_one()) {
             constexpr uint32_t id2 = idesc_bf16(128, 64);
             const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
             const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
@@ -1298,6 +1403,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                               (combo | ks) != 0);
             }
             umma_commit(mbar_d);
+        }
+        // stage 5, while the tensor core works: the next unit's decay tables, its path rows (the v rows they
+        // land on are dead) and the scalars of the path
+        if (next_ok) {
+            path_decay((iter + 1) & 1);
+            fetch_path_rows(nh, nhk, (iter + 1) & 1, false);
+            if constexpr (FUSED) {
+                if (warp == 4 && lane < q_len)
+                    reinterpret_cast<float2 *>(smem + SM_PATH + ((iter + 1) & 1) * 256 + 128)[lane] =
+                        make_float2(expf(__uint_as_float((uint32_t)q_g << 16)), __uint_as_float((uint32_t)q_be << 16));
+            }
         }
         if (tid == 0 && !mbar_wait_bounded(mbar_d, par)) *flag = 1;
         __syncthreads();
