@@ -1263,14 +1263,15 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             if (q_mine) q_n = p.path[q_pp0 + lane];
         }
     }
-    if (tid == 0 && !mbar_wait_bounded(mbar_p, par)) *flag = 1;
-    __syncthreads();
+    bool unit_done_ok = false;
+    // From here to the output staging every thread waits on the barriers of the tensor core and of TMA itself;
+    // an expired wait only raises the flag, which is looked at behind the next CTA barrier (uniform decision).
+    if (!mbar_wait_bounded(mbar_p, par)) *flag = 1;
     tc_fence_after();
-    bool ok = *flag == 0;
     GDN_TRACE_MARK_U(unit, 8);
     warm_l2_state(3);
 
-    if (ok) {
+    {
         // (7) both operand tiles are dead now: the tree's v rows go over the state operand, and z is
         // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path) over the k/q tile
         if (warp == 0 && elect_one()) {
@@ -1314,8 +1315,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
-        if (tid == 0 && !mbar_wait_bounded(mbar_v, par)) *flag = 1;   // the v rows have landed
-        __syncthreads();
+        if (!mbar_wait_bounded(mbar_v, par)) *flag = 1;   // the v rows have landed
         GDN_TRACE_MARK_U(unit, 9);
         // stage 4: the path is checked (a chain from a root inside the previous tree) and published; the
         // per-step scalars of its nodes are asked for
@@ -1415,15 +1415,13 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                         make_float2(expf(__uint_as_float((uint32_t)q_g << 16)), __uint_as_float((uint32_t)q_be << 16));
             }
         }
-        if (tid == 0 && !mbar_wait_bounded(mbar_d, par)) *flag = 1;
-        __syncthreads();
+        if (!mbar_wait_bounded(mbar_d, par)) *flag = 1;
         tc_fence_after();
-        ok = *flag == 0;
         GDN_TRACE_MARK_U(unit, 11);
 
         // (10) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i]), staged through shared memory (over the
         // dead R^T tiles) so that global memory sees 16-byte stores of whole rows
-        if (ok) {
+        {
             const int c = (warp & 3) * 32 + lane;
             const int half = warp >> 2;
             const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
@@ -1446,7 +1444,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
         __syncthreads();
-        if (*flag == 0) {
+        unit_done_ok = *flag == 0;
+        if (unit_done_ok) {
             constexpr int ROW_CHUNKS = FV_D * (int)sizeof(TOut) / 16;   // 16-byte pieces per output row
             uint8_t *o = static_cast<uint8_t *>(p.o);
             for (int idx = tid; idx < T * ROW_CHUNKS; idx += FV_THREADS) {
@@ -1465,7 +1464,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     }
 #endif
     ++done_units;
-    if (*flag != 0) break;   // a bounded wait expired: stop, report, release
+    if (!unit_done_ok) break;   // a bounded wait expired: stop, report, release
     if (next_ok) issue_gram((uint32_t)(done_units & 1));   // the next unit's Gram block, as soon as its tile is there
     b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
     }   // unit loop
