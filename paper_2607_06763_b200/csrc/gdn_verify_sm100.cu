@@ -1150,24 +1150,25 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
-        // the committed state: the only state write of the step
-        float *S = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float *dst = S + (size_t)(warp * 16 + i * 4 + r4) * FV_D + l8 * 8;
-#pragma unroll
-            for (int kh = 0; kh < 2; ++kh) stg_v8(dst + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
-        }
         }
         __syncthreads();   // the path rows sit where the state operand is about to be written
     }
 
-    // (4) fp32 -> bf16 hi + lo, written as the A operand
+    // (4) fp32 -> bf16 hi + lo, written as the A operand.  FUSED: the committed state -- the only state write of
+    // the step -- goes out from the same registers, one 32-byte store in front of each piece's conversion so
+    // that the stores drain while the arithmetic runs.
+    float *S_out = nullptr;
+    if constexpr (FUSED) {
+        if (path_len > 0) S_out = p.S_rw + (size_t)(b * p.h_v + h) * FV_D * FV_D;
+    }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int row = warp * 16 + i * 4 + r4;
 #pragma unroll
         for (int kh = 0; kh < 2; ++kh) {
+            if constexpr (FUSED) {
+                if (S_out) stg_v8(S_out + (size_t)row * FV_D + l8 * 8 + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
+            }
             const float4 u = x[i][kh * 2 + 0], w = x[i][kh * 2 + 1];
             const float f[8] = {u.x, u.y, u.z, u.w, w.x, w.y, w.z, w.w};
             uint32_t hi[4], lo[4];
