@@ -44,6 +44,8 @@ constexpr int SM_GRAM = 0;                       // fp32 [128][64], column j of 
 constexpr int SM_RT_HI = 0;                      // then R^T hi: [128 rows = components][64 nodes] bf16, swizzled
 constexpr int SM_RT_LO = 16384;                  //      R^T lo
 constexpr int SM_V = 32768;                      // v rows of the tree, bf16 [64][128]
+constexpr int SM_VE = 40960;                     // persistent kernel: the v rows land here at the top of a unit (free until
+                                                 // the state operand is written) and move into registers before that
 constexpr int SM_Z_HI = 49152;                   // Z hi: [64 rows = nodes i][64 nodes j] bf16, swizzled
 constexpr int SM_Z_LO = 57344;                   // Z lo
 constexpr int SM_X = 98304;                      // fp32 [64][16]  X(i, t-th path node)
@@ -791,7 +793,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     float *xs = reinterpret_cast<float *>(smem + SM_X);
     float *ys = reinterpret_cast<float *>(smem + SM_Y);
     float *gram = reinterpret_cast<float *>(smem + SM_GRAM);
-    const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(smem + SM_V);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM_TMEM);
     volatile uint32_t *flag = reinterpret_cast<volatile uint32_t *>(smem + SM_FLAG);
     const uint32_t mbar_g = sbase + SM_MBAR, mbar_p = mbar_g + 8, mbar_d = mbar_g + 16;
@@ -1027,9 +1028,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
         }
     }
-    // this tree's v rows are wanted in shared memory only after the first MMA group: ask L2 for them now
-    if (tid >= 192 && tid - 192 < T)
-        prefetch_l2_bulk(p.v + ((size_t)(base + tid - 192) * p.h_v + h) * FV_D, FV_D * 2);
+    // this tree's v rows: one TMA box into an area that stays free until the state operand is written
+    if (warp == 0 && elect_one()) {
+        mbar_expect_tx(mbar_v, FV_T * FV_D * 2);
+        tma_load_3d(sbase + SM_VE, &p.tm_v, 0, h, base, mbar_v);
+    }
     // fused commit: this tree's accepted path of the previous step was fetched one unit ahead
     const float2 *ab_path = reinterpret_cast<const float2 *>(smem + SM_PATH + (iter & 1) * 256 + 128);
     int path_len = 0;
@@ -1151,8 +1154,19 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
         }
-        __syncthreads();   // the path rows sit where the state operand is about to be written
     }
+    // The v rows move into registers in the orientation of the R phase (component c = TMEM lane of this
+    // thread, its 32 nodes, two bf16 per register): they are about to be overwritten by the state operand.
+    uint32_t vreg[16];
+    {
+        if (!mbar_wait_bounded(mbar_v, par)) *flag = 1;
+        const uint16_t *ve = reinterpret_cast<const uint16_t *>(smem + SM_VE) + ((warp >> 2) * 32) * FV_D +
+                             (warp & 3) * 32 + lane;
+#pragma unroll
+        for (int m = 0; m < 16; ++m)
+            vreg[m] = (uint32_t)ve[(2 * m) * FV_D] | ((uint32_t)ve[(2 * m + 1) * FV_D] << 16);
+    }
+    __syncthreads();   // the v rows and (FUSED) the path rows sit where the state operand is about to be written
 
     // (4) fp32 -> bf16 hi + lo, written as the A operand.  FUSED: the committed state -- the only state write of
     // the step -- goes out from the same registers, one 32-byte store in front of each piece's conversion so
@@ -1273,12 +1287,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     warm_l2_state(3);
 
     {
-        // (7) both operand tiles are dead now: the tree's v rows go over the state operand, and z is
-        // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path) over the k/q tile
-        if (warp == 0 && elect_one()) {
-            mbar_expect_tx(mbar_v, FV_T * FV_D * 2);
-            tma_load_3d(sbase + SM_V, &p.tm_v, 0, h, base, mbar_v);
-        }
+        // (7) both operand tiles are dead now: z is scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off
+        // the root path) over the state operand
         // the k/q tile is dead: start on the next unit of this CTA (its k/q tile, its tables), to be
         // consumed after the loop comes round
         if (next_ok) {
@@ -1316,8 +1326,50 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
-        if (!mbar_wait_bounded(mbar_v, par)) *flag = 1;   // the v rows have landed
         GDN_TRACE_MARK_U(unit, 9);
+
+        // (8) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
+        // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
+        {
+            const int c = (warp & 3) * 32 + lane;
+            const int half = warp >> 2;
+            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+#pragma unroll 1
+            for (int part = 0; part < 2; ++part) {
+                const int j0 = half * 32 + part * 16;
+                uint32_t rr[16];
+                GDN_TMEM_LD16(taddr + j0, rr);   // columns j0 .. j0+15: p^k of 16 nodes
+                float vv[16], aj[16], bj[16];
+                uint32_t vpart[8];
+#pragma unroll
+                for (int m = 0; m < 8; ++m) vpart[m] = part ? vreg[8 + m] : vreg[m];
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) {
+                    const uint32_t vw = vpart[jj >> 1];
+                    vv[jj] = __uint_as_float((jj & 1) ? (vw & 0xFFFF0000u) : (vw << 16));
+                    const float4 gj = gab[j0 + jj];
+                    aj[jj] = gj.y;
+                    bj[jj] = gj.z;
+                }
+                tmem_wait_ld();
+                uint32_t hi[8], lo[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    // nodes beyond the tree hold another tree's rows: their r is forced to an exact zero
+                    const float r0 = j0 + 2 * e < T ? bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[2 * e])) : 0.f;
+                    const float r1 = j0 + 2 * e + 1 < T
+                                         ? bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[2 * e + 1]))
+                                         : 0.f;
+                    split_pack_bf16(r0, r1, hi[e], lo[e]);
+                }
+#pragma unroll
+                for (int oct = 0; oct < 2; ++oct) {
+                    const uint32_t off = sw128_row_offset(c, half * 4 + part * 2 + oct);
+                    *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = make_uint4(hi[4 * oct], hi[4 * oct + 1], hi[4 * oct + 2], hi[4 * oct + 3]);
+                    *reinterpret_cast<uint4 *>(smem + SM_RT_LO + off) = make_uint4(lo[4 * oct], lo[4 * oct + 1], lo[4 * oct + 2], lo[4 * oct + 3]);
+                }
+            }
+        }
         // stage 4: the path is checked (a chain from a root inside the previous tree) and published; the
         // per-step scalars of its nodes are asked for
         if constexpr (FUSED) {
@@ -1347,44 +1399,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
 
-        // (8) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
-        // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
-        {
-            const int c = (warp & 3) * 32 + lane;
-            const int half = warp >> 2;
-            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-#pragma unroll 1
-            for (int part = 0; part < 2; ++part) {
-                const int j0 = half * 32 + part * 16;
-                uint32_t rr[16];
-                GDN_TMEM_LD16(taddr + j0, rr);   // columns j0 .. j0+15: p^k of 16 nodes
-                float vv[16], aj[16], bj[16];
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) {
-                    vv[jj] = __bfloat162float(vs[(j0 + jj) * FV_D + c]);
-                    const float4 gj = gab[j0 + jj];
-                    aj[jj] = gj.y;
-                    bj[jj] = gj.z;
-                }
-                tmem_wait_ld();
-                uint32_t hi[8], lo[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    // nodes beyond the tree hold another tree's rows: their r is forced to an exact zero
-                    const float r0 = j0 + 2 * e < T ? bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[2 * e])) : 0.f;
-                    const float r1 = j0 + 2 * e + 1 < T
-                                         ? bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[2 * e + 1]))
-                                         : 0.f;
-                    split_pack_bf16(r0, r1, hi[e], lo[e]);
-                }
-#pragma unroll
-                for (int oct = 0; oct < 2; ++oct) {
-                    const uint32_t off = sw128_row_offset(c, half * 4 + part * 2 + oct);
-                    *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = make_uint4(hi[4 * oct], hi[4 * oct + 1], hi[4 * oct + 2], hi[4 * oct + 3]);
-                    *reinterpret_cast<uint4 *>(smem + SM_RT_LO + off) = make_uint4(lo[4 * oct], lo[4 * oct + 1], lo[4 * oct + 2], lo[4 * oct + 3]);
-                }
-            }
-        }
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
@@ -1410,11 +1424,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if (next_ok) {
             path_decay((iter + 1) & 1);
             fetch_path_rows(nh, nhk, (iter + 1) & 1, false);
-            if constexpr (FUSED) {
-                if (warp == 4 && lane < q_len)
-                    reinterpret_cast<float2 *>(smem + SM_PATH + ((iter + 1) & 1) * 256 + 128)[lane] =
-                        make_float2(expf(__uint_as_float((uint32_t)q_g << 16)), __uint_as_float((uint32_t)q_be << 16));
-            }
         }
         if (!mbar_wait_bounded(mbar_d, par)) *flag = 1;
         tc_fence_after();
@@ -1445,6 +1454,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
         __syncthreads();
+        if constexpr (FUSED) {   // stage 6: the scalars of the next unit's path (asked for two phases ago)
+            if (next_ok && warp == 4 && lane < q_len)
+                reinterpret_cast<float2 *>(smem + SM_PATH + ((iter + 1) & 1) * 256 + 128)[lane] =
+                    make_float2(expf(__uint_as_float((uint32_t)q_g << 16)), __uint_as_float((uint32_t)q_be << 16));
+        }
         unit_done_ok = *flag == 0;
         if (unit_done_ok) {
             constexpr int ROW_CHUNKS = FV_D * (int)sizeof(TOut) / 16;   // 16-byte pieces per output row
