@@ -1,26 +1,27 @@
-// Tree-verify fast path for sm_100a: d_k = d_v = 128, bf16 inputs, root paths of at most 16 nodes,
-// trees of at most 64 nodes per CTA (larger trees are cut into ancestor-closed groups, one CTA each).  It evaluates the triangular form of Section 3.4.1 (Eq. 9-11)
-// restricted to real ancestors, with the W S0 term folded into the right-hand side as in
-// Section 3.4.2, and turns all of the per-component work into two dense contractions on the
+// Tree-verify fast path for sm_100a: d_k = d_v = 128, bf16 inputs, root paths of at most 16 nodes, trees of at
+// most 64 nodes per CTA (larger trees are cut into ancestor-closed groups, one CTA each).  It evaluates the
+// triangular form of Section 3.4.1 (Eq. 9-11) restricted to real ancestors, with the W S0 term folded into the
+// right-hand side as in Section 3.4.2, and turns all of the per-component work into dense contractions on the
 // 5th-generation tensor cores (tcgen05.mma, bf16 operands, fp32 accumulators in tensor memory):
 //
-//   (1) P [d_v x 2T] = S0 [d_v x d_k] . [k_0;q_0;k_1;q_1;...]^T      the S0 projections of Eq. 11 / Eq. 13
-//       Gr [2T x 2T] = [k;q rows] . [k;q rows]^T                     k_i.k_j and q_i.k_j of Eq. 9
-//   (2) D [d_v x T]  = R^T [d_v x T] . Z^T [T x T]                   the whole masked solve + output
+//   (1) P  [d_v x 2T] = S0 [d_v x d_k] . [k rows; q rows]^T          the S0 projections of Eq. 11 / Eq. 13
+//       Gr [2T x T]   = [k rows; q rows] . [k rows]^T                k_i.k_j and q_i.k_j of Eq. 9
+//   (2) D  [d_v x T]  = R^T [d_v x T] . Z^T [T x T]                  the whole masked solve + output
 //
 // where r_j = beta_j (v_j - a_j S0^T k_j) is the folded right-hand side and row i of Z is
-// z_i^T = y_i^T (I + X_path(i))^-1: because the ancestors of a node form a chain, the inverse
-// restricted to one root path is a back-substitution with at most 16 unknowns that each node
-// can run on its own (one thread per node, no dependence between nodes).  Then
+// z_i^T = y_i^T (I + X_path(i))^-1: because the ancestors of a node form a chain, the inverse restricted to one
+// root path is a back-substitution with at most 16 unknowns that each node can run on its own (four threads per
+// node, no dependence between nodes).  Then
 //   o_i = scale (a_i S0^T q_i + sum_{j on the root path of i} Z_ij r_j),
 // which is Eq. 11 with U - W S0 eliminated; no per-component sequential substitution is left.
-// fp32 quantities that feed the tensor cores are split into two bf16 terms (x = hi + lo,
-// |x - hi - lo| <= 2^-16 |x|): S0 for (1), R and Z for (2), all four cross terms accumulated.
+// fp32 quantities that feed the tensor cores are split into two bf16 terms (x = hi + lo, |x - hi - lo| <= 2^-16 |x|):
+// S0 for (1), R and Z for (2); the lo.lo term of (2) is dropped.
 //
-// Operand orientation: d_v on the TMEM lanes, nodes on the TMEM columns, so every thread of a
-// warp owns one value component.  One CTA per (tree, value head), 256 threads, about 106 KB of
-// shared memory and 256 TMEM columns, so two CTAs share an SM: while one streams its 64 KB
-// state tile from HBM the other computes.
+// Operand orientation: d_v on the TMEM lanes, nodes on the TMEM columns, so every thread of a warp owns one value
+// component.  256 threads, about 112 KB of shared memory and 256 TMEM columns per CTA, so two CTAs share an SM.
+// Two kernels: a persistent one for trees that fit one CTA (TMA tiles on mbarriers, a software pipeline across
+// the units of a CTA, optionally the commit of the previous step fused in front), and a one-shot one for the
+// groups of larger trees (row gathers through a node table).
 #include <cuda.h>   // CUtensorMap and the cuTensorMapEncodeTiled prototype (resolved at run time, no libcuda link)
 
 #include "gdn_internal.cuh"
@@ -33,12 +34,14 @@ constexpr int FV_THREADS = 256;
 constexpr int FV_D = 128;           // d_k = d_v
 constexpr int FV_T = 64;            // max nodes per tree
 constexpr int FV_MD = 16;           // max nodes on a root path
-constexpr int FV_TMEM_COLS = 256;   // P: columns [0,128) (2i: k_i, 2i+1: q_i); Gram: [128,256), later D: [128,192)
+constexpr int FV_TMEM_COLS = 256;   // P: columns [0,128); D (one-shot kernel: first the Gram block): [128,192);
+                                    // persistent kernel: Gram block of the unit to come in [192,256)
 
 // shared memory map (bytes from a 1024-byte aligned base)
 constexpr int SM_A_HI = 0;                       // S0 hi: [2][128 rows][128 B], 128B-swizzled, K-major
 constexpr int SM_A_LO = 32768;                   // S0 lo
-constexpr int SM_B_KQ = 65536;                   // row 2i = k of node i, row 2i+1 = q of node i; same layout
+constexpr int SM_B_KQ = 65536;                   // k and q rows, same layout (one-shot kernel: row 2i = k_i, 2i+1 = q_i;
+                                                 // persistent kernel: rows 0..63 = k, 64..127 = q)
 // after the first MMA group the operand tiles are dead and are reused:
 constexpr int SM_GRAM = 0;                       // fp32 [128][64], column j of row r stored at j ^ (r & 31)
 constexpr int SM_RT_HI = 0;                      // then R^T hi: [128 rows = components][64 nodes] bf16, swizzled
@@ -773,17 +776,19 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
 }
 
-// Persistent form of the kernel above for trees that fit one CTA, with the optional fused commit
-// In this kernel the k/q tile holds the k rows first and the q rows second (rows i and 64 + i), so P has
-// p^k in columns 0..63 and p^q in columns 64..127, and the Gram block needs only N = 64.
-// (FUSED: Eq. 7 replayed along the previous step's accepted path on the state tile while it sits in
-// registers -- per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c), the eight lanes that share a row
-// reducing k.s_c with three shuffles -- written back as the only state write of the step, and the new tree
-// verified against it): a CTA keeps its tensor memory and walks over
-// the units blockIdx.x, blockIdx.x + gridDim.x, ...  While it finishes one unit (R, second GEMM, outputs) the
-// next unit's k/q tile streams into the freed operand tile and its per-node tables into the other table buffer,
-// so that a unit starts on the tensor core at once; the state tile is asked for at the top of the unit and is
-// only needed after the Gram / coefficient phases.
+// Persistent form of the kernel above for trees that fit one CTA, with the optional fused commit.  The k/q tile
+// holds the k rows first and the q rows second (rows i and 64 + i), so P has p^k in columns 0..63 and p^q in
+// columns 64..127, and the Gram block needs only N = 64.
+// FUSED: Eq. 7 is replayed along the previous step's accepted path on the state tile while it sits in registers
+// -- per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c), the eight lanes that share a row reducing k.s_c with
+// three shuffles -- the tile is written back as the only state write of the step, and the new tree is verified
+// against it.
+// A CTA keeps its tensor memory and walks over the units blockIdx.x, blockIdx.x + gridDim.x, ...  Nothing a unit
+// can know in advance is waited for inside it: the next unit's k/q tile streams into the operand tile as soon as the
+// first MMA group has released it, its Gram block is issued at the end of the current unit into spare TMEM columns,
+// and its per-node tables, decay tables and accepted path are fetched in stages, each global load one phase before
+// its value is used.  The state tile is asked for at the top of the unit and is needed only after the Gram /
+// coefficient phases; the v rows land by TMA in an area that is free until the state operand is written.
 template <typename TOut, bool FUSED>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const __grid_constant__ VerifyFastParams p)
 {
