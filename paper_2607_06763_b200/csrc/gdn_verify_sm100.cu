@@ -1130,15 +1130,18 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             // the four rows of this thread advance together: four independent FMA chains, then their
             // shuffle reductions back to back, then the four updates
             float dot[4];
+            float2 kf2[8];   // the same values as packed pairs for the two-wide fp32 FMA
+#pragma unroll
+            for (int e = 0; e < 8; ++e) kf2[e] = make_float2(kf[2 * e], kf[2 * e + 1]);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                float d0 = 0.f, d1 = 0.f;
+                float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
-                    d0 = fmaf(kf[q4 * 4 + 0], x[i][q4].x, d0); d1 = fmaf(kf[q4 * 4 + 1], x[i][q4].y, d1);
-                    d0 = fmaf(kf[q4 * 4 + 2], x[i][q4].z, d0); d1 = fmaf(kf[q4 * 4 + 3], x[i][q4].w, d1);
+                    acc = __ffma2_rn(kf2[q4 * 2 + 0], make_float2(x[i][q4].x, x[i][q4].y), acc);
+                    acc = __ffma2_rn(kf2[q4 * 2 + 1], make_float2(x[i][q4].z, x[i][q4].w), acc);
                 }
-                dot[i] = d0 + d1;
+                dot[i] = acc.x + acc.y;
             }
 #pragma unroll
             for (int m = 1; m < 8; m <<= 1)
@@ -1149,12 +1152,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 const int row = warp * 16 + i * 4 + r4;
                 const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
                 const float w = ab.y * (vc - ab.x * dot[i]);
+                const float2 w2 = make_float2(w, w), a2 = make_float2(ab.x, ab.x);
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
-                    x[i][q4].x = fmaf(kf[q4 * 4 + 0], w, ab.x * x[i][q4].x);
-                    x[i][q4].y = fmaf(kf[q4 * 4 + 1], w, ab.x * x[i][q4].y);
-                    x[i][q4].z = fmaf(kf[q4 * 4 + 2], w, ab.x * x[i][q4].z);
-                    x[i][q4].w = fmaf(kf[q4 * 4 + 3], w, ab.x * x[i][q4].w);
+                    const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, __fmul2_rn(a2, make_float2(x[i][q4].x, x[i][q4].y)));
+                    const float2 hi = __ffma2_rn(kf2[q4 * 2 + 1], w2, __fmul2_rn(a2, make_float2(x[i][q4].z, x[i][q4].w)));
+                    x[i][q4] = make_float4(lo.x, lo.y, hi.x, hi.y);
                 }
             }
         }
