@@ -162,7 +162,8 @@ def run_reference(args, w: synth.Workload):
 
 def workload_config(w: synth.Workload, args):
     sizes = np.diff(w.node_offsets)
-    return {"workload": args.workload, "mode": getattr(args, "mode", "fused"), "name": w.name, "n_seq_or_layer_slots": w.n_seq, "h_qk": w.h_qk, "h_v": w.h_v,
+    return {"workload": args.workload, "mode": getattr(args, "mode", "fused"),
+            "launch": "cuda graph replay" if getattr(args, "graph", False) else "api call per step", "name": w.name, "n_seq_or_layer_slots": w.n_seq, "h_qk": w.h_qk, "h_v": w.h_v,
             "d_k": w.d_k, "d_v": w.d_v, "tree_nodes": int(sizes.max()), "total_nodes": w.total_nodes,
             "in_dtype": w.in_dtype, "state_dtype": "f32", "out_dtype": w.out_dtype,
             "accepted_path_len_mean": float(np.diff(w.path_offsets).mean()),
@@ -181,6 +182,8 @@ def main():
     ap.add_argument("--oracle-slots", type=int, default=48, help="layer slots / sequences in the oracle's sample")
     ap.add_argument("--mode", default="fused", choices=["fused", "separate"],
                     help="fused: one gdn_tree_commit_verify call per step; separate: gdn_tree_verify + gdn_tree_commit")
+    ap.add_argument("--graph", action="store_true",
+                    help="fused mode: capture one step per buffer set in a CUDA graph and time replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--layers", type=int, default=48, help="layer slots of the stack workloads (profiling: fewer)")
@@ -232,7 +235,7 @@ def main():
                                  d["path"], d["path_offsets"], status, stream)
         assert rc == 0, gdn.gdn_status_string(rc)
 
-    def step_fused(d):
+    def step_fused(d, stream=stream):
         # one decode iteration as the paper schedules it: commit the previous step's accepted path, then verify
         # the new tree against the advanced state (here the previous and the new tree carry the same tensors)
         rc = gdn.gdn_tree_commit_verify(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
@@ -251,6 +254,18 @@ def main():
     for i in range(args.warmup):
         step(sets[i % n_sets])
     barrier()
+    graphs = None
+    if args.graph and args.mode == "fused":
+        # one captured step per buffer set (the launches of a call, dependent-launch edge included)
+        graphs, side = [], torch.cuda.Stream()
+        for d in sets:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                step_fused(d, torch.cuda.current_stream())
+            graphs.append(g)
+        for i in range(args.warmup):
+            graphs[i % n_sets].replay()
+        barrier()
     assert int(status.item()) == 0, gdn.gdn_status_string(int(status.item()))
 
     # ---- timed region: K steps, device timing with events on the launching stream
@@ -267,7 +282,10 @@ def main():
         if args.mode == "fused":
             # nothing but the calls themselves inside the timed region: an event between two steps would
             # keep the next call's first kernel from being launched under the tail of this one
-            step_fused(d)
+            if graphs is not None:
+                graphs[(args.warmup + i) % n_sets].replay()
+            else:
+                step_fused(d)
             continue
         ev[i][0].record()
         rc = gdn.gdn_tree_verify(shape, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], d["parent"],

@@ -391,3 +391,60 @@ def test_rows_of_a_neighbouring_tree_never_leak(tl):
 def torch_isfinite(t):
     import torch
     return torch.isfinite(t).all()
+
+
+def test_calls_are_cuda_graph_capturable(tl):
+    """The library allocates nothing, never synchronises and launches only on the given stream, so a decode step
+    can be captured once and replayed (Section 3.4.2 runs the verify under CUDA graphs)."""
+    import torch
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(91)
+    prev_trees = [synth.tree_geo(rng, 64), synth.tree_geo(rng, 30)]
+    paths = [synth.longest_path(prev_trees[0]), synth.longest_path(prev_trees[1])]
+    prev = synth.random_case(92, prev_trees, 2, 4, 128, 128, synth.BF16, synth.BF16, paths=paths, name="prev")
+    new = synth.random_case(93, [synth.tree_geo(rng, 64), synth.tree_geo(rng, 50)], 2, 4, 128, 128, synth.BF16,
+                            synth.BF16, name="new")
+    dp, dn = tl.DeviceCase(prev), tl.DeviceCase(new)
+    S = dp.S0.clone()
+
+    def call(stream):
+        return gdn.gdn_tree_commit_verify(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets,
+                                          dp.path, dp.path_offsets, dn.q, dn.k, dn.v, dn.g, dn.beta, dn.parent,
+                                          dn.node_offsets, dn.o, dn.ws, dn.ws_bytes, dn.status, stream)
+
+    assert call(None) == 0 and dn.device_status() == 0   # eager once (also loads the kernels before the capture)
+    S_eager, o_eager = S.clone(), dn.o.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    S.copy_(dp.S0)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        rc = call(torch.cuda.current_stream())
+    assert rc == 0
+    for _ in range(2):   # the captured step replays on a restored state, bit for bit like the eager call
+        S.copy_(dp.S0)
+        dn.o.zero_()
+        graph.replay()
+        assert dn.device_status() == 0
+        assert bool((S == S_eager).all()) and bool((dn.o == o_eager).all())
+    S_ref = tl.oracle_commit(prev)
+    tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what="graph replay S_new")
+    from oracle import gdn_oracle as orc
+    o_ref = orc.verify(S_ref, new.f64("q"), new.f64("k"), new.f64("v"), new.f64("g"), new.f64("beta"), new.parent,
+                       new.node_offsets, new.scale)
+    tl.assert_close_per_head(dn.o_host(), o_ref, new.node_offsets, "graph replay o", bf16_out=True)
+    # the separate entry points under one capture as well
+    S2 = dn.S0.clone()
+    graph2 = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph2, stream=side):
+        st = torch.cuda.current_stream()
+        rc1 = dn.verify(stream=st)
+        rc2 = gdn.gdn_tree_commit(dn.shape, S2, dn.k, dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets, dn.path,
+                                  dn.path_offsets, dn.status, st)
+    assert rc1 == 0 and rc2 == 0
+    dn.o.zero_()
+    graph2.replay()
+    assert dn.device_status() == 0
+    tl.assert_close_per_head(dn.o_host(), tl.oracle_verify(new), new.node_offsets, "graph verify o", bf16_out=True)
+    tl.assert_state_close(S2.cpu().numpy().astype(np.float64), tl.oracle_commit(new), what="graph commit")
