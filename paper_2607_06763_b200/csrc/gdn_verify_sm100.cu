@@ -820,6 +820,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // warp-uniform by construction
     // Launched with programmatic stream serialization: everything above overlaps the tail of the kernel
     // in front (the tree-metadata kernel); nothing below may run before that kernel's writes are visible.
+    // The first unit's state tile is an input of the call, not of that kernel: L2 is asked for it meanwhile.
+    if (tid < 4 && (int)blockIdx.x < p.n_units)
+        prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // unit -> (tree, head, first node, size); a unit whose tree was rejected or is empty is skipped
