@@ -56,11 +56,13 @@ constexpr int SM_Y = SM_X + 4096;                // fp32 [64][16]  Y(i, t-th pat
 constexpr int SM_ANC = SM_Y + 4096;              // u8   [64][16]  root-path node ids (0xFF = unused)
 constexpr int SM_GAB = SM_ANC + 1024;            // float4 [64]: (G_i = log a_i, a_i, beta_i, g_i)
 constexpr int SM_DEPTH = SM_GAB + 1024;          // u8 [64] (0 beyond T)
-constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit, two slots of 256 B: int [16] path node ids, int length (0 = no
-                                                 // replay), int first node of the tree; at +128 float2 [16] (alpha, beta)
+constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit, two slots of 384 B: int [16] path node ids, int length (0 = no
+                                                 // replay), int first node of the tree; at +128 float4 [16] (A_t = decay of the
+                                                 // path up to and including step t, beta_t, alpha_t, 1 / A_t)
+constexpr int SM_PATH_SLOT = 384;
 constexpr int SM_PK = 32768;                     // fused commit: k rows of the accepted path, bf16 [16][128], parked in the
 constexpr int SM_PV = 36864;                     // state-operand area until the replay is over; v rows likewise
-constexpr int SM_VNODE = SM_PATH + 512;          // grouped mode: u16 [64] node id of virtual index u
+constexpr int SM_VNODE = SM_PATH + 2 * SM_PATH_SLOT;          // grouped mode: u16 [64] node id of virtual index u
 constexpr int SM_TABLE2 = SM_VNODE + 128;        // persistent kernel: second copy of ANC / GAB / DEPTH (2112 B)
 constexpr int SM_TABLE_STRIDE = SM_TABLE2 - SM_ANC;   // table buffer tb lives SM_TABLE_STRIDE * tb further on
 constexpr int SM_MBAR = SM_TABLE2 + 2176;        // 5 x u64: Gram done, P done, D done, k/q tile landed, v tile landed
@@ -876,7 +878,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     auto fetch_path = [&](int ub, int ps) {
         if constexpr (FUSED) {
             if (warp == 4) {
-                int *slot = reinterpret_cast<int *>(smem + SM_PATH + ps * 256);
+                int *slot = reinterpret_cast<int *>(smem + SM_PATH + ps * SM_PATH_SLOT);
                 const int pp0 = p.path_offsets[ub];
                 int len = p.path_offsets[ub + 1] - pp0;   // 0 leaves the state alone
                 int pb = 0;
@@ -914,8 +916,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // slot: issued by everybody once the slot is readable and the parking area is free
     auto fetch_path_rows = [&](int uh, int uhk, int ps, bool scalars) {
         if constexpr (FUSED) {
-            const int *slot = reinterpret_cast<const int *>(smem + SM_PATH + ps * 256);
-            float2 *ab = reinterpret_cast<float2 *>(smem + SM_PATH + ps * 256 + 128);
+            const int *slot = reinterpret_cast<const int *>(smem + SM_PATH + ps * SM_PATH_SLOT);
+            float4 *ab = reinterpret_cast<float4 *>(smem + SM_PATH + ps * SM_PATH_SLOT + 128);
             const int len = slot[16], pb = slot[17];
             for (int idx = tid; idx < len * 32; idx += FV_THREADS) {
                 const int t = idx >> 5, c16 = idx & 15;
@@ -926,9 +928,14 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                     cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + uhk) * FV_D + c16 * 8, true);
             }
             if (scalars && tid < len) {
+                float gsum = 0.f, gt = 0.f;
+                for (int t = 0; t <= tid; ++t) {
+                    gt = __bfloat162float(p.pg[((size_t)pb + slot[t]) * p.h_v + uh]);
+                    gsum += gt;
+                }
                 const size_t n = (size_t)pb + slot[tid];
-                ab[tid] = make_float2(expf(__bfloat162float(p.pg[n * p.h_v + uh])),
-                                      __bfloat162float(p.pbeta[n * p.h_v + uh]));
+                const float A = expf(gsum);
+                ab[tid] = make_float4(A, __bfloat162float(p.pbeta[n * p.h_v + uh]), expf(gt), 1.f / A);
             }
         }
     };
@@ -1042,9 +1049,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         tma_load_3d(sbase + SM_VE, &p.tm_v, 0, h, base, mbar_v);
     }
     // fused commit: this tree's accepted path of the previous step was fetched one unit ahead
-    const float2 *ab_path = reinterpret_cast<const float2 *>(smem + SM_PATH + (iter & 1) * 256 + 128);
+    const float4 *ab_path = reinterpret_cast<const float4 *>(smem + SM_PATH + (iter & 1) * SM_PATH_SLOT + 128);
     int path_len = 0;
-    if constexpr (FUSED) path_len = reinterpret_cast<const int *>(smem + SM_PATH + (iter & 1) * 256)[16];
+    if constexpr (FUSED) path_len = reinterpret_cast<const int *>(smem + SM_PATH + (iter & 1) * SM_PATH_SLOT)[16];
     GDN_TRACE_MARK_U(unit, 1);
 
     // Everything that depends only on q, k, g, beta runs now, under the latency of the state loads.  The Gram
@@ -1115,6 +1122,10 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             const int L = path_len;
         const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
         const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
+        // Scaled form: with A_t = alpha_1 .. alpha_t and s~ = s / A_t a step is s~ += k beta_t (v / A_t - k.s~)
+        // (the decay costs nothing), and s = A_L s~ at the end.  It is taken unless the path decays below 2^-80:
+        // then 1 / A_t could overflow and the plain form alpha s + k w is used.
+        const bool scaled = ab_path[L - 1].x > 8.3e-25f;
 #pragma unroll 1
         for (int t = 0; t < L; ++t) {
             // this thread's sixteen key positions: 64*kh + 8*l8 + e
@@ -1129,7 +1140,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                     kf[kh * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
                 }
             }
-            const float2 ab = ab_path[t];
+            const float4 ab = ab_path[t];   // (A_t, beta_t, alpha_t, 1 / A_t)
             // the four rows of this thread advance together: four independent FMA chains, then their
             // shuffle reductions back to back, then the four updates
             float dot[4];
@@ -1150,19 +1161,44 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             for (int m = 1; m < 8; m <<= 1)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) dot[i] += __shfl_xor_sync(0xffffffffu, dot[i], m);
+            if (scaled) {
+                // x holds s / A_t: s~ += k beta_t (v / A_t - k.s~), one packed FMA per pair
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = warp * 16 + i * 4 + r4;
-                const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
-                const float w = ab.y * (vc - ab.x * dot[i]);
-                const float2 w2 = make_float2(w, w), a2 = make_float2(ab.x, ab.x);
+                for (int i = 0; i < 4; ++i) {
+                    const int row = warp * 16 + i * 4 + r4;
+                    const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
+                    const float w = ab.y * fmaf(vc, ab.w, -dot[i]);
+                    const float2 w2 = make_float2(w, w);
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, __fmul2_rn(a2, make_float2(x[i][q4].x, x[i][q4].y)));
-                    const float2 hi = __ffma2_rn(kf2[q4 * 2 + 1], w2, __fmul2_rn(a2, make_float2(x[i][q4].z, x[i][q4].w)));
-                    x[i][q4] = make_float4(lo.x, lo.y, hi.x, hi.y);
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, make_float2(x[i][q4].x, x[i][q4].y));
+                        const float2 hi = __ffma2_rn(kf2[q4 * 2 + 1], w2, make_float2(x[i][q4].z, x[i][q4].w));
+                        x[i][q4] = make_float4(lo.x, lo.y, hi.x, hi.y);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = warp * 16 + i * 4 + r4;
+                    const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
+                    const float w = ab.y * (vc - ab.z * dot[i]);
+                    const float2 w2 = make_float2(w, w), a2 = make_float2(ab.z, ab.z);
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, __fmul2_rn(a2, make_float2(x[i][q4].x, x[i][q4].y)));
+                        const float2 hi = __ffma2_rn(kf2[q4 * 2 + 1], w2, __fmul2_rn(a2, make_float2(x[i][q4].z, x[i][q4].w)));
+                        x[i][q4] = make_float4(lo.x, lo.y, hi.x, hi.y);
+                    }
                 }
             }
+        }
+        if (scaled) {   // back to s = A_L s~
+            const float aL = ab_path[L - 1].x;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    x[i][q4] = make_float4(aL * x[i][q4].x, aL * x[i][q4].y, aL * x[i][q4].z, aL * x[i][q4].w);
         }
         }
     }
@@ -1385,7 +1421,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         // per-step scalars of its nodes are asked for
         if constexpr (FUSED) {
             if (next_ok && warp == 4) {
-                int *slot = reinterpret_cast<int *>(smem + SM_PATH + ((iter + 1) & 1) * 256);
+                int *slot = reinterpret_cast<int *>(smem + SM_PATH + ((iter + 1) & 1) * SM_PATH_SLOT);
                 const int n_up = __shfl_up_sync(0xffffffffu, q_n, 1);
                 bool bad = false;
                 if (q_mine) {
@@ -1466,9 +1502,20 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
         __syncthreads();
         if constexpr (FUSED) {   // stage 6: the scalars of the next unit's path (asked for two phases ago)
-            if (next_ok && warp == 4 && lane < q_len)
-                reinterpret_cast<float2 *>(smem + SM_PATH + ((iter + 1) & 1) * 256 + 128)[lane] =
-                    make_float2(expf(__uint_as_float((uint32_t)q_g << 16)), __uint_as_float((uint32_t)q_be << 16));
+            if (next_ok && warp == 4) {   // lane t: decay of the path up to and including step t by a prefix sum
+                const float gt = lane < q_len ? __uint_as_float((uint32_t)q_g << 16) : 0.f;
+                float gsum = gt;
+#pragma unroll
+                for (int off = 1; off < FV_MD; off <<= 1) {
+                    const float up = __shfl_up_sync(0xffffffffu, gsum, off);
+                    if (lane >= off) gsum += up;
+                }
+                if (lane < q_len) {
+                    const float A = expf(gsum);
+                    reinterpret_cast<float4 *>(smem + SM_PATH + ((iter + 1) & 1) * SM_PATH_SLOT + 128)[lane] =
+                        make_float4(A, __uint_as_float((uint32_t)q_be << 16), expf(gt), 1.f / A);
+                }
+            }
         }
         unit_done_ok = *flag == 0;
         if (unit_done_ok) {
