@@ -12,6 +12,7 @@
 // are issued before anything else so that the path checks and the k-row staging run under their
 // latency, and the kernel keeps to 64 registers so that two CTAs (32 warps) share an SM.
 #include "gdn_internal.cuh"
+#include "gdn_replay.cuh"
 
 namespace gdn {
 
@@ -141,6 +142,113 @@ __global__ void __launch_bounds__(CM_THREADS, 2) commit_generic_kernel(const Com
     }
 }
 
+// Fast form for d_k = d_v = 128, bf16 inputs, paths of at most 16 nodes: 256 threads hold the tile as the
+// tensor-core verify kernel does (eight lanes per row, 32-byte accesses) and replay the path in the scaled form
+// (gdn_replay.cuh).  One CTA per (tree, value head), two CTAs per SM; the state loads go first, the path is fetched
+// and checked by one warp with shuffles, its k/v rows arrive by cp.async.
+constexpr int CF_THREADS = 256;
+constexpr int CF_MD = 16;
+
+__device__ __forceinline__ void cf_cp_async_16(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+__global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const CommitParams p)
+{
+    __shared__ __align__(16) uint16_t pk_s[CF_MD * GDN_TILE_D];
+    __shared__ __align__(16) uint16_t pv_s[CF_MD * GDN_TILE_D];
+    __shared__ __align__(16) float4 ab_s[CF_MD];
+    __shared__ int path_s[CF_MD];
+    __shared__ int len_s;
+
+    const int b = blockIdx.x / p.h_v, h = blockIdx.x % p.h_v;
+    const int hk = h / (p.h_v / p.h_qk);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r4 = lane >> 3, l8 = lane & 7;
+    const int pp0 = p.path_offsets[b];
+    int len = p.path_offsets[b + 1] - pp0;
+    if (len == 0) return;   // nothing accepted from this tree: state untouched
+
+    // the state tile first: its latency covers the path fetch below
+    float *S = p.S + (size_t)(b * p.h_v + h) * GDN_TILE_D * GDN_TILE_D;
+    float4 x[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float *src = S + (size_t)(warp * 16 + i * 4 + r4) * GDN_TILE_D + l8 * 8;
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
+    }
+
+    const int pb = p.node_offsets[b];
+    const int pT = p.node_offsets[b + 1] - pb;
+    const __nv_bfloat16 *k = static_cast<const __nv_bfloat16 *>(p.k), *v = static_cast<const __nv_bfloat16 *>(p.v);
+    const __nv_bfloat16 *g = static_cast<const __nv_bfloat16 *>(p.g), *beta = static_cast<const __nv_bfloat16 *>(p.beta);
+    if (warp == 0) {
+        // lane t: entry t of the path and that node's parent; the path must be a chain from a root inside the tree
+        const bool shape_ok = len > 0 && len <= CF_MD && len <= p.max_depth && pT > 0 && pp0 >= 0;
+        const bool mine = shape_ok && lane < len;
+        int n = -1, parent_n = -2;
+        if (mine) {
+            n = p.path[pp0 + lane];
+            if (p.parent && n >= 0 && n < pT) parent_n = p.parent[pb + n];
+        }
+        const int n_up = __shfl_up_sync(0xffffffffu, n, 1);
+        bool bad = false;
+        if (mine) {
+            if (n < 0 || n >= pT) bad = true;
+            else if (p.parent) bad = parent_n != (lane ? n_up : -1);
+            else if (lane && n <= n_up) bad = true;   // without parent[] only the topological order can be checked
+        }
+        if (__any_sync(0xffffffffu, bad) || !shape_ok) {
+            if (lane == 0) report_status(p.status_dev, GDN_ERR_PATH);
+            len = 0;
+        }
+        // per-step scalars: decay of the path up to and including step t by a prefix sum over the lanes
+        float gt = 0.f, be = 0.f;
+        if (lane < len) {
+            gt = __bfloat162float(g[((size_t)pb + n) * p.h_v + h]);
+            be = __bfloat162float(beta[((size_t)pb + n) * p.h_v + h]);
+        }
+        float gsum = gt;
+#pragma unroll
+        for (int off = 1; off < CF_MD; off <<= 1) {
+            const float up = __shfl_up_sync(0xffffffffu, gsum, off);
+            if (lane >= off) gsum += up;
+        }
+        if (lane < len) {
+            const float A = expf(gsum);
+            path_s[lane] = n;
+            ab_s[lane] = make_float4(A, be, expf(gt), 1.f / A);
+        }
+        if (lane == 0) len_s = len;
+    }
+    __syncthreads();
+    len = len_s;
+    if (len == 0) return;   // rejected path: this state stays as it was
+    for (int idx = tid; idx < len * 32; idx += CF_THREADS) {
+        const int t = idx >> 5, c16 = idx & 15;
+        const size_t n = (size_t)pb + path_s[t];
+        if (idx & 16)
+            cf_cp_async_16((uint32_t)__cvta_generic_to_shared(pv_s + t * GDN_TILE_D + c16 * 8),
+                           v + (n * p.h_v + h) * GDN_TILE_D + c16 * 8);
+        else
+            cf_cp_async_16((uint32_t)__cvta_generic_to_shared(pk_s + t * GDN_TILE_D + c16 * 8),
+                           k + (n * p.h_qk + hk) * GDN_TILE_D + c16 * 8);
+    }
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+
+    replay_path_on_tile(x, len, pk_s, pv_s, ab_s, warp, r4, l8);
+
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float *dst = S + (size_t)(warp * 16 + i * 4 + r4) * GDN_TILE_D + l8 * 8;
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh) stg_v8(dst + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k, const void *v,
@@ -152,6 +260,10 @@ cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k,
     if (grid == 0) return cudaSuccess;
     CommitParams p{s.h_qk, s.h_v, s.d_k, s.d_v, s.max_depth, S, k, v, g, beta,
                    parent, node_offsets, path, path_offsets, status_dev};
+    if (s.d_k == GDN_TILE_D && s.d_v == GDN_TILE_D && s.in_dtype == GDN_BF16 && s.max_depth <= CF_MD) {
+        commit_tile128_kernel<<<grid, CF_THREADS, 0, stream>>>(p);
+        return cudaGetLastError();
+    }
     const size_t smem = sizeof(float) * ((size_t)s.max_depth * CM_DK + 4 * (size_t)s.max_depth);
     cudaError_t e;
     if (s.in_dtype == GDN_BF16) {

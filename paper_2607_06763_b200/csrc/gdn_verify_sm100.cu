@@ -25,6 +25,7 @@
 #include <cuda.h>   // CUtensorMap and the cuTensorMapEncodeTiled prototype (resolved at run time, no libcuda link)
 
 #include "gdn_internal.cuh"
+#include "gdn_replay.cuh"
 
 namespace gdn {
 
@@ -146,20 +147,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
 {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
                  ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar)
-                 : "memory");
-}
-// 32-byte global accesses (one instruction per eight floats: half the load/store instructions of float4).
-__device__ __forceinline__ void ldg_v8(const float *p, float4 &a, float4 &b)
-{
-    asm volatile("ld.global.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w), "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w)
-                 : "l"(p)
-                 : "memory");
-}
-__device__ __forceinline__ void stg_v8(float *p, const float4 &a, const float4 &b)
-{
-    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
-                 ::"l"(p), "f"(a.x), "f"(a.y), "f"(a.z), "f"(a.w), "f"(b.x), "f"(b.y), "f"(b.z), "f"(b.w)
                  : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all()
@@ -1118,89 +1105,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // Per row c (one value component): s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that
     // share a row reduce k.s_c with three shuffles.  The path's k/v rows were fetched above.
     if constexpr (FUSED) {
-        if (path_len > 0) {
-            const int L = path_len;
-        const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
-        const uint16_t *pvs = reinterpret_cast<const uint16_t *>(smem + SM_PV);
-        // Scaled form: with A_t = alpha_1 .. alpha_t and s~ = s / A_t a step is s~ += k beta_t (v / A_t - k.s~)
-        // (the decay costs nothing), and s = A_L s~ at the end.  It is taken unless the path decays below 2^-80:
-        // then 1 / A_t could overflow and the plain form alpha s + k w is used.
-        const bool scaled = ab_path[L - 1].x > 8.3e-25f;
-#pragma unroll 1
-        for (int t = 0; t < L; ++t) {
-            // this thread's sixteen key positions: 64*kh + 8*l8 + e
-            float kf[16];
-#pragma unroll
-            for (int kh = 0; kh < 2; ++kh) {
-                const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
-                const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    kf[kh * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
-                    kf[kh * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
-                }
-            }
-            const float4 ab = ab_path[t];   // (A_t, beta_t, alpha_t, 1 / A_t)
-            // the four rows of this thread advance together: four independent FMA chains, then their
-            // shuffle reductions back to back, then the four updates
-            float dot[4];
-            float2 kf2[8];   // the same values as packed pairs for the two-wide fp32 FMA
-#pragma unroll
-            for (int e = 0; e < 8; ++e) kf2[e] = make_float2(kf[2 * e], kf[2 * e + 1]);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float2 acc = make_float2(0.f, 0.f);
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    acc = __ffma2_rn(kf2[q4 * 2 + 0], make_float2(x[i][q4].x, x[i][q4].y), acc);
-                    acc = __ffma2_rn(kf2[q4 * 2 + 1], make_float2(x[i][q4].z, x[i][q4].w), acc);
-                }
-                dot[i] = acc.x + acc.y;
-            }
-#pragma unroll
-            for (int m = 1; m < 8; m <<= 1)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) dot[i] += __shfl_xor_sync(0xffffffffu, dot[i], m);
-            if (scaled) {
-                // x holds s / A_t: s~ += k beta_t (v / A_t - k.s~), one packed FMA per pair
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = warp * 16 + i * 4 + r4;
-                    const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
-                    const float w = ab.y * fmaf(vc, ab.w, -dot[i]);
-                    const float2 w2 = make_float2(w, w);
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, make_float2(x[i][q4].x, x[i][q4].y));
-                        const float2 hi = __ffma2_rn(kf2[q4 * 2 + 1], w2, make_float2(x[i][q4].z, x[i][q4].w));
-                        x[i][q4] = make_float4(lo.x, lo.y, hi.x, hi.y);
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = warp * 16 + i * 4 + r4;
-                    const float vc = __uint_as_float((uint32_t)pvs[t * FV_D + row] << 16);
-                    const float w = ab.y * (vc - ab.z * dot[i]);
-                    const float2 w2 = make_float2(w, w), a2 = make_float2(ab.z, ab.z);
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, __fmul2_rn(a2, make_float2(x[i][q4].x, x[i][q4].y)));
-                        const float2 hi = __ffma2_rn(kf2[q4 * 2 + 1], w2, __fmul2_rn(a2, make_float2(x[i][q4].z, x[i][q4].w)));
-                        x[i][q4] = make_float4(lo.x, lo.y, hi.x, hi.y);
-                    }
-                }
-            }
-        }
-        if (scaled) {   // back to s = A_L s~
-            const float aL = ab_path[L - 1].x;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4)
-                    x[i][q4] = make_float4(aL * x[i][q4].x, aL * x[i][q4].y, aL * x[i][q4].z, aL * x[i][q4].w);
-        }
-        }
+        if (path_len > 0)
+            replay_path_on_tile(x, path_len, reinterpret_cast<const uint16_t *>(smem + SM_PK),
+                                reinterpret_cast<const uint16_t *>(smem + SM_PV), ab_path, warp, r4, l8);
     }
     // The v rows move into registers in the orientation of the R phase (component c = TMEM lane of this
     // thread, its 32 nodes, two bf16 per register): they are about to be overwritten by the state operand.
