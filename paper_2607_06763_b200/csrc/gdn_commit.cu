@@ -159,7 +159,6 @@ __global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const Com
     __shared__ __align__(16) uint16_t pk_s[CF_MD * GDN_TILE_D];
     __shared__ __align__(16) uint16_t pv_s[CF_MD * GDN_TILE_D];
     __shared__ __align__(16) float4 ab_s[CF_MD];
-    __shared__ int path_s[CF_MD];
     __shared__ int len_s;
 
     const int b = blockIdx.x / p.h_v, h = blockIdx.x % p.h_v;
@@ -184,9 +183,25 @@ __global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const Com
     const int pT = p.node_offsets[b + 1] - pb;
     const __nv_bfloat16 *k = static_cast<const __nv_bfloat16 *>(p.k), *v = static_cast<const __nv_bfloat16 *>(p.v);
     const __nv_bfloat16 *g = static_cast<const __nv_bfloat16 *>(p.g), *beta = static_cast<const __nv_bfloat16 *>(p.beta);
+    const bool shape_ok = len > 0 && len <= CF_MD && len <= p.max_depth && pT > 0 && pp0 >= 0;
+    // Every thread reads the path entry whose row piece it fetches (no hand-over through shared memory in front of
+    // the row fetch); an entry outside the tree is skipped here and reported by the check below.
+    if (shape_ok) {
+        for (int idx = tid; idx < len * 32; idx += CF_THREADS) {
+            const int t = idx >> 5, c16 = idx & 15;
+            const int nt = p.path[pp0 + t];
+            if (nt < 0 || nt >= pT) continue;
+            const size_t n = (size_t)pb + nt;
+            if (idx & 16)
+                cf_cp_async_16((uint32_t)__cvta_generic_to_shared(pv_s + t * GDN_TILE_D + c16 * 8),
+                               v + (n * p.h_v + h) * GDN_TILE_D + c16 * 8);
+            else
+                cf_cp_async_16((uint32_t)__cvta_generic_to_shared(pk_s + t * GDN_TILE_D + c16 * 8),
+                               k + (n * p.h_qk + hk) * GDN_TILE_D + c16 * 8);
+        }
+    }
     if (warp == 0) {
         // lane t: entry t of the path and that node's parent; the path must be a chain from a root inside the tree
-        const bool shape_ok = len > 0 && len <= CF_MD && len <= p.max_depth && pT > 0 && pp0 >= 0;
         const bool mine = shape_ok && lane < len;
         int n = -1, parent_n = -2;
         if (mine) {
@@ -218,26 +233,14 @@ __global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const Com
         }
         if (lane < len) {
             const float A = expf(gsum);
-            path_s[lane] = n;
             ab_s[lane] = make_float4(A, be, expf(gt), 1.f / A);
         }
         if (lane == 0) len_s = len;
     }
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     len = len_s;
     if (len == 0) return;   // rejected path: this state stays as it was
-    for (int idx = tid; idx < len * 32; idx += CF_THREADS) {
-        const int t = idx >> 5, c16 = idx & 15;
-        const size_t n = (size_t)pb + path_s[t];
-        if (idx & 16)
-            cf_cp_async_16((uint32_t)__cvta_generic_to_shared(pv_s + t * GDN_TILE_D + c16 * 8),
-                           v + (n * p.h_v + h) * GDN_TILE_D + c16 * 8);
-        else
-            cf_cp_async_16((uint32_t)__cvta_generic_to_shared(pk_s + t * GDN_TILE_D + c16 * 8),
-                           k + (n * p.h_qk + hk) * GDN_TILE_D + c16 * 8);
-    }
-    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
 
     replay_path_on_tile(x, len, pk_s, pv_s, ab_s, warp, r4, l8);
 
