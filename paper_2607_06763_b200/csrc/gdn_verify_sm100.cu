@@ -393,12 +393,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         const float *S = p.S0 + (size_t)(b * p.h_v + h) * FV_D * FV_D;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float4 *src = reinterpret_cast<const float4 *>(S + (size_t)(warp * 16 + i * 4 + r4) * FV_D);
+            const float *src = S + (size_t)(warp * 16 + i * 4 + r4) * FV_D + l8 * 8;
 #pragma unroll
-            for (int kh = 0; kh < 2; ++kh) {
-                x[i][kh * 2 + 0] = __ldg(src + kh * 16 + l8 * 2 + 0);
-                x[i][kh * 2 + 1] = __ldg(src + kh * 16 + l8 * 2 + 1);
-            }
+            for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
         }
     }
     // (2) k and q rows -> B operand tile (rows beyond T are zero-filled)
@@ -459,12 +456,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
+    const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // warp-uniform by construction
     GDN_TRACE_MARK(2);
 
     // (4) Everything that depends only on q, k, g, beta runs now, under the latency of the state loads:
     // Gram = [k;q].[k;q]^T on the tensor core, G_i / a_i tables, then X and Y of Eq. 9.
-    if (tid == 0) {
+    if (warp == 0 && elect_one()) {
         const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
         constexpr uint32_t id = idesc_bf16(128, 128);
 #pragma unroll
@@ -568,7 +565,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     warm_l2_state(2);
 
     // (5) P = S0.[k;q]^T (hi then lo) on the tensor core; meanwhile the back-substitution below
-    if (tid == 0) {
+    if (warp == 0 && elect_one()) {
         const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
         const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
         constexpr uint32_t id = idesc_bf16(128, 128);
@@ -695,7 +692,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         warm_l2_rows();
 
         // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
-        if (tid == 0) {
+        if (warp == 0 && elect_one()) {
             constexpr uint32_t id2 = idesc_bf16(128, 64);
             const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
             const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
