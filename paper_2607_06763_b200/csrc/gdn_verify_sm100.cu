@@ -775,7 +775,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 // and its per-node tables, decay tables and accepted path are fetched in stages, each global load one phase before
 // its value is used.  The state tile is asked for at the top of the unit and is needed only after the Gram /
 // coefficient phases; the v rows land by TMA in an area that is free until the state operand is written.
-template <typename TOut, bool FUSED>
+// SMALL (every tree of the call has at most 32 nodes): the R and output phases skip the 16-node pieces beyond the tree.
+template <typename TOut, bool FUSED, bool SMALL>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const __grid_constant__ VerifyFastParams p)
 {
     extern __shared__ uint8_t fv_smem_raw[];
@@ -1288,6 +1289,16 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 #pragma unroll 1
             for (int part = 0; part < 2; ++part) {
                 const int j0 = half * 32 + part * 16;
+                if (SMALL && j0 >= T) {   // no node of the tree in this 16-column piece: exact zeros for the D GEMM
+                    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                    for (int oct = 0; oct < 2; ++oct) {
+                        const uint32_t off = sw128_row_offset(c, half * 4 + part * 2 + oct);
+                        *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = zero4;
+                        *reinterpret_cast<uint4 *>(smem + SM_RT_LO + off) = zero4;
+                    }
+                    continue;
+                }
                 uint32_t rr[16];
                 GDN_TMEM_LD16(taddr + j0, rr);   // columns j0 .. j0+15: p^k of 16 nodes
                 float vv[16], aj[16], bj[16];
@@ -1390,6 +1401,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 #pragma unroll 1
             for (int part = 0; part < 2; ++part) {
                 const int i0 = half * 32 + part * 16;
+                if constexpr (SMALL) {
+                    if (i0 >= T) continue;   // rows beyond the tree are never stored
+                }
                 uint32_t pp[16], dd[16];
                 GDN_TMEM_LD16(trow + 64 + i0, pp);    // p^q of 16 nodes
                 GDN_TMEM_LD16(trow + 128 + i0, dd);
@@ -1500,8 +1514,9 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
             !make_row_tensor_map(&pt.tm_q, p.q, s.total_nodes, s.h_qk, 64, true) ||
             !make_row_tensor_map(&pt.tm_v, p.v, s.total_nodes, s.h_v, FV_D, false))
             return cudaErrorNotSupported;
-        cudaError_t e = cudaFuncSetAttribute(verify_sm100_persistent_kernel<TOut, FUSED>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
+        const bool small = s.max_tree_nodes <= 32;
+        auto kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true> : verify_sm100_persistent_kernel<TOut, FUSED, false>;
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
         if (e != cudaSuccess) return e;
         const int grid = p.n_units < p.prefetch_dist ? p.n_units : p.prefetch_dist;
         cudaLaunchConfig_t cfg{};
@@ -1514,7 +1529,7 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, verify_sm100_persistent_kernel<TOut, FUSED>, pt);
+        return cudaLaunchKernelEx(&cfg, kernel, pt);
     }
     return cudaGetLastError();
 }
