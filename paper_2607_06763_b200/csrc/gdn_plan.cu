@@ -26,8 +26,10 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     __shared__ uint8_t dfirst_s[GDN_GROUPED_MAX_NODES / GDN_GROUP_NODES + 1];   // depth of each group's first node
     // parent[] of this tree, staged once so that the root-path walks below run out of shared memory
     __shared__ int32_t par_s[GDN_MAX_TREE_NODES];
-    // The kernel behind this one may be launched early (programmatic stream serialization); it waits for
-    // this grid to finish before it reads anything written here.
+    // Programmatic stream serialization on both sides: this grid may have been launched under the tail of the
+    // kernel in front of it (nothing is read before that kernel has completed), and the kernel behind this one
+    // may be launched early in turn; it waits for this grid to finish before it reads anything written here.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
     const int b = blockIdx.x;
     const int lo = node_offsets[b], hi = node_offsets[b + 1];
@@ -129,10 +131,19 @@ cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32
                         const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream)
 {
     if (s.n_seq == 0) return cudaSuccess;
-    plan_kernel<<<s.n_seq, PLAN_THREADS, 0, stream>>>(s.n_seq, s.total_nodes, s.max_tree_nodes,
-                                                      s.max_depth, parent, node_offsets, plan.tree_ok,
-                                                      plan.depth, plan.anc, plan.anc8, plan.dfs_node, plan.dfs_depth, plan.dfs_anc8, status_dev);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)s.n_seq);
+    cfg.blockDim = dim3(PLAN_THREADS);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, plan_kernel, s.n_seq, s.total_nodes, s.max_tree_nodes, s.max_depth, parent,
+                              node_offsets, plan.tree_ok, plan.depth, plan.anc, plan.anc8, plan.dfs_node,
+                              plan.dfs_depth, plan.dfs_anc8, status_dev);
 }
 
 }  // namespace gdn

@@ -811,6 +811,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (tid < 4 && (int)blockIdx.x < p.n_units)
         prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // ... and whatever is launched behind this grid with the same attribute (the next call's tree-metadata kernel,
+    // which itself waits for this grid to complete before it reads or writes anything) may be made resident now.
+    asm volatile("griddepcontrol.launch_dependents;");
 
     // unit -> (tree, head, first node, size); a unit whose tree was rejected or is empty is skipped
     auto decode = [&](int u, int &ub, int &uh, int &uhk, int &ubase, int &uT) -> bool {
