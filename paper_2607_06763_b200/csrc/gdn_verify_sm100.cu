@@ -823,7 +823,15 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         uhk = uh / (p.h_v / p.h_qk);
         ubase = p.node_offsets[ub];
         uT = p.node_offsets[ub + 1] - ubase;
-        return p.tree_ok[ub] && uT > 0 && uT <= FV_T;
+        const bool tree_good = p.tree_ok[ub] && uT > 0 && uT <= FV_T;
+        if (FUSED && !tree_good) {
+            // the commit of the previous step does not depend on the new tree: the unit runs as a tree of no
+            // nodes (every node masked, nothing stored), so that its accepted path is still replayed
+            ubase = 0;
+            uT = 0;
+            return true;
+        }
+        return tree_good;
     };
     // k and q rows -> B operand tile by TMA: four 64-row x 64-column boxes (k and q, either K half), 128-byte
     // swizzled, completing on mbar_kq.  A box always spans 64 nodes: rows beyond the tree belong to the next tree

@@ -448,3 +448,113 @@ def test_calls_are_cuda_graph_capturable(tl):
     assert dn.device_status() == 0
     tl.assert_close_per_head(dn.o_host(), tl.oracle_verify(new), new.node_offsets, "graph verify o", bf16_out=True)
     tl.assert_state_close(S2.cpu().numpy().astype(np.float64), tl.oracle_commit(new), what="graph commit")
+
+
+def test_persistent_pipeline_with_rejected_and_empty_trees(tl):
+    """640 units, so that a persistent CTA walks two or three of them: rejected trees, empty trees and rejected
+    accepted paths sit at the first, the middle and the last place of a CTA's walk.  Every good tree must come out
+    right (the prefetch pipeline and its barrier phases stay consistent across skipped units), every rejected
+    tree must write nothing, and a rejected path must leave its state alone."""
+    import torch
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(123)
+    n_seq = 160
+    sizes = rng.integers(1, 65, n_seq)
+    bad_tree = {0, 5, 75, 76, 149, 150, 151}       # parent[] made non-topological below
+    empty_tree = {2, 77, 152, 9}
+    bad_path = {1, 78, 153, 10}
+    prev_trees, new_trees, paths = [], [], []
+    for b in range(n_seq):
+        tp = synth.tree_geo(rng, int(rng.integers(2, 65)))
+        prev_trees.append(tp)
+        pth = synth.root_path(tp, int(rng.integers(0, len(tp))))
+        if b % 7 == 3:
+            pth = np.zeros(0, np.int32)             # nothing accepted
+        if b in bad_path:
+            pth = np.array([0, len(tp) - 1, 1], np.int32) if len(tp) > 2 else np.array([1, 0], np.int32)
+        paths.append(pth)
+        new_trees.append(np.zeros(0, np.int32) if b in empty_tree else synth.tree_geo(rng, max(int(sizes[b]), 3)))
+    prev = synth.random_case(124, prev_trees, 2, 4, 128, 128, synth.BF16, synth.F32, paths=paths, name="prev")
+    new = synth.random_case(125, new_trees, 2, 4, 128, 128, synth.BF16, synth.F32, name="new")
+    good_new = new.parent.copy()
+    for b in bad_tree:
+        lo = int(new.node_offsets[b])
+        new.parent[lo + 1] = 2                      # parent index >= node index: rejected on the device
+    dp, dn = tl.DeviceCase(prev), tl.DeviceCase(new)
+    S = dp.S0.clone()
+    dn.o.fill_(77.0)
+    rc = gdn.gdn_tree_commit_verify(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path,
+                                    dp.path_offsets, dn.q, dn.k, dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets,
+                                    dn.o, dn.ws, dn.ws_bytes, dn.status)
+    assert rc == 0
+    assert dn.device_status() in (-7, -9)           # GDN_ERR_TREE or GDN_ERR_PATH, whichever was seen first
+    # reference: rejected paths count as empty, rejected trees are left out of the comparison
+    ref_paths = [np.zeros(0, np.int32) if b in bad_path else paths[b] for b in range(n_seq)]
+    prev_ref = synth.random_case(124, prev_trees, 2, 4, 128, 128, synth.BF16, synth.F32, paths=ref_paths)
+    S_ref = tl.oracle_commit(prev_ref)
+    S_host = S.cpu().numpy().astype(np.float64)
+    tl.assert_state_close(S_host, S_ref, what="pipeline S_new")
+    for b in bad_path:
+        assert bool((S[b] == dp.S0[b]).all()), "a rejected path must leave its state untouched"
+    from oracle import gdn_oracle as orc
+    new.parent = good_new
+    o_ref = orc.verify(S_ref, new.f64("q"), new.f64("k"), new.f64("v"), new.f64("g"), new.f64("beta"), new.parent,
+                       new.node_offsets, new.scale)
+    o = dn.o_host()
+    for b in range(n_seq):
+        lo, hi = int(new.node_offsets[b]), int(new.node_offsets[b + 1])
+        if b in bad_tree:
+            assert np.all(o[lo:hi] == 77.0), f"rejected tree {b} wrote outputs"
+        elif hi > lo:
+            tl.assert_close_per_head(o[lo:hi], o_ref[lo:hi], np.array([0, hi - lo]), f"pipeline o, tree {b}")
+    # the plain verify walks the same units and skips the rejected / empty ones altogether
+    dn.o.fill_(55.0)
+    dn.status.zero_()
+    before = dn.S0.clone()
+    assert dn.verify() == 0 and dn.device_status() == -7
+    assert bool((dn.S0 == before).all()), "verify must not touch the state"
+    o_ref = tl.oracle_verify(new)
+    o = dn.o_host()
+    for b in range(n_seq):
+        lo, hi = int(new.node_offsets[b]), int(new.node_offsets[b + 1])
+        if b in bad_tree:
+            assert np.all(o[lo:hi] == 55.0), f"rejected tree {b} wrote outputs"
+        elif hi > lo:
+            tl.assert_close_per_head(o[lo:hi], o_ref[lo:hi], np.array([0, hi - lo]), f"pipeline verify o, tree {b}")
+
+
+def test_commit_tile_kernel_paths(tl):
+    """d = 128 / bf16 commit kernel: longest legal path, empty path, and every way a path can be rejected."""
+    trees = [synth.tree_chain(16), synth.tree_chain(16), synth.tree_star(9), synth.tree_chain(5), synth.tree_chain(5),
+             synth.tree_chain(5), synth.tree_star(6)]
+    paths = [np.arange(16, dtype=np.int32),            # 0: all 16 nodes
+             np.zeros(0, np.int32),                    # 1: nothing accepted
+             np.array([0, 7], np.int32),               # 2: root and one leaf of a star
+             np.array([0, 1, 9], np.int32),            # 3: node id outside the tree        -> rejected
+             np.array([1, 2], np.int32),               # 4: does not start at a root        -> rejected
+             np.array([0, 2], np.int32),               # 5: skips a node                    -> rejected
+             np.array([0, 3], np.int32)]               # 6: fine
+    w = synth.random_case(41, trees, 2, 4, 128, 128, synth.BF16, synth.BF16, paths=paths)
+    rejected = {3, 4, 5}
+    ref_paths = [np.zeros(0, np.int32) if b in rejected else paths[b] for b in range(len(trees))]
+    w_ref = synth.random_case(41, trees, 2, 4, 128, 128, synth.BF16, synth.BF16, paths=ref_paths)
+    dc = tl.DeviceCase(w)
+    before = dc.S0.clone()
+    assert dc.commit() == 0 and dc.device_status() == -9
+    tl.assert_state_close(dc.S0.cpu().numpy().astype(np.float64), tl.oracle_commit(w_ref), what="tile commit")
+    for b in rejected | {1}:
+        assert bool((dc.S0[b] == before[b]).all())
+    # without parent[] only the topological order of the path can be checked: 0,2 passes, 2,1 does not
+    w2 = synth.random_case(42, [synth.tree_chain(5), synth.tree_chain(5)], 1, 2, 128, 128, synth.BF16, synth.BF16,
+                           paths=[np.array([0, 2], np.int32), np.array([2, 1], np.int32)])
+    d2 = tl.DeviceCase(w2)
+    before2 = d2.S0.clone()
+    assert d2.commit(parent=False) == 0 and d2.device_status() == -9
+    assert bool((d2.S0[1] == before2[1]).all()) and not bool((d2.S0[0] == before2[0]).all())
+    # a path longer than max_depth is rejected as a whole
+    w3 = synth.random_case(43, [synth.tree_chain(12)], 1, 2, 128, 128, synth.BF16, synth.BF16,
+                           paths=[np.arange(10, dtype=np.int32)])
+    d3 = tl.DeviceCase(w3, max_depth=8)
+    before3 = d3.S0.clone()
+    assert d3.commit() == 0 and d3.device_status() == -9
+    assert bool((d3.S0 == before3).all())
