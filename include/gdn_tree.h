@@ -161,7 +161,8 @@ int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k, const voi
  *   q, k, v, g, beta, parent, node_offsets, o, workspace, workspace_bytes, status_dev :
  *                  the new tree, exactly as for gdn_tree_verify
  * A rejected path (GDN_ERR_PATH) leaves that state unchanged and the new tree is verified
- * against the unchanged state.
+ * against the unchanged state.  A rejected or empty NEW tree (GDN_ERR_TREE / GDN_ERR_DEPTH, or no
+ * nodes) writes no outputs; the commit of the previous step's path happens all the same.
  */
 int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
                            const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
