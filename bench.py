@@ -44,10 +44,10 @@ def measured_peaks():
 
 def ncu_traffic(args, w, fused):
     """DRAM bytes per launch of the dominant kernel from the committed ncu capture
-    (profiles/verify_sm100_fused_stack24_T64.md: 85.7 MB for 24 layer slots), scaled by layer slots; only
+    (profiles/verify_sm100_fused_stack24_T64.md: 85.5 MB for 24 layer slots), scaled by layer slots; only
     quoted for the workload and mode that capture covers."""
     if args.workload == "stack48_T64" and fused:
-        return 85.7e6 / 24.0 * w.n_seq
+        return 85.5e6 / 24.0 * w.n_seq
     return None
 
 
