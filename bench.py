@@ -366,7 +366,7 @@ def main():
             kernel_name = "verify_sm100_persistent_kernel<fused commit>" if fused else "verify_sm100_persistent_kernel"
             launches_per_step = 2 if fused else 3
         else:   # larger trees: grouped verify kernel; the fused call runs commit and verify back to back
-            kernel_name = "commit_generic_kernel + verify_sm100_kernel<grouped>" if fused else "verify_sm100_kernel<grouped>"
+            kernel_name = "commit_tile128_kernel + verify_sm100_kernel<grouped>" if fused else "verify_sm100_kernel<grouped>"
             launches_per_step = 3
         achieved = dom_bytes / (v_avg * 1e-3) / 1e9
         out = {
