@@ -53,7 +53,7 @@ def ncu_traffic(args, w, fused):
 
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -64,12 +64,15 @@ class ClockSampler:
         try:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.file,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.file,
                                          stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
+        """Median SM clock over the samples taken inside the wall-clock window [t0, t1] (the timed region); all
+        samples if none fell inside."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -80,20 +83,29 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, reasons, inside = [], [], set(), []
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for line in self.file.read().splitlines():
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 8:
+            if len(parts) < 9:
                 continue
             try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
+                stamp = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
             except ValueError:
                 continue
-            for name, val in zip(names, parts[4:8]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
+            under_load = t0 is not None and t1 is not None and t0 <= stamp <= t1
+            inside.append(under_load)
+            if under_load or t0 is None:
+                for name, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        if any(inside):
+            sm = [v for v, keep in zip(sm, inside) if keep]
+            out["window"] = "timed region"
+        elif sm:
+            out["window"] = "whole run (no sample fell inside the timed region)"
         self.file.close()
         os.unlink(self.file.name)
         if sm:
@@ -173,8 +185,8 @@ def workload_config(w: synth.Workload, args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=60)
-    ap.add_argument("--warmup", type=int, default=6)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="stack48_T64", choices=sorted(WORKLOADS))
     ap.add_argument("--sets", type=int, default=0, help="buffer sets to rotate over (0 = enough to exceed 2x L2)")
@@ -272,10 +284,11 @@ def main():
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.25)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)] if args.mode != "fused" else []
     barrier()
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
     t_start.record()
     for i in range(args.steps):
         d = sets[(args.warmup + i) % n_sets]
@@ -297,9 +310,10 @@ def main():
         ev[i][2].record()
     t_end.record()
     barrier()
+    wall1 = time.time()
     total_ms = t_start.elapsed_time(t_end)
     time.sleep(0.15)
-    clocks = sampler.stop()
+    clocks = sampler.stop(wall0, wall1)
     assert int(status.item()) == 0, gdn.gdn_status_string(int(status.item()))
     if args.mode == "fused":
         # one call per step and one dominant kernel per call: its average launch duration over the timed
