@@ -329,7 +329,9 @@ def main():
 
     # ---- end-to-end: host buffers through the *_host entry points (copies inside the timed region)
     L = int(w.path_offsets[-1])
-    arena_bytes = gdn.gdn_tree_host_arena_bytes(shape, L)
+    fused_e2e = args.mode == "fused"
+    arena_bytes = (gdn.gdn_tree_commit_verify_host_arena_bytes(shape, w.total_nodes, L) if fused_e2e
+                   else gdn.gdn_tree_host_arena_bytes(shape, L))
     arena = torch.empty(arena_bytes, dtype=torch.uint8, device="cuda")
     pin = {n: torch.from_numpy(np.ascontiguousarray(getattr(w, n)).view(np.int16) if getattr(w, n).dtype == np.uint16
                                else np.ascontiguousarray(getattr(w, n))).pin_memory()
@@ -339,6 +341,16 @@ def main():
     o_pin = torch.empty(w.total_nodes * w.h_v * w.d_v * osz, dtype=torch.uint8).pin_memory()
 
     def e2e_step():
+        if fused_e2e:
+            # the user's call for one decode iteration: commit of the previous step's paths + verify of the tree,
+            # every tensor in pinned host memory (here the previous and the new tree carry the same tensors)
+            rc = gdn.gdn_tree_commit_verify_host(shape, pin["S0"], w.total_nodes, pin["k"], pin["v"], pin["g"],
+                                                 pin["beta"], pin["parent"], pin["node_offsets"], pin["path"],
+                                                 pin["path_offsets"], L, pin["q"], pin["k"], pin["v"], pin["g"],
+                                                 pin["beta"], pin["parent"], pin["node_offsets"], o_pin, arena,
+                                                 arena_bytes, stream)
+            assert rc == 0, gdn.gdn_status_string(rc)
+            return
         rc = gdn.gdn_tree_verify_host(shape, pin["S0"], pin["q"], pin["k"], pin["v"], pin["g"], pin["beta"],
                                       pin["parent"], pin["node_offsets"], o_pin, arena, arena_bytes, stream)
         assert rc == 0, gdn.gdn_status_string(rc)
@@ -351,8 +363,12 @@ def main():
     state_b = w.n_seq * w.h_v * w.d_v * w.d_k * 4
     qk_b, v_b, gb_b = w.total_nodes * w.h_qk * w.d_k * isz, w.total_nodes * w.h_v * w.d_v * isz, w.total_nodes * w.h_v * isz
     idx_b = 4 * (w.total_nodes + 2 * (w.n_seq + 1) + (w.n_seq + 1) + L)
-    h2d = (state_b + 2 * qk_b + v_b + 2 * gb_b) + (state_b + qk_b + v_b + 2 * gb_b) + idx_b
-    d2h = w.total_nodes * w.h_v * w.d_v * osz + state_b + 8
+    if fused_e2e:   # state up once; the previous step's k, v, g, beta and the new tree's q, k, v, g, beta
+        h2d = state_b + (qk_b + v_b + 2 * gb_b) + (2 * qk_b + v_b + 2 * gb_b) + idx_b + 4 * (w.total_nodes + w.n_seq + 1)
+        d2h = w.total_nodes * w.h_v * w.d_v * osz + state_b + 4
+    else:
+        h2d = (state_b + 2 * qk_b + v_b + 2 * gb_b) + (state_b + qk_b + v_b + 2 * gb_b) + idx_b
+        d2h = w.total_nodes * w.h_v * w.d_v * osz + state_b + 8
     e2e_s = float("nan")
     if not args.no_e2e:
         for _ in range(2):

@@ -194,6 +194,28 @@ int gdn_tree_commit_host(const gdn_shape_t *shape, float *S_h, const void *k_h, 
                          size_t arena_bytes, void *cuda_stream);
 
 /*
+ * Host-buffer variant of gdn_tree_commit_verify: one decode iteration as Section 3.4 schedules it
+ * (the commit of the previous step's accepted paths, then the verification of the new trees), with
+ * the state copied to the device once and copied back once.  prev_total_nodes = number of rows of
+ * the previous step's packed tensors (node_offsets_prev[n_seq]); the other arguments as for the
+ * two entry points above.  `dev_arena`: [device], 256-byte aligned, at least
+ * gdn_tree_commit_verify_host_arena_bytes(shape, prev_total_nodes, total_path_len) bytes.
+ * S_h is written back only if total_path_len > 0 (otherwise no state changes); o_h receives the
+ * outputs of the new trees.  Returns the host-side status, or the device-side status if non-zero.
+ */
+size_t gdn_tree_commit_verify_host_arena_bytes(const gdn_shape_t *shape, int32_t prev_total_nodes,
+                                               int32_t total_path_len);
+
+int gdn_tree_commit_verify_host(const gdn_shape_t *shape, float *S_h, int32_t prev_total_nodes,
+                                const void *k_prev_h, const void *v_prev_h, const void *g_prev_h,
+                                const void *beta_prev_h, const int32_t *parent_prev_h,
+                                const int32_t *node_offsets_prev_h, const int32_t *path_h,
+                                const int32_t *path_offsets_h, int32_t total_path_len, const void *q_h,
+                                const void *k_h, const void *v_h, const void *g_h, const void *beta_h,
+                                const int32_t *parent_h, const int32_t *node_offsets_h, void *o_h,
+                                void *dev_arena, size_t arena_bytes, void *cuda_stream);
+
+/*
  * Tree verification without a caller-provided workspace, for callers that cannot allocate device
  * memory at all (a server whose own pool owns every free byte, a latency-critical loop that must
  * not hit cudaMalloc's device-wide synchronisation, a plug-in that is forbidden to allocate).

@@ -26,6 +26,8 @@ EXPORTS = (
     "gdn_tree_host_arena_bytes",
     "gdn_tree_verify_host",
     "gdn_tree_commit_host",
+    "gdn_tree_commit_verify_host_arena_bytes",
+    "gdn_tree_commit_verify_host",
     "gdn_tree_verify_static",
     "gdn_tree_commit_verify",
 )
@@ -90,6 +92,11 @@ def load_library():
         lib.gdn_tree_verify_host.argtypes = [sp] + [vp] * 10 + [ctypes.c_size_t, vp]
         lib.gdn_tree_commit_host.restype = ctypes.c_int
         lib.gdn_tree_commit_host.argtypes = [sp] + [vp] * 9 + [ctypes.c_int32, vp, ctypes.c_size_t, vp]
+        lib.gdn_tree_commit_verify_host_arena_bytes.restype = ctypes.c_size_t
+        lib.gdn_tree_commit_verify_host_arena_bytes.argtypes = [sp, ctypes.c_int32, ctypes.c_int32]
+        lib.gdn_tree_commit_verify_host.restype = ctypes.c_int
+        lib.gdn_tree_commit_verify_host.argtypes = ([sp, vp, ctypes.c_int32] + [vp] * 8 + [ctypes.c_int32] + [vp] * 8 +
+                                                    [vp, ctypes.c_size_t, vp])
         lib.gdn_tree_commit_verify.restype = ctypes.c_int
         lib.gdn_tree_commit_verify.argtypes = [sp] + [vp] * 18 + [ctypes.c_size_t, vp, vp]
         lib.gdn_tree_verify_static.restype = ctypes.c_int
@@ -172,6 +179,21 @@ def gdn_tree_commit_host(shape: GdnShape, S, k, v, g, beta, parent, node_offsets
                                                     _ptr(beta), _ptr(parent), _ptr(node_offsets), _ptr(path),
                                                     _ptr(path_offsets), int(total_path_len), _ptr(dev_arena),
                                                     int(arena_bytes), _stream(stream)))
+
+
+def gdn_tree_commit_verify_host_arena_bytes(shape: GdnShape, prev_total_nodes: int, total_path_len: int) -> int:
+    return int(load_library().gdn_tree_commit_verify_host_arena_bytes(ctypes.byref(shape), int(prev_total_nodes),
+                                                                      int(total_path_len)))
+
+
+def gdn_tree_commit_verify_host(shape: GdnShape, S, prev_total_nodes, k_prev, v_prev, g_prev, beta_prev, parent_prev,
+                                node_offsets_prev, path, path_offsets, total_path_len, q, k, v, g, beta, parent,
+                                node_offsets, o, dev_arena, arena_bytes, stream=None) -> int:
+    return int(load_library().gdn_tree_commit_verify_host(
+        ctypes.byref(shape), _ptr(S), int(prev_total_nodes), _ptr(k_prev), _ptr(v_prev), _ptr(g_prev), _ptr(beta_prev),
+        _ptr(parent_prev), _ptr(node_offsets_prev), _ptr(path), _ptr(path_offsets), int(total_path_len), _ptr(q),
+        _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(parent), _ptr(node_offsets), _ptr(o), _ptr(dev_arena),
+        int(arena_bytes), _stream(stream)))
 
 
 def gdn_tree_verify_static(shape: GdnShape, S0, q, k, v, g, beta, parent, node_offsets, o, status_dev,

@@ -335,3 +335,94 @@ extern "C" int gdn_tree_commit_host(const gdn_shape_t *shape, float *S_h, const 
     GDN_CUDA_TRY(cudaStreamSynchronize(stream));
     return status_h;
 }
+
+extern "C" size_t gdn_tree_commit_verify_host_arena_bytes(const gdn_shape_t *shape, int32_t prev_total_nodes,
+                                                          int32_t total_path_len)
+{
+    if (check_shape(shape) != GDN_OK || total_path_len < 0 || prev_total_nodes < 0) return 0;
+    gdn_shape_t prev = *shape;
+    prev.total_nodes = prev_total_nodes;
+    const TensorBytes t = tensor_bytes(*shape), tp = tensor_bytes(prev);
+    size_t n = 0;
+    n += align256(t.state) + 2 * align256(t.qk) + align256(t.v) + 2 * align256(t.gb) + align256(t.o);
+    n += align256(t.parent) + align256(t.offsets);
+    n += align256(tp.qk) + align256(tp.v) + 2 * align256(tp.gb) + align256(tp.parent) + 2 * align256(tp.offsets);
+    n += align256((size_t)total_path_len * sizeof(int32_t) + 4) + align256(sizeof(int32_t));
+    n += workspace_layout(*shape).total;
+    return n + 256;
+}
+
+extern "C" int gdn_tree_commit_verify_host(const gdn_shape_t *shape, float *S_h, int32_t prev_total_nodes,
+                                           const void *k_prev_h, const void *v_prev_h, const void *g_prev_h,
+                                           const void *beta_prev_h, const int32_t *parent_prev_h,
+                                           const int32_t *node_offsets_prev_h, const int32_t *path_h,
+                                           const int32_t *path_offsets_h, int32_t total_path_len, const void *q_h,
+                                           const void *k_h, const void *v_h, const void *g_h, const void *beta_h,
+                                           const int32_t *parent_h, const int32_t *node_offsets_h, void *o_h,
+                                           void *dev_arena, size_t arena_bytes, void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0) return GDN_OK;
+    if (total_path_len < 0 || prev_total_nodes < 0) return GDN_ERR_SHAPE;
+    if (!S_h || !node_offsets_prev_h || !path_offsets_h || !node_offsets_h) return GDN_ERR_NULL;
+    if (total_path_len > 0 && (!k_prev_h || !v_prev_h || !g_prev_h || !beta_prev_h || !path_h)) return GDN_ERR_NULL;
+    if (s.total_nodes > 0 && (!q_h || !k_h || !v_h || !g_h || !beta_h || !parent_h || !o_h)) return GDN_ERR_NULL;
+    if (!dev_arena || arena_bytes < gdn_tree_commit_verify_host_arena_bytes(shape, prev_total_nodes, total_path_len))
+        return GDN_ERR_WORKSPACE;
+    if (!aligned256(dev_arena)) return GDN_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    gdn_shape_t prev = s;
+    prev.total_nodes = prev_total_nodes;
+    const TensorBytes t = tensor_bytes(s), tp = tensor_bytes(prev);
+    const WorkspaceLayout lay = workspace_layout(s);
+    Arena a{static_cast<char *>(dev_arena), 0, arena_bytes};
+    float *S = static_cast<float *>(a.take(t.state));
+    void *q = a.take(t.qk), *k = a.take(t.qk), *v = a.take(t.v), *g = a.take(t.gb), *beta = a.take(t.gb);
+    void *o = a.take(t.o);
+    int32_t *parent = static_cast<int32_t *>(a.take(t.parent));
+    int32_t *offs = static_cast<int32_t *>(a.take(t.offsets));
+    void *kp = a.take(tp.qk), *vp = a.take(tp.v), *gp = a.take(tp.gb), *bp = a.take(tp.gb);
+    int32_t *parent_p = parent_prev_h ? static_cast<int32_t *>(a.take(tp.parent)) : nullptr;
+    int32_t *offs_p = static_cast<int32_t *>(a.take(tp.offsets));
+    int32_t *poffs = static_cast<int32_t *>(a.take(tp.offsets));
+    const size_t path_bytes = (size_t)total_path_len * sizeof(int32_t);
+    int32_t *path = static_cast<int32_t *>(a.take(path_bytes + 4));
+    int32_t *status = static_cast<int32_t *>(a.take(sizeof(int32_t)));
+    void *ws = a.take(lay.total);
+    if (!ws) return GDN_ERR_WORKSPACE;
+    GDN_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
+    // one copy of the state for both halves of the step: it goes up once and comes back once
+    GDN_CUDA_TRY(cudaMemcpyAsync(S, S_h, t.state, cudaMemcpyHostToDevice, stream));
+    if (total_path_len > 0) {
+        GDN_CUDA_TRY(cudaMemcpyAsync(kp, k_prev_h, tp.qk, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(vp, v_prev_h, tp.v, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(gp, g_prev_h, tp.gb, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(bp, beta_prev_h, tp.gb, cudaMemcpyHostToDevice, stream));
+        if (parent_p) GDN_CUDA_TRY(cudaMemcpyAsync(parent_p, parent_prev_h, tp.parent, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(path, path_h, path_bytes, cudaMemcpyHostToDevice, stream));
+    }
+    GDN_CUDA_TRY(cudaMemcpyAsync(offs_p, node_offsets_prev_h, tp.offsets, cudaMemcpyHostToDevice, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(poffs, path_offsets_h, tp.offsets, cudaMemcpyHostToDevice, stream));
+    if (s.total_nodes > 0) {
+        GDN_CUDA_TRY(cudaMemcpyAsync(q, q_h, t.qk, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(k, k_h, t.qk, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(v, v_h, t.v, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(g, g_h, t.gb, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(beta, beta_h, t.gb, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(parent, parent_h, t.parent, cudaMemcpyHostToDevice, stream));
+    }
+    GDN_CUDA_TRY(cudaMemcpyAsync(offs, node_offsets_h, t.offsets, cudaMemcpyHostToDevice, stream));
+    if (total_path_len > 0 || s.total_nodes > 0) {
+        rc = gdn_tree_commit_verify(shape, S, kp, vp, gp, bp, parent_p, offs_p, path, poffs, q, k, v, g, beta, parent,
+                                    offs, o, ws, lay.total, status, cuda_stream);
+        if (rc != GDN_OK) return rc;
+    }
+    int32_t status_h = 0;
+    if (s.total_nodes > 0) GDN_CUDA_TRY(cudaMemcpyAsync(o_h, o, t.o, cudaMemcpyDeviceToHost, stream));
+    if (total_path_len > 0) GDN_CUDA_TRY(cudaMemcpyAsync(S_h, S, t.state, cudaMemcpyDeviceToHost, stream));
+    GDN_CUDA_TRY(cudaMemcpyAsync(&status_h, status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    GDN_CUDA_TRY(cudaStreamSynchronize(stream));
+    return status_h;
+}

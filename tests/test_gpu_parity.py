@@ -248,6 +248,28 @@ def test_host_buffer_entry_points(tl):
                                   w.path_offsets, L, arena, arena_bytes)
     assert rc == 0
     tl.assert_state_close(S_h.astype(np.float64), tl.oracle_commit(w), what="commit_host S_new")
+    # one decode iteration through host buffers: commit of the previous step's path + verify of a new tree
+    new = synth.config(1, 1)
+    shape_new = gdn.GdnShape.from_workload(new)
+    fb = gdn.gdn_tree_commit_verify_host_arena_bytes(shape_new, w.total_nodes, L)
+    assert fb > 0
+    arena2 = torch.empty(fb, dtype=torch.uint8, device="cuda")
+    S2 = w.S0.copy()
+    o2 = np.zeros((new.total_nodes, new.h_v, new.d_v), dtype=np.uint16)
+    rc = gdn.gdn_tree_commit_verify_host(shape_new, S2, w.total_nodes, w.k, w.v, w.g, w.beta, w.parent,
+                                         w.node_offsets, w.path, w.path_offsets, L, new.q, new.k, new.v, new.g,
+                                         new.beta, new.parent, new.node_offsets, o2, arena2, fb)
+    assert rc == 0
+    S_ref = tl.oracle_commit(w)
+    tl.assert_state_close(S2.astype(np.float64), S_ref, what="commit_verify_host S_new")
+    from oracle import gdn_oracle as orc
+    o_ref = orc.verify(S_ref, new.f64("q"), new.f64("k"), new.f64("v"), new.f64("g"), new.f64("beta"), new.parent,
+                       new.node_offsets, new.scale)
+    tl.assert_close_per_head(synth.bf16_bits_to_f32(o2).astype(np.float64), o_ref, new.node_offsets,
+                             "commit_verify_host o", bf16_out=True)
+    assert gdn.gdn_tree_commit_verify_host(shape_new, S2, w.total_nodes, w.k, w.v, w.g, w.beta, w.parent,
+                                           w.node_offsets, w.path, w.path_offsets, L, new.q, new.k, new.v, new.g,
+                                           new.beta, new.parent, new.node_offsets, o2, arena2, fb - 4096) == -10   # GDN_ERR_WORKSPACE
 
 
 # ------------------------------------------------------------------ fused commit + verify
