@@ -153,7 +153,14 @@ def run_reference(args, w: synth.Workload):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    run, nodes, n_slots, cores, _ = oracle_sample(w, args.oracle_slots)
+    # A step is a bounded sample of the workload: as many layer slots / sequences as keep the whole
+    # --steps/--warmup run near two minutes of host time (at least one), found from one probe slot.
+    probe, _, _, _, _ = oracle_sample(w, 1)
+    probe()
+    t_slot = min(probe(), probe())
+    budget_s = 120.0
+    fit = int(budget_s / max((args.steps + args.warmup) * t_slot, 1e-9))
+    run, nodes, n_slots, cores, _ = oracle_sample(w, max(1, min(fit, args.oracle_slots)))
     for _ in range(args.warmup):
         run()
     t0 = time.perf_counter()
@@ -161,7 +168,8 @@ def run_reference(args, w: synth.Workload):
         run()
     dt = (time.perf_counter() - t0) / args.steps
     value = nodes / dt
-    sample = f"first {n_slots} of {w.n_seq} layer slots/sequences ({nodes} nodes) per step, verify + commit"
+    sample = (f"first {n_slots} of {w.n_seq} layer slots/sequences ({nodes} nodes) per step, verify + commit; "
+              f"sample sized for about {budget_s:.0f} s over {args.steps}+{args.warmup} steps")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
