@@ -580,3 +580,14 @@ def test_commit_tile_kernel_paths(tl):
     before3 = d3.S0.clone()
     assert d3.commit() == 0 and d3.device_status() == -9
     assert bool((d3.S0 == before3).all())
+
+
+def test_fused_call_on_large_trees(tl):
+    """Trees beyond one CTA tile: the fused entry point runs the commit tile kernel and the grouped verify kernel back
+    to back; results as for the small-tree kernel."""
+    rng = np.random.default_rng(131)
+    prev_trees = [synth.tree_geo(rng, 200), synth.tree_geo(rng, 70), synth.tree_chain(16)]
+    new_trees = [synth.tree_geo(rng, 256), synth.tree_geo(rng, 20), synth.tree_geo(rng, 130)]
+    prev = synth.random_case(132, prev_trees, 2, 4, 128, 128, synth.BF16, synth.BF16, name="prev")
+    new = synth.random_case(133, new_trees, 2, 4, 128, 128, synth.BF16, synth.BF16, name="new")
+    _fused_case(tl, prev, new, "fused, large trees")
