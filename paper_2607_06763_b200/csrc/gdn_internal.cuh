@@ -18,20 +18,25 @@ namespace gdn {
 //                                          tree has <= 256 nodes; unused entries are 0xFF)
 // Grouped verification of trees with more than 64 nodes (filled when max_depth <= 16 and the tree has at
 // most GDN_GROUPED_MAX_NODES nodes).  "Position" = index in the depth-first pre-order of the tree (children
-// by increasing id).  The positions are cut into groups of GDN_GROUP_NODES; a group together with the proper
-// ancestors of its first node (at most 15, all outside the group) is closed under "ancestor of", so it can
-// be verified as a tree of at most 63 nodes: virtual index = depth-1 for those ancestors, n_prefix + offset
-// in the group for the group's own nodes.
+// by increasing id).  The positions are cut into consecutive groups; a group together with the proper
+// ancestors of its first node (n_prefix <= 15 of them, all outside the group) is closed under "ancestor of", so it
+// can be verified as a tree of its own: virtual index = depth-1 for those ancestors, n_prefix + offset in the
+// group for the group's own nodes.  A group takes as many positions as the 64-node tile leaves after its prefix
+// (64 - n_prefix, i.e. at least GDN_GROUP_MIN_NODES).
+//   group_start uint16[n_seq][GDN_MAX_GROUPS + 1]  first position of group k of tree b; entries behind the
+//                                          last group hold the tree's size
 //   dfs_node  uint16[N]                    node id at position r
 //   dfs_depth uint8 [N]                    depth of that node
 //   dfs_anc8  uint8 [N][16]                its root path in virtual indices of its group (0xFF = unused)
 //   utilde   float [N][h_v][d_v]           solve result u~ (Eq. 10 with the W S0 term folded in)
 struct WorkspaceLayout {
-    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, utilde, total;
+    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, group_start, utilde, total;
 };
 
-constexpr int GDN_GROUP_NODES = 48;           // own nodes of a group
+constexpr int GDN_GROUP_TILE = 64;            // nodes of a group and its prefix together
+constexpr int GDN_GROUP_MIN_NODES = 49;       // own nodes a group has at least (prefix of 15)
 constexpr int GDN_GROUPED_MAX_NODES = 1024;   // largest tree the grouped tensor-core path takes
+constexpr int GDN_MAX_GROUPS = (GDN_GROUPED_MAX_NODES + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;   // 21
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -47,6 +52,7 @@ inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
     w.dfs_node = off; off = align256(off + 2 * N);
     w.dfs_depth = off; off = align256(off + N);
     w.dfs_anc8 = off; off = align256(off + 16 * N);
+    w.group_start = off; off = align256(off + sizeof(uint16_t) * (size_t)s.n_seq * (GDN_MAX_GROUPS + 1));
     w.utilde = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
     w.total = off;
     return w;
@@ -59,6 +65,7 @@ struct PlanPtrs {
     uint8_t *anc8;
     uint16_t *dfs_node;
     uint8_t *dfs_depth, *dfs_anc8;
+    uint16_t *group_start;
     float *utilde;
 };
 
@@ -68,7 +75,8 @@ inline PlanPtrs plan_ptrs(void *workspace, const WorkspaceLayout &w)
     return {reinterpret_cast<int32_t *>(b + w.tree_ok), reinterpret_cast<uint8_t *>(b + w.depth),
             reinterpret_cast<uint16_t *>(b + w.anc), reinterpret_cast<uint8_t *>(b + w.anc8),
             reinterpret_cast<uint16_t *>(b + w.dfs_node), reinterpret_cast<uint8_t *>(b + w.dfs_depth),
-            reinterpret_cast<uint8_t *>(b + w.dfs_anc8), reinterpret_cast<float *>(b + w.utilde)};
+            reinterpret_cast<uint8_t *>(b + w.dfs_anc8), reinterpret_cast<uint16_t *>(b + w.group_start),
+            reinterpret_cast<float *>(b + w.utilde)};
 }
 
 // Host launchers (each returns the cudaError_t of its launch).

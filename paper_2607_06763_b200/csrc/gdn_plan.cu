@@ -18,12 +18,13 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
             const int32_t *__restrict__ parent, const int32_t *__restrict__ node_offsets,
             int32_t *__restrict__ tree_ok, uint8_t *__restrict__ depth, uint16_t *__restrict__ anc,
             uint8_t *__restrict__ anc8, uint16_t *__restrict__ dfs_node, uint8_t *__restrict__ dfs_depth,
-            uint8_t *__restrict__ dfs_anc8, int32_t *status_dev)
+            uint8_t *__restrict__ dfs_anc8, uint16_t *__restrict__ group_start, int32_t *status_dev)
 {
     __shared__ int size_s[GDN_GROUPED_MAX_NODES];        // subtree sizes
     __shared__ uint16_t left_s[GDN_GROUPED_MAX_NODES];   // nodes in the subtrees of earlier siblings
     __shared__ uint16_t pos_s[GDN_GROUPED_MAX_NODES];    // pre-order position of node i
-    __shared__ uint8_t dfirst_s[GDN_GROUPED_MAX_NODES / GDN_GROUP_NODES + 1];   // depth of each group's first node
+    __shared__ uint8_t depth_at_s[GDN_GROUPED_MAX_NODES];   // depth of the node at pre-order position r
+    __shared__ uint16_t gstart_s[GDN_MAX_GROUPS + 1];        // first position of each group (then the tree's size)
     // parent[] of this tree, staged once so that the root-path walks below run out of shared memory
     __shared__ int32_t par_s[GDN_MAX_TREE_NODES];
     // Programmatic stream serialization on both sides: this grid may have been launched under the tail of the
@@ -103,9 +104,21 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
         pos_s[i] = (uint16_t)pos;
         dfs_node[lo + pos] = (uint16_t)i;
         dfs_depth[lo + pos] = (uint8_t)d;
-        if (pos % GDN_GROUP_NODES == 0) dfirst_s[pos / GDN_GROUP_NODES] = (uint8_t)d;
+        depth_at_s[pos] = (uint8_t)d;
     }
     __syncthreads();
+    // Groups: each takes as many positions as the tile leaves after the proper ancestors of its first node
+    if (threadIdx.x == 0) {
+        int start = 0, k = 0;
+        while (start < T && k < GDN_MAX_GROUPS) {
+            gstart_s[k++] = (uint16_t)start;
+            start += GDN_GROUP_TILE - (depth_at_s[start] - 1);
+        }
+        for (; k <= GDN_MAX_GROUPS; ++k) gstart_s[k] = (uint16_t)T;
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k <= GDN_MAX_GROUPS; k += PLAN_THREADS)
+        group_start[(size_t)b * (GDN_MAX_GROUPS + 1) + k] = gstart_s[k];
     // Root path of every node in the virtual indices of its group: an ancestor before the group's first
     // position is an ancestor of the group's first node and gets index depth-1; one inside the group gets
     // n_prefix + its offset in the group, n_prefix = depth(first node) - 1.
@@ -113,8 +126,10 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
         const uint16_t *row = anc + (size_t)(lo + i) * max_depth;
         const int d = depth[lo + i];
         const int pos = pos_s[i];
-        const int g0 = pos / GDN_GROUP_NODES * GDN_GROUP_NODES;
-        const int n_prefix = dfirst_s[pos / GDN_GROUP_NODES] - 1;
+        int k = 0;
+        while (gstart_s[k + 1] <= pos) ++k;   // the group of this position (at most GDN_MAX_GROUPS steps)
+        const int g0 = gstart_s[k];
+        const int n_prefix = depth_at_s[g0] - 1;
         uint32_t w[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
         for (int t = 0; t < d; ++t) {
             const int pa = pos_s[row[t]];
@@ -143,7 +158,7 @@ cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, plan_kernel, s.n_seq, s.total_nodes, s.max_tree_nodes, s.max_depth, parent,
                               node_offsets, plan.tree_ok, plan.depth, plan.anc, plan.anc8, plan.dfs_node,
-                              plan.dfs_depth, plan.dfs_anc8, status_dev);
+                              plan.dfs_depth, plan.dfs_anc8, plan.group_start, status_dev);
 }
 
 }  // namespace gdn

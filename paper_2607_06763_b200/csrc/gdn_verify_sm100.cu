@@ -114,7 +114,7 @@ struct VerifyFastParams {
     int32_t *status_dev;
     // grouped verification of trees with more than 64 nodes (only read by the GROUPED instantiation)
     int groups_per_tree, anc_stride;                   // CTAs per (tree, head); entries per row of anc16
-    const uint16_t *anc16, *dfs_node;
+    const uint16_t *anc16, *dfs_node, *group_start;
     const uint8_t *dfs_depth, *dfs_anc8;
     // fused commit of the previous step's accepted paths (only read by the FUSED instantiation)
     float *S_rw;                                       // same tensor as S0, written in place
@@ -308,12 +308,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (T_tree <= 0) return;
     if (!GROUPED && T_tree > FV_T) return;   // larger trees never reach that instantiation (host-side dispatch)
     const bool ident = !GROUPED || T_tree <= FV_T;
-    const int g0 = grp * GDN_GROUP_NODES;
-    if (GROUPED && (ident ? grp > 0 : g0 >= T_tree)) return;   // no such group in this tree
+    int g0 = 0, n_own = T_tree;
+    if (GROUPED && !ident) {
+        const uint16_t *gs = p.group_start + (size_t)b * (GDN_MAX_GROUPS + 1);
+        g0 = grp <= GDN_MAX_GROUPS - 1 ? gs[grp] : T_tree;
+        n_own = (grp <= GDN_MAX_GROUPS - 1 ? gs[grp + 1] : T_tree) - g0;
+    }
+    if (GROUPED && (ident ? grp > 0 : n_own <= 0)) return;   // no such group in this tree
     int n_prefix = 0, T = T_tree;
     if (GROUPED && !ident) {
         n_prefix = p.dfs_depth[base + g0] - 1;
-        T = n_prefix + min(GDN_GROUP_NODES, T_tree - g0);
+        T = n_prefix + n_own;
     }
 
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fv_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -1560,9 +1565,11 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     p.beta = static_cast<const __nv_bfloat16 *>(beta);
     p.node_offsets = node_offsets; p.o = o;
     p.tree_ok = plan.tree_ok; p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
-    p.groups_per_tree = (s.max_tree_nodes + GDN_GROUP_NODES - 1) / GDN_GROUP_NODES;
+    p.groups_per_tree = (s.max_tree_nodes + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;   // upper bound; a CTA
+                                                                                            // without a group leaves at once
     p.anc_stride = s.max_depth;
     p.anc16 = plan.anc; p.dfs_node = plan.dfs_node; p.dfs_depth = plan.dfs_depth; p.dfs_anc8 = plan.dfs_anc8;
+    p.group_start = plan.group_start;
     return p;
 }
 
