@@ -1070,13 +1070,16 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             const int row = (warp & 3) * 32 + lane;
             const int half = warp >> 2;   // TMEM columns 192 + 32*half .. : k_j for j = 32*half ..
             const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 192 + half * 32;
-            uint32_t ra[32];
-            GDN_TMEM_LD32(taddr, ra);
-            tmem_wait_ld();
+            // SMALL: only rows k_0..k_31, q_0..q_31 against columns k_0..k_31 can belong to the tree
+            if (!SMALL || (half == 0 && (warp & 1) == 0)) {
+                uint32_t ra[32];
+                GDN_TMEM_LD32(taddr, ra);
+                tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int col = half * 32 + j;
-                gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[j]);
+                for (int j = 0; j < 32; ++j) {
+                    const int col = half * 32 + j;
+                    gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[j]);
+                }
             }
         }
         tc_fence_before();
