@@ -954,7 +954,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         G += __shfl_xor_sync(0xffffffffu, G, 2);
         if (s4 == 0) {
             gab_t[i].x = G;
-            gab_t[i].y = d ? expf(G) : 0.f;
+            gab_t[i].y = d ? __expf(G) : 0.f;
         }
     };
     // Gram = [k;q].k^T of the tile in the k/q operand area, into TMEM columns 192..255, which nothing else uses:
@@ -1107,7 +1107,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int idx = u * FV_THREADS + tid;
-                const float dec = expf(gdiff[u]);
+                const float dec = __expf(gdiff[u]);
                 ys[idx] = on[u] ? dec * gq[u] : 0.f;
                 xs[idx] = onx[u] ? bi[u] * dec * gk[u] : 0.f;
             }
