@@ -44,7 +44,7 @@ def measured_peaks():
 
 def ncu_traffic(args, w, fused):
     """DRAM bytes per launch of the dominant kernel from the committed ncu capture
-    (profiles/verify_sm100_fused_stack24_T64.md: 85.5 MB for 24 layer slots), scaled by layer slots; only
+    (the summary under profiles/ for the fused kernel on a 24-slot slice: 85.5 MB), scaled by layer slots; only
     quoted for the workload and mode that capture covers."""
     if args.workload == "stack48_T64" and fused:
         return 85.5e6 / 24.0 * w.n_seq
