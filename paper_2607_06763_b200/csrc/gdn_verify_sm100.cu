@@ -1351,6 +1351,26 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        GDN_TRACE_MARK_U(unit, 10);
+
+        // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
+        if (warp == 0 && elect_one()) {
+            constexpr uint32_t id2 = idesc_bf16(128, 64);
+            const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
+            const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
+#pragma unroll
+            for (int combo = 0; combo < 3; ++combo) {   // hi.hi, lo.hi, hi.lo; lo.lo is below 2^-18 of the result
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16(tmem + 128, a2[combo & 1] + (uint64_t)(ks * 2), b2[combo >> 1] + (uint64_t)(ks * 2), id2,
+                              (combo | ks) != 0);
+            }
+            umma_commit(mbar_d);
+        }
         // stage 4: the path is checked (a chain from a root inside the previous tree) and published; the
         // per-step scalars of its nodes are asked for
         if constexpr (FUSED) {
@@ -1380,32 +1400,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
 
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        GDN_TRACE_MARK_U(unit, 10);
-
-        // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
-        if (warp == 0 && elect_one()) {
-            constexpr uint32_t id2 = idesc_bf16(128, 64);
-            const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
-            const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
-#pragma unroll
-            for (int combo = 0; combo < 3; ++combo) {   // hi.hi, lo.hi, hi.lo; lo.lo is below 2^-18 of the result
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_bf16(tmem + 128, a2[combo & 1] + (uint64_t)(ks * 2), b2[combo >> 1] + (uint64_t)(ks * 2), id2,
-                              (combo | ks) != 0);
-            }
-            umma_commit(mbar_d);
-        }
-        // stage 5, while the tensor core works: the next unit's decay tables, its path rows (the v rows they
-        // land on are dead) and the scalars of the path
-        if (next_ok) {
-            path_decay((iter + 1) & 1);
-            fetch_path_rows(nh, nhk, (iter + 1) & 1, false);
-        }
+        // stage 5, while the tensor core works: the next unit's decay tables
+        if (next_ok) path_decay((iter + 1) & 1);
         if (!mbar_wait_bounded(mbar_d, par)) *flag = 1;
         tc_fence_after();
         GDN_TRACE_MARK_U(unit, 11);
@@ -1438,7 +1434,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
         __syncthreads();
-        if constexpr (FUSED) {   // stage 6: the scalars of the next unit's path (asked for two phases ago)
+        // stage 6: the next unit's path rows (published above, behind a barrier now; the area they land in is free)
+        if (next_ok) fetch_path_rows(nh, nhk, (iter + 1) & 1, false);
+        if constexpr (FUSED) {   // ... and the scalars of that path (asked for a phase ago)
             if (next_ok && warp == 4) {   // lane t: decay of the path up to and including step t by a prefix sum
                 const float gt = lane < q_len ? __uint_as_float((uint32_t)q_g << 16) : 0.f;
                 float gsum = gt;
