@@ -44,7 +44,8 @@ constexpr int SM_A_LO = 32768;                   // S0 lo
 constexpr int SM_B_KQ = 65536;                   // k and q rows, same layout (one-shot kernel: row 2i = k_i, 2i+1 = q_i;
                                                  // persistent kernel: rows 0..63 = k, 64..127 = q)
 // after the first MMA group the operand tiles are dead and are reused:
-constexpr int SM_GRAM = 0;                       // fp32 [128][64], column j of row r stored at j ^ (r & 31)
+constexpr int SM_GRAM = 0;                       // fp32 [128][64]; one-shot kernel: column j of row r stored at j ^ (r & 31);
+                                                 // persistent kernel: four-column piece c of row r at position c ^ (r & 15)
 constexpr int SM_RT_HI = 0;                      // then R^T hi: [128 rows = components][64 nodes] bf16, swizzled
 constexpr int SM_RT_LO = 16384;                  //      R^T lo
 constexpr int SM_V = 32768;                      // v rows of the tree, bf16 [64][128]
@@ -1075,11 +1076,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 uint32_t ra[32];
                 GDN_TMEM_LD32(taddr, ra);
                 tmem_wait_ld();
+                // row r of the copy: 16 pieces of four columns, piece c stored at position c ^ (r & 15), so that the
+                // 16-byte stores of a quarter-warp (eight consecutive rows, same piece) hit all the banks once
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int col = half * 32 + j;
-                    gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[j]);
-                }
+                for (int c4 = 0; c4 < 8; ++c4)
+                    *reinterpret_cast<uint4 *>(gram + row * 64 + (((half * 8 + c4) ^ (row & 15)) << 2)) =
+                        make_uint4(ra[4 * c4], ra[4 * c4 + 1], ra[4 * c4 + 2], ra[4 * c4 + 3]);
             }
         }
         tc_fence_before();
@@ -1101,8 +1103,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 const float4 gi = gab[i];
                 gdiff[u] = gi.x - gab[j].x;
                 bi[u] = gi.z;
-                gq[u] = gram[(64 + i) * 64 + (j ^ (i & 31))];   // row 64 + i: q_i
-                gk[u] = gram[i * 64 + (j ^ (i & 31))];          // row i: k_i
+                const int jpos = (((j >> 2) ^ (i & 15)) << 2) | (j & 3);   // rows i and 64 + i share i & 15
+                gq[u] = gram[(64 + i) * 64 + jpos];   // row 64 + i: q_i
+                gk[u] = gram[i * 64 + jpos];          // row i: k_i
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
