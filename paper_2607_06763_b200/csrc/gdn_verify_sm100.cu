@@ -44,8 +44,7 @@ constexpr int SM_A_LO = 32768;                   // S0 lo
 constexpr int SM_B_KQ = 65536;                   // k and q rows, same layout (one-shot kernel: row 2i = k_i, 2i+1 = q_i;
                                                  // persistent kernel: rows 0..63 = k, 64..127 = q)
 // after the first MMA group the operand tiles are dead and are reused:
-constexpr int SM_GRAM = 0;                       // fp32 [128][64]; one-shot kernel: column j of row r stored at j ^ (r & 31);
-                                                 // persistent kernel: four-column piece c of row r at position c ^ (r & 15)
+constexpr int SM_GRAM = 0;                       // fp32 [128][64]: four-column piece c of row r at position c ^ (r & 15)
 constexpr int SM_RT_HI = 0;                      // then R^T hi: [128 rows = components][64 nodes] bf16, swizzled
 constexpr int SM_RT_LO = 16384;                  //      R^T lo
 constexpr int SM_V = 32768;                      // v rows of the tree, bf16 [64][128]
@@ -504,11 +503,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
                 uint32_t ra[32];
                 GDN_TMEM_LD32(taddr + part * 32, ra);
                 tmem_wait_ld();
+                // four-column piece c of row r goes to position c ^ (r & 15): 16-byte stores, conflict-free
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int col = half * 32 + part * 16 + j;
-                    gram[row * 64 + (col ^ (row & 31))] = __uint_as_float(ra[2 * j]);
-                }
+                for (int c4 = 0; c4 < 4; ++c4)
+                    *reinterpret_cast<uint4 *>(gram + row * 64 + (((half * 8 + part * 4 + c4) ^ (row & 15)) << 2)) =
+                        make_uint4(ra[8 * c4], ra[8 * c4 + 2], ra[8 * c4 + 4], ra[8 * c4 + 6]);
             }
         }
         tc_fence_before();
@@ -530,8 +529,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
                 const float4 gi = gab[i];
                 gdiff[u] = gi.x - gab[j].x;
                 bi[u] = gi.z;
-                gq[u] = gram[(2 * i + 1) * 64 + (j ^ ((2 * i + 1) & 31))];
-                gk[u] = gram[(2 * i) * 64 + (j ^ ((2 * i) & 31))];
+                gq[u] = gram[(2 * i + 1) * 64 + ((((j >> 2) ^ ((2 * i + 1) & 15)) << 2) | (j & 3))];
+                gk[u] = gram[(2 * i) * 64 + ((((j >> 2) ^ ((2 * i) & 15)) << 2) | (j & 3))];
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
