@@ -591,3 +591,40 @@ def test_fused_call_on_large_trees(tl):
     prev = synth.random_case(132, prev_trees, 2, 4, 128, 128, synth.BF16, synth.BF16, name="prev")
     new = synth.random_case(133, new_trees, 2, 4, 128, 128, synth.BF16, synth.BF16, name="new")
     _fused_case(tl, prev, new, "fused, large trees")
+
+
+@pytest.mark.parametrize("seed", list(range(10)))
+def test_fused_randomized_shapes(tl, seed):
+    """Random batches on the tensor-core path: head counts and ratios, tree kinds and sizes from 1 to 64 nodes, root
+    paths up to 16 nodes (bushy, chains, stars), accepted paths from empty to 16 nodes, both output types."""
+    rng = np.random.default_rng(1000 + seed)
+    n_seq = int(rng.integers(1, 41))
+    h_qk = int(rng.choice([1, 2, 4]))
+    h_v = h_qk * int(rng.choice([1, 2, 4]))
+    out_dtype = synth.BF16 if seed % 2 else synth.F32
+
+    def tree():
+        kind = int(rng.integers(0, 4))
+        n = int(rng.integers(1, 65))
+        if kind == 0:
+            return synth.tree_geo(rng, n)
+        if kind == 1:
+            return synth.tree_chain(min(n, 16))
+        if kind == 2:
+            return synth.tree_star(n)
+        return synth.tree_bestfirst(rng, n) if n >= 4 else synth.tree_geo(rng, n)
+
+    prev_trees = [tree() for _ in range(n_seq)]
+    new_trees = [tree() for _ in range(n_seq)]
+    paths = []
+    for t in prev_trees:
+        r = int(rng.integers(0, 4))
+        if r == 0:
+            paths.append(np.zeros(0, np.int32))
+        elif r == 1:
+            paths.append(synth.longest_path(t))
+        else:
+            paths.append(synth.root_path(t, int(rng.integers(0, len(t)))))
+    prev = synth.random_case(2000 + seed, prev_trees, h_qk, h_v, 128, 128, synth.BF16, out_dtype, paths=paths, name="prev")
+    new = synth.random_case(3000 + seed, new_trees, h_qk, h_v, 128, 128, synth.BF16, out_dtype, name="new")
+    _fused_case(tl, prev, new, f"randomized {seed}")
