@@ -628,3 +628,28 @@ def test_fused_randomized_shapes(tl, seed):
     prev = synth.random_case(2000 + seed, prev_trees, h_qk, h_v, 128, 128, synth.BF16, out_dtype, paths=paths, name="prev")
     new = synth.random_case(3000 + seed, new_trees, h_qk, h_v, 128, 128, synth.BF16, out_dtype, name="new")
     _fused_case(tl, prev, new, f"randomized {seed}")
+
+
+@pytest.mark.parametrize("seed", list(range(6)))
+def test_verify_and_commit_randomized_shapes(tl, seed):
+    """Random batches through the plain entry points: even seeds keep every tree within one CTA tile (persistent
+    kernel), odd seeds mix in trees of up to 300 nodes (grouped kernel, groups of 49 to 64 nodes)."""
+    rng = np.random.default_rng(5000 + seed)
+    n_seq = int(rng.integers(1, 25))
+    h_qk = int(rng.choice([1, 2, 4]))
+    h_v = h_qk * int(rng.choice([1, 2]))
+    big = seed % 2 == 1
+    trees = []
+    for _ in range(n_seq):
+        n = int(rng.integers(1, 301 if big else 65))
+        kind = int(rng.integers(0, 3))
+        trees.append(synth.tree_geo(rng, n) if kind == 0 else synth.tree_bestfirst(rng, n) if kind == 1 and n >= 4
+                     else synth.tree_star(min(n, 200)))
+    w = synth.random_case(6000 + seed, trees, h_qk, h_v, 128, 128, synth.BF16, synth.F32)
+    dc = tl.DeviceCase(w)
+    before = dc.S0.clone()
+    assert dc.verify() == 0 and dc.device_status() == 0
+    assert bool((dc.S0 == before).all())
+    tl.assert_close_per_head(dc.o_host(), tl.oracle_verify(w), w.node_offsets, f"randomized verify {seed}")
+    assert dc.commit() == 0 and dc.device_status() == 0
+    tl.assert_state_close(dc.S0.cpu().numpy().astype(np.float64), tl.oracle_commit(w), what=f"randomized commit {seed}")
