@@ -815,10 +815,10 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // The first unit's state tile is an input of the call, not of that kernel: L2 is asked for it meanwhile.
     if (tid < 4 && (int)blockIdx.x < p.n_units)
         prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    // ... and whatever is launched behind this grid with the same attribute (the next call's tree-metadata kernel,
-    // which itself waits for this grid to complete before it reads or writes anything) may be made resident now.
-    asm volatile("griddepcontrol.launch_dependents;");
+    // A call of at most one unit per CTA is all latency: there (fused form, where every unit runs whatever the
+    // metadata kernel finds) the first unit's k/q tile and accepted path, inputs of the call as well, are asked for
+    // before that kernel has finished.
+    const bool early_inputs = FUSED && p.n_units <= (int)gridDim.x;
 
     // unit -> (tree, head, first node, size); a unit whose tree was rejected or is empty is skipped
     auto decode = [&](int u, int &ub, int &uh, int &uhk, int &ubase, int &uT) -> bool {
@@ -975,11 +975,22 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     };
 
     int b = 0, h = 0, hk = 0, base = 0, T = 0;
+    if (early_inputs) {
+        const int ub = blockIdx.x / p.h_v, uh = blockIdx.x % p.h_v;
+        issue_kq(ub, uh / (p.h_v / p.h_qk), p.node_offsets[ub], 0);
+        fetch_path(ub, 0);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // ... and whatever is launched behind this grid with the same attribute (the next call's tree-metadata kernel,
+    // which itself waits for this grid to complete before it reads or writes anything) may be made resident now.
+    asm volatile("griddepcontrol.launch_dependents;");
     bool cur_ok = decode(blockIdx.x, b, h, hk, base, T);
     if (cur_ok) {
-        issue_kq(b, hk, base, T);
+        if (!early_inputs) {
+            issue_kq(b, hk, base, T);
+            fetch_path(b, 0);
+        }
         load_tables(b, h, base, T, 0);
-        fetch_path(b, 0);
     }
     __syncthreads();
     if (cur_ok) {
