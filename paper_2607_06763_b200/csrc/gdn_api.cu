@@ -153,9 +153,12 @@ extern "C" int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const 
     if (workspace_bytes < lay.total) return GDN_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const PlanPtrs plan = plan_ptrs(workspace, lay);
-    if (launch_plan(s, parent, node_offsets, plan, status_dev, stream) != cudaSuccess) return GDN_ERR_CUDA;
+    // trees of at most 64 nodes on the tensor-core path: that kernel builds the tree metadata itself
+    if (!verify_sm100_single_group(s) &&
+        launch_plan(s, parent, node_offsets, plan, status_dev, stream) != cudaSuccess)
+        return GDN_ERR_CUDA;
     const cudaError_t e = verify_sm100_supported(s)
-                              ? launch_verify_sm100(s, S0, q, k, v, g, beta, node_offsets, o, plan, status_dev, stream)
+                              ? launch_verify_sm100(s, S0, q, k, v, g, beta, parent, node_offsets, o, plan, status_dev, stream)
                               : launch_verify_generic(s, S0, q, k, v, g, beta, node_offsets, o, plan, stream);
     if (e != cudaSuccess) return GDN_ERR_CUDA;
     return GDN_OK;
@@ -219,10 +222,8 @@ extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const 
     const WorkspaceLayout lay = workspace_layout(s);
     if (workspace_bytes < lay.total) return GDN_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const PlanPtrs plan = plan_ptrs(workspace, lay);
-    if (launch_plan(s, parent, node_offsets, plan, status_dev, stream) != cudaSuccess) return GDN_ERR_CUDA;
     if (launch_commit_verify_sm100(s, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
-                                   path_offsets, q, k, v, g, beta, node_offsets, o, plan, status_dev,
+                                   path_offsets, q, k, v, g, beta, parent, node_offsets, o, status_dev,
                                    stream) != cudaSuccess)
         return GDN_ERR_CUDA;
     return GDN_OK;

@@ -91,8 +91,10 @@ cudaError_t launch_verify_generic(const gdn_shape_t &s, const float *S0, const v
 // Tensor-core fast path (d_k = d_v = 128, bf16 inputs, trees <= 64 nodes, root paths <= 16 nodes).
 bool verify_sm100_supported(const gdn_shape_t &s);
 bool verify_sm100_single_group(const gdn_shape_t &s);   // every tree fits one CTA (<= 64 nodes): fusable with commit
+// Trees of at most 64 nodes: the kernel builds the tree metadata itself from parent[] (`plan` is not read);
+// larger trees: `plan` must have been filled by launch_plan on the same stream.
 cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
-                                const void *v, const void *g, const void *beta,
+                                const void *v, const void *g, const void *beta, const int32_t *parent,
                                 const int32_t *node_offsets, void *o, const PlanPtrs &plan,
                                 int32_t *status_dev, cudaStream_t stream);
 
@@ -103,8 +105,9 @@ cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const voi
                                        const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
                                        const int32_t *node_offsets_prev, const int32_t *path,
                                        const int32_t *path_offsets, const void *q, const void *k, const void *v,
-                                       const void *g, const void *beta, const int32_t *node_offsets, void *o,
-                                       const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream);
+                                       const void *g, const void *beta, const int32_t *parent,
+                                       const int32_t *node_offsets, void *o, int32_t *status_dev,
+                                       cudaStream_t stream);
 
 cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k, const void *v,
                                   const void *g, const void *beta, const int32_t *parent,

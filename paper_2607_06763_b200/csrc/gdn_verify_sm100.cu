@@ -69,7 +69,9 @@ constexpr int SM_TABLE_STRIDE = SM_TABLE2 - SM_ANC;   // table buffer tb lives S
 constexpr int SM_MBAR = SM_TABLE2 + 2176;        // 5 x u64: Gram done, P done, D done, k/q tile landed, v tile landed
 constexpr int SM_TMEM = SM_MBAR + 40;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
-constexpr int SM_BYTES = SM_FLAG + 4;
+constexpr int SM_PAR = SM_FLAG + 4;              // persistent kernel: s8 [64] parent[] of the tree whose tables are being built
+constexpr int SM_BAD = SM_PAR + FV_T;            // persistent kernel: int [2], tree of table buffer tb was rejected
+constexpr int SM_BYTES = SM_BAD + 8;
 constexpr int SM_ALLOC = SM_BYTES + 1024;        // slack for the 1024-byte alignment of the base
 
 // Development aid: with -DGDN_TRACE thread 0 of every CTA records clock64() at each phase boundary into a
@@ -82,7 +84,7 @@ __device__ long long *g_trace_buf = nullptr;
     } while (0)
 #define GDN_TRACE_MARK_U(u, k)                                                       \
     do {                                                                             \
-        if (threadIdx.x == 0 && g_trace_buf) g_trace_buf[(u) * 16 + (k)] = clock64(); \
+        if (threadIdx.x == 0 && g_trace_buf) g_trace_buf[(p.trace_call * p.n_units + (u)) * 16 + (k)] = clock64(); \
     } while (0)
 #define GDN_TRACE_MARK_T(t, k)                                                       \
     do {                                                                             \
@@ -100,13 +102,15 @@ struct VerifyFastParams {
     alignas(64) CUtensorMap tm_q;
     alignas(64) CUtensorMap tm_v;
     int h_qk, h_v;
-    int skew_ns;        // persistent kernel: start delay of the second half of the grid
+    int trace_call;
     int n_units;        // n_seq * h_v
     int prefetch_dist;  // a CTA warms L2 for unit blockIdx.x + prefetch_dist (about one wave ahead)
     float scale;
     const float *S0;
     const __nv_bfloat16 *q, *k, *v, *g, *beta;
     const int32_t *node_offsets;
+    const int32_t *parent;                             // persistent kernel: it builds the tree metadata itself
+    int n_seq, total_nodes, max_tree_nodes, max_depth;
     void *o;
     const int32_t *tree_ok;
     const uint8_t *depth;
@@ -815,20 +819,24 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // The first unit's state tile is an input of the call, not of that kernel: L2 is asked for it meanwhile.
     if (tid < 4 && (int)blockIdx.x < p.n_units)
         prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
-    // A call of at most one unit per CTA is all latency: there (fused form, where every unit runs whatever the
-    // metadata kernel finds) the first unit's k/q tile and accepted path, inputs of the call as well, are asked for
-    // before that kernel has finished.
-    const bool early_inputs = FUSED && p.n_units <= (int)gridDim.x;
+    signed char *par_s = reinterpret_cast<signed char *>(smem + SM_PAR);
+    volatile int *bad_s = reinterpret_cast<volatile int *>(smem + SM_BAD);
 
-    // unit -> (tree, head, first node, size); a unit whose tree was rejected or is empty is skipped
+    // unit -> (tree, head, first node, size); a unit whose node_offsets[] are inconsistent (reported) or whose tree
+    // is empty is skipped.  parent[] itself is checked when the unit's tables are built.
     auto decode = [&](int u, int &ub, int &uh, int &uhk, int &ubase, int &uT) -> bool {
         if (u >= p.n_units) return false;
         ub = u / p.h_v;
         uh = u % p.h_v;
         uhk = uh / (p.h_v / p.h_qk);
         ubase = p.node_offsets[ub];
-        uT = p.node_offsets[ub + 1] - ubase;
-        const bool tree_good = p.tree_ok[ub] && uT > 0 && uT <= FV_T;
+        const int uend = p.node_offsets[ub + 1];
+        uT = uend - ubase;
+        bool off_ok = ubase >= 0 && uT >= 0 && uT <= FV_T && uT <= p.max_tree_nodes && uend <= p.total_nodes;
+        if (ub == 0) off_ok = off_ok && ubase == 0;
+        if (ub == p.n_seq - 1) off_ok = off_ok && uend == p.total_nodes;
+        if (!off_ok && tid == 0) report_status(p.status_dev, GDN_ERR_TREE);
+        const bool tree_good = off_ok && uT > 0;
         if (FUSED && !tree_good) {
             // the commit of the previous step does not depend on the new tree: the unit runs as a tree of no
             // nodes (every node masked, nothing stored), so that its accepted path is still replayed
@@ -852,24 +860,63 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
     };
-    // per-node tables: depth, root-path ids, g, beta (zeros beyond T), into table buffer `tb`
-    auto load_tables = [&](int ub, int uh, int ubase, int uT, int tb) {
-        (void)ub;
+    // Tree metadata of Section 3.4.2 for one tree of at most 64 nodes, built by the CTA itself one unit ahead of
+    // its use: depth and root-path list (root first, node last, 0xFF beyond) of every node.  put_parent() stages
+    // parent[] in shared memory (entries outside [-1, i) are reported and cut); after a CTA barrier walk_tables()
+    // lets thread i climb from node i to its root, shifting each id into a 16-byte row from below, so that the
+    // root ends up in byte 0.  A tree with a bad parent[] or a root path of more than max_depth nodes is flagged in
+    // bad_s[tb]; the unit then runs as a tree of no nodes.
+    auto put_parent = [&](int uT, int par, int tb) -> bool {
+        bool bad = false;
         if (tid < FV_T) {
-            int d = 0;
-            uint4 row = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
-            float gi = 0.f, be = 0.f;
+            int pv = -1;
             if (tid < uT) {
-                const int n = ubase + tid;
-                d = p.depth[n];
-                row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)n * 16));
-                gi = __bfloat162float(p.g[(size_t)n * p.h_v + uh]);
-                be = __bfloat162float(p.beta[(size_t)n * p.h_v + uh]);
+                pv = par;
+                if (pv < -1 || pv >= tid) { bad = true; pv = -1; }
+            }
+            par_s[tid] = (signed char)pv;
+        }
+        if (tid == FV_T) bad_s[tb] = 0;
+        return bad;
+    };
+    auto walk_tables = [&](int uT, int tb, uint32_t g_bits, uint32_t be_bits, bool my_bad) {
+        if (tid < FV_T) {
+            int d = 0, err = my_bad ? GDN_ERR_TREE : 0;
+            uint32_t w0 = 0xFFFFFFFFu, w1 = 0xFFFFFFFFu, w2 = 0xFFFFFFFFu, w3 = 0xFFFFFFFFu;
+            if (tid < uT && !err) {
+                int cur = tid;
+                while (cur >= 0) {
+                    if (++d > p.max_depth) { err = GDN_ERR_DEPTH; break; }
+                    w3 = __funnelshift_l(w2, w3, 8);
+                    w2 = __funnelshift_l(w1, w2, 8);
+                    w1 = __funnelshift_l(w0, w1, 8);
+                    w0 = (w0 << 8) | (uint32_t)cur;
+                    cur = par_s[cur];
+                }
+            }
+            if (err) {
+                d = 0;
+                report_status(p.status_dev, err);
+                bad_s[tb] = 1;
             }
             (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[tid] = (uint8_t)d;
-            *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + tid * 16) = row;
-            reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[tid] = make_float4(0.f, 0.f, be, gi);
+            *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + tid * 16) = make_uint4(w0, w1, w2, w3);
+            reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[tid] =
+                make_float4(0.f, 0.f, __uint_as_float(be_bits << 16), __uint_as_float(g_bits << 16));
         }
+    };
+    // the same two steps with the loads issued on the spot (first unit of a CTA, and behind a skipped unit)
+    auto load_parent = [&](int ubase, int uT, int tb) -> bool {
+        return put_parent(uT, tid < uT ? p.parent[ubase + tid] : -1, tb);
+    };
+    auto load_tables = [&](int uh, int ubase, int uT, int tb, bool my_bad) {
+        uint32_t gb = 0, bb = 0;
+        if (tid < uT) {
+            const size_t n = (size_t)(ubase + tid);
+            gb = __ldg(reinterpret_cast<const unsigned short *>(p.g) + n * p.h_v + uh);
+            bb = __ldg(reinterpret_cast<const unsigned short *>(p.beta) + n * p.h_v + uh);
+        }
+        walk_tables(uT, tb, gb, bb, my_bad);
     };
 
     // Fused commit: the accepted path of tree `ub` in the previous step goes to path slot `ps`.  One warp
@@ -886,7 +933,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 if (len != 0) {
                     pb = p.pnode_offsets[ub];
                     const int pT = p.pnode_offsets[ub + 1] - pb;
-                    const bool shape_ok = len > 0 && len <= FV_MD && pT > 0 && pp0 >= 0;
+                    const bool shape_ok = len > 0 && len <= FV_MD && len <= p.max_depth && pT > 0 && pp0 >= 0;
                     const bool mine = shape_ok && lane < len;
                     int n = -1, parent_n = -2;
                     if (mine) {
@@ -975,23 +1022,19 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     };
 
     int b = 0, h = 0, hk = 0, base = 0, T = 0;
-    if (early_inputs) {
-        const int ub = blockIdx.x / p.h_v, uh = blockIdx.x % p.h_v;
-        issue_kq(ub, uh / (p.h_v / p.h_qk), p.node_offsets[ub], 0);
-        fetch_path(ub, 0);
-    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // ... and whatever is launched behind this grid with the same attribute (the next call's tree-metadata kernel,
     // which itself waits for this grid to complete before it reads or writes anything) may be made resident now.
     asm volatile("griddepcontrol.launch_dependents;");
     bool cur_ok = decode(blockIdx.x, b, h, hk, base, T);
+    bool par_bad = false;
     if (cur_ok) {
-        if (!early_inputs) {
-            issue_kq(b, hk, base, T);
-            fetch_path(b, 0);
-        }
-        load_tables(b, h, base, T, 0);
+        issue_kq(b, hk, base, T);
+        fetch_path(b, 0);
+        par_bad = load_parent(base, T, 0);
     }
+    __syncthreads();
+    if (cur_ok) load_tables(h, base, T, 0, par_bad);
     __syncthreads();
     if (cur_ok) {
         path_decay(0);
@@ -1011,11 +1054,14 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     uint8_t *depth_s = smem + SM_DEPTH + (iter & 1) * SM_TABLE_STRIDE;
     if (!unit_ok) {   // nothing to compute here: only keep the pipeline fed
         __syncthreads();
+        bool nbad = false;
         if (next_ok) {
             issue_kq(nb, nhk, nbase, nT);
-            load_tables(nb, nh, nbase, nT, (iter + 1) & 1);
+            nbad = load_parent(nbase, nT, (iter + 1) & 1);
             fetch_path(nb, (iter + 1) & 1);
         }
+        __syncthreads();
+        if (next_ok) load_tables(nh, nbase, nT, (iter + 1) & 1, nbad);
         __syncthreads();
         if (next_ok) {
             path_decay((iter + 1) & 1);
@@ -1032,8 +1078,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         unsigned long long gt;
         asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-        g_trace_buf[unit * 16 + 14] = smid;
-        g_trace_buf[unit * 16 + 15] = (long long)gt;
+        g_trace_buf[(p.trace_call * p.n_units + unit) * 16 + 14] = smid;
+        g_trace_buf[(p.trace_call * p.n_units + unit) * 16 + 15] = (long long)gt;
     }
 #endif
     // L2 warming for this CTA's next unit, in slices at phase boundaries
@@ -1043,6 +1089,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             prefetch_l2_bulk(p.S0 + (size_t)u_next * FV_D * FV_D + (size_t)slice * 4096, 16384);
     };
 
+    // a tree whose parent[] was rejected while its tables were built runs as a tree of no nodes: nothing of it
+    // is stored (fused form: its accepted path of the previous step is committed all the same)
+    if (bad_s[iter & 1]) {
+        T = 0;
+        if (tid < FV_T) depth_s[tid] = 0;
+    }
     // (1) state tile loads: a warp instruction covers four rows; the eight lanes of a row each own one
     // 16-byte bf16 piece of either K half.  Needed only after the Gram / coefficient phases.
     float4 x[4][4];   // [row i][kh*2 + half]
@@ -1186,8 +1238,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // The next unit's tables and accepted path are fetched in stages, each load issued one phase before its
     // value is used, so that no global-memory latency is paid in front of a barrier.
     // stage 1: table entries of node `tid` and the path bounds (registers only)
-    int t_depth = 0;
-    uint4 t_row = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+    int t_par = -1;
+    bool t_bad = false;
     unsigned short t_g = 0, t_be = 0;
     int q_pp0 = 0, q_len = 0, q_pb = 0, q_pT = 0, q_n = -1, q_par = -2;
     unsigned short q_g = 0, q_be = 0;
@@ -1195,8 +1247,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (next_ok) {
         if (tid < nT) {
             const int n = nbase + tid;
-            t_depth = p.depth[n];
-            t_row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)n * 16));
+            t_par = __ldg(p.parent + n);
             t_g = __ldg(reinterpret_cast<const unsigned short *>(p.g) + (size_t)n * p.h_v + nh);
             t_be = __ldg(reinterpret_cast<const unsigned short *>(p.beta) + (size_t)n * p.h_v + nh);
         }
@@ -1257,7 +1308,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if (next_ok && warp == 4) {
             q_len -= q_pp0;
             q_pT -= q_pb;
-            q_shape_ok = q_len > 0 && q_len <= FV_MD && q_pT > 0 && q_pp0 >= 0;
+            q_shape_ok = q_len > 0 && q_len <= FV_MD && q_len <= p.max_depth && q_pT > 0 && q_pp0 >= 0;
             q_mine = q_shape_ok && lane < q_len;
             if (q_mine) q_n = p.path[q_pp0 + lane];
         }
@@ -1277,14 +1328,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         // consumed after the loop comes round
         if (next_ok) {
             issue_kq(nb, nhk, nbase, nT);
-            // stage 3: the table entries go to the other table buffer; the parents of the path entries are asked for
-            if (tid < FV_T) {
-                const int tb = (iter + 1) & 1;
-                (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[tid] = (uint8_t)t_depth;
-                *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + tid * 16) = t_row;
-                reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[tid] =
-                    make_float4(0.f, 0.f, __uint_as_float((uint32_t)t_be << 16), __uint_as_float((uint32_t)t_g << 16));
-            }
+            // stage 3: parent[] of the next tree is staged for the walk behind the next CTA barrier; the parents of
+            // the path entries are asked for
+            t_bad = put_parent(nT, t_par, (iter + 1) & 1);
             if constexpr (FUSED) {
                 if (warp == 4 && q_mine && p.pparent && q_n >= 0 && q_n < q_pT) q_par = p.pparent[q_pb + q_n];
             }
@@ -1413,8 +1459,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
 
-        // stage 5, while the tensor core works: the next unit's decay tables
-        if (next_ok) path_decay((iter + 1) & 1);
+        // stage 5, while the tensor core works: the next unit's tables (depth, root paths) from the staged parent[]
+        if (next_ok) walk_tables(nT, (iter + 1) & 1, t_g, t_be, t_bad);
         if (!mbar_wait_bounded(mbar_d, par)) *flag = 1;
         tc_fence_after();
         GDN_TRACE_MARK_U(unit, 11);
@@ -1447,7 +1493,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
         __syncthreads();
-        // stage 6: the next unit's path rows (published above, behind a barrier now; the area they land in is free)
+        // stage 6: the next unit's decay tables, and its path rows (published above, behind a barrier now; the area
+        // they land in is free)
+        if (next_ok) path_decay((iter + 1) & 1);
         if (next_ok) fetch_path_rows(nh, nhk, (iter + 1) & 1, false);
         if constexpr (FUSED) {   // ... and the scalars of that path (asked for a phase ago)
             if (next_ok && warp == 4) {   // lane t: decay of the path up to and including step t by a prefix sum
@@ -1481,7 +1529,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (threadIdx.x == 0 && g_trace_buf) {
         unsigned long long gt;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-        g_trace_buf[unit * 16 + 13] = (long long)gt;
+        g_trace_buf[(p.trace_call * p.n_units + unit) * 16 + 13] = (long long)gt;
     }
 #endif
     ++done_units;
@@ -1540,6 +1588,10 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
     } else {
         // trees that fit one CTA: persistent CTAs, two per SM, pipelined across units
         VerifyFastParams pt = p;
+#ifdef GDN_TRACE
+        static int trace_calls = 0;
+        pt.trace_call = trace_calls++ % 8;
+#endif
         if (!make_row_tensor_map(&pt.tm_k, p.k, s.total_nodes, s.h_qk, 64, true) ||
             !make_row_tensor_map(&pt.tm_q, p.q, s.total_nodes, s.h_qk, 64, true) ||
             !make_row_tensor_map(&pt.tm_v, p.v, s.total_nodes, s.h_v, FV_D, false))
@@ -1572,12 +1624,12 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     VerifyFastParams p{};
     p.h_qk = s.h_qk; p.h_v = s.h_v; p.n_units = s.n_seq * s.h_v; p.prefetch_dist = 2 * sms; p.scale = s.scale;
-    p.skew_ns = 0;   // measured: a staggered start of the two CTAs of an SM does not help (138 vs 140 us)
     p.S0 = S0;
     p.q = static_cast<const __nv_bfloat16 *>(q); p.k = static_cast<const __nv_bfloat16 *>(k);
     p.v = static_cast<const __nv_bfloat16 *>(v); p.g = static_cast<const __nv_bfloat16 *>(g);
     p.beta = static_cast<const __nv_bfloat16 *>(beta);
     p.node_offsets = node_offsets; p.o = o;
+    p.n_seq = s.n_seq; p.total_nodes = s.total_nodes; p.max_tree_nodes = s.max_tree_nodes; p.max_depth = s.max_depth;
     p.tree_ok = plan.tree_ok; p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
     p.groups_per_tree = (s.max_tree_nodes + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;   // upper bound; a CTA
                                                                                             // without a group leaves at once
@@ -1598,12 +1650,13 @@ bool verify_sm100_supported(const gdn_shape_t &s)
 bool verify_sm100_single_group(const gdn_shape_t &s) { return verify_sm100_supported(s) && s.max_tree_nodes <= FV_T; }
 
 cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
-                                const void *v, const void *g, const void *beta,
+                                const void *v, const void *g, const void *beta, const int32_t *parent,
                                 const int32_t *node_offsets, void *o, const PlanPtrs &plan,
                                 int32_t *status_dev, cudaStream_t stream)
 {
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
-    const VerifyFastParams p = make_params(s, S0, q, k, v, g, beta, node_offsets, o, plan, status_dev);
+    VerifyFastParams p = make_params(s, S0, q, k, v, g, beta, node_offsets, o, plan, status_dev);
+    p.parent = parent;
     if (s.max_tree_nodes > FV_T) {
         if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false, true>(s, p, stream);
         return launch_fast_typed<float, false, true>(s, p, stream);
@@ -1616,11 +1669,13 @@ cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const voi
                                        const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
                                        const int32_t *node_offsets_prev, const int32_t *path,
                                        const int32_t *path_offsets, const void *q, const void *k, const void *v,
-                                       const void *g, const void *beta, const int32_t *node_offsets, void *o,
-                                       const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream)
+                                       const void *g, const void *beta, const int32_t *parent,
+                                       const int32_t *node_offsets, void *o, int32_t *status_dev,
+                                       cudaStream_t stream)
 {
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
-    VerifyFastParams p = make_params(s, S, q, k, v, g, beta, node_offsets, o, plan, status_dev);
+    VerifyFastParams p = make_params(s, S, q, k, v, g, beta, node_offsets, o, PlanPtrs{}, status_dev);
+    p.parent = parent;
     p.S_rw = S;
     p.pk = static_cast<const __nv_bfloat16 *>(k_prev); p.pv = static_cast<const __nv_bfloat16 *>(v_prev);
     p.pg = static_cast<const __nv_bfloat16 *>(g_prev); p.pbeta = static_cast<const __nv_bfloat16 *>(beta_prev);
