@@ -800,6 +800,10 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     const uint32_t mbar_kq = mbar_g + 24, mbar_v = mbar_g + 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r4 = lane >> 3, l8 = lane & 7;
+    // The asynchronous work of a unit is issued by one elected lane each of four warps, so that no single warp
+    // carries all of it: warp 0 the projection MMA group, warp 1 the D group, warp 2 the Gram block of the unit to
+    // come, warp 3 the TMA loads.  Every issuer commits its own MMAs to an mbarrier.
+    constexpr int W_MMA_P = 0, W_MMA_D = 1, W_MMA_G = 2, W_TMA = 3;
 
     if (warp == 0) tmem_alloc(sbase + SM_TMEM, FV_TMEM_COLS);
     if (tid == 32) {
@@ -851,7 +855,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // (or are zero past the end of the tensor); every use of them is masked further down.
     auto issue_kq = [&](int ub, int uhk, int ubase, int uT) {
         (void)ub; (void)uT;
-        if (warp == 0 && elect_one()) {
+        if (warp == W_TMA && elect_one()) {
             mbar_expect_tx(mbar_kq, 32768);
 #pragma unroll
             for (int kh = 0; kh < 2; ++kh) {
@@ -866,25 +870,28 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // lets thread i climb from node i to its root, shifting each id into a 16-byte row from below, so that the
     // root ends up in byte 0.  A tree with a bad parent[] or a root path of more than max_depth nodes is flagged in
     // bad_s[tb]; the unit then runs as a tree of no nodes.
+    // Node i is handled by thread FV_T + i (warps 2 and 3; warps 0 and 1 issue MMAs at the same time).
+    const int tnode = tid - FV_T;
+    const bool tbl_thread = tid >= FV_T && tid < 2 * FV_T;
     auto put_parent = [&](int uT, int par, int tb) -> bool {
         bool bad = false;
-        if (tid < FV_T) {
+        if (tbl_thread) {
             int pv = -1;
-            if (tid < uT) {
+            if (tnode < uT) {
                 pv = par;
-                if (pv < -1 || pv >= tid) { bad = true; pv = -1; }
+                if (pv < -1 || pv >= tnode) { bad = true; pv = -1; }
             }
-            par_s[tid] = (signed char)pv;
+            par_s[tnode] = (signed char)pv;
         }
-        if (tid == FV_T) bad_s[tb] = 0;
+        if (tid == 0) bad_s[tb] = 0;
         return bad;
     };
     auto walk_tables = [&](int uT, int tb, uint32_t g_bits, uint32_t be_bits, bool my_bad) {
-        if (tid < FV_T) {
+        if (tbl_thread) {
             int d = 0, err = my_bad ? GDN_ERR_TREE : 0;
             uint32_t w0 = 0xFFFFFFFFu, w1 = 0xFFFFFFFFu, w2 = 0xFFFFFFFFu, w3 = 0xFFFFFFFFu;
-            if (tid < uT && !err) {
-                int cur = tid;
+            if (tnode < uT && !err) {
+                int cur = tnode;
                 while (cur >= 0) {
                     if (++d > p.max_depth) { err = GDN_ERR_DEPTH; break; }
                     w3 = __funnelshift_l(w2, w3, 8);
@@ -899,20 +906,20 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 report_status(p.status_dev, err);
                 bad_s[tb] = 1;
             }
-            (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[tid] = (uint8_t)d;
-            *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + tid * 16) = make_uint4(w0, w1, w2, w3);
-            reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[tid] =
+            (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[tnode] = (uint8_t)d;
+            *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + tnode * 16) = make_uint4(w0, w1, w2, w3);
+            reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[tnode] =
                 make_float4(0.f, 0.f, __uint_as_float(be_bits << 16), __uint_as_float(g_bits << 16));
         }
     };
     // the same two steps with the loads issued on the spot (first unit of a CTA, and behind a skipped unit)
     auto load_parent = [&](int ubase, int uT, int tb) -> bool {
-        return put_parent(uT, tid < uT ? p.parent[ubase + tid] : -1, tb);
+        return put_parent(uT, tbl_thread && tnode < uT ? p.parent[ubase + tnode] : -1, tb);
     };
     auto load_tables = [&](int uh, int ubase, int uT, int tb, bool my_bad) {
         uint32_t gb = 0, bb = 0;
-        if (tid < uT) {
-            const size_t n = (size_t)(ubase + tid);
+        if (tbl_thread && tnode < uT) {
+            const size_t n = (size_t)(ubase + tnode);
             gb = __ldg(reinterpret_cast<const unsigned short *>(p.g) + n * p.h_v + uh);
             bb = __ldg(reinterpret_cast<const unsigned short *>(p.beta) + n * p.h_v + uh);
         }
@@ -1007,7 +1014,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // Gram = [k;q].k^T of the tile in the k/q operand area, into TMEM columns 192..255, which nothing else uses:
     // issued by one thread as soon as the tile has landed, one unit ahead of its use.
     auto issue_gram = [&](uint32_t kq_parity) {
-        if (warp == 0 && elect_one()) {
+        if (warp == W_MMA_G && elect_one()) {
             if (!mbar_wait_bounded(mbar_kq, kq_parity)) *flag = 1;
             tc_fence_after();
             const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
@@ -1108,7 +1115,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
     }
     // this tree's v rows: one TMA box into an area that stays free until the state operand is written
-    if (warp == 0 && elect_one()) {
+    if (warp == W_TMA && elect_one()) {
         mbar_expect_tx(mbar_v, FV_T * FV_D * 2);
         tma_load_3d(sbase + SM_VE, &p.tm_v, 0, h, base, mbar_v);
     }
@@ -1245,8 +1252,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     unsigned short q_g = 0, q_be = 0;
     bool q_shape_ok = false, q_mine = false;
     if (next_ok) {
-        if (tid < nT) {
-            const int n = nbase + tid;
+        if (tbl_thread && tnode < nT) {
+            const int n = nbase + tnode;
             t_par = __ldg(p.parent + n);
             t_g = __ldg(reinterpret_cast<const unsigned short *>(p.g) + (size_t)n * p.h_v + nh);
             t_be = __ldg(reinterpret_cast<const unsigned short *>(p.beta) + (size_t)n * p.h_v + nh);
@@ -1262,7 +1269,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     }
 
     // (5) P = S0.[k;q]^T (hi then lo) on the tensor core; meanwhile the back-substitution below
-    if (warp == 0 && elect_one()) {
+    if (warp == W_MMA_P && elect_one()) {
         const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
         const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
         constexpr uint32_t id = idesc_bf16(128, 128);
@@ -1417,7 +1424,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         GDN_TRACE_MARK_U(unit, 10);
 
         // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
-        if (warp == 0 && elect_one()) {
+        if (warp == W_MMA_D && elect_one()) {
             constexpr uint32_t id2 = idesc_bf16(128, 64);
             const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
             const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
