@@ -228,8 +228,11 @@ int gdn_tree_commit_verify_host(const gdn_shape_t *shape, float *S_h, int32_t pr
  *   - Limit: gdn_tree_workspace_bytes(shape) must not exceed GDN_STATIC_SCRATCH_BYTES (about
  *     one layer of 32 value heads x 128 with a tree of up to ~250 nodes); larger problems get
  *     GDN_ERR_WORKSPACE and nothing is launched.
- *   - The first call on each device resolves the array's device address (with that device
- *     current); make that first call before starting any stream capture.
+ *   - The first call on each device does one-time set-up with that device current: the CUDA
+ *     runtime loads the library's device code (which is when the array itself comes into being),
+ *     the array's device address is resolved, the kernels' shared-memory attributes are set and the
+ *     driver entry point for tensor maps is looked up.  Make that first call before starting any
+ *     stream capture; the calls after it do none of this.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in
  *     it (verify rewrites every part it later reads, so nothing needs clearing).  Two calls
  *     whose kernels overlap on the GPU -- different streams, or the same stream from two threads

@@ -60,6 +60,38 @@ struct Arena {
     }
 };
 
+// Host-side argument checks of gdn_tree_verify (everything that can be refused before a launch).
+int check_verify_args(const gdn_shape_t &s, const float *S0, const void *q, const void *k, const void *v,
+                      const void *g, const void *beta, const int32_t *parent, const int32_t *node_offsets,
+                      const void *o, const void *workspace, size_t workspace_bytes, const int32_t *status_dev)
+{
+    if (!S0 || !q || !k || !v || !g || !beta || !parent || !node_offsets || !o || !status_dev)
+        return GDN_ERR_NULL;
+    if (!workspace) return GDN_ERR_WORKSPACE;
+    if (!aligned16(S0) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) ||
+        !aligned16(beta) || !aligned16(o) || !aligned256(workspace) ||
+        (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(node_offsets) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    if (workspace_bytes < workspace_layout(s).total) return GDN_ERR_WORKSPACE;
+    return GDN_OK;
+}
+
+// Host-side argument checks of gdn_tree_commit.
+int check_commit_args(const gdn_shape_t &s, const float *S, const void *k, const void *v, const void *g,
+                      const void *beta, const int32_t *parent, const int32_t *node_offsets, const int32_t *path,
+                      const int32_t *path_offsets, const int32_t *status_dev)
+{
+    if (!S || !node_offsets || !path_offsets || !status_dev) return GDN_ERR_NULL;
+    if (s.total_nodes > 0 && (!k || !v || !g || !beta || !path)) return GDN_ERR_NULL;
+    if (!aligned16(S) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(node_offsets) & 3u) ||
+        (reinterpret_cast<uintptr_t>(path) & 3u) || (reinterpret_cast<uintptr_t>(path_offsets) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    return GDN_OK;
+}
+
 }  // namespace
 
 extern "C" const char *gdn_status_string(int status)
@@ -141,16 +173,9 @@ extern "C" int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const 
     if (rc != GDN_OK) return rc;
     const gdn_shape_t &s = *shape;
     if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
-    if (!S0 || !q || !k || !v || !g || !beta || !parent || !node_offsets || !o || !status_dev)
-        return GDN_ERR_NULL;
-    if (!workspace) return GDN_ERR_WORKSPACE;
-    if (!aligned16(S0) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) ||
-        !aligned16(beta) || !aligned16(o) || !aligned256(workspace) ||
-        (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(node_offsets) & 3u) ||
-        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
-        return GDN_ERR_ALIGN;
+    rc = check_verify_args(s, S0, q, k, v, g, beta, parent, node_offsets, o, workspace, workspace_bytes, status_dev);
+    if (rc != GDN_OK) return rc;
     const WorkspaceLayout lay = workspace_layout(s);
-    if (workspace_bytes < lay.total) return GDN_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const PlanPtrs plan = plan_ptrs(workspace, lay);
     // trees of at most 64 nodes on the tensor-core path: that kernel builds the tree metadata itself
@@ -173,13 +198,8 @@ extern "C" int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k
     if (rc != GDN_OK) return rc;
     const gdn_shape_t &s = *shape;
     if (s.n_seq == 0) return GDN_OK;
-    if (!S || !node_offsets || !path_offsets || !status_dev) return GDN_ERR_NULL;
-    if (s.total_nodes > 0 && (!k || !v || !g || !beta || !path)) return GDN_ERR_NULL;
-    if (!aligned16(S) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
-        (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(node_offsets) & 3u) ||
-        (reinterpret_cast<uintptr_t>(path) & 3u) || (reinterpret_cast<uintptr_t>(path_offsets) & 3u) ||
-        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
-        return GDN_ERR_ALIGN;
+    rc = check_commit_args(s, S, k, v, g, beta, parent, node_offsets, path, path_offsets, status_dev);
+    if (rc != GDN_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (launch_commit_generic(s, S, k, v, g, beta, parent, node_offsets, path, path_offsets, status_dev,
                               stream) != cudaSuccess)
@@ -202,7 +222,16 @@ extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const 
     if (!S || !node_offsets_prev || !path_offsets || !status_dev) return GDN_ERR_NULL;
     if (!verify_sm100_single_group(s) || s.total_nodes == 0) {
         // general shapes: the two kernels back to back on the stream (the shape's node counts are
-        // not used by commit, so the new tree's shape serves for the previous tree as well)
+        // not used by commit, so the new tree's shape serves for the previous tree as well).  Both
+        // halves are checked before the first launch: a refused call must leave the state as it was.
+        rc = check_commit_args(s, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
+                               path_offsets, status_dev);
+        if (rc != GDN_OK) return rc;
+        if (s.total_nodes > 0) {
+            rc = check_verify_args(s, S, q, k, v, g, beta, parent, node_offsets, o, workspace, workspace_bytes,
+                                   status_dev);
+            if (rc != GDN_OK) return rc;
+        }
         rc = gdn_tree_commit(shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
                              path_offsets, status_dev, cuda_stream);
         if (rc != GDN_OK) return rc;

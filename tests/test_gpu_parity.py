@@ -335,6 +335,58 @@ def test_fused_commit_verify_general_shapes_and_rejected_path(tl):
     tl.assert_close_per_head(dn.o_host(), o_ref, new2.node_offsets, "fused, rejected path o")
 
 
+def test_refused_fused_call_launches_nothing(tl):
+    """A fused call that is refused on the host (here: workspace too small, then a NULL output) must not have
+    committed anything: state bit-identical, device status word untouched -- also on shapes that run as two kernels."""
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(91)
+    for trees_prev, trees_new in (([synth.tree_geo(rng, 40)], [synth.tree_geo(rng, 100)]),      # grouped: two kernels
+                                  ([synth.tree_geo(rng, 40)], [synth.tree_geo(rng, 50)])):      # one fused kernel
+        prev = synth.random_case(92, trees_prev, 2, 4, 128, 128, synth.BF16, synth.F32)
+        new = synth.random_case(93, trees_new, 2, 4, 128, 128, synth.BF16, synth.F32)
+        dp, dn = tl.DeviceCase(prev), tl.DeviceCase(new)
+        S = dp.S0.clone()
+        args = (dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path, dp.path_offsets, dn.q,
+                dn.k, dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets)
+        assert gdn.gdn_tree_commit_verify(*args, dn.o, dn.ws, dn.ws_bytes - 256, dn.status) == -10
+        assert gdn.gdn_tree_commit_verify(*args, None, dn.ws, dn.ws_bytes, dn.status) == -1
+        assert dn.device_status() == 0
+        assert bool((S == dp.S0).all()), "a refused call must leave the state as it was"
+        assert gdn.gdn_tree_commit_verify(*args, dn.o, dn.ws, dn.ws_bytes, dn.status) == 0
+        assert dn.device_status() == 0
+        tl.assert_state_close(S.cpu().numpy().astype(np.float64), tl.oracle_commit(prev), what="after the retry")
+
+
+def test_path_longer_than_max_depth_is_rejected_by_both_entry_points(tl):
+    """max_depth = 8 and an accepted path of 12 nodes: the separate commit and the fused call must agree
+    (GDN_ERR_PATH, state unchanged)."""
+    import paper_2607_06763_b200 as gdn
+    prev = synth.random_case(94, [synth.tree_chain(12)], 2, 4, 128, 128, synth.BF16, synth.F32,
+                             paths=[np.arange(12, dtype=np.int32)])
+    new = synth.random_case(95, [synth.tree_star(8)], 2, 4, 128, 128, synth.BF16, synth.F32)
+    dp16 = tl.DeviceCase(prev)
+    dn = tl.DeviceCase(new, max_depth=8)
+    S = dp16.S0.clone()
+    rc = gdn.gdn_tree_commit(dn.shape, S, dp16.k, dp16.v, dp16.g, dp16.beta, dp16.parent, dp16.node_offsets,
+                             dp16.path, dp16.path_offsets, dn.status)
+    assert rc == 0 and dn.device_status() == -9
+    assert bool((S == dp16.S0).all())
+    dn.status.zero_()
+    rc = gdn.gdn_tree_commit_verify(dn.shape, S, dp16.k, dp16.v, dp16.g, dp16.beta, dp16.parent, dp16.node_offsets,
+                                    dp16.path, dp16.path_offsets, dn.q, dn.k, dn.v, dn.g, dn.beta, dn.parent,
+                                    dn.node_offsets, dn.o, dn.ws, dn.ws_bytes, dn.status)
+    assert rc == 0 and dn.device_status() == -9
+    assert bool((S == dp16.S0).all())
+    # the new tree is verified against the unchanged state all the same
+    tl.assert_close_per_head(dn.o_host(), tl.oracle_verify(dataclass_replace_S0(new, prev.S0)), new.node_offsets,
+                             "verify on the unchanged state")
+
+
+def dataclass_replace_S0(w, S0):
+    import dataclasses
+    return dataclasses.replace(w, S0=S0)
+
+
 def test_fused_commit_verify_full_stack_sampled(tl):
     import paper_2607_06763_b200 as gdn
     prev, new = synth.config(5, 0), synth.config(5, 1)
