@@ -127,6 +127,20 @@ int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const void *q, co
                     int32_t *status_dev, void *cuda_stream);
 
 /*
+ * Per-branch recurrent verification: the baseline that Section 3.4 describes as "sequential scans
+ * along tree branches" and that Section 5.2 / Figure 5 times against the fused kernel.  For every
+ * leaf of every tree the state is copied and Eq. 7 is run token by token down the leaf's root path,
+ * writing o_i (Eq. 8) for each node passed; prefixes shared by several branches are recomputed
+ * once per branch.  Same arguments and results as gdn_tree_verify (fp32 arithmetic on CUDA cores,
+ * any d_k, d_v <= 128), but no workspace.  A branch whose parent[] chain is broken or longer than
+ * max_depth reports GDN_ERR_TREE / GDN_ERR_DEPTH and writes nothing; other branches still do.
+ * It is here as a comparator and as an independent GPU check of the triangular-form kernels.
+ */
+int gdn_tree_verify_recurrent(const gdn_shape_t *shape, const float *S0, const void *q, const void *k,
+                              const void *v, const void *g, const void *beta, const int32_t *parent,
+                              const int32_t *node_offsets, void *o, int32_t *status_dev, void *cuda_stream);
+
+/*
  * Commit (Section 3.4: the state write is postponed until the accepted branch is known and
  * is then a short recurrence over that branch; Section 3.4.2, end: it is the only state
  * write of a decode step): for every tree b, S[b] <- Eq. 7 replayed over

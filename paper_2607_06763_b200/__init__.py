@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     gdn_tree_validate_host,
     gdn_tree_verify,
     gdn_tree_verify_host,
+    gdn_tree_verify_recurrent,
     gdn_tree_verify_static,
     gdn_tree_workspace_bytes,
     library_path,

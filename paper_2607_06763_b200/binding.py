@@ -30,6 +30,7 @@ EXPORTS = (
     "gdn_tree_commit_verify_host",
     "gdn_tree_verify_static",
     "gdn_tree_commit_verify",
+    "gdn_tree_verify_recurrent",
 )
 
 GDN_STATIC_SCRATCH_BYTES = 4 << 20
@@ -101,6 +102,8 @@ def load_library():
         lib.gdn_tree_commit_verify.argtypes = [sp] + [vp] * 18 + [ctypes.c_size_t, vp, vp]
         lib.gdn_tree_verify_static.restype = ctypes.c_int
         lib.gdn_tree_verify_static.argtypes = [sp] + [vp] * 11
+        lib.gdn_tree_verify_recurrent.restype = ctypes.c_int
+        lib.gdn_tree_verify_recurrent.argtypes = [sp] + [vp] * 11
         _lib = lib
     return _lib
 
@@ -194,6 +197,13 @@ def gdn_tree_commit_verify_host(shape: GdnShape, S, prev_total_nodes, k_prev, v_
         _ptr(parent_prev), _ptr(node_offsets_prev), _ptr(path), _ptr(path_offsets), int(total_path_len), _ptr(q),
         _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(parent), _ptr(node_offsets), _ptr(o), _ptr(dev_arena),
         int(arena_bytes), _stream(stream)))
+
+
+def gdn_tree_verify_recurrent(shape, S0, q, k, v, g, beta, parent, node_offsets, o, status_dev, stream=None) -> int:
+    """``gdn_tree_verify_recurrent``: the per-branch recurrent baseline (same results as ``gdn_tree_verify``)."""
+    return int(load_library().gdn_tree_verify_recurrent(ctypes.byref(shape), _ptr(S0), _ptr(q), _ptr(k), _ptr(v),
+                                                         _ptr(g), _ptr(beta), _ptr(parent), _ptr(node_offsets),
+                                                         _ptr(o), _ptr(status_dev), _stream(stream)))
 
 
 def gdn_tree_verify_static(shape: GdnShape, S0, q, k, v, g, beta, parent, node_offsets, o, status_dev,

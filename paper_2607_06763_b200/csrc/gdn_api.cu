@@ -189,6 +189,26 @@ extern "C" int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const 
     return GDN_OK;
 }
 
+extern "C" int gdn_tree_verify_recurrent(const gdn_shape_t *shape, const float *S0, const void *q, const void *k,
+                                         const void *v, const void *g, const void *beta, const int32_t *parent,
+                                         const int32_t *node_offsets, void *o, int32_t *status_dev,
+                                         void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
+    if (!S0 || !q || !k || !v || !g || !beta || !parent || !node_offsets || !o || !status_dev) return GDN_ERR_NULL;
+    if (!aligned16(S0) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        !aligned16(o) || (reinterpret_cast<uintptr_t>(parent) & 3u) ||
+        (reinterpret_cast<uintptr_t>(node_offsets) & 3u) || (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    if (launch_verify_recurrent(s, S0, q, k, v, g, beta, parent, node_offsets, o, status_dev,
+                                static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
 extern "C" int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k, const void *v,
                                const void *g, const void *beta, const int32_t *parent,
                                const int32_t *node_offsets, const int32_t *path,

@@ -109,6 +109,11 @@ cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const voi
                                        const int32_t *node_offsets, void *o, int32_t *status_dev,
                                        cudaStream_t stream);
 
+// Per-branch recurrent verification (the baseline of Section 5.2 / Figure 5): no workspace, no tree plan.
+cudaError_t launch_verify_recurrent(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
+                                    const void *v, const void *g, const void *beta, const int32_t *parent,
+                                    const int32_t *node_offsets, void *o, int32_t *status_dev, cudaStream_t stream);
+
 cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k, const void *v,
                                   const void *g, const void *beta, const int32_t *parent,
                                   const int32_t *node_offsets, const int32_t *path,

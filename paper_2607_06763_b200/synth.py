@@ -318,6 +318,14 @@ def config(idx: int, rep: int = 0, out_dtype: str | None = None, n_layers: int =
     raise ValueError(f"unknown configuration {idx}")
 
 
+def layer_sweep(T: int, rep: int = 0, out_dtype: str = BF16) -> Workload:
+    """One layer with configuration 1's head shapes and a GEO tree of ``T`` nodes (the tree-size sweep of the
+    paper's Table 1 / Figure 5: budgets 32..512); accepted path = longest root path."""
+    rng = np.random.Generator(np.random.PCG64(SEED_BASE + 101 * 6 + 7 * T + rep))
+    t = tree_geo(rng, T)
+    return make_workload(f"layer_T{T}", [t], [longest_path(t)], 16, 32, 128, 128, BF16, out_dtype, rng)
+
+
 def random_case(seed: int, trees, h_qk, h_v, d_k, d_v, in_dtype=F32, out_dtype=F32, paths=None, name="case"):
     """A free-form case for tests: given trees, random accepted root paths unless ``paths`` is given."""
     rng = np.random.Generator(np.random.PCG64(seed))

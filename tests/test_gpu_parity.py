@@ -705,3 +705,49 @@ def test_verify_and_commit_randomized_shapes(tl, seed):
     tl.assert_close_per_head(dc.o_host(), tl.oracle_verify(w), w.node_offsets, f"randomized verify {seed}")
     assert dc.commit() == 0 and dc.device_status() == 0
     tl.assert_state_close(dc.S0.cpu().numpy().astype(np.float64), tl.oracle_commit(w), what=f"randomized commit {seed}")
+
+
+# ------------------------------------------------------------------ per-branch recurrent comparator (Section 5.2, Figure 5)
+@pytest.mark.parametrize("cfg", [0, 1])
+def test_recurrent_comparator_matches_oracle(tl, cfg):
+    import paper_2607_06763_b200 as gdn
+    for rep in range(3):
+        w = synth.config(cfg, rep, out_dtype=synth.F32)
+        dc = tl.DeviceCase(w)
+        S_before = dc.S0.clone()
+        rc = gdn.gdn_tree_verify_recurrent(dc.shape, dc.S0, dc.q, dc.k, dc.v, dc.g, dc.beta, dc.parent, dc.node_offsets,
+                                           dc.o, dc.status)
+        assert rc == 0 and dc.device_status() == 0
+        assert bool((dc.S0 == S_before).all()), "verify must not write the state"
+        tl.assert_close_per_head(dc.o_host(), tl.oracle_verify(w), w.node_offsets, f"recurrent cfg{cfg} rep{rep}")
+
+
+def test_recurrent_comparator_agrees_with_the_tensor_core_path_on_a_ragged_batch(tl):
+    """Two structurally different GPU evaluations (token-by-token replay per branch; triangular form on the tensor
+    core) of the same trees, both against the oracle: forests, chains, a 300-node tree, bf16 outputs."""
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(123)
+    a, b2 = synth.tree_geo(rng, 30), synth.tree_geo(rng, 20)
+    forest = np.concatenate([a, np.where(b2 < 0, -1, b2 + 30)]).astype(np.int32)
+    trees = [synth.tree_geo(rng, 64), forest, synth.tree_chain(16), synth.tree_bestfirst(rng, 300, width=4),
+             synth.tree_star(9)]
+    w = synth.random_case(124, trees, 2, 4, 128, 128, synth.BF16, synth.BF16, name="recurrent_ragged")
+    ref = tl.oracle_verify(w)
+    dc = tl.DeviceCase(w)
+    assert gdn.gdn_tree_verify_recurrent(dc.shape, dc.S0, dc.q, dc.k, dc.v, dc.g, dc.beta, dc.parent, dc.node_offsets,
+                                         dc.o, dc.status) == 0
+    assert dc.device_status() == 0
+    tl.assert_close_per_head(dc.o_host(), ref, w.node_offsets, "recurrent ragged", bf16_out=True)
+    dc.o.zero_()
+    assert dc.verify() == 0 and dc.device_status() == 0
+    tl.assert_close_per_head(dc.o_host(), ref, w.node_offsets, "tensor-core ragged", bf16_out=True)
+
+
+def test_recurrent_comparator_rejects_a_broken_branch(tl):
+    import paper_2607_06763_b200 as gdn
+    w = synth.random_case(125, [synth.tree_chain(20)], 1, 2, 64, 64, synth.F32, synth.F32)
+    dc = tl.DeviceCase(w)     # max_depth 16 < 20 nodes on the only branch
+    dc.o.fill_(7.0)
+    assert gdn.gdn_tree_verify_recurrent(dc.shape, dc.S0, dc.q, dc.k, dc.v, dc.g, dc.beta, dc.parent, dc.node_offsets,
+                                         dc.o, dc.status) == 0
+    assert dc.device_status() == -8 and bool((dc.o == 7.0).all())
