@@ -36,13 +36,15 @@ METRIC = "verified tree-nodes/sec per GDN layer"
 UNIT = "nodes/s"
 CONFIG_WORKLOADS = {"stack48_T64": 5, "layer_T64": 1, "stack48_T256": 2, "ragged32": 3, "chains64x16": 4}
 SWEEP_T = (32, 64, 128, 256, 512)
-WORKLOADS = sorted(CONFIG_WORKLOADS) + [f"sweep_T{t}" for t in SWEEP_T]
+WORKLOADS = sorted(CONFIG_WORKLOADS) + [f"sweep_T{t}" for t in SWEEP_T] + ["stack48_T64_deep"]
 DTYPE = "bf16 inputs/outputs, fp32 state; contractions as bf16 hi+lo splits on tcgen05 with fp32 accumulation"
 
 
 def make_workload(args) -> synth.Workload:
     if args.workload in CONFIG_WORKLOADS:
         return synth.config(CONFIG_WORKLOADS[args.workload], 0, n_layers=args.layers)
+    if args.workload == "stack48_T64_deep":
+        return synth.deep_stack(args.path_len, n_layers=args.layers)
     return synth.layer_sweep(int(args.workload.split("_T")[1]))
 
 
@@ -258,6 +260,11 @@ def main():
     ap.add_argument("--mode", default="fused", choices=["fused", "separate", "verify"],
                     help="fused: one gdn_tree_commit_verify call per step; separate: gdn_tree_verify + gdn_tree_commit; "
                          "verify: gdn_tree_verify alone (no commit; for kernel comparisons)")
+    ap.add_argument("--path-len", type=int, default=16,
+                    help="workload stack48_T64_deep: nodes on the accepted path (0..16)")
+    ap.add_argument("--commit", default="replay", choices=["cached", "replay"],
+                    help="fused mode: cached = gdn_tree_commit_verify_cached (the commit reads the projections the "
+                         "previous step's call left in its workspace); replay = gdn_tree_commit_verify")
     ap.add_argument("--graph", action="store_true",
                     help="fused mode: capture one step per buffer set in a CUDA graph and time replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -274,6 +281,8 @@ def main():
         return
     if args.impl == "recurrent":
         args.mode = "verify"
+    if args.graph:
+        args.commit = "replay"   # a captured step has its workspace baked in; the cached form alternates two
 
     w = make_workload(args)
     if args.impl == "reference":
@@ -306,7 +315,10 @@ def main():
         d["path"] = to_dev(w.path if w.path.size else np.zeros(1, np.int32))
         odt = torch.float32 if w.out_dtype == synth.F32 else torch.bfloat16
         d["o"] = torch.empty((w.total_nodes, w.h_v, w.d_v), dtype=odt, device="cuda")
-        d["ws"] = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        # two workspaces per set: a step reads the projection cache of the step before it and writes its own
+        d["ws2"] = [torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        d["ws"] = d["ws2"][0]
+        d["visits"] = 0
         sets.append(d)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
@@ -329,10 +341,20 @@ def main():
     def step_fused(d, stream=stream):
         # one decode iteration as the paper schedules it: commit the previous step's accepted path, then verify
         # the new tree against the advanced state (here the previous and the new tree carry the same tensors)
-        rc = gdn.gdn_tree_commit_verify(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
-                                        d["node_offsets"], d["path"], d["path_offsets"], d["q"], d["k"], d["v"],
-                                        d["g"], d["beta"], d["parent"], d["node_offsets"], d["o"], d["ws"], ws_bytes,
-                                        status, stream)
+        if args.commit == "replay":
+            rc = gdn.gdn_tree_commit_verify(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
+                                            d["node_offsets"], d["path"], d["path_offsets"], d["q"], d["k"], d["v"],
+                                            d["g"], d["beta"], d["parent"], d["node_offsets"], d["o"], d["ws"],
+                                            ws_bytes, status, stream)
+        else:
+            # the state of this set was last verified (against exactly what it holds now) by the previous step on
+            # this set, which left its projection cache in the other workspace
+            prev_ws, ws = d["ws2"][(d["visits"] + 1) & 1], d["ws2"][d["visits"] & 1]
+            d["visits"] += 1
+            rc = gdn.gdn_tree_commit_verify_cached(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
+                                                   d["node_offsets"], d["path"], d["path_offsets"], prev_ws,
+                                                   w.total_nodes, d["q"], d["k"], d["v"], d["g"], d["beta"],
+                                                   d["parent"], d["node_offsets"], d["o"], ws, ws_bytes, status, stream)
         assert rc == 0, gdn.gdn_status_string(rc)
 
     step = {"fused": step_fused, "separate": step_separate, "verify": step_verify}[args.mode]
@@ -496,6 +518,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": DTYPE if w.in_dtype == synth.BF16 else "f32", "data": "synthetic",
             "config": workload_config(w, args), "mode": args.mode, "impl": args.impl,
+            "commit": args.commit if args.mode == "fused" else "replay",
             "timing": {"regions": len(region_ms), "steps_per_region": args.steps,
                        "ms_per_step_median_region": med_region / args.steps,
                        "ms_per_step_fastest_region": min_region / args.steps,

@@ -92,10 +92,12 @@ typedef struct gdn_shape {
 const char *gdn_status_string(int status);
 
 /*
- * Bytes of device scratch gdn_tree_verify needs for this shape (tree metadata
- * of Section 3.4.2 -- per node its depth and ancestor list -- plus the cached
- * solve result u~ [N][h_v][d_v] fp32, the quantity "u_j - w_j^T S0" that the
- * substitution of Eq. 13 returns).  Returns 0 if the shape is invalid.
+ * Bytes of device scratch gdn_tree_verify needs for this shape: tree metadata
+ * of Section 3.4.2 (per node its depth and ancestor list), the solve result
+ * u~ [N][h_v][d_v] fp32 of the general kernel (the quantity "u_j - w_j^T S0"
+ * that the substitution of Eq. 13 returns), and the projection cache
+ * [N][h_v][d_v] fp32 that gdn_tree_commit_verify_cached reads one step later.
+ * Returns 0 if the shape is invalid.
  */
 size_t gdn_tree_workspace_bytes(const gdn_shape_t *shape);
 
@@ -118,7 +120,8 @@ int gdn_tree_validate_host(const gdn_shape_t *shape, const int32_t *parent_h,
  *   S0, q, k, v, g, beta, parent, node_offsets : [device], read-only
  *   o            : [device], written for every node of every valid tree
  *   workspace    : [device], >= gdn_tree_workspace_bytes(shape) bytes, 256-byte aligned;
- *                  contents after the call: the tree metadata and u~ (reused by nothing else)
+ *                  contents after the call: tree metadata, u~, and on the tensor-core path the
+ *                  projection cache (see gdn_tree_commit_verify_cached)
  *   status_dev   : [device] one int32, see "Return value" above
  */
 int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const void *q, const void *k,
@@ -185,6 +188,40 @@ int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_pre
                            const void *g, const void *beta, const int32_t *parent,
                            const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
                            int32_t *status_dev, void *cuda_stream);
+
+/*
+ * gdn_tree_commit_verify with the commit taken from what the previous verification cached
+ * (Section 3.4.1, Eq. 12: the end state of an accepted node follows directly from quantities the
+ * verification pass has already computed, so the commit needs no second pass over the prefix).
+ * Every verification on the tensor-core path (gdn_tree_verify, gdn_tree_commit_verify[_cached]; trees
+ * of at most 64 nodes, d_k = d_v = 128, bf16 inputs) leaves in its workspace the projections
+ * S^T k_n of the state it verified against onto the key of every node n.  Given that workspace, the
+ * commit of an accepted path n_1..n_L is Eq. 12 restricted to the path: with A_t the decay up to
+ * step t,   (I + M) w = r,  r_t = beta_t (v_t / A_t - S^T k_{n_t}),  M_tj = beta_t k_t.k_j (j < t),
+ *           S_new = A_L (S + sum_t w_t k_t^T),
+ * a rank-L update with no recurrence over d_k; results equal gdn_tree_commit_verify within the same
+ * tolerances (the projections carry the 2^-16 relative error of the tensor-core operand split).
+ *   prev_workspace    : [device] or NULL: the workspace given to the call that verified the PREVIOUS
+ *                       trees (whose accepted paths are committed now), untouched since; read-only
+ *                       here and different from `workspace`.  That call must have verified exactly
+ *                       the trees described by k_prev .. node_offsets_prev against exactly the state
+ *                       S holds now -- the sequence verify(t), commit_verify(t+1), ... of Section 3.4
+ *                       guarantees it.  The cache is tagged with the shape of the call that wrote it;
+ *                       NULL, a tag that does not match (n_seq, h_v, prev_total_nodes), a call that ran
+ *                       on another kernel, or a path that decays below 2^-80 make the commit fall back
+ *                       to the step-by-step replay of gdn_tree_commit_verify.
+ *   prev_total_nodes  : rows of the previous step's packed tensors (node_offsets_prev[n_seq])
+ * Other arguments, error reporting and the treatment of rejected paths and trees as for
+ * gdn_tree_commit_verify.  On shapes outside the tensor-core path the cache is ignored.
+ */
+int gdn_tree_commit_verify_cached(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
+                                  const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                  const int32_t *node_offsets_prev, const int32_t *path,
+                                  const int32_t *path_offsets, const void *prev_workspace,
+                                  int32_t prev_total_nodes, const void *q, const void *k, const void *v,
+                                  const void *g, const void *beta, const int32_t *parent,
+                                  const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
+                                  int32_t *status_dev, void *cuda_stream);
 
 /*
  * Host-buffer variants: same operations with every tensor in [host] memory

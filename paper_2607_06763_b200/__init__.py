@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     gdn_tree_commit,
     gdn_tree_commit_host,
     gdn_tree_commit_verify,
+    gdn_tree_commit_verify_cached,
     gdn_tree_commit_verify_host,
     gdn_tree_commit_verify_host_arena_bytes,
     gdn_tree_host_arena_bytes,

@@ -227,19 +227,23 @@ extern "C" int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k
     return GDN_OK;
 }
 
-extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
-                                      const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
-                                      const int32_t *node_offsets_prev, const int32_t *path,
-                                      const int32_t *path_offsets, const void *q, const void *k, const void *v,
-                                      const void *g, const void *beta, const int32_t *parent,
-                                      const int32_t *node_offsets, void *o, void *workspace,
-                                      size_t workspace_bytes, int32_t *status_dev, void *cuda_stream)
+namespace {
+
+int commit_verify_impl(bool cached, const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
+                       const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                       const int32_t *node_offsets_prev, const int32_t *path, const int32_t *path_offsets,
+                       const void *prev_workspace, int32_t prev_total_nodes, const void *q, const void *k,
+                       const void *v, const void *g, const void *beta, const int32_t *parent,
+                       const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
+                       int32_t *status_dev, void *cuda_stream)
 {
     int rc = check_shape(shape);
     if (rc != GDN_OK) return rc;
     const gdn_shape_t &s = *shape;
     if (s.n_seq == 0) return GDN_OK;
     if (!S || !node_offsets_prev || !path_offsets || !status_dev) return GDN_ERR_NULL;
+    if (prev_workspace && (prev_total_nodes < 0 || !aligned256(prev_workspace))) return GDN_ERR_ALIGN;
+    if (prev_workspace && prev_workspace == workspace) return GDN_ERR_WORKSPACE;   // the cache is read while the new one is written
     if (!verify_sm100_single_group(s) || s.total_nodes == 0) {
         // general shapes: the two kernels back to back on the stream (the shape's node counts are
         // not used by commit, so the new tree's shape serves for the previous tree as well).  Both
@@ -271,11 +275,52 @@ extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const 
     const WorkspaceLayout lay = workspace_layout(s);
     if (workspace_bytes < lay.total) return GDN_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const PlanPtrs plan = plan_ptrs(workspace, lay);
+    const float *pcache_prev = nullptr;
+    const int32_t *tag_prev = nullptr;
+    if (prev_workspace) {   // the previous trees' workspace has the layout of their shape
+        gdn_shape_t prev = s;
+        prev.total_nodes = prev_total_nodes;
+        const WorkspaceLayout pl = workspace_layout(prev);
+        const char *pb = static_cast<const char *>(prev_workspace);
+        pcache_prev = reinterpret_cast<const float *>(pb + pl.pcache);
+        tag_prev = reinterpret_cast<const int32_t *>(pb + pl.cache_tag);
+    }
     if (launch_commit_verify_sm100(s, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
-                                   path_offsets, q, k, v, g, beta, parent, node_offsets, o, status_dev,
-                                   stream) != cudaSuccess)
+                                   path_offsets, q, k, v, g, beta, parent, node_offsets, o, plan, pcache_prev,
+                                   tag_prev, prev_total_nodes, cached, status_dev, stream) != cudaSuccess)
         return GDN_ERR_CUDA;
     return GDN_OK;
+}
+
+}  // namespace
+
+extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
+                                      const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                      const int32_t *node_offsets_prev, const int32_t *path,
+                                      const int32_t *path_offsets, const void *q, const void *k, const void *v,
+                                      const void *g, const void *beta, const int32_t *parent,
+                                      const int32_t *node_offsets, void *o, void *workspace,
+                                      size_t workspace_bytes, int32_t *status_dev, void *cuda_stream)
+{
+    return commit_verify_impl(false, shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
+                              path_offsets, nullptr, 0, q, k, v, g, beta, parent, node_offsets, o, workspace,
+                              workspace_bytes, status_dev, cuda_stream);
+}
+
+extern "C" int gdn_tree_commit_verify_cached(const gdn_shape_t *shape, float *S, const void *k_prev,
+                                             const void *v_prev, const void *g_prev, const void *beta_prev,
+                                             const int32_t *parent_prev, const int32_t *node_offsets_prev,
+                                             const int32_t *path, const int32_t *path_offsets,
+                                             const void *prev_workspace, int32_t prev_total_nodes, const void *q,
+                                             const void *k, const void *v, const void *g, const void *beta,
+                                             const int32_t *parent, const int32_t *node_offsets, void *o,
+                                             void *workspace, size_t workspace_bytes, int32_t *status_dev,
+                                             void *cuda_stream)
+{
+    return commit_verify_impl(true, shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
+                              path_offsets, prev_workspace, prev_total_nodes, q, k, v, g, beta, parent, node_offsets,
+                              o, workspace, workspace_bytes, status_dev, cuda_stream);
 }
 
 extern "C" size_t gdn_tree_host_arena_bytes(const gdn_shape_t *shape, int32_t total_path_len)

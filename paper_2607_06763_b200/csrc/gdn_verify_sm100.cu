@@ -22,6 +22,8 @@
 // Two kernels: a persistent one for trees that fit one CTA (TMA tiles on mbarriers, a software pipeline across
 // the units of a CTA, optionally the commit of the previous step fused in front), and a one-shot one for the
 // groups of larger trees (row gathers through a node table).
+#include <cstdlib>
+#include <type_traits>
 #include <cuda.h>   // CUtensorMap and the cuTensorMapEncodeTiled prototype (resolved at run time, no libcuda link)
 
 #include "gdn_internal.cuh"
@@ -71,7 +73,11 @@ constexpr int SM_TMEM = SM_MBAR + 40;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
 constexpr int SM_PAR = SM_FLAG + 4;              // persistent kernel: s8 [64] parent[] of the tree whose tables are being built
 constexpr int SM_BAD = SM_PAR + FV_T;            // persistent kernel: int [2], tree of table buffer tb was rejected
-constexpr int SM_BYTES = SM_BAD + 8;
+constexpr int SM_GM = (SM_BAD + 8 + 15) & ~15;   // fused commit from the cache: fp32 k_t . k_j of the path, j < t, at t (t - 1) / 2 + j
+constexpr int SM_NM = SM_GM + 480;               //   fp32 N = (I + M)^-1, M_tj = beta_t k_t . k_j: N_tj, j <= t, at t (t + 1) / 2 + j
+constexpr int SM_BYTES = SM_NM + 544;
+constexpr int SM_PC = 57344;                     // fused commit from the cache: fp32 [16][128] cached projections of the path's
+                                                 // nodes, then (in place) the update coefficients w; in the state-operand area
 constexpr int SM_ALLOC = SM_BYTES + 1024;        // slack for the 1024-byte alignment of the base
 
 // Development aid: with -DGDN_TRACE thread 0 of every CTA records clock64() at each phase boundary into a
@@ -116,6 +122,9 @@ struct VerifyFastParams {
     const uint8_t *depth;
     const uint8_t *anc8;
     int32_t *status_dev;
+    // projection cache (persistent kernel): rows S^T k_n of every node, left for the commit of the next step
+    float *pcache_out;
+    int32_t *cache_tag_out;
     // grouped verification of trees with more than 64 nodes (only read by the GROUPED instantiation)
     int groups_per_tree, anc_stride;                   // CTAs per (tree, head); entries per row of anc16
     const uint16_t *anc16, *dfs_node, *group_start;
@@ -124,6 +133,10 @@ struct VerifyFastParams {
     float *S_rw;                                       // same tensor as S0, written in place
     const __nv_bfloat16 *pk, *pv, *pg, *pbeta;         // the previous tree's k, v, g, beta
     const int32_t *pparent, *pnode_offsets, *path, *path_offsets;
+    const float *pcache_prev;                          // projection cache of the previous trees (may be NULL)
+    const int32_t *cache_tag_prev;
+    int prev_total_nodes;
+    int cached_min_len;                                // shortest accepted path that is committed from the cache
 };
 
 // ---------------------------------------------------------------------------------------- PTX
@@ -774,10 +787,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 // Persistent form of the kernel above for trees that fit one CTA, with the optional fused commit.  The k/q tile
 // holds the k rows first and the q rows second (rows i and 64 + i), so P has p^k in columns 0..63 and p^q in
 // columns 64..127, and the Gram block needs only N = 64.
-// FUSED: Eq. 7 is replayed along the previous step's accepted path on the state tile while it sits in registers
-// -- per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c), the eight lanes that share a row reducing k.s_c with
-// three shuffles -- the tile is written back as the only state write of the step, and the new tree is verified
-// against it.
+// FUSED: the previous step's accepted path is committed on the state tile while it sits in registers, the tile is
+// written back as the only state write of the step, and the new tree is verified against it.  Two forms:
+//  - replay: per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c) step by step, the eight lanes that share a row
+//    reducing k.s_c with three shuffles;
+//  - from the projection cache (the masked end-state formula, Eq. 12, restricted to the accepted path).  Every
+//    verification leaves p_n = S^T k_n of all its nodes in its workspace (they are in registers in the R phase
+//    anyway).  With A_t = alpha_1..alpha_t and S~_t = S_t / A_t, Eq. 7 reads S~_t = S~_{t-1} + w_t k_t^T with
+//        (I + M) w = r,   r_t = beta_t (v_t / A_t - p_{n_t}),   M_tj = beta_t (k_t . k_j) for j < t,
+//    an L x L triangular system shared by all 128 value components: its inverse N is formed once per unit (sixteen
+//    threads, one column each), w = N r by all threads, and the commit is the rank-L update S_new = A_L (S0 + sum_t
+//    w_t k_t^T) on the registers: no dot product over d_k, no shuffle, no step that waits for the one before.
 // A CTA keeps its tensor memory and walks over the units blockIdx.x, blockIdx.x + gridDim.x, ...  Nothing a unit
 // can know in advance is waited for inside it: the next unit's k/q tile streams into the operand tile as soon as the
 // first MMA group has released it, its Gram block is issued at the end of the current unit into spare TMEM columns,
@@ -785,7 +805,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 // its value is used.  The state tile is asked for at the top of the unit and is needed only after the Gram /
 // coefficient phases; the v rows land by TMA in an area that is free until the state operand is written.
 // SMALL (every tree of the call has at most 32 nodes): the R and output phases skip the 16-node pieces beyond the tree.
-template <typename TOut, bool FUSED, bool SMALL>
+template <typename TOut, bool FUSED, bool SMALL, bool CACHED>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const __grid_constant__ VerifyFastParams p)
 {
     extern __shared__ uint8_t fv_smem_raw[];
@@ -823,6 +843,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // The first unit's state tile is an input of the call, not of that kernel: L2 is asked for it meanwhile.
     if (tid < 4 && (int)blockIdx.x < p.n_units)
         prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
+    bool use_cache = false;   // FUSED: commit from the projection cache (decided once per call, below)
     signed char *par_s = reinterpret_cast<signed char *>(smem + SM_PAR);
     volatile int *bad_s = reinterpret_cast<volatile int *>(smem + SM_BAD);
 
@@ -963,17 +984,18 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 if (lane == 0) {
                     slot[16] = len;
                     slot[17] = pb;
+                    slot[18] = len;
                 }
             }
         }
     };
-    // k and v rows of that path (bf16, 256 B each) into their parking area and the per-step scalars into the
-    // slot: issued by everybody once the slot is readable and the parking area is free
-    auto fetch_path_rows = [&](int uh, int uhk, int ps, bool scalars) {
+    // k and v rows of that path (bf16, 256 B each) into their parking area: issued by everybody once the slot is
+    // readable and the parking area is free.  Only node ids that have been range-checked are used (slot[18] =
+    // length of the path as far as it has been checked when the rows are asked for).
+    auto fetch_path_kv = [&](int uh, int uhk, int ps) {
         if constexpr (FUSED) {
             const int *slot = reinterpret_cast<const int *>(smem + SM_PATH + ps * SM_PATH_SLOT);
-            float4 *ab = reinterpret_cast<float4 *>(smem + SM_PATH + ps * SM_PATH_SLOT + 128);
-            const int len = slot[16], pb = slot[17];
+            const int len = slot[18], pb = slot[17];
             for (int idx = tid; idx < len * 32; idx += FV_THREADS) {
                 const int t = idx >> 5, c16 = idx & 15;
                 const size_t n = (size_t)pb + slot[t];
@@ -982,7 +1004,29 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 else
                     cp_async_16(sbase + SM_PK + t * 256 + c16 * 16, p.pk + (n * p.h_qk + uhk) * FV_D + c16 * 8, true);
             }
-            if (scalars && tid < len) {
+        }
+    };
+    // cached projections of the path's nodes (fp32, 512 B each) into their parking area
+    auto fetch_path_pc = [&](int uh, int ps) {
+        if constexpr (FUSED && CACHED) {
+            if (use_cache) {
+                const int *slot = reinterpret_cast<const int *>(smem + SM_PATH + ps * SM_PATH_SLOT);
+                const int len = slot[16], pb = slot[17];
+                for (int idx = tid; idx < len * 32; idx += FV_THREADS) {
+                    const int t = idx >> 5, c16 = idx & 31;
+                    const size_t n = (size_t)pb + slot[t];
+                    cp_async_16(sbase + SM_PC + t * 512 + c16 * 16, p.pcache_prev + (n * p.h_v + uh) * FV_D + c16 * 4, true);
+                }
+            }
+        }
+    };
+    // per-step scalars of the path, computed on the spot (first unit of a CTA, and behind a skipped unit)
+    auto path_scalars_direct = [&](int uh, int ps) {
+        if constexpr (FUSED) {
+            const int *slot = reinterpret_cast<const int *>(smem + SM_PATH + ps * SM_PATH_SLOT);
+            float4 *ab = reinterpret_cast<float4 *>(smem + SM_PATH + ps * SM_PATH_SLOT + 128);
+            const int len = slot[16], pb = slot[17];
+            if (tid < len) {
                 float gsum = 0.f, gt = 0.f;
                 for (int t = 0; t <= tid; ++t) {
                     gt = __bfloat162float(p.pg[((size_t)pb + slot[t]) * p.h_v + uh]);
@@ -991,6 +1035,38 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 const size_t n = (size_t)pb + slot[tid];
                 const float A = expf(gsum);
                 ab[tid] = make_float4(A, __bfloat162float(p.pbeta[n * p.h_v + uh]), expf(gt), 1.f / A);
+            }
+        }
+    };
+    // k_t . k_j for the pairs j < t of the path whose k rows have landed: eight lanes per pair, 32 pairs per round
+    auto path_gram = [&](int ps) {
+        if constexpr (FUSED && CACHED) {
+            if (use_cache) {
+                float *gm = reinterpret_cast<float *>(smem + SM_GM);
+                const int len = reinterpret_cast<const int *>(smem + SM_PATH + ps * SM_PATH_SLOT)[16];
+                const int n_pairs = len * (len - 1) / 2;
+                for (int pi0 = warp * 4; pi0 < n_pairs; pi0 += FV_THREADS / 8) {   // warp-uniform trip count
+                    const int pi = min(pi0 + r4, n_pairs - 1);
+                    int t = 1, j = pi;
+                    while (j >= t) { j -= t; ++t; }
+                    const uint16_t *pk = reinterpret_cast<const uint16_t *>(smem + SM_PK);
+                    float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+                    for (int kh = 0; kh < 2; ++kh) {
+                        const uint4 a = *reinterpret_cast<const uint4 *>(pk + t * FV_D + kh * 64 + l8 * 8);
+                        const uint4 c = *reinterpret_cast<const uint4 *>(pk + j * FV_D + kh * 64 + l8 * 8);
+                        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            acc = __ffma2_rn(make_float2(__uint_as_float(aw[e] << 16), __uint_as_float(aw[e] & 0xFFFF0000u)),
+                                             make_float2(__uint_as_float(cw[e] << 16), __uint_as_float(cw[e] & 0xFFFF0000u)), acc);
+                    }
+                    float dot = acc.x + acc.y;
+                    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+                    if (l8 == 0 && pi0 + r4 < n_pairs) gm[pi] = dot;
+                }
             }
         }
     };
@@ -1033,6 +1109,16 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // ... and whatever is launched behind this grid with the same attribute (the next call's tree-metadata kernel,
     // which itself waits for this grid to complete before it reads or writes anything) may be made resident now.
     asm volatile("griddepcontrol.launch_dependents;");
+    if constexpr (FUSED && CACHED) {
+        // the projection cache of the previous trees is used if the call that left it had their shape
+        if (p.pcache_prev && p.cache_tag_prev) {
+            const int4 tg = __ldg(reinterpret_cast<const int4 *>(p.cache_tag_prev));
+            use_cache = tg.x == GDN_CACHE_MAGIC && tg.y == p.prev_total_nodes && tg.z == p.h_v && tg.w == p.n_seq;
+        }
+    }
+    if (blockIdx.x == 0 && tid == 0 && p.cache_tag_out)
+        *reinterpret_cast<int4 *>(p.cache_tag_out) =
+            CACHED && p.pcache_out ? make_int4(GDN_CACHE_MAGIC, p.total_nodes, p.h_v, p.n_seq) : make_int4(0, 0, 0, 0);
     bool cur_ok = decode(blockIdx.x, b, h, hk, base, T);
     bool par_bad = false;
     if (cur_ok) {
@@ -1045,8 +1131,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     __syncthreads();
     if (cur_ok) {
         path_decay(0);
-        fetch_path_rows(h, hk, 0, true);
+        fetch_path_kv(h, hk, 0);
+        fetch_path_pc(h, 0);
+        path_scalars_direct(h, 0);
         issue_gram(0);
+    }
+    if constexpr (FUSED && CACHED) {
+        if (use_cache) {   // (call-uniform) the k rows have to be there for the path's Gram block
+            cp_async_wait_all();
+            __syncthreads();
+            if (cur_ok) path_gram(0);
+        }
     }
 
     int done_units = 0;
@@ -1072,8 +1167,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         __syncthreads();
         if (next_ok) {
             path_decay((iter + 1) & 1);
-            fetch_path_rows(nh, nhk, (iter + 1) & 1, true);
+            fetch_path_kv(nh, nhk, (iter + 1) & 1);
+            fetch_path_pc(nh, (iter + 1) & 1);
+            path_scalars_direct(nh, (iter + 1) & 1);
             issue_gram(par);   // no unit was processed in between: the tile's barrier phase is this one
+        }
+        if constexpr (FUSED && CACHED) {
+            if (use_cache) {
+                cp_async_wait_all();
+                __syncthreads();
+                if (next_ok) path_gram((iter + 1) & 1);
+            }
         }
         b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
         continue;
@@ -1130,11 +1234,47 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // flags the error and everybody falls through to the clean-up).
     if (!mbar_wait_bounded(mbar_g, par)) *flag = 1;
     GDN_TRACE_MARK_U(unit, 2);
+    if constexpr (CACHED) {
+        if (use_cache) cp_async_wait_all();   // the path's cached projections, asked for one unit ahead
+    }
     tc_fence_after();
     __syncthreads();
     GDN_TRACE_MARK_U(unit, 3);
     warm_l2_state(0);
+    // Form of the commit (unit-uniform; the path's scalars were written behind the last barrier of the unit before
+    // and are readable from here on): from the cache unless the path decays below 2^-80 (1 / A_t could overflow).
+    bool cached_commit = false;
+    if constexpr (FUSED && CACHED)
+        cached_commit = use_cache && path_len >= p.cached_min_len && path_len > 0 && ab_path[path_len - 1].x > 8.3e-25f;
     if (*flag == 0) {
+        if constexpr (FUSED && CACHED) {
+            // N = (I + M)^-1, M_tj = beta_t (k_t . k_j): lane j of warp 4 builds column j (u_m = N_{j+m,j})
+            if (cached_commit && warp == 4 && lane < path_len) {
+                const float *gm = reinterpret_cast<const float *>(smem + SM_GM);
+                float *nm = reinterpret_cast<float *>(smem + SM_NM);
+                const int j = lane;
+                nm[j * (j + 1) / 2 + j] = 1.f;
+                auto column = [&](auto lb) {   // unrolled for paths of at most LB nodes
+                    constexpr int LB = decltype(lb)::value;
+                    float u[LB];
+                    u[0] = 1.f;
+#pragma unroll
+                    for (int m = 1; m < LB; ++m) {
+                        const int t = j + m;
+                        float acc = 0.f;
+                        if (t < path_len) {
+#pragma unroll
+                            for (int n = 0; n < m; ++n) acc = fmaf(gm[t * (t - 1) / 2 + j + n], u[n], acc);
+                            acc *= -ab_path[t].y;
+                            nm[t * (t + 1) / 2 + j] = acc;
+                        }
+                        u[m] = acc;
+                    }
+                };
+                if (path_len <= 8) column(std::integral_constant<int, 8>{});
+                else column(std::integral_constant<int, 16>{});
+            }
+        }
         // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
         {
             const int row = (warp & 3) * 32 + lane;
@@ -1184,6 +1324,43 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 xs[idx] = onx[u] ? bi[u] * dec * gk[u] : 0.f;
             }
         }
+        if constexpr (FUSED && CACHED) {
+            // w = N r for value component c = tid / 2, r_j = beta_j (v_j[c] / A_j - p_j[c]); the two threads of a
+            // component take the even and the odd steps, and w replaces p in place (every r is in registers before
+            // either of them stores: __syncwarp)
+            if (cached_commit) {
+                const float *nm = reinterpret_cast<const float *>(smem + SM_NM);
+                float *pc = reinterpret_cast<float *>(smem + SM_PC);
+                const uint16_t *pv = reinterpret_cast<const uint16_t *>(smem + SM_PV);
+                const int c = tid >> 1, hf = tid & 1;
+                auto coefficients = [&](auto lb) {   // unrolled for paths of at most LB nodes
+                    constexpr int LB = decltype(lb)::value;
+                    float r[LB];
+#pragma unroll
+                    for (int j = 0; j < LB; ++j) {
+                        r[j] = 0.f;
+                        if (j < path_len) {
+                            const float4 ab = ab_path[j];
+                            r[j] = ab.y * fmaf(__uint_as_float((uint32_t)pv[j * FV_D + c] << 16), ab.w, -pc[j * FV_D + c]);
+                        }
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int tt = 0; tt < LB / 2; ++tt) {
+                        const int t = 2 * tt + hf;
+                        if (2 * tt < path_len) {   // warp-uniform
+                            float acc = 0.f;
+#pragma unroll
+                            for (int j = 0; j <= 2 * tt + 1; ++j)
+                                if (j <= t) acc = fmaf(nm[t * (t + 1) / 2 + j], r[j], acc);
+                            if (t < path_len) pc[t * FV_D + c] = acc;
+                        }
+                    }
+                };
+                if (path_len <= 8) coefficients(std::integral_constant<int, 8>{});
+                else coefficients(std::integral_constant<int, 16>{});
+            }
+        }
     }
     cp_async_wait_all();
     __syncthreads();   // X and Y complete; the Gram copy is dead and its area can take the state operand
@@ -1193,10 +1370,46 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // sits in registers, write it back, and let everything below verify the new tree against it.
     // Per row c (one value component): s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that
     // share a row reduce k.s_c with three shuffles.  The path's k/v rows were fetched above.
+    const bool healthy = *flag == 0;   // uniform: every write of the flag so far lies before the barrier above
     if constexpr (FUSED) {
-        if (path_len > 0)
+        if (!healthy) path_len = 0;    // a wait expired: this state is left as it was
+        if (cached_commit && healthy) {
+            // S_new = A_L (S0 + sum_t w_t k_t^T): rank-L update of the registers
+            const float *wcol = reinterpret_cast<const float *>(smem + SM_PC) + warp * 16 + r4;
+            const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
+#pragma unroll 1
+            for (int t = 0; t < path_len; ++t) {
+                float2 kf2[8];
+#pragma unroll
+                for (int kh = 0; kh < 2; ++kh) {
+                    const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
+                    const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        kf2[kh * 4 + e] = make_float2(__uint_as_float(w4[e] << 16), __uint_as_float(w4[e] & 0xFFFF0000u));
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float wv = wcol[t * FV_D + i * 4];
+                    const float2 w2 = make_float2(wv, wv);
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, make_float2(x[i][q4].x, x[i][q4].y));
+                        const float2 hi = __ffma2_rn(kf2[q4 * 2 + 1], w2, make_float2(x[i][q4].z, x[i][q4].w));
+                        x[i][q4] = make_float4(lo.x, lo.y, hi.x, hi.y);
+                    }
+                }
+            }
+            const float aL = ab_path[path_len - 1].x;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    x[i][q4] = make_float4(aL * x[i][q4].x, aL * x[i][q4].y, aL * x[i][q4].z, aL * x[i][q4].w);
+        } else if (path_len > 0) {
             replay_path_on_tile(x, path_len, reinterpret_cast<const uint16_t *>(smem + SM_PK),
                                 reinterpret_cast<const uint16_t *>(smem + SM_PV), ab_path, warp, r4, l8);
+        }
     }
     // The v rows move into registers in the orientation of the R phase (component c = TMEM lane of this
     // thread, its 32 nodes, two bf16 per register): they are about to be overwritten by the state operand.
@@ -1339,7 +1552,19 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             // the path entries are asked for
             t_bad = put_parent(nT, t_par, (iter + 1) & 1);
             if constexpr (FUSED) {
-                if (warp == 4 && q_mine && p.pparent && q_n >= 0 && q_n < q_pT) q_par = p.pparent[q_pb + q_n];
+                if (warp == 4) {
+                    // the entries are published as far as they are checked (inside the previous tree), so that
+                    // their rows can be asked for behind the next barrier; whether they form a chain is decided then
+                    int *slot = reinterpret_cast<int *>(smem + SM_PATH + ((iter + 1) & 1) * SM_PATH_SLOT);
+                    const bool in_range = q_mine && q_n >= 0 && q_n < q_pT;
+                    const bool all_in = __all_sync(0xffffffffu, !q_mine || in_range);
+                    if (lane < FV_MD) slot[lane] = in_range ? q_n : 0;
+                    if (lane == 0) {
+                        slot[17] = q_pb;
+                        slot[18] = q_shape_ok && all_in ? q_len : 0;
+                    }
+                    if (in_range && p.pparent) q_par = p.pparent[q_pb + q_n];
+                }
             }
         }
         {
@@ -1399,6 +1624,13 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                     bj[jj] = gj.z;
                 }
                 tmem_wait_ld();
+                // the projections S^T k_j go to the cache that a later commit of a path of this tree reads
+                if (CACHED && p.pcache_out) {
+                    float *dst = p.pcache_out + ((size_t)(base + j0) * p.h_v + h) * FV_D + c;
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj)
+                        if (j0 + jj < T) dst[(size_t)jj * p.h_v * FV_D] = __uint_as_float(rr[jj]);
+                }
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -1445,7 +1677,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 const int n_up = __shfl_up_sync(0xffffffffu, q_n, 1);
                 bool bad = false;
                 if (q_mine) {
-                    slot[lane] = q_n;
                     if (q_n < 0 || q_n >= q_pT) bad = true;
                     else if (p.pparent) bad = q_par != (lane ? n_up : -1);
                     else if (lane && q_n <= n_up) bad = true;
@@ -1466,6 +1697,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
 
+        if (use_cache && next_ok) fetch_path_kv(nh, nhk, (iter + 1) & 1);   // into an area that is free from now on
         // stage 5, while the tensor core works: the next unit's tables (depth, root paths) from the staged parent[]
         if (next_ok) walk_tables(nT, (iter + 1) & 1, t_g, t_be, t_bad);
         if (!mbar_wait_bounded(mbar_d, par)) *flag = 1;
@@ -1499,11 +1731,14 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
+        if (use_cache) cp_async_wait_all();   // the path's k and v rows, needed for their Gram block below
         __syncthreads();
-        // stage 6: the next unit's decay tables, and its path rows (published above, behind a barrier now; the area
-        // they land in is free)
+        // stage 6: the next unit's decay tables; the cached projections of its path (whose final length was
+        // published behind the barrier before this one) are asked for, and the Gram block of the path's keys is formed
         if (next_ok) path_decay((iter + 1) & 1);
-        if (next_ok) fetch_path_rows(nh, nhk, (iter + 1) & 1, false);
+        if (!use_cache && next_ok) fetch_path_kv(nh, nhk, (iter + 1) & 1);
+        if (next_ok) fetch_path_pc(nh, (iter + 1) & 1);
+        if (next_ok) path_gram((iter + 1) & 1);
         if constexpr (FUSED) {   // ... and the scalars of that path (asked for a phase ago)
             if (next_ok && warp == 4) {   // lane t: decay of the path up to and including step t by a prefix sum
                 const float gt = lane < q_len ? __uint_as_float((uint32_t)q_g << 16) : 0.f;
@@ -1604,7 +1839,15 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
             !make_row_tensor_map(&pt.tm_v, p.v, s.total_nodes, s.h_v, FV_D, false))
             return cudaErrorNotSupported;
         const bool small = s.max_tree_nodes <= 32;
-        auto kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true> : verify_sm100_persistent_kernel<TOut, FUSED, false>;
+        // the instantiation with the projection cache (read and/or written) exists for the fused form only
+        const bool cached = FUSED && (p.pcache_out || p.pcache_prev);
+        auto kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true, false>
+                            : verify_sm100_persistent_kernel<TOut, FUSED, false, false>;
+        if constexpr (FUSED) {
+            if (cached)
+                kernel = small ? verify_sm100_persistent_kernel<TOut, true, true, true>
+                               : verify_sm100_persistent_kernel<TOut, true, false, true>;
+        }
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
         if (e != cudaSuccess) return e;
         const int grid = p.n_units < p.prefetch_dist ? p.n_units : p.prefetch_dist;
@@ -1638,6 +1881,7 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     p.node_offsets = node_offsets; p.o = o;
     p.n_seq = s.n_seq; p.total_nodes = s.total_nodes; p.max_tree_nodes = s.max_tree_nodes; p.max_depth = s.max_depth;
     p.tree_ok = plan.tree_ok; p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
+    p.cache_tag_out = plan.cache_tag;   // the projection cache is written on request only (the tag says so)
     p.groups_per_tree = (s.max_tree_nodes + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;   // upper bound; a CTA
                                                                                             // without a group leaves at once
     p.anc_stride = s.max_depth;
@@ -1677,12 +1921,20 @@ cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const voi
                                        const int32_t *node_offsets_prev, const int32_t *path,
                                        const int32_t *path_offsets, const void *q, const void *k, const void *v,
                                        const void *g, const void *beta, const int32_t *parent,
-                                       const int32_t *node_offsets, void *o, int32_t *status_dev,
-                                       cudaStream_t stream)
+                                       const int32_t *node_offsets, void *o, const PlanPtrs &plan,
+                                       const float *pcache_prev, const int32_t *cache_tag_prev, int prev_total_nodes,
+                                       bool write_cache, int32_t *status_dev, cudaStream_t stream)
 {
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
-    VerifyFastParams p = make_params(s, S, q, k, v, g, beta, node_offsets, o, PlanPtrs{}, status_dev);
+    VerifyFastParams p = make_params(s, S, q, k, v, g, beta, node_offsets, o, plan, status_dev);
     p.parent = parent;
+    p.pcache_prev = pcache_prev; p.cache_tag_prev = cache_tag_prev; p.prev_total_nodes = prev_total_nodes;
+    if (write_cache) p.pcache_out = plan.pcache;
+    // Paths shorter than this are replayed even when the cache is there: inside this instantiation the cached form
+    // is the faster one from two nodes on (measured on B200; GDN_CACHED_MIN_LEN overrides the threshold, e.g. to
+    // time either form at every length).
+    p.cached_min_len = 2;
+    if (const char *e = getenv("GDN_CACHED_MIN_LEN")) p.cached_min_len = atoi(e);
     p.S_rw = S;
     p.pk = static_cast<const __nv_bfloat16 *>(k_prev); p.pv = static_cast<const __nv_bfloat16 *>(v_prev);
     p.pg = static_cast<const __nv_bfloat16 *>(g_prev); p.pbeta = static_cast<const __nv_bfloat16 *>(beta_prev);

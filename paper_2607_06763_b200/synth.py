@@ -326,6 +326,18 @@ def layer_sweep(T: int, rep: int = 0, out_dtype: str = BF16) -> Workload:
     return make_workload(f"layer_T{T}", [t], [longest_path(t)], 16, 32, 128, 128, BF16, out_dtype, rng)
 
 
+def deep_stack(path_len: int, n_layers: int = 48, rep: int = 0, out_dtype: str = BF16) -> Workload:
+    """Configuration "1x48" with a 64-node best-first tree that reaches depth 16 and an accepted path of exactly
+    ``path_len`` nodes (the first nodes of its deepest root path; 0..16): the accepted-length sweep of the commit."""
+    rng = np.random.Generator(np.random.PCG64(SEED_BASE + 101 * 7 + rep))
+    # a spine of 16 nodes (one accepted candidate per depth) with the rest of the 64-node budget hanging off its first
+    # 15 nodes as rejected siblings, three or four each: the shape of a deep, narrow best-first tree
+    t = bfs_renumber(np.asarray([i - 1 for i in range(16)] + [i % 15 for i in range(48)], np.int32))
+    p = longest_path(t)[:path_len]
+    return make_workload(f"stack{n_layers}_T64_deep_L{path_len}", [t] * n_layers, [p] * n_layers, 16, 32, 128, 128, BF16,
+                         out_dtype, rng, {"layers": n_layers})
+
+
 def random_case(seed: int, trees, h_qk, h_v, d_k, d_v, in_dtype=F32, out_dtype=F32, paths=None, name="case"):
     """A free-form case for tests: given trees, random accepted root paths unless ``paths`` is given."""
     rng = np.random.Generator(np.random.PCG64(seed))
