@@ -42,5 +42,5 @@ def build_library(force: bool = False, verbose: bool = False, extra_flags=()) ->
 
 
 if __name__ == "__main__":
-    flags = (["-Xptxas", "-v"] if "-v" in sys.argv else []) + (["-DGDN_TRACE"] if "--trace" in sys.argv else [])
+    flags = ["-Xptxas", "-v"] if "-v" in sys.argv else []
     print(build_library(force=True, verbose=True, extra_flags=flags))

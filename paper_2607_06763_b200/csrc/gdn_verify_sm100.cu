@@ -80,35 +80,12 @@ constexpr int SM_PC = 57344;                     // fused commit from the cache:
                                                  // nodes, then (in place) the update coefficients w; in the state-operand area
 constexpr int SM_ALLOC = SM_BYTES + 1024;        // slack for the 1024-byte alignment of the base
 
-// Development aid: with -DGDN_TRACE thread 0 of every CTA records clock64() at each phase boundary into a
-// buffer registered through gdn_trace_set_buffer(); normal builds compile none of it.
-#ifdef GDN_TRACE
-__device__ long long *g_trace_buf = nullptr;
-#define GDN_TRACE_MARK(k)                                                            \
-    do {                                                                             \
-        if (threadIdx.x == 0 && g_trace_buf) g_trace_buf[blockIdx.x * 16 + (k)] = clock64(); \
-    } while (0)
-#define GDN_TRACE_MARK_U(u, k)                                                       \
-    do {                                                                             \
-        if (threadIdx.x == 0 && g_trace_buf) g_trace_buf[(p.trace_call * p.n_units + (u)) * 16 + (k)] = clock64(); \
-    } while (0)
-#define GDN_TRACE_MARK_T(t, k)                                                       \
-    do {                                                                             \
-        if (threadIdx.x == (t) && g_trace_buf) g_trace_buf[blockIdx.x * 16 + (k)] = clock64(); \
-    } while (0)
-#else
-#define GDN_TRACE_MARK(k) do {} while (0)
-#define GDN_TRACE_MARK_U(u, k) do {} while (0)
-#define GDN_TRACE_MARK_T(t, k) do {} while (0)
-#endif
-
 struct VerifyFastParams {
     // TMA descriptors of the packed k, q, v tensors viewed as [N][heads][128] bf16 (persistent kernel only)
     alignas(64) CUtensorMap tm_k;
     alignas(64) CUtensorMap tm_q;
     alignas(64) CUtensorMap tm_v;
     int h_qk, h_v;
-    int trace_call;
     int n_units;        // n_seq * h_v
     int prefetch_dist;  // a CTA warms L2 for unit blockIdx.x + prefetch_dist (about one wave ahead)
     float scale;
@@ -370,17 +347,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         __syncthreads();
     }
     auto node_of = [&](int u) -> int { return GROUPED ? (int)vnode_s[u] : u; };
-    GDN_TRACE_MARK(0);
-#ifdef GDN_TRACE
-    if (threadIdx.x == 0 && g_trace_buf) {
-        unsigned smid;
-        unsigned long long gt;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-        g_trace_buf[blockIdx.x * 16 + 14] = smid;
-        g_trace_buf[blockIdx.x * 16 + 15] = (long long)gt;
-    }
-#endif
 
     // L2 warming for the unit that a CTA will pick up about one wave from now, issued in slices at
     // phase boundaries (one thread, a few instructions each) so that HBM keeps streaming while the resident
@@ -471,7 +437,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         *reinterpret_cast<uint4 *>(anc_s + tid * 16) = row;
         gab[tid] = make_float4(0.f, 0.f, be, gi);
     }
-    GDN_TRACE_MARK(1);
 
     cp_async_wait_all();
     fence_proxy_async();   // the k/q tile (cp.async) becomes visible to the tensor core
@@ -479,7 +444,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // warp-uniform by construction
-    GDN_TRACE_MARK(2);
 
     // (4) Everything that depends only on q, k, g, beta runs now, under the latency of the state loads:
     // Gram = [k;q].[k;q]^T on the tensor core, G_i / a_i tables, then X and Y of Eq. 9.
@@ -507,7 +471,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (tid == 0 && !mbar_wait_bounded(mbar_g, 0)) *flag = 1;
     __syncthreads();
     tc_fence_after();
-    GDN_TRACE_MARK(3);
     warm_l2_state(0);
     if (*flag == 0) {
         // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
@@ -529,7 +492,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         }
         tc_fence_before();
         __syncthreads();
-        GDN_TRACE_MARK(4);
         warm_l2_state(1);
         // X and Y for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
         {
@@ -560,7 +522,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     }
     cp_async_wait_all();
     __syncthreads();   // X and Y complete; the Gram copy is dead and its area can take the state operand
-    GDN_TRACE_MARK(5);
 
 
     // (4) fp32 -> bf16 hi + lo, written as the A operand
@@ -583,7 +544,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    GDN_TRACE_MARK(6);
     warm_l2_state(2);
 
     // (5) P = S0.[k;q]^T (hi then lo) on the tensor core; meanwhile the back-substitution below
@@ -627,12 +587,10 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
                 }
             }
         }
-    GDN_TRACE_MARK(7);
     if (tid == 0 && !mbar_wait_bounded(mbar_p, 0)) *flag = 1;
     __syncthreads();
     tc_fence_after();
     bool ok = *flag == 0;
-    GDN_TRACE_MARK(8);
     warm_l2_state(3);
 
     if (ok) {
@@ -669,7 +627,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         }
         cp_async_wait_all();
         __syncthreads();
-        GDN_TRACE_MARK(9);
 
         // (8) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
         // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
@@ -710,7 +667,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        GDN_TRACE_MARK(10);
         warm_l2_rows();
 
         // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
@@ -731,7 +687,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
         __syncthreads();
         tc_fence_after();
         ok = *flag == 0;
-        GDN_TRACE_MARK(11);
 
         // (10) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i]), staged through shared memory (over the
         // dead R^T tiles) so that global memory sees 16-byte stores of whole rows
@@ -771,14 +726,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     }
     if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
 
-    GDN_TRACE_MARK(12);
-#ifdef GDN_TRACE
-    if (threadIdx.x == 0 && g_trace_buf) {
-        unsigned long long gt;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-        g_trace_buf[blockIdx.x * 16 + 13] = (long long)gt;
-    }
-#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
@@ -1182,17 +1129,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
         continue;
     }
-    GDN_TRACE_MARK_U(unit, 0);
-#ifdef GDN_TRACE
-    if (threadIdx.x == 0 && g_trace_buf) {
-        unsigned smid;
-        unsigned long long gt;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-        g_trace_buf[(p.trace_call * p.n_units + unit) * 16 + 14] = smid;
-        g_trace_buf[(p.trace_call * p.n_units + unit) * 16 + 15] = (long long)gt;
-    }
-#endif
     // L2 warming for this CTA's next unit, in slices at phase boundaries
     const int u_next = unit + gridDim.x;
     auto warm_l2_state = [&](int slice) {
@@ -1227,19 +1163,16 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     const float4 *ab_path = reinterpret_cast<const float4 *>(smem + SM_PATH + (iter & 1) * SM_PATH_SLOT + 128);
     int path_len = 0;
     if constexpr (FUSED) path_len = reinterpret_cast<const int *>(smem + SM_PATH + (iter & 1) * SM_PATH_SLOT)[16];
-    GDN_TRACE_MARK_U(unit, 1);
 
     // Everything that depends only on q, k, g, beta runs now, under the latency of the state loads.  The Gram
     // block of this unit was issued one unit ahead; every thread waits for it on its own (bounded: on expiry it
     // flags the error and everybody falls through to the clean-up).
     if (!mbar_wait_bounded(mbar_g, par)) *flag = 1;
-    GDN_TRACE_MARK_U(unit, 2);
     if constexpr (CACHED) {
         if (use_cache) cp_async_wait_all();   // the path's cached projections, asked for one unit ahead
     }
     tc_fence_after();
     __syncthreads();
-    GDN_TRACE_MARK_U(unit, 3);
     warm_l2_state(0);
     // Form of the commit (unit-uniform; the path's scalars were written behind the last barrier of the unit before
     // and are readable from here on): from the cache unless the path decays below 2^-80 (1 / A_t could overflow).
@@ -1295,7 +1228,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
         tc_fence_before();
         __syncthreads();
-        GDN_TRACE_MARK_U(unit, 4);
         warm_l2_state(1);
         // X and Y for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
         {
@@ -1364,7 +1296,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     }
     cp_async_wait_all();
     __syncthreads();   // X and Y complete; the Gram copy is dead and its area can take the state operand
-    GDN_TRACE_MARK_U(unit, 5);
 
     // (3') fused commit: replay Eq. 7 along the previous step's accepted path on the state tile while it
     // sits in registers, write it back, and let everything below verify the new tree against it.
@@ -1453,7 +1384,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    GDN_TRACE_MARK_U(unit, 6);
     warm_l2_state(2);
     // The next unit's tables and accepted path are fetched in stages, each load issued one phase before its
     // value is used, so that no global-memory latency is paid in front of a barrier.
@@ -1522,7 +1452,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
-    GDN_TRACE_MARK_U(unit, 7);
     // stage 2: the path entries
     if constexpr (FUSED) {
         if (next_ok && warp == 4) {
@@ -1538,7 +1467,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // an expired wait only raises the flag, which is looked at behind the next CTA barrier (uniform decision).
     if (!mbar_wait_bounded(mbar_p, par)) *flag = 1;
     tc_fence_after();
-    GDN_TRACE_MARK_U(unit, 8);
     warm_l2_state(3);
 
     {
@@ -1588,7 +1516,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
-        GDN_TRACE_MARK_U(unit, 9);
 
         // (8) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
         // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
@@ -1653,7 +1580,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        GDN_TRACE_MARK_U(unit, 10);
 
         // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
         if (warp == W_MMA_D && elect_one()) {
@@ -1702,7 +1628,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if (next_ok) walk_tables(nT, (iter + 1) & 1, t_g, t_be, t_bad);
         if (!mbar_wait_bounded(mbar_d, par)) *flag = 1;
         tc_fence_after();
-        GDN_TRACE_MARK_U(unit, 11);
 
         // (10) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i]), staged through shared memory (over the
         // dead R^T tiles) so that global memory sees 16-byte stores of whole rows
@@ -1766,14 +1691,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
     }
-    GDN_TRACE_MARK_U(unit, 12);
-#ifdef GDN_TRACE
-    if (threadIdx.x == 0 && g_trace_buf) {
-        unsigned long long gt;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-        g_trace_buf[(p.trace_call * p.n_units + unit) * 16 + 13] = (long long)gt;
-    }
-#endif
     ++done_units;
     if (!unit_done_ok) break;   // a bounded wait expired: stop, report, release
     if (next_ok) issue_gram((uint32_t)(done_units & 1));   // the next unit's Gram block, as soon as its tile is there
@@ -1830,10 +1747,6 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
     } else {
         // trees that fit one CTA: persistent CTAs, two per SM, pipelined across units
         VerifyFastParams pt = p;
-#ifdef GDN_TRACE
-        static int trace_calls = 0;
-        pt.trace_call = trace_calls++ % 8;
-#endif
         if (!make_row_tensor_map(&pt.tm_k, p.k, s.total_nodes, s.h_qk, 64, true) ||
             !make_row_tensor_map(&pt.tm_q, p.q, s.total_nodes, s.h_qk, 64, true) ||
             !make_row_tensor_map(&pt.tm_v, p.v, s.total_nodes, s.h_v, FV_D, false))
@@ -1943,11 +1856,5 @@ cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const voi
     return launch_fast_typed<float, true, false>(s, p, stream);
 }
 
-#ifdef GDN_TRACE
-extern "C" int gdn_trace_set_buffer(long long *buf)
-{
-    return cudaMemcpyToSymbol(g_trace_buf, &buf, sizeof(buf)) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 }  // namespace gdn

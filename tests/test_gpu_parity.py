@@ -60,28 +60,30 @@ def test_config1_single_layer(tl, rep, out_dtype):
     _check_full(tl, synth.config(1, rep, out_dtype=out_dtype), f"cfg1 rep{rep} {out_dtype}")
 
 
-def test_config5_stack48_T64_sampled(tl):
-    w = synth.config(5, 0)
-    _check_sampled(tl, w, [0, 17, 47], "cfg1x48")
+# The four large configurations, whole: every layer slot / sequence of every repetition goes through the oracle, by
+# the separate entry points (verify, then commit) and by the fused one (the same repetition as the previous step,
+# the next repetition as the new trees); repetition 0 also with fp32 outputs.
+BIG_CONFIGS = {"cfg1x48": 5, "cfg2": 2, "cfg3": 3, "cfg4": 4}
 
 
-def test_config2_stack48_T256_sampled(tl):
-    w = synth.config(2, 0)
-    _check_sampled(tl, w, [3, 47], "cfg2")
+@pytest.mark.parametrize("rep", [0, 1, 2])
+@pytest.mark.parametrize("name", sorted(BIG_CONFIGS))
+def test_big_config_whole_workload_separate_calls(tl, name, rep):
+    _check_full(tl, synth.config(BIG_CONFIGS[name], rep), f"{name} rep{rep}")
 
 
-def test_config3_ragged_sampled(tl):
-    w = synth.config(3, 0)
-    sizes = np.diff(w.node_offsets)
-    seqs = sorted({0, int(np.argmin(sizes)), int(np.argmax(sizes)), 31})
-    _check_sampled(tl, w, seqs, "cfg3")
+@pytest.mark.parametrize("rep", [0, 1, 2])
+@pytest.mark.parametrize("name", sorted(BIG_CONFIGS))
+def test_big_config_whole_workload_fused_call(tl, name, rep):
+    prev, new = synth.config(BIG_CONFIGS[name], rep), synth.config(BIG_CONFIGS[name], (rep + 1) % 3)
+    if prev.n_seq != new.n_seq:
+        pytest.skip("repetitions differ in batch size")
+    _fused_case(tl, prev, new, f"fused {name} rep{rep}")
 
 
-def test_config4_chains_sampled(tl):
-    w = synth.config(4, 0)
-    L = np.diff(w.path_offsets)
-    seqs = sorted({0, int(np.argmin(L)), int(np.argmax(L)), 63})
-    _check_sampled(tl, w, seqs, "cfg4")
+@pytest.mark.parametrize("name", sorted(BIG_CONFIGS))
+def test_big_config_whole_workload_fp32_outputs(tl, name):
+    _check_full(tl, synth.config(BIG_CONFIGS[name], 0, out_dtype=synth.F32), f"{name} f32 out")
 
 
 # ------------------------------------------------------------------ edge shapes
@@ -385,26 +387,6 @@ def test_path_longer_than_max_depth_is_rejected_by_both_entry_points(tl):
 def dataclass_replace_S0(w, S0):
     import dataclasses
     return dataclasses.replace(w, S0=S0)
-
-
-def test_fused_commit_verify_full_stack_sampled(tl):
-    import paper_2607_06763_b200 as gdn
-    prev, new = synth.config(5, 0), synth.config(5, 1)
-    dp, dn = tl.DeviceCase(prev), tl.DeviceCase(new)
-    S = dp.S0.clone()
-    rc = gdn.gdn_tree_commit_verify(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path,
-                                    dp.path_offsets, dn.q, dn.k, dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets,
-                                    dn.o, dn.ws, dn.ws_bytes, dn.status)
-    assert rc == 0 and dn.device_status() == 0
-    seqs = [0, 23, 47]
-    psub, _ = tl.sub_workload(prev, seqs)
-    nsub, nodes = tl.sub_workload(new, seqs)
-    S_ref = tl.oracle_commit(psub)
-    tl.assert_state_close(S.cpu().numpy().astype(np.float64)[seqs], S_ref, what="fused 1x48 S_new")
-    from oracle import gdn_oracle as orc
-    o_ref = orc.verify(S_ref, nsub.f64("q"), nsub.f64("k"), nsub.f64("v"), nsub.f64("g"), nsub.f64("beta"),
-                       nsub.parent, nsub.node_offsets, nsub.scale)
-    tl.assert_close_per_head(dn.o_host()[nodes], o_ref, nsub.node_offsets, "fused 1x48 o", bf16_out=True)
 
 
 # ------------------------------------------------------------------ trees larger than one CTA tile (grouped path)
