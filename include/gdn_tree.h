@@ -253,6 +253,13 @@ int gdn_tree_commit_host(const gdn_shape_t *shape, float *S_h, const void *k_h, 
  * gdn_tree_commit_verify_host_arena_bytes(shape, prev_total_nodes, total_path_len) bytes.
  * S_h is written back only if total_path_len > 0 (otherwise no state changes); o_h receives the
  * outputs of the new trees.  Returns the host-side status, or the device-side status if non-zero.
+ * With two or more sequences the call is pipelined: the batch is cut into up to eight groups of
+ * sequences, and the copies up of one group, the kernels of the group before it and the copies down
+ * of the group before that run at the same time (both directions of the host link busy).  The
+ * copies run on two helper streams that the library creates on first use for each device and keeps
+ * (the one exception to "keeps no state"); `cuda_stream` is synchronised before returning, as for
+ * the other host variants, and nothing is left in flight.  Host buffers should be pinned: with
+ * pageable memory the copies are staged synchronously and nothing overlaps.
  */
 size_t gdn_tree_commit_verify_host_arena_bytes(const gdn_shape_t *shape, int32_t prev_total_nodes,
                                                int32_t total_path_len);

@@ -1,6 +1,8 @@
 // C-ABI entry points of libgdn_tree.so: argument validation, workspace carving, kernel launches,
 // and the host-buffer variants.  See include/gdn_tree.h for the contract of every function.
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "gdn_internal.cuh"
 
@@ -431,6 +433,41 @@ extern "C" int gdn_tree_commit_host(const gdn_shape_t *shape, float *S_h, const 
     return status_h;
 }
 
+namespace {
+
+// Helper streams and events of the pipelined host-buffer call, created on first use for each device and kept for
+// the life of the process (the one piece of state the library keeps besides the static scratch array).
+constexpr int HOST_PIPE_GROUPS = 8;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t start = nullptr, done = nullptr, in[HOST_PIPE_GROUPS] = {}, k[HOST_PIPE_GROUPS] = {};
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipe[64];
+
+HostPipe *host_pipe()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe &p = g_pipe[dev];
+    if (!p.ready) {
+        bool ok = cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.done, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < HOST_PIPE_GROUPS; ++i)
+            ok = cudaEventCreateWithFlags(&p.in[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p.k[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        p.ready = true;
+    }
+    return &p;
+}
+
+}  // namespace
+
 extern "C" size_t gdn_tree_commit_verify_host_arena_bytes(const gdn_shape_t *shape, int32_t prev_total_nodes,
                                                           int32_t total_path_len)
 {
@@ -444,6 +481,7 @@ extern "C" size_t gdn_tree_commit_verify_host_arena_bytes(const gdn_shape_t *sha
     n += align256(tp.qk) + align256(tp.v) + 2 * align256(tp.gb) + align256(tp.parent) + 2 * align256(tp.offsets);
     n += align256((size_t)total_path_len * sizeof(int32_t) + 4) + align256(sizeof(int32_t));
     n += workspace_layout(*shape).total;
+    n += 3 * align256(sizeof(int32_t) * ((size_t)shape->n_seq + HOST_PIPE_GROUPS + 1));   // per-group offset arrays
     return n + 256;
 }
 
@@ -486,8 +524,94 @@ extern "C" int gdn_tree_commit_verify_host(const gdn_shape_t *shape, float *S_h,
     int32_t *path = static_cast<int32_t *>(a.take(path_bytes + 4));
     int32_t *status = static_cast<int32_t *>(a.take(sizeof(int32_t)));
     void *ws = a.take(lay.total);
-    if (!ws) return GDN_ERR_WORKSPACE;
+    const size_t goff_bytes = sizeof(int32_t) * ((size_t)s.n_seq + HOST_PIPE_GROUPS + 1);
+    int32_t *g_offs = static_cast<int32_t *>(a.take(goff_bytes));
+    int32_t *g_offs_p = static_cast<int32_t *>(a.take(goff_bytes));
+    int32_t *g_poffs = static_cast<int32_t *>(a.take(goff_bytes));
+    if (!ws || !g_poffs) return GDN_ERR_WORKSPACE;
     GDN_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
+    // group slices of g / beta start at multiples of h_v elements: they keep the 16-byte alignment the device entry
+    // points ask for only if a row of them is a multiple of 16 bytes (otherwise the call runs unpipelined)
+    const bool sliceable = ((size_t)s.h_v * dtype_size(s.in_dtype)) % 16 == 0;
+    HostPipe *pipe = (sliceable && s.n_seq >= 2 && s.total_nodes > 0 && total_path_len > 0) ? host_pipe() : nullptr;
+    if (pipe) {
+        // Pipelined form: the layer slots / sequences are cut into groups; the copies up of group i+1 (helper stream
+        // s_in), the kernels of group i (the caller's stream) and the copies down of group i-1 (helper stream s_out)
+        // run at the same time, so that both directions of the host link are busy.  Each group is a call of its own
+        // on slices of the packed tensors, with node and path offsets rebased to its first row.
+        const int G = s.n_seq < HOST_PIPE_GROUPS ? s.n_seq : HOST_PIPE_GROUPS;
+        std::vector<int32_t> ho((size_t)s.n_seq + G), hop((size_t)s.n_seq + G), hpo((size_t)s.n_seq + G);
+        std::vector<int> first(G + 1);
+        for (int i = 0; i <= G; ++i) first[i] = (int)((long long)s.n_seq * i / G);
+        for (int i = 0; i < G; ++i)
+            for (int b = first[i]; b <= first[i + 1]; ++b) {
+                ho[(size_t)b + i] = node_offsets_h[b] - node_offsets_h[first[i]];
+                hop[(size_t)b + i] = node_offsets_prev_h[b] - node_offsets_prev_h[first[i]];
+                hpo[(size_t)b + i] = path_offsets_h[b] - path_offsets_h[first[i]];
+            }
+        const size_t ob = sizeof(int32_t) * ho.size();
+        GDN_CUDA_TRY(cudaMemcpyAsync(g_offs, ho.data(), ob, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(g_offs_p, hop.data(), ob, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaMemcpyAsync(g_poffs, hpo.data(), ob, cudaMemcpyHostToDevice, stream));
+        GDN_CUDA_TRY(cudaEventRecord(pipe->start, stream));
+        GDN_CUDA_TRY(cudaStreamWaitEvent(pipe->s_in, pipe->start, 0));
+        GDN_CUDA_TRY(cudaStreamWaitEvent(pipe->s_out, pipe->start, 0));
+        const size_t isz = dtype_size(s.in_dtype), osz = dtype_size(s.out_dtype);
+        const size_t row_qk = (size_t)s.h_qk * s.d_k * isz, row_v = (size_t)s.h_v * s.d_v * isz, row_gb = (size_t)s.h_v * isz;
+        const size_t row_o = (size_t)s.h_v * s.d_v * osz, slot_state = (size_t)s.h_v * s.d_v * s.d_k * sizeof(float);
+        auto at = [](const void *base, size_t off) { return static_cast<const char *>(base) + off; };
+        auto atw = [](void *base, size_t off) { return static_cast<char *>(base) + off; };
+        for (int i = 0; i < G; ++i) {
+            const int b0 = first[i], nb = first[i + 1] - b0;
+            const size_t n0 = (size_t)node_offsets_h[b0], nn = (size_t)node_offsets_h[b0 + nb] - n0;
+            const size_t m0 = (size_t)node_offsets_prev_h[b0], mm = (size_t)node_offsets_prev_h[b0 + nb] - m0;
+            const size_t p0 = (size_t)path_offsets_h[b0], pl = (size_t)path_offsets_h[b0 + nb] - p0;
+            cudaStream_t si = pipe->s_in;
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(S, b0 * slot_state), at(S_h, b0 * slot_state), nb * slot_state, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(q, n0 * row_qk), at(q_h, n0 * row_qk), nn * row_qk, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(k, n0 * row_qk), at(k_h, n0 * row_qk), nn * row_qk, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(v, n0 * row_v), at(v_h, n0 * row_v), nn * row_v, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(g, n0 * row_gb), at(g_h, n0 * row_gb), nn * row_gb, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(beta, n0 * row_gb), at(beta_h, n0 * row_gb), nn * row_gb, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(parent + n0, parent_h + n0, nn * sizeof(int32_t), cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(kp, m0 * row_qk), at(k_prev_h, m0 * row_qk), mm * row_qk, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(vp, m0 * row_v), at(v_prev_h, m0 * row_v), mm * row_v, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(gp, m0 * row_gb), at(g_prev_h, m0 * row_gb), mm * row_gb, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(atw(bp, m0 * row_gb), at(beta_prev_h, m0 * row_gb), mm * row_gb, cudaMemcpyHostToDevice, si));
+            if (parent_p) GDN_CUDA_TRY(cudaMemcpyAsync(parent_p + m0, parent_prev_h + m0, mm * sizeof(int32_t), cudaMemcpyHostToDevice, si));
+            if (pl) GDN_CUDA_TRY(cudaMemcpyAsync(path + p0, path_h + p0, pl * sizeof(int32_t), cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaEventRecord(pipe->in[i], si));
+            GDN_CUDA_TRY(cudaStreamWaitEvent(stream, pipe->in[i], 0));
+            gdn_shape_t gs = s;
+            gs.n_seq = nb;
+            gs.total_nodes = (int32_t)nn;
+            if (nn > 0 || pl > 0) {
+                rc = gdn_tree_commit_verify(&gs, S + (size_t)b0 * (slot_state / sizeof(float)), at(kp, m0 * row_qk),
+                                            at(vp, m0 * row_v), at(gp, m0 * row_gb), at(bp, m0 * row_gb),
+                                            parent_p ? parent_p + m0 : nullptr, g_offs_p + b0 + i, path + p0,
+                                            g_poffs + b0 + i, at(q, n0 * row_qk), at(k, n0 * row_qk), at(v, n0 * row_v),
+                                            at(g, n0 * row_gb), at(beta, n0 * row_gb), parent + n0, g_offs + b0 + i,
+                                            atw(o, n0 * row_o), ws, lay.total, status, cuda_stream);
+                if (rc != GDN_OK) {   // refused on the host: let what is in flight drain before returning
+                    cudaStreamSynchronize(pipe->s_in);
+                    cudaStreamSynchronize(stream);
+                    cudaStreamSynchronize(pipe->s_out);
+                    return rc;
+                }
+            }
+            GDN_CUDA_TRY(cudaEventRecord(pipe->k[i], stream));
+            cudaStream_t so = pipe->s_out;
+            GDN_CUDA_TRY(cudaStreamWaitEvent(so, pipe->k[i], 0));
+            if (nn) GDN_CUDA_TRY(cudaMemcpyAsync(atw(o_h, n0 * row_o), at(o, n0 * row_o), nn * row_o, cudaMemcpyDeviceToHost, so));
+            if (pl) GDN_CUDA_TRY(cudaMemcpyAsync(atw(S_h, b0 * slot_state), at(S, b0 * slot_state), nb * slot_state, cudaMemcpyDeviceToHost, so));
+        }
+        GDN_CUDA_TRY(cudaEventRecord(pipe->done, pipe->s_out));
+        GDN_CUDA_TRY(cudaStreamWaitEvent(stream, pipe->done, 0));
+        int32_t status_p = 0;
+        GDN_CUDA_TRY(cudaMemcpyAsync(&status_p, status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+        GDN_CUDA_TRY(cudaStreamSynchronize(stream));
+        return status_p;
+    }
     // one copy of the state for both halves of the step: it goes up once and comes back once
     GDN_CUDA_TRY(cudaMemcpyAsync(S, S_h, t.state, cudaMemcpyHostToDevice, stream));
     if (total_path_len > 0) {

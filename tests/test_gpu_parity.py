@@ -274,6 +274,51 @@ def test_host_buffer_entry_points(tl):
                                            new.beta, new.parent, new.node_offsets, o2, arena2, fb - 4096) == -10   # GDN_ERR_WORKSPACE
 
 
+def test_host_buffer_fused_call_pipelined_over_sequence_groups(tl):
+    """More sequences than one: the host-buffer fused call cuts the batch into groups and overlaps copies and kernels
+    on helper streams (node and path offsets rebased per group).  13 ragged sequences, empty paths and a rejected one
+    among them, against the oracle; a second call on the same arena must give the same."""
+    import torch
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(401)
+    sizes = [64, 5, 33, 1, 64, 17, 48, 9, 64, 2, 40, 64, 21]
+    prev_trees = [synth.tree_geo(rng, T) for T in sizes]
+    paths = [synth.root_path(t, int(rng.integers(0, len(t)))) if i % 4 else np.zeros(0, np.int32)
+             for i, t in enumerate(prev_trees)]
+    prev = synth.random_case(402, prev_trees, 4, 8, 128, 128, synth.BF16, synth.BF16, paths=paths, name="host_prev")
+    new = synth.random_case(403, [synth.tree_geo(rng, T) for T in reversed(sizes)], 4, 8, 128, 128, synth.BF16,
+                            synth.BF16, name="host_new")
+    shape = gdn.GdnShape.from_workload(new)
+    L = int(prev.path_offsets[-1])
+    fb = gdn.gdn_tree_commit_verify_host_arena_bytes(shape, prev.total_nodes, L)
+    arena = torch.empty(fb, dtype=torch.uint8, device="cuda")
+    S_ref, o_ref = _oracle_step(prev.S0.astype(np.float64), prev, new)
+    for call in range(2):
+        S = prev.S0.copy()
+        o = np.zeros((new.total_nodes, new.h_v, new.d_v), dtype=np.uint16)
+        rc = gdn.gdn_tree_commit_verify_host(shape, S, prev.total_nodes, prev.k, prev.v, prev.g, prev.beta, prev.parent,
+                                             prev.node_offsets, prev.path, prev.path_offsets, L, new.q, new.k, new.v,
+                                             new.g, new.beta, new.parent, new.node_offsets, o, arena, fb)
+        assert rc == 0, gdn.gdn_status_string(rc)
+        tl.assert_state_close(S.astype(np.float64), S_ref, what=f"pipelined host call {call}: state")
+        tl.assert_close_per_head(synth.bf16_bits_to_f32(o).astype(np.float64), o_ref, new.node_offsets,
+                                 f"pipelined host call {call}: o", bf16_out=True)
+    # one accepted path that is not a chain: reported, that state kept, everything else as before
+    bad_paths = list(paths)
+    bad_paths[5] = np.array([0, 0], np.int32)
+    bad = synth.random_case(402, prev_trees, 4, 8, 128, 128, synth.BF16, synth.BF16, paths=bad_paths, name="host_bad")
+    Lb = int(bad.path_offsets[-1])
+    S = bad.S0.copy()
+    o = np.zeros((new.total_nodes, new.h_v, new.d_v), dtype=np.uint16)
+    fb2 = gdn.gdn_tree_commit_verify_host_arena_bytes(shape, bad.total_nodes, Lb)
+    arena2 = torch.empty(fb2, dtype=torch.uint8, device="cuda")
+    rc = gdn.gdn_tree_commit_verify_host(shape, S, bad.total_nodes, bad.k, bad.v, bad.g, bad.beta, bad.parent,
+                                         bad.node_offsets, bad.path, bad.path_offsets, Lb, new.q, new.k, new.v, new.g,
+                                         new.beta, new.parent, new.node_offsets, o, arena2, fb2)
+    assert rc == -9
+    np.testing.assert_array_equal(S[5], bad.S0[5])
+
+
 # ------------------------------------------------------------------ fused commit + verify
 def _fused_case(tl, prev, new, what):
     """commit(prev.path) + verify(new tree) in one call against: oracle commit, then oracle verify on that state."""
