@@ -34,10 +34,18 @@
  *   path      : [path_offsets[n_seq]] local node ids, root first
  * Value head h reads key head h / (h_v / h_qk).
  *
+ *   - Gate activations ("scalars" stage of Section 3.4.2 / Table 1, which
+ *     forms the write strengths beta and the log-decays from the layer's raw
+ *     gate inputs; the paper does not print the activation, the reading is
+ *     the Gated DeltaNet one that the input recipe also uses):
+ *         g = -softplus(a) = -log(1 + e^a),   beta = sigmoid(b) = 1 / (1 + e^-b).
+ *
  * Parity pins (tests/test_oracle_pins.py): dense-matrix brute force, the
  * triangular-solve form of Eq. 9-11, the masked closed form of Eq. 12,
  * chain == sequential decoding, sibling-order invariance, hand example,
- * closed forms for beta = 0 / orthonormal keys / scalar recurrence.
+ * closed forms for beta = 0 / orthonormal keys / scalar recurrence; the
+ * gate activations against their functional equations, their limits and
+ * independent library routines.
  */
 #include <math.h>
 #include <stdint.h>
@@ -192,4 +200,18 @@ int gdn_oracle_commit(int n_seq, int h_qk, int h_v, int d_k, int d_v, const doub
         free(ktS);
     }
     return failed ? GDN_ORACLE_NOMEM : GDN_ORACLE_OK;
+}
+
+
+/* Gate activations of n raw gate pairs: g = -softplus(a), beta = sigmoid(b)
+ * (the "scalars" stage of Section 3.4.2).  Written in the forms that do not
+ * overflow for large |x|. */
+void gdn_oracle_gates(int64_t n, const double *a_raw, const double *b_raw, double *g_out, double *beta_out)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        const double a = a_raw[i], b = b_raw[i];
+        const double softplus = a > 0.0 ? a + log1p(exp(-a)) : log1p(exp(a));
+        g_out[i] = -softplus;
+        beta_out[i] = b >= 0.0 ? 1.0 / (1.0 + exp(-b)) : exp(b) / (1.0 + exp(b));
+    }
 }

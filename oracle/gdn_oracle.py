@@ -48,6 +48,8 @@ def _load():
                                                                                             ctypes.c_int, ctypes.c_int]
         lib.gdn_oracle_commit.restype = ctypes.c_int
         lib.gdn_oracle_commit.argtypes = [ctypes.c_int] * 5 + [dp] * 5 + [ip] * 4 + [dp]
+        lib.gdn_oracle_gates.restype = None
+        lib.gdn_oracle_gates.argtypes = [ctypes.c_int64, dp, dp, dp, dp]
         _lib = lib
     return _lib
 
@@ -129,3 +131,68 @@ def commit(S0, k, v, g, beta, parent, node_offsets, path, path_offsets):
     if rc != 0:
         raise ValueError(f"gdn_oracle_commit failed with code {rc}")
     return S_new
+
+
+def gates(a_raw, b_raw):
+    """Gate activations of the "scalars" stage (Section 3.4.2): ``g = -softplus(a_raw)``, ``beta = sigmoid(b_raw)``,
+    elementwise in fp64.  Returns ``(g, beta)`` with the shape of the inputs."""
+    lib = _load()
+    a = np.ascontiguousarray(a_raw, dtype=np.float64)
+    b = np.ascontiguousarray(b_raw, dtype=np.float64)
+    assert a.shape == b.shape
+    g, beta = np.empty_like(a), np.empty_like(b)
+    lib.gdn_oracle_gates(a.size, _dp(a), _dp(b), _dp(g), _dp(beta))
+    return g, beta
+
+
+def _unpad(n_slots, n_trees, t_pad, n_nodes, parent_pad):
+    """Row indices (into the flattened ``[n_slots * t_pad]`` node axis), packed ``parent`` and ``node_offsets`` of the
+    padded layout of Section 3.4.2: slot ``s`` carries tree ``s % n_trees`` in its first ``n_nodes[tree]`` rows."""
+    n_nodes = np.asarray(n_nodes, dtype=np.int64)
+    parent_pad = np.asarray(parent_pad, dtype=np.int32).reshape(n_trees, t_pad)
+    rows, parents, offs = [], [], [0]
+    for s in range(n_slots):
+        tr = s % n_trees
+        T = int(n_nodes[tr])
+        assert 0 <= T <= t_pad
+        rows.append(np.arange(s * t_pad, s * t_pad + T, dtype=np.int64))
+        parents.append(parent_pad[tr, :T])
+        offs.append(offs[-1] + T)
+    return (np.concatenate(rows) if rows else np.zeros(0, np.int64),
+            np.concatenate(parents).astype(np.int32) if parents else np.zeros(0, np.int32),
+            np.asarray(offs, dtype=np.int32))
+
+
+def verify_padded(S0, q, k, v, g_in, beta_in, parent_pad, n_nodes, scale, raw_gates):
+    """Verification in the padded layout of Section 3.4.2: ``q,k [B,T,H_k,d_k]``, ``v [B,T,H_v,d_v]``, ``g_in, beta_in
+    [B,T,H_v]`` (raw gate inputs if ``raw_gates``), ``parent_pad [n_trees,T]``, ``n_nodes [n_trees]``; slot ``s`` carries
+    tree ``s % n_trees``.  Returns ``o [B,T,H_v,d_v]`` (rows beyond a tree's node count are zero).  The padded tensors
+    are unpacked to the ragged form and handed to :func:`verify`: only indices move here."""
+    B, T = np.shape(q)[:2]
+    n_trees = len(n_nodes)
+    rows, parent, offs = _unpad(B, n_trees, T, n_nodes, parent_pad)
+    flat = lambda x: np.asarray(x, dtype=np.float64).reshape((B * T,) + tuple(np.shape(x)[2:]))[rows]
+    g, beta = flat(g_in), flat(beta_in)
+    if raw_gates:
+        g, beta = gates(g, beta)
+    o_r = verify(S0, flat(q), flat(k), flat(v), g, beta, parent, offs, scale)
+    o = np.zeros((B * T,) + o_r.shape[1:], dtype=np.float64)
+    o[rows] = o_r
+    return o.reshape((B, T) + o_r.shape[1:])
+
+
+def commit_padded(S0, k, v, g_in, beta_in, parent_pad, n_nodes, path_pad, path_len, raw_gates):
+    """Commit in the padded layout: ``path_pad [n_trees, max_depth]``, ``path_len [n_trees]`` (every slot of a tree
+    commits that tree's accepted path).  Returns ``S_new``."""
+    B, T = np.shape(k)[:2]
+    n_trees = len(n_nodes)
+    rows, parent, offs = _unpad(B, n_trees, T, n_nodes, parent_pad)
+    flat = lambda x: np.asarray(x, dtype=np.float64).reshape((B * T,) + tuple(np.shape(x)[2:]))[rows]
+    g, beta = flat(g_in), flat(beta_in)
+    if raw_gates:
+        g, beta = gates(g, beta)
+    path_pad = np.asarray(path_pad, dtype=np.int32).reshape(n_trees, -1)
+    paths = [path_pad[s % n_trees, : int(path_len[s % n_trees])] for s in range(B)]
+    poffs = np.concatenate([[0], np.cumsum([len(p) for p in paths])]).astype(np.int32)
+    path = np.concatenate(paths).astype(np.int32) if paths else np.zeros(0, np.int32)
+    return commit(S0, flat(k), flat(v), g, beta, parent, offs, path, poffs)

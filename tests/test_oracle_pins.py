@@ -318,3 +318,100 @@ def test_sequence_sampling_matches_full_run():
     lo, hi = int(w.node_offsets[1]), int(w.node_offsets[3])
     np.testing.assert_array_equal(part[lo:hi], full[lo:hi])
     assert not part[:lo].any() and not part[hi:].any()
+
+
+# ------------------------------------------------------------------ gate activations and the padded layout
+def test_gate_activations_functional_equations_and_limits():
+    """g = -softplus(a), beta = sigmoid(b): pinned by what fixes the two functions -- values at 0, the reflection
+    identities, the derivative relation softplus' = sigmoid, and the asymptotes for large arguments."""
+    x = np.linspace(-30.0, 30.0, 2401)
+    g, beta = orc.gates(x, x)
+    sp = -g
+    g_neg, beta_neg = orc.gates(-x, -x)
+    assert orc.gates(np.zeros(1), np.zeros(1))[0][0] == pytest.approx(-np.log(2.0), abs=1e-16)
+    assert orc.gates(np.zeros(1), np.zeros(1))[1][0] == 0.5
+    np.testing.assert_allclose(beta + beta_neg, 1.0, rtol=0, atol=5e-16)            # sigmoid(-x) = 1 - sigmoid(x)
+    np.testing.assert_allclose(sp - (-g_neg), x, rtol=0, atol=1e-13)                # softplus(x) - softplus(-x) = x
+    np.testing.assert_allclose(np.exp(-sp), beta_neg, rtol=1e-13, atol=1e-300)      # e^{-softplus(x)} = sigmoid(-x)
+    h = x[1] - x[0]
+    np.testing.assert_allclose((sp[2:] - sp[:-2]) / (2 * h), beta[1:-1], rtol=0, atol=2e-5)   # d softplus = sigmoid
+    big = np.array([50.0, 200.0, 745.0])
+    gb, bb = orc.gates(big, big)
+    np.testing.assert_allclose(-gb, big, rtol=1e-15)
+    assert np.all(bb == 1.0) or np.all(1.0 - bb < 1e-20)
+    gs, bs = orc.gates(-big, -big)
+    np.testing.assert_allclose(-gs, np.exp(-big), rtol=1e-12, atol=0)
+    np.testing.assert_allclose(bs, np.exp(-big), rtol=1e-12, atol=0)
+    assert np.all(np.isfinite(orc.gates(np.array([-1e4, 1e4]), np.array([-1e4, 1e4]))[0]))
+
+
+def test_gate_activations_against_library_routines():
+    scipy_special = pytest.importorskip("scipy.special")
+    rng = np.random.default_rng(3)
+    x = rng.normal(size=4000) * 6.0
+    g, beta = orc.gates(x, x)
+    np.testing.assert_allclose(-g, np.logaddexp(0.0, x), rtol=1e-14, atol=1e-300)
+    np.testing.assert_allclose(beta, scipy_special.expit(x), rtol=1e-14, atol=1e-300)
+
+
+def test_hand_worked_scalar_tree_through_raw_gates_and_padded_layout():
+    """The hand example again, now entering through the raw gate inputs and the padded [slots, T, ...] layout with
+    three slots sharing the one tree (T padded to 6).  alpha = .5 <-> a = 0 (softplus(0) = ln 2), alpha = .25 <-> a =
+    ln 3, beta = .5 <-> b = 0; alpha = 1 and beta in {0, 1} are reached in the limit, here |raw| = 40 (off by 4e-18)."""
+    ex = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "scalar_tree_example.json")))
+    a_raw = {0.5: 0.0, 1.0: -40.0, 0.25: np.log(3.0)}
+    b_raw = {0.5: 0.0, 1.0: 40.0, 0.0: -40.0}
+    T, B = 6, 3
+    pad = lambda vals, fill=0.0: np.array(list(vals) + [fill] * (T - len(vals)))
+    a = np.tile(pad([a_raw[x] for x in ex["alpha"]], 7.0)[None, :, None], (B, 1, 1))
+    b = np.tile(pad([b_raw[x] for x in ex["beta"]], -3.0)[None, :, None], (B, 1, 1))
+    k = np.tile(pad(ex["k"], 5.0)[None, :, None, None], (B, 1, 1, 1))
+    v = np.tile(pad(ex["v"], 5.0)[None, :, None, None], (B, 1, 1, 1))
+    q = np.tile(pad(ex["q"], 5.0)[None, :, None, None], (B, 1, 1, 1))
+    parent = np.array([ex["parent"] + [0, 0]], dtype=np.int32)      # the padding rows carry garbage parents
+    S0 = np.full((B, 1, 1, 1), ex["S0"])
+    o = orc.verify_padded(S0, q, k, v, a, b, parent, [4], 1.0, raw_gates=True)
+    for s in range(B):
+        np.testing.assert_allclose(o[s, :4, 0, 0], ex["o"], rtol=0, atol=1e-15)
+        assert np.all(o[s, 4:] == 0.0)
+    for key, want in ex["commit"].items():
+        path = json.loads(key)
+        S = orc.commit_padded(S0, k, v, a, b, parent, [4], np.array([path + [0] * (16 - len(path))]), [len(path)],
+                              raw_gates=True)
+        np.testing.assert_allclose(S[:, 0, 0, 0], want, rtol=0, atol=1e-15)
+
+
+def test_padded_layout_equals_ragged_layout():
+    """Two trees shared by five slots, T padded to 24: the padded front end must give exactly what the ragged calls give
+    on the unpacked tensors (with the activations applied by hand through independent library routines)."""
+    scipy_special = pytest.importorskip("scipy.special")
+    rng = np.random.default_rng(11)
+    trees = [synth.tree_geo(rng, 17), synth.tree_geo(rng, 24)]
+    B, T, hk, hv, d = 5, 24, 2, 4, 8
+    parent = np.full((2, T), 99, np.int32)
+    for i, t in enumerate(trees):
+        parent[i, : len(t)] = t
+    q, k = rng.normal(size=(B, T, hk, d)), rng.normal(size=(B, T, hk, d))
+    v = rng.normal(size=(B, T, hv, d))
+    a, b = rng.normal(size=(B, T, hv)), rng.normal(size=(B, T, hv))
+    S0 = rng.normal(size=(B, hv, d, d)) * 0.1
+    n_nodes = [17, 24]
+    o = orc.verify_padded(S0, q, k, v, a, b, parent, n_nodes, 0.3, raw_gates=True)
+    paths = np.zeros((2, 16), np.int32)
+    plen = []
+    for i, t in enumerate(trees):
+        p = synth.longest_path(t)
+        paths[i, : len(p)] = p
+        plen.append(len(p))
+    S_new = orc.commit_padded(S0, k, v, a, b, parent, n_nodes, paths, plen, raw_gates=True)
+    for s in range(B):
+        tr = s % 2
+        n = n_nodes[tr]
+        g, beta = -np.logaddexp(0.0, a[s, :n]), scipy_special.expit(b[s, :n])
+        offs = np.array([0, n], np.int32)
+        o_ref = orc.verify(S0[s:s + 1], q[s, :n], k[s, :n], v[s, :n], g, beta, trees[tr], offs, 0.3)
+        np.testing.assert_allclose(o[s, :n], o_ref, rtol=1e-13, atol=1e-14)
+        assert np.all(o[s, n:] == 0.0)
+        S_ref = orc.commit(S0[s:s + 1], k[s, :n], v[s, :n], g, beta, trees[tr], offs, paths[tr, : plen[tr]],
+                           np.array([0, plen[tr]], np.int32))
+        np.testing.assert_allclose(S_new[s], S_ref[0], rtol=1e-13, atol=1e-14)
