@@ -262,9 +262,6 @@ def main():
                          "verify: gdn_tree_verify alone (no commit; for kernel comparisons)")
     ap.add_argument("--path-len", type=int, default=16,
                     help="workload stack48_T64_deep: nodes on the accepted path (0..16)")
-    ap.add_argument("--commit", default="replay", choices=["cached", "replay"],
-                    help="fused mode: cached = gdn_tree_commit_verify_cached (the commit reads the projections the "
-                         "previous step's call left in its workspace); replay = gdn_tree_commit_verify")
     ap.add_argument("--graph", action="store_true",
                     help="fused mode: capture one step per buffer set in a CUDA graph and time replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -281,8 +278,6 @@ def main():
         return
     if args.impl == "recurrent":
         args.mode = "verify"
-    if args.graph:
-        args.commit = "replay"   # a captured step has its workspace baked in; the cached form alternates two
 
     w = make_workload(args)
     if args.impl == "reference":
@@ -315,10 +310,7 @@ def main():
         d["path"] = to_dev(w.path if w.path.size else np.zeros(1, np.int32))
         odt = torch.float32 if w.out_dtype == synth.F32 else torch.bfloat16
         d["o"] = torch.empty((w.total_nodes, w.h_v, w.d_v), dtype=odt, device="cuda")
-        # two workspaces per set: a step reads the projection cache of the step before it and writes its own
-        d["ws2"] = [torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda") for _ in range(2)]
-        d["ws"] = d["ws2"][0]
-        d["visits"] = 0
+        d["ws"] = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
         sets.append(d)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
@@ -341,20 +333,10 @@ def main():
     def step_fused(d, stream=stream):
         # one decode iteration as the paper schedules it: commit the previous step's accepted path, then verify
         # the new tree against the advanced state (here the previous and the new tree carry the same tensors)
-        if args.commit == "replay":
-            rc = gdn.gdn_tree_commit_verify(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
-                                            d["node_offsets"], d["path"], d["path_offsets"], d["q"], d["k"], d["v"],
-                                            d["g"], d["beta"], d["parent"], d["node_offsets"], d["o"], d["ws"],
-                                            ws_bytes, status, stream)
-        else:
-            # the state of this set was last verified (against exactly what it holds now) by the previous step on
-            # this set, which left its projection cache in the other workspace
-            prev_ws, ws = d["ws2"][(d["visits"] + 1) & 1], d["ws2"][d["visits"] & 1]
-            d["visits"] += 1
-            rc = gdn.gdn_tree_commit_verify_cached(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
-                                                   d["node_offsets"], d["path"], d["path_offsets"], prev_ws,
-                                                   w.total_nodes, d["q"], d["k"], d["v"], d["g"], d["beta"],
-                                                   d["parent"], d["node_offsets"], d["o"], ws, ws_bytes, status, stream)
+        rc = gdn.gdn_tree_commit_verify(shape, d["S0"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
+                                        d["node_offsets"], d["path"], d["path_offsets"], d["q"], d["k"], d["v"],
+                                        d["g"], d["beta"], d["parent"], d["node_offsets"], d["o"], d["ws"], ws_bytes,
+                                        status, stream)
         assert rc == 0, gdn.gdn_status_string(rc)
 
     step = {"fused": step_fused, "separate": step_separate, "verify": step_verify}[args.mode]
@@ -518,7 +500,6 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": DTYPE if w.in_dtype == synth.BF16 else "f32", "data": "synthetic",
             "config": workload_config(w, args), "mode": args.mode, "impl": args.impl,
-            "commit": args.commit if args.mode == "fused" else "replay",
             "timing": {"regions": len(region_ms), "steps_per_region": args.steps,
                        "ms_per_step_median_region": med_region / args.steps,
                        "ms_per_step_fastest_region": min_region / args.steps,

@@ -93,11 +93,10 @@ const char *gdn_status_string(int status);
 
 /*
  * Bytes of device scratch gdn_tree_verify needs for this shape: tree metadata
- * of Section 3.4.2 (per node its depth and ancestor list), the solve result
+ * of Section 3.4.2 (per node its depth and ancestor list; used for trees of
+ * more than 64 nodes and by the general kernel) and the solve result
  * u~ [N][h_v][d_v] fp32 of the general kernel (the quantity "u_j - w_j^T S0"
- * that the substitution of Eq. 13 returns), and the projection cache
- * [N][h_v][d_v] fp32 that gdn_tree_commit_verify_cached reads one step later.
- * Returns 0 if the shape is invalid.
+ * that the substitution of Eq. 13 returns).  Returns 0 if the shape is invalid.
  */
 size_t gdn_tree_workspace_bytes(const gdn_shape_t *shape);
 
@@ -120,14 +119,52 @@ int gdn_tree_validate_host(const gdn_shape_t *shape, const int32_t *parent_h,
  *   S0, q, k, v, g, beta, parent, node_offsets : [device], read-only
  *   o            : [device], written for every node of every valid tree
  *   workspace    : [device], >= gdn_tree_workspace_bytes(shape) bytes, 256-byte aligned;
- *                  contents after the call: tree metadata, u~, and on the tensor-core path the
- *                  projection cache (see gdn_tree_commit_verify_cached)
+ *                  contents after the call: the tree metadata and u~ (reused by nothing else)
  *   status_dev   : [device] one int32, see "Return value" above
  */
 int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const void *q, const void *k,
                     const void *v, const void *g, const void *beta, const int32_t *parent,
                     const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
                     int32_t *status_dev, void *cuda_stream);
+
+/*
+ * Padded, shape-static entry points (Section 3.4.2: dense [N, T, H, d] inputs with T the padded tree
+ * size, so that every shape is independent of the tree's contents and the call can be captured once
+ * in a CUDA graph and replayed for every tree; "the proposal tree is shared by every GDN layer, so its
+ * verification metadata is computed once per decode step"; Table 1, stage "scalars": the write
+ * strengths and log-decays are formed inside the kernel from the layer's gate inputs).
+ *   shape        : n_seq = number of slots (a (sequence, layer) pair), max_tree_nodes = T = rows per
+ *                  slot (<= 64), total_nodes = n_seq * T, d_k = d_v = 128, in_dtype = GDN_BF16,
+ *                  max_depth <= 16; anything else returns GDN_ERR_UNSUPPORTED
+ *   n_trees      : number of distinct trees; n_seq % n_trees == 0 and slot b carries tree b % n_trees
+ *                  (with one sequence and 48 layers: n_trees = 1, n_seq = 48 -- the tree is given once
+ *                  and each CTA derives its metadata from it on chip, no metadata kernel runs)
+ *   raw_gates    : 0: g = log(alpha) and beta as for gdn_tree_verify; non-zero: `g` and `beta` hold
+ *                  the raw gate inputs a, b of the layer and the kernel forms g = -softplus(a),
+ *                  beta = sigmoid(b) in fp32 (the Gated DeltaNet activations; the paper does not print them)
+ *   q, k         : [n_seq][T][h_qk][d_k]       v, o : [n_seq][T][h_v][d_v]       g, beta : [n_seq][T][h_v]
+ *   parent       : [device] int32 [n_trees][T], entries beyond a tree's node count are ignored
+ *   n_nodes      : [device] int32 [n_trees], 0 .. T; rows of `o` beyond the count are never written
+ * The fused form commits, for every slot, the accepted path of its tree in the PREVIOUS step
+ * (prev_t_pad rows per slot; k_prev, v_prev, g_prev, beta_prev, parent_prev [n_trees][prev_t_pad],
+ * n_nodes_prev [n_trees] in the same layout; parent_prev may be NULL) and verifies the new tree against
+ * the advanced state, exactly as gdn_tree_commit_verify:
+ *   path         : [device] int32 [n_trees][max_depth], node ids root first
+ *   path_len     : [device] int32 [n_trees], 0 .. max_depth (0 leaves the states of that tree's slots alone)
+ * Everything data-dependent (tree, node counts, paths) lives in device arrays: a captured call can be
+ * replayed after they have been overwritten in place.  No workspace.  Errors as for gdn_tree_verify.
+ */
+int gdn_tree_verify_padded(const gdn_shape_t *shape, int32_t n_trees, int32_t raw_gates, const float *S0,
+                           const void *q, const void *k, const void *v, const void *g, const void *beta,
+                           const int32_t *parent, const int32_t *n_nodes, void *o, int32_t *status_dev,
+                           void *cuda_stream);
+
+int gdn_tree_commit_verify_padded(const gdn_shape_t *shape, int32_t n_trees, int32_t raw_gates, float *S,
+                                  int32_t prev_t_pad, const void *k_prev, const void *v_prev, const void *g_prev,
+                                  const void *beta_prev, const int32_t *parent_prev, const int32_t *n_nodes_prev,
+                                  const int32_t *path, const int32_t *path_len, const void *q, const void *k,
+                                  const void *v, const void *g, const void *beta, const int32_t *parent,
+                                  const int32_t *n_nodes, void *o, int32_t *status_dev, void *cuda_stream);
 
 /*
  * Per-branch recurrent verification: the baseline that Section 3.4 describes as "sequential scans
@@ -188,40 +225,6 @@ int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_pre
                            const void *g, const void *beta, const int32_t *parent,
                            const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
                            int32_t *status_dev, void *cuda_stream);
-
-/*
- * gdn_tree_commit_verify with the commit taken from what the previous verification cached
- * (Section 3.4.1, Eq. 12: the end state of an accepted node follows directly from quantities the
- * verification pass has already computed, so the commit needs no second pass over the prefix).
- * Every verification on the tensor-core path (gdn_tree_verify, gdn_tree_commit_verify[_cached]; trees
- * of at most 64 nodes, d_k = d_v = 128, bf16 inputs) leaves in its workspace the projections
- * S^T k_n of the state it verified against onto the key of every node n.  Given that workspace, the
- * commit of an accepted path n_1..n_L is Eq. 12 restricted to the path: with A_t the decay up to
- * step t,   (I + M) w = r,  r_t = beta_t (v_t / A_t - S^T k_{n_t}),  M_tj = beta_t k_t.k_j (j < t),
- *           S_new = A_L (S + sum_t w_t k_t^T),
- * a rank-L update with no recurrence over d_k; results equal gdn_tree_commit_verify within the same
- * tolerances (the projections carry the 2^-16 relative error of the tensor-core operand split).
- *   prev_workspace    : [device] or NULL: the workspace given to the call that verified the PREVIOUS
- *                       trees (whose accepted paths are committed now), untouched since; read-only
- *                       here and different from `workspace`.  That call must have verified exactly
- *                       the trees described by k_prev .. node_offsets_prev against exactly the state
- *                       S holds now -- the sequence verify(t), commit_verify(t+1), ... of Section 3.4
- *                       guarantees it.  The cache is tagged with the shape of the call that wrote it;
- *                       NULL, a tag that does not match (n_seq, h_v, prev_total_nodes), a call that ran
- *                       on another kernel, or a path that decays below 2^-80 make the commit fall back
- *                       to the step-by-step replay of gdn_tree_commit_verify.
- *   prev_total_nodes  : rows of the previous step's packed tensors (node_offsets_prev[n_seq])
- * Other arguments, error reporting and the treatment of rejected paths and trees as for
- * gdn_tree_commit_verify.  On shapes outside the tensor-core path the cache is ignored.
- */
-int gdn_tree_commit_verify_cached(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
-                                  const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
-                                  const int32_t *node_offsets_prev, const int32_t *path,
-                                  const int32_t *path_offsets, const void *prev_workspace,
-                                  int32_t prev_total_nodes, const void *q, const void *k, const void *v,
-                                  const void *g, const void *beta, const int32_t *parent,
-                                  const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
-                                  int32_t *status_dev, void *cuda_stream);
 
 /*
  * Host-buffer variants: same operations with every tensor in [host] memory

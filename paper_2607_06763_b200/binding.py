@@ -31,7 +31,8 @@ EXPORTS = (
     "gdn_tree_verify_static",
     "gdn_tree_commit_verify",
     "gdn_tree_verify_recurrent",
-    "gdn_tree_commit_verify_cached",
+    "gdn_tree_verify_padded",
+    "gdn_tree_commit_verify_padded",
 )
 
 GDN_STATIC_SCRATCH_BYTES = 4 << 20
@@ -101,9 +102,11 @@ def load_library():
                                                     [vp, ctypes.c_size_t, vp])
         lib.gdn_tree_commit_verify.restype = ctypes.c_int
         lib.gdn_tree_commit_verify.argtypes = [sp] + [vp] * 18 + [ctypes.c_size_t, vp, vp]
-        lib.gdn_tree_commit_verify_cached.restype = ctypes.c_int
-        lib.gdn_tree_commit_verify_cached.argtypes = ([sp] + [vp] * 10 + [ctypes.c_int32] + [vp] * 9 +
-                                                      [ctypes.c_size_t, vp, vp])
+        lib.gdn_tree_verify_padded.restype = ctypes.c_int
+        lib.gdn_tree_verify_padded.argtypes = [sp, ctypes.c_int32, ctypes.c_int32] + [vp] * 11
+        lib.gdn_tree_commit_verify_padded.restype = ctypes.c_int
+        lib.gdn_tree_commit_verify_padded.argtypes = ([sp, ctypes.c_int32, ctypes.c_int32, vp, ctypes.c_int32] +
+                                                      [vp] * 18)
         lib.gdn_tree_verify_static.restype = ctypes.c_int
         lib.gdn_tree_verify_static.argtypes = [sp] + [vp] * 11
         lib.gdn_tree_verify_recurrent.restype = ctypes.c_int
@@ -203,15 +206,23 @@ def gdn_tree_commit_verify_host(shape: GdnShape, S, prev_total_nodes, k_prev, v_
         int(arena_bytes), _stream(stream)))
 
 
-def gdn_tree_commit_verify_cached(shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
-                                  path_offsets, prev_workspace, prev_total_nodes, q, k, v, g, beta, parent,
-                                  node_offsets, o, workspace, workspace_bytes, status_dev, stream=None) -> int:
-    """``gdn_tree_commit_verify_cached``: the fused step with the commit taken from the previous call's workspace."""
-    return int(load_library().gdn_tree_commit_verify_cached(
-        ctypes.byref(shape), _ptr(S), _ptr(k_prev), _ptr(v_prev), _ptr(g_prev), _ptr(beta_prev), _ptr(parent_prev),
-        _ptr(node_offsets_prev), _ptr(path), _ptr(path_offsets), _ptr(prev_workspace), int(prev_total_nodes), _ptr(q),
-        _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(parent), _ptr(node_offsets), _ptr(o), _ptr(workspace),
-        int(workspace_bytes), _ptr(status_dev), _stream(stream)))
+def gdn_tree_verify_padded(shape, n_trees, raw_gates, S0, q, k, v, g, beta, parent, n_nodes, o, status_dev,
+                           stream=None) -> int:
+    """``gdn_tree_verify_padded``: dense ``[slots, T, ...]`` inputs, trees shared by slots, optional raw gates."""
+    return int(load_library().gdn_tree_verify_padded(
+        ctypes.byref(shape), int(n_trees), int(bool(raw_gates)), _ptr(S0), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta),
+        _ptr(parent), _ptr(n_nodes), _ptr(o), _ptr(status_dev), _stream(stream)))
+
+
+def gdn_tree_commit_verify_padded(shape, n_trees, raw_gates, S, prev_t_pad, k_prev, v_prev, g_prev, beta_prev,
+                                  parent_prev, n_nodes_prev, path, path_len, q, k, v, g, beta, parent, n_nodes, o,
+                                  status_dev, stream=None) -> int:
+    """``gdn_tree_commit_verify_padded``: the fused step in the padded layout."""
+    return int(load_library().gdn_tree_commit_verify_padded(
+        ctypes.byref(shape), int(n_trees), int(bool(raw_gates)), _ptr(S), int(prev_t_pad), _ptr(k_prev), _ptr(v_prev),
+        _ptr(g_prev), _ptr(beta_prev), _ptr(parent_prev), _ptr(n_nodes_prev), _ptr(path), _ptr(path_len), _ptr(q),
+        _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(parent), _ptr(n_nodes), _ptr(o), _ptr(status_dev),
+        _stream(stream)))
 
 
 def gdn_tree_verify_recurrent(shape, S0, q, k, v, g, beta, parent, node_offsets, o, status_dev, stream=None) -> int:

@@ -191,6 +191,74 @@ extern "C" int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const 
     return GDN_OK;
 }
 
+namespace {
+
+// Shape rules of the padded entry points: rows per slot = max_tree_nodes, total_nodes = n_seq * rows, every tree
+// shared by n_seq / n_trees slots; they run on the persistent tensor-core kernel only.
+int check_padded_shape(const gdn_shape_t &s, int32_t n_trees)
+{
+    if (n_trees < 1 || s.n_seq % n_trees != 0) return GDN_ERR_SHAPE;
+    if ((long long)s.n_seq * s.max_tree_nodes != s.total_nodes) return GDN_ERR_SHAPE;
+    if (!verify_sm100_single_group(s)) return GDN_ERR_UNSUPPORTED;
+    return GDN_OK;
+}
+
+}  // namespace
+
+extern "C" int gdn_tree_verify_padded(const gdn_shape_t *shape, int32_t n_trees, int32_t raw_gates, const float *S0,
+                                      const void *q, const void *k, const void *v, const void *g, const void *beta,
+                                      const int32_t *parent, const int32_t *n_nodes, void *o, int32_t *status_dev,
+                                      void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
+    rc = check_padded_shape(s, n_trees);
+    if (rc != GDN_OK) return rc;
+    if (!S0 || !q || !k || !v || !g || !beta || !parent || !n_nodes || !o || !status_dev) return GDN_ERR_NULL;
+    if (!aligned16(S0) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        !aligned16(o) || (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(n_nodes) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    if (launch_verify_sm100_padded(s, n_trees, raw_gates != 0, S0, q, k, v, g, beta, parent, n_nodes, o, status_dev,
+                                   static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
+extern "C" int gdn_tree_commit_verify_padded(const gdn_shape_t *shape, int32_t n_trees, int32_t raw_gates, float *S,
+                                             int32_t prev_t_pad, const void *k_prev, const void *v_prev,
+                                             const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                             const int32_t *n_nodes_prev, const int32_t *path,
+                                             const int32_t *path_len, const void *q, const void *k, const void *v,
+                                             const void *g, const void *beta, const int32_t *parent,
+                                             const int32_t *n_nodes, void *o, int32_t *status_dev, void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
+    rc = check_padded_shape(s, n_trees);
+    if (rc != GDN_OK) return rc;
+    if (prev_t_pad < 1 || prev_t_pad > GDN_MAX_TREE_NODES) return GDN_ERR_SHAPE;
+    if (!S || !k_prev || !v_prev || !g_prev || !beta_prev || !n_nodes_prev || !path || !path_len || !q || !k || !v ||
+        !g || !beta || !parent || !n_nodes || !o || !status_dev)
+        return GDN_ERR_NULL;
+    if (!aligned16(S) || !aligned16(k_prev) || !aligned16(v_prev) || !aligned16(g_prev) || !aligned16(beta_prev) ||
+        !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) || !aligned16(o) ||
+        (reinterpret_cast<uintptr_t>(parent_prev) & 3u) || (reinterpret_cast<uintptr_t>(n_nodes_prev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(path) & 3u) || (reinterpret_cast<uintptr_t>(path_len) & 3u) ||
+        (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(n_nodes) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    if (launch_commit_verify_sm100_padded(s, n_trees, raw_gates != 0, S, prev_t_pad, k_prev, v_prev, g_prev, beta_prev,
+                                          parent_prev, n_nodes_prev, path, path_len, q, k, v, g, beta, parent, n_nodes,
+                                          o, status_dev, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
 extern "C" int gdn_tree_verify_recurrent(const gdn_shape_t *shape, const float *S0, const void *q, const void *k,
                                          const void *v, const void *g, const void *beta, const int32_t *parent,
                                          const int32_t *node_offsets, void *o, int32_t *status_dev,
@@ -229,23 +297,19 @@ extern "C" int gdn_tree_commit(const gdn_shape_t *shape, float *S, const void *k
     return GDN_OK;
 }
 
-namespace {
-
-int commit_verify_impl(bool cached, const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
-                       const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
-                       const int32_t *node_offsets_prev, const int32_t *path, const int32_t *path_offsets,
-                       const void *prev_workspace, int32_t prev_total_nodes, const void *q, const void *k,
-                       const void *v, const void *g, const void *beta, const int32_t *parent,
-                       const int32_t *node_offsets, void *o, void *workspace, size_t workspace_bytes,
-                       int32_t *status_dev, void *cuda_stream)
+extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
+                                      const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                      const int32_t *node_offsets_prev, const int32_t *path,
+                                      const int32_t *path_offsets, const void *q, const void *k, const void *v,
+                                      const void *g, const void *beta, const int32_t *parent,
+                                      const int32_t *node_offsets, void *o, void *workspace,
+                                      size_t workspace_bytes, int32_t *status_dev, void *cuda_stream)
 {
     int rc = check_shape(shape);
     if (rc != GDN_OK) return rc;
     const gdn_shape_t &s = *shape;
     if (s.n_seq == 0) return GDN_OK;
     if (!S || !node_offsets_prev || !path_offsets || !status_dev) return GDN_ERR_NULL;
-    if (prev_workspace && (prev_total_nodes < 0 || !aligned256(prev_workspace))) return GDN_ERR_ALIGN;
-    if (prev_workspace && prev_workspace == workspace) return GDN_ERR_WORKSPACE;   // the cache is read while the new one is written
     if (!verify_sm100_single_group(s) || s.total_nodes == 0) {
         // general shapes: the two kernels back to back on the stream (the shape's node counts are
         // not used by commit, so the new tree's shape serves for the previous tree as well).  Both
@@ -277,52 +341,11 @@ int commit_verify_impl(bool cached, const gdn_shape_t *shape, float *S, const vo
     const WorkspaceLayout lay = workspace_layout(s);
     if (workspace_bytes < lay.total) return GDN_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const PlanPtrs plan = plan_ptrs(workspace, lay);
-    const float *pcache_prev = nullptr;
-    const int32_t *tag_prev = nullptr;
-    if (prev_workspace) {   // the previous trees' workspace has the layout of their shape
-        gdn_shape_t prev = s;
-        prev.total_nodes = prev_total_nodes;
-        const WorkspaceLayout pl = workspace_layout(prev);
-        const char *pb = static_cast<const char *>(prev_workspace);
-        pcache_prev = reinterpret_cast<const float *>(pb + pl.pcache);
-        tag_prev = reinterpret_cast<const int32_t *>(pb + pl.cache_tag);
-    }
     if (launch_commit_verify_sm100(s, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
-                                   path_offsets, q, k, v, g, beta, parent, node_offsets, o, plan, pcache_prev,
-                                   tag_prev, prev_total_nodes, cached, status_dev, stream) != cudaSuccess)
+                                   path_offsets, q, k, v, g, beta, parent, node_offsets, o, status_dev,
+                                   stream) != cudaSuccess)
         return GDN_ERR_CUDA;
     return GDN_OK;
-}
-
-}  // namespace
-
-extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const void *k_prev, const void *v_prev,
-                                      const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
-                                      const int32_t *node_offsets_prev, const int32_t *path,
-                                      const int32_t *path_offsets, const void *q, const void *k, const void *v,
-                                      const void *g, const void *beta, const int32_t *parent,
-                                      const int32_t *node_offsets, void *o, void *workspace,
-                                      size_t workspace_bytes, int32_t *status_dev, void *cuda_stream)
-{
-    return commit_verify_impl(false, shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
-                              path_offsets, nullptr, 0, q, k, v, g, beta, parent, node_offsets, o, workspace,
-                              workspace_bytes, status_dev, cuda_stream);
-}
-
-extern "C" int gdn_tree_commit_verify_cached(const gdn_shape_t *shape, float *S, const void *k_prev,
-                                             const void *v_prev, const void *g_prev, const void *beta_prev,
-                                             const int32_t *parent_prev, const int32_t *node_offsets_prev,
-                                             const int32_t *path, const int32_t *path_offsets,
-                                             const void *prev_workspace, int32_t prev_total_nodes, const void *q,
-                                             const void *k, const void *v, const void *g, const void *beta,
-                                             const int32_t *parent, const int32_t *node_offsets, void *o,
-                                             void *workspace, size_t workspace_bytes, int32_t *status_dev,
-                                             void *cuda_stream)
-{
-    return commit_verify_impl(true, shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
-                              path_offsets, prev_workspace, prev_total_nodes, q, k, v, g, beta, parent, node_offsets,
-                              o, workspace, workspace_bytes, status_dev, cuda_stream);
 }
 
 extern "C" size_t gdn_tree_host_arena_bytes(const gdn_shape_t *shape, int32_t total_path_len)

@@ -29,15 +29,9 @@ namespace gdn {
 //   dfs_depth uint8 [N]                    depth of that node
 //   dfs_anc8  uint8 [N][16]                its root path in virtual indices of its group (0xFF = unused)
 //   utilde   float [N][h_v][d_v]           solve result u~ (Eq. 10 with the W S0 term folded in; general kernel)
-//   pcache   float [N][h_v][d_v]           projection cache: row (n, h) = S^T k_n of the state S the tree was verified
-//                                          against (written by the persistent tensor-core kernel; what a later
-//                                          commit of an accepted path of this tree needs from the old state)
-//   cache_tag int32[4]                     {GDN_CACHE_MAGIC, total_nodes, h_v, n_seq} once pcache has been written
-//                                          by a call of that shape; zeroed by the calls that do not write it
 struct WorkspaceLayout {
-    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, group_start, utilde, pcache, cache_tag, total;
+    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, group_start, utilde, total;
 };
-constexpr int32_t GDN_CACHE_MAGIC = 0x47444E43;
 
 constexpr int GDN_GROUP_TILE = 64;            // nodes of a group and its prefix together
 constexpr int GDN_GROUP_MIN_NODES = 49;       // own nodes a group has at least (prefix of 15)
@@ -60,8 +54,6 @@ inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
     w.dfs_anc8 = off; off = align256(off + 16 * N);
     w.group_start = off; off = align256(off + sizeof(uint16_t) * (size_t)s.n_seq * (GDN_MAX_GROUPS + 1));
     w.utilde = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
-    w.pcache = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
-    w.cache_tag = off; off = align256(off + 4 * sizeof(int32_t));
     w.total = off;
     return w;
 }
@@ -75,8 +67,6 @@ struct PlanPtrs {
     uint8_t *dfs_depth, *dfs_anc8;
     uint16_t *group_start;
     float *utilde;
-    float *pcache;
-    int32_t *cache_tag;
 };
 
 inline PlanPtrs plan_ptrs(void *workspace, const WorkspaceLayout &w)
@@ -86,8 +76,7 @@ inline PlanPtrs plan_ptrs(void *workspace, const WorkspaceLayout &w)
             reinterpret_cast<uint16_t *>(b + w.anc), reinterpret_cast<uint8_t *>(b + w.anc8),
             reinterpret_cast<uint16_t *>(b + w.dfs_node), reinterpret_cast<uint8_t *>(b + w.dfs_depth),
             reinterpret_cast<uint8_t *>(b + w.dfs_anc8), reinterpret_cast<uint16_t *>(b + w.group_start),
-            reinterpret_cast<float *>(b + w.utilde), reinterpret_cast<float *>(b + w.pcache),
-            reinterpret_cast<int32_t *>(b + w.cache_tag)};
+            reinterpret_cast<float *>(b + w.utilde)};
 }
 
 // Host launchers (each returns the cudaError_t of its launch).
@@ -111,17 +100,31 @@ cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const voi
 
 // Same kernel with the commit of the previous step's accepted paths fused in front of the verify:
 // the state tile is read once, advanced along the path (Eq. 7), written back, and the new tree is
-// verified against the advanced state.  pcache_prev / cache_tag_prev (may be NULL): the projection cache that
-// the verification of the previous trees left in its workspace; with it the commit is a rank-L update.
-// write_cache: leave the projections of the new trees in `plan` for the step after this one.
+// verified against the advanced state.
 cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const void *k_prev, const void *v_prev,
                                        const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
                                        const int32_t *node_offsets_prev, const int32_t *path,
                                        const int32_t *path_offsets, const void *q, const void *k, const void *v,
                                        const void *g, const void *beta, const int32_t *parent,
-                                       const int32_t *node_offsets, void *o, const PlanPtrs &plan,
-                                       const float *pcache_prev, const int32_t *cache_tag_prev, int prev_total_nodes,
-                                       bool write_cache, int32_t *status_dev, cudaStream_t stream);
+                                       const int32_t *node_offsets, void *o, int32_t *status_dev,
+                                       cudaStream_t stream);
+
+// Padded layout of Section 3.4.2 on the persistent tensor-core kernel (s.max_tree_nodes = rows per slot, s.total_nodes =
+// n_seq * rows per slot, trees of at most 64 nodes): slot b carries tree b % n_trees; parent [n_trees][t_pad], n_nodes
+// [n_trees]; raw_gates: g / beta are raw gate inputs.  The fused form takes the previous step in the same layout
+// (prev_t_pad rows per slot) and one accepted path per tree: path [n_trees][max_depth], path_len [n_trees].
+cudaError_t launch_verify_sm100_padded(const gdn_shape_t &s, int n_trees, bool raw_gates, const float *S0,
+                                       const void *q, const void *k, const void *v, const void *g, const void *beta,
+                                       const int32_t *parent, const int32_t *n_nodes, void *o, int32_t *status_dev,
+                                       cudaStream_t stream);
+cudaError_t launch_commit_verify_sm100_padded(const gdn_shape_t &s, int n_trees, bool raw_gates, float *S,
+                                              int prev_t_pad, const void *k_prev, const void *v_prev,
+                                              const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                              const int32_t *n_nodes_prev, const int32_t *path,
+                                              const int32_t *path_len, const void *q, const void *k, const void *v,
+                                              const void *g, const void *beta, const int32_t *parent,
+                                              const int32_t *n_nodes, void *o, int32_t *status_dev,
+                                              cudaStream_t stream);
 
 // Per-branch recurrent verification (the baseline of Section 5.2 / Figure 5): no workspace, no tree plan.
 cudaError_t launch_verify_recurrent(const gdn_shape_t &s, const float *S0, const void *q, const void *k,

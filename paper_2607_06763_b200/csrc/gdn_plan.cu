@@ -18,8 +18,7 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
             const int32_t *__restrict__ parent, const int32_t *__restrict__ node_offsets,
             int32_t *__restrict__ tree_ok, uint8_t *__restrict__ depth, uint16_t *__restrict__ anc,
             uint8_t *__restrict__ anc8, uint16_t *__restrict__ dfs_node, uint8_t *__restrict__ dfs_depth,
-            uint8_t *__restrict__ dfs_anc8, uint16_t *__restrict__ group_start, int32_t *__restrict__ cache_tag,
-            int32_t *status_dev)
+            uint8_t *__restrict__ dfs_anc8, uint16_t *__restrict__ group_start, int32_t *status_dev)
 {
     __shared__ int size_s[GDN_GROUPED_MAX_NODES];        // subtree sizes
     __shared__ uint16_t left_s[GDN_GROUPED_MAX_NODES];   // nodes in the subtrees of earlier siblings
@@ -34,8 +33,6 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
     const int b = blockIdx.x;
-    // the kernels that run behind this one do not fill the projection cache of this workspace: mark it empty
-    if (b == 0 && threadIdx.x == 0) cache_tag[0] = 0;
     const int lo = node_offsets[b], hi = node_offsets[b + 1];
     const int T = hi - lo;
     bool offsets_ok = lo >= 0 && T >= 0 && T <= max_tree_nodes && hi <= total_nodes;
@@ -161,7 +158,7 @@ cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, plan_kernel, s.n_seq, s.total_nodes, s.max_tree_nodes, s.max_depth, parent,
                               node_offsets, plan.tree_ok, plan.depth, plan.anc, plan.anc8, plan.dfs_node,
-                              plan.dfs_depth, plan.dfs_anc8, plan.group_start, plan.cache_tag, status_dev);
+                              plan.dfs_depth, plan.dfs_anc8, plan.group_start, status_dev);
 }
 
 }  // namespace gdn

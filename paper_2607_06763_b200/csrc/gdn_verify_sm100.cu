@@ -22,8 +22,6 @@
 // Two kernels: a persistent one for trees that fit one CTA (TMA tiles on mbarriers, a software pipeline across
 // the units of a CTA, optionally the commit of the previous step fused in front), and a one-shot one for the
 // groups of larger trees (row gathers through a node table).
-#include <cstdlib>
-#include <type_traits>
 #include <cuda.h>   // CUtensorMap and the cuTensorMapEncodeTiled prototype (resolved at run time, no libcuda link)
 
 #include "gdn_internal.cuh"
@@ -73,11 +71,7 @@ constexpr int SM_TMEM = SM_MBAR + 40;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
 constexpr int SM_PAR = SM_FLAG + 4;              // persistent kernel: s8 [64] parent[] of the tree whose tables are being built
 constexpr int SM_BAD = SM_PAR + FV_T;            // persistent kernel: int [2], tree of table buffer tb was rejected
-constexpr int SM_GM = (SM_BAD + 8 + 15) & ~15;   // fused commit from the cache: fp32 k_t . k_j of the path, j < t, at t (t - 1) / 2 + j
-constexpr int SM_NM = SM_GM + 480;               //   fp32 N = (I + M)^-1, M_tj = beta_t k_t . k_j: N_tj, j <= t, at t (t + 1) / 2 + j
-constexpr int SM_BYTES = SM_NM + 544;
-constexpr int SM_PC = 57344;                     // fused commit from the cache: fp32 [16][128] cached projections of the path's
-                                                 // nodes, then (in place) the update coefficients w; in the state-operand area
+constexpr int SM_BYTES = SM_BAD + 8;
 constexpr int SM_ALLOC = SM_BYTES + 1024;        // slack for the 1024-byte alignment of the base
 
 struct VerifyFastParams {
@@ -99,9 +93,6 @@ struct VerifyFastParams {
     const uint8_t *depth;
     const uint8_t *anc8;
     int32_t *status_dev;
-    // projection cache (persistent kernel): rows S^T k_n of every node, left for the commit of the next step
-    float *pcache_out;
-    int32_t *cache_tag_out;
     // grouped verification of trees with more than 64 nodes (only read by the GROUPED instantiation)
     int groups_per_tree, anc_stride;                   // CTAs per (tree, head); entries per row of anc16
     const uint16_t *anc16, *dfs_node, *group_start;
@@ -110,10 +101,12 @@ struct VerifyFastParams {
     float *S_rw;                                       // same tensor as S0, written in place
     const __nv_bfloat16 *pk, *pv, *pg, *pbeta;         // the previous tree's k, v, g, beta
     const int32_t *pparent, *pnode_offsets, *path, *path_offsets;
-    const float *pcache_prev;                          // projection cache of the previous trees (may be NULL)
-    const int32_t *cache_tag_prev;
-    int prev_total_nodes;
-    int cached_min_len;                                // shortest accepted path that is committed from the cache
+    // Padded layout of Section 3.4.2 (persistent kernel; t_pad = 0: ragged packing by node_offsets[]): slot b keeps
+    // its nodes in rows b * t_pad .. and carries tree b % n_trees, whose parent[] row and node count are shared by
+    // all the slots (layers) of that tree; the accepted paths are per tree as well.
+    int t_pad, n_trees, pt_pad, path_stride;
+    const int32_t *n_nodes, *pn_nodes, *path_len;
+    int raw_gates;                                     // g / beta arrive as raw gate inputs ("scalars" stage on chip)
 };
 
 // ---------------------------------------------------------------------------------------- PTX
@@ -731,20 +724,30 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
 }
 
+// Gate activations of the "scalars" stage (Section 3.4.2; Table 1 row "scalars"): the kernel takes either the
+// finished log-decay g and write strength beta, or the layer's raw gate inputs a, b, for which
+// g = -softplus(a) = -log(1 + e^a) and beta = sigmoid(b) are formed here (fp32, never rounded to the input type).
+__device__ __forceinline__ float gate_log_decay(uint32_t bf16_bits, bool raw)
+{
+    const float x = __uint_as_float(bf16_bits << 16);
+    if (!raw) return x;
+    return x > 0.f ? -(x + log1pf(expf(-x))) : -log1pf(expf(x));
+}
+__device__ __forceinline__ float gate_beta(uint32_t bf16_bits, bool raw)
+{
+    const float x = __uint_as_float(bf16_bits << 16);
+    if (!raw) return x;
+    const float e = expf(-fabsf(x));
+    return x >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
+}
+
 // Persistent form of the kernel above for trees that fit one CTA, with the optional fused commit.  The k/q tile
 // holds the k rows first and the q rows second (rows i and 64 + i), so P has p^k in columns 0..63 and p^q in
 // columns 64..127, and the Gram block needs only N = 64.
-// FUSED: the previous step's accepted path is committed on the state tile while it sits in registers, the tile is
-// written back as the only state write of the step, and the new tree is verified against it.  Two forms:
-//  - replay: per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c) step by step, the eight lanes that share a row
-//    reducing k.s_c with three shuffles;
-//  - from the projection cache (the masked end-state formula, Eq. 12, restricted to the accepted path).  Every
-//    verification leaves p_n = S^T k_n of all its nodes in its workspace (they are in registers in the R phase
-//    anyway).  With A_t = alpha_1..alpha_t and S~_t = S_t / A_t, Eq. 7 reads S~_t = S~_{t-1} + w_t k_t^T with
-//        (I + M) w = r,   r_t = beta_t (v_t / A_t - p_{n_t}),   M_tj = beta_t (k_t . k_j) for j < t,
-//    an L x L triangular system shared by all 128 value components: its inverse N is formed once per unit (sixteen
-//    threads, one column each), w = N r by all threads, and the commit is the rank-L update S_new = A_L (S0 + sum_t
-//    w_t k_t^T) on the registers: no dot product over d_k, no shuffle, no step that waits for the one before.
+// FUSED: Eq. 7 is replayed along the previous step's accepted path on the state tile while it sits in registers
+// -- per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c), the eight lanes that share a row reducing k.s_c with
+// three shuffles -- the tile is written back as the only state write of the step, and the new tree is verified
+// against it.
 // A CTA keeps its tensor memory and walks over the units blockIdx.x, blockIdx.x + gridDim.x, ...  Nothing a unit
 // can know in advance is waited for inside it: the next unit's k/q tile streams into the operand tile as soon as the
 // first MMA group has released it, its Gram block is issued at the end of the current unit into spare TMEM columns,
@@ -752,7 +755,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 // its value is used.  The state tile is asked for at the top of the unit and is needed only after the Gram /
 // coefficient phases; the v rows land by TMA in an area that is free until the state operand is written.
 // SMALL (every tree of the call has at most 32 nodes): the R and output phases skip the 16-node pieces beyond the tree.
-template <typename TOut, bool FUSED, bool SMALL, bool CACHED>
+template <typename TOut, bool FUSED, bool SMALL, bool PADDED>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const __grid_constant__ VerifyFastParams p)
 {
     extern __shared__ uint8_t fv_smem_raw[];
@@ -790,23 +793,32 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // The first unit's state tile is an input of the call, not of that kernel: L2 is asked for it meanwhile.
     if (tid < 4 && (int)blockIdx.x < p.n_units)
         prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
-    bool use_cache = false;   // FUSED: commit from the projection cache (decided once per call, below)
     signed char *par_s = reinterpret_cast<signed char *>(smem + SM_PAR);
     volatile int *bad_s = reinterpret_cast<volatile int *>(smem + SM_BAD);
 
     // unit -> (tree, head, first node, size); a unit whose node_offsets[] are inconsistent (reported) or whose tree
     // is empty is skipped.  parent[] itself is checked when the unit's tables are built.
-    auto decode = [&](int u, int &ub, int &uh, int &uhk, int &ubase, int &uT) -> bool {
+    auto decode = [&](int u, int &ub, int &uh, int &uhk, int &ubase, int &uT, int &upar) -> bool {
         if (u >= p.n_units) return false;
         ub = u / p.h_v;
         uh = u % p.h_v;
         uhk = uh / (p.h_v / p.h_qk);
-        ubase = p.node_offsets[ub];
-        const int uend = p.node_offsets[ub + 1];
-        uT = uend - ubase;
-        bool off_ok = ubase >= 0 && uT >= 0 && uT <= FV_T && uT <= p.max_tree_nodes && uend <= p.total_nodes;
-        if (ub == 0) off_ok = off_ok && ubase == 0;
-        if (ub == p.n_seq - 1) off_ok = off_ok && uend == p.total_nodes;
+        bool off_ok;
+        if (PADDED && p.t_pad) {   // padded layout: rows of the slot, node count and parent[] row of its tree
+            const int tree = ub % p.n_trees;
+            ubase = ub * p.t_pad;
+            uT = p.n_nodes[tree];
+            upar = tree * p.t_pad;
+            off_ok = uT >= 0 && uT <= FV_T && uT <= p.t_pad;
+        } else {
+            ubase = p.node_offsets[ub];
+            const int uend = p.node_offsets[ub + 1];
+            uT = uend - ubase;
+            upar = ubase;
+            off_ok = ubase >= 0 && uT >= 0 && uT <= FV_T && uT <= p.max_tree_nodes && uend <= p.total_nodes;
+            if (ub == 0) off_ok = off_ok && ubase == 0;
+            if (ub == p.n_seq - 1) off_ok = off_ok && uend == p.total_nodes;
+        }
         if (!off_ok && tid == 0) report_status(p.status_dev, GDN_ERR_TREE);
         const bool tree_good = off_ok && uT > 0;
         if (FUSED && !tree_good) {
@@ -814,6 +826,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             // nodes (every node masked, nothing stored), so that its accepted path is still replayed
             ubase = 0;
             uT = 0;
+            upar = 0;
             return true;
         }
         return tree_good;
@@ -877,12 +890,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[tnode] = (uint8_t)d;
             *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + tnode * 16) = make_uint4(w0, w1, w2, w3);
             reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[tnode] =
-                make_float4(0.f, 0.f, __uint_as_float(be_bits << 16), __uint_as_float(g_bits << 16));
+                make_float4(0.f, 0.f, gate_beta(be_bits, PADDED && p.raw_gates), gate_log_decay(g_bits, PADDED && p.raw_gates));
         }
     };
     // the same two steps with the loads issued on the spot (first unit of a CTA, and behind a skipped unit)
-    auto load_parent = [&](int ubase, int uT, int tb) -> bool {
-        return put_parent(uT, tbl_thread && tnode < uT ? p.parent[ubase + tnode] : -1, tb);
+    auto load_parent = [&](int upar, int uT, int tb) -> bool {
+        return put_parent(uT, tbl_thread && tnode < uT ? p.parent[upar + tnode] : -1, tb);
     };
     auto load_tables = [&](int uh, int ubase, int uT, int tb, bool my_bad) {
         uint32_t gb = 0, bb = 0;
@@ -902,18 +915,30 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if constexpr (FUSED) {
             if (warp == 4) {
                 int *slot = reinterpret_cast<int *>(smem + SM_PATH + ps * SM_PATH_SLOT);
-                const int pp0 = p.path_offsets[ub];
-                int len = p.path_offsets[ub + 1] - pp0;   // 0 leaves the state alone
-                int pb = 0;
+                int pp0, len, pb = 0, pT = 0, ppar = 0;   // len 0 leaves the state alone
+                if (PADDED && p.t_pad) {
+                    const int tree = ub % p.n_trees;
+                    pp0 = tree * p.path_stride;
+                    len = p.path_len[tree];
+                    pb = ub * p.pt_pad;
+                    pT = min(p.pn_nodes[tree], p.pt_pad);
+                    ppar = tree * p.pt_pad;
+                } else {
+                    pp0 = p.path_offsets[ub];
+                    len = p.path_offsets[ub + 1] - pp0;
+                    if (len != 0) {
+                        pb = p.pnode_offsets[ub];
+                        pT = p.pnode_offsets[ub + 1] - pb;
+                        ppar = pb;
+                    }
+                }
                 if (len != 0) {
-                    pb = p.pnode_offsets[ub];
-                    const int pT = p.pnode_offsets[ub + 1] - pb;
                     const bool shape_ok = len > 0 && len <= FV_MD && len <= p.max_depth && pT > 0 && pp0 >= 0;
                     const bool mine = shape_ok && lane < len;
                     int n = -1, parent_n = -2;
                     if (mine) {
                         n = p.path[pp0 + lane];
-                        if (p.pparent && n >= 0 && n < pT) parent_n = p.pparent[pb + n];
+                        if (p.pparent && n >= 0 && n < pT) parent_n = p.pparent[ppar + n];
                         slot[lane] = n;
                     }
                     const int n_up = __shfl_up_sync(0xffffffffu, n, 1);
@@ -953,20 +978,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
     };
-    // cached projections of the path's nodes (fp32, 512 B each) into their parking area
-    auto fetch_path_pc = [&](int uh, int ps) {
-        if constexpr (FUSED && CACHED) {
-            if (use_cache) {
-                const int *slot = reinterpret_cast<const int *>(smem + SM_PATH + ps * SM_PATH_SLOT);
-                const int len = slot[16], pb = slot[17];
-                for (int idx = tid; idx < len * 32; idx += FV_THREADS) {
-                    const int t = idx >> 5, c16 = idx & 31;
-                    const size_t n = (size_t)pb + slot[t];
-                    cp_async_16(sbase + SM_PC + t * 512 + c16 * 16, p.pcache_prev + (n * p.h_v + uh) * FV_D + c16 * 4, true);
-                }
-            }
-        }
-    };
     // per-step scalars of the path, computed on the spot (first unit of a CTA, and behind a skipped unit)
     auto path_scalars_direct = [&](int uh, int ps) {
         if constexpr (FUSED) {
@@ -975,45 +986,15 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             const int len = slot[16], pb = slot[17];
             if (tid < len) {
                 float gsum = 0.f, gt = 0.f;
+                const unsigned short *pg = reinterpret_cast<const unsigned short *>(p.pg);
+                const unsigned short *pbe = reinterpret_cast<const unsigned short *>(p.pbeta);
                 for (int t = 0; t <= tid; ++t) {
-                    gt = __bfloat162float(p.pg[((size_t)pb + slot[t]) * p.h_v + uh]);
+                    gt = gate_log_decay(pg[((size_t)pb + slot[t]) * p.h_v + uh], PADDED && p.raw_gates);
                     gsum += gt;
                 }
                 const size_t n = (size_t)pb + slot[tid];
                 const float A = expf(gsum);
-                ab[tid] = make_float4(A, __bfloat162float(p.pbeta[n * p.h_v + uh]), expf(gt), 1.f / A);
-            }
-        }
-    };
-    // k_t . k_j for the pairs j < t of the path whose k rows have landed: eight lanes per pair, 32 pairs per round
-    auto path_gram = [&](int ps) {
-        if constexpr (FUSED && CACHED) {
-            if (use_cache) {
-                float *gm = reinterpret_cast<float *>(smem + SM_GM);
-                const int len = reinterpret_cast<const int *>(smem + SM_PATH + ps * SM_PATH_SLOT)[16];
-                const int n_pairs = len * (len - 1) / 2;
-                for (int pi0 = warp * 4; pi0 < n_pairs; pi0 += FV_THREADS / 8) {   // warp-uniform trip count
-                    const int pi = min(pi0 + r4, n_pairs - 1);
-                    int t = 1, j = pi;
-                    while (j >= t) { j -= t; ++t; }
-                    const uint16_t *pk = reinterpret_cast<const uint16_t *>(smem + SM_PK);
-                    float2 acc = make_float2(0.f, 0.f);
-#pragma unroll
-                    for (int kh = 0; kh < 2; ++kh) {
-                        const uint4 a = *reinterpret_cast<const uint4 *>(pk + t * FV_D + kh * 64 + l8 * 8);
-                        const uint4 c = *reinterpret_cast<const uint4 *>(pk + j * FV_D + kh * 64 + l8 * 8);
-                        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, cw[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            acc = __ffma2_rn(make_float2(__uint_as_float(aw[e] << 16), __uint_as_float(aw[e] & 0xFFFF0000u)),
-                                             make_float2(__uint_as_float(cw[e] << 16), __uint_as_float(cw[e] & 0xFFFF0000u)), acc);
-                    }
-                    float dot = acc.x + acc.y;
-                    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-                    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-                    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-                    if (l8 == 0 && pi0 + r4 < n_pairs) gm[pi] = dot;
-                }
+                ab[tid] = make_float4(A, gate_beta(pbe[n * p.h_v + uh], PADDED && p.raw_gates), expf(gt), 1.f / A);
             }
         }
     };
@@ -1051,27 +1032,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
     };
 
-    int b = 0, h = 0, hk = 0, base = 0, T = 0;
+    int b = 0, h = 0, hk = 0, base = 0, T = 0, par0 = 0;
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // ... and whatever is launched behind this grid with the same attribute (the next call's tree-metadata kernel,
     // which itself waits for this grid to complete before it reads or writes anything) may be made resident now.
     asm volatile("griddepcontrol.launch_dependents;");
-    if constexpr (FUSED && CACHED) {
-        // the projection cache of the previous trees is used if the call that left it had their shape
-        if (p.pcache_prev && p.cache_tag_prev) {
-            const int4 tg = __ldg(reinterpret_cast<const int4 *>(p.cache_tag_prev));
-            use_cache = tg.x == GDN_CACHE_MAGIC && tg.y == p.prev_total_nodes && tg.z == p.h_v && tg.w == p.n_seq;
-        }
-    }
-    if (blockIdx.x == 0 && tid == 0 && p.cache_tag_out)
-        *reinterpret_cast<int4 *>(p.cache_tag_out) =
-            CACHED && p.pcache_out ? make_int4(GDN_CACHE_MAGIC, p.total_nodes, p.h_v, p.n_seq) : make_int4(0, 0, 0, 0);
-    bool cur_ok = decode(blockIdx.x, b, h, hk, base, T);
+    bool cur_ok = decode(blockIdx.x, b, h, hk, base, T, par0);
     bool par_bad = false;
     if (cur_ok) {
         issue_kq(b, hk, base, T);
         fetch_path(b, 0);
-        par_bad = load_parent(base, T, 0);
+        par_bad = load_parent(par0, T, 0);
     }
     __syncthreads();
     if (cur_ok) load_tables(h, base, T, 0, par_bad);
@@ -1079,25 +1050,16 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (cur_ok) {
         path_decay(0);
         fetch_path_kv(h, hk, 0);
-        fetch_path_pc(h, 0);
         path_scalars_direct(h, 0);
         issue_gram(0);
     }
-    if constexpr (FUSED && CACHED) {
-        if (use_cache) {   // (call-uniform) the k rows have to be there for the path's Gram block
-            cp_async_wait_all();
-            __syncthreads();
-            if (cur_ok) path_gram(0);
-        }
-    }
-
     int done_units = 0;
 #pragma unroll 1
     for (int unit = blockIdx.x, iter = 0; unit < p.n_units; unit += gridDim.x, ++iter) {
     const bool unit_ok = cur_ok;
     const uint32_t par = (uint32_t)(done_units & 1);   // every barrier completes once per processed unit
-    int nb = 0, nh = 0, nhk = 0, nbase = 0, nT = 0;
-    const bool next_ok = decode(unit + gridDim.x, nb, nh, nhk, nbase, nT);
+    int nb = 0, nh = 0, nhk = 0, nbase = 0, nT = 0, npar0 = 0;
+    const bool next_ok = decode(unit + gridDim.x, nb, nh, nhk, nbase, nT, npar0);
     float4 *gab = reinterpret_cast<float4 *>(smem + SM_GAB + (iter & 1) * SM_TABLE_STRIDE);
     uint8_t *anc_s = smem + SM_ANC + (iter & 1) * SM_TABLE_STRIDE;
     uint8_t *depth_s = smem + SM_DEPTH + (iter & 1) * SM_TABLE_STRIDE;
@@ -1106,7 +1068,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         bool nbad = false;
         if (next_ok) {
             issue_kq(nb, nhk, nbase, nT);
-            nbad = load_parent(nbase, nT, (iter + 1) & 1);
+            nbad = load_parent(npar0, nT, (iter + 1) & 1);
             fetch_path(nb, (iter + 1) & 1);
         }
         __syncthreads();
@@ -1115,16 +1077,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if (next_ok) {
             path_decay((iter + 1) & 1);
             fetch_path_kv(nh, nhk, (iter + 1) & 1);
-            fetch_path_pc(nh, (iter + 1) & 1);
             path_scalars_direct(nh, (iter + 1) & 1);
             issue_gram(par);   // no unit was processed in between: the tile's barrier phase is this one
-        }
-        if constexpr (FUSED && CACHED) {
-            if (use_cache) {
-                cp_async_wait_all();
-                __syncthreads();
-                if (next_ok) path_gram((iter + 1) & 1);
-            }
         }
         b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
         continue;
@@ -1168,46 +1122,10 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // block of this unit was issued one unit ahead; every thread waits for it on its own (bounded: on expiry it
     // flags the error and everybody falls through to the clean-up).
     if (!mbar_wait_bounded(mbar_g, par)) *flag = 1;
-    if constexpr (CACHED) {
-        if (use_cache) cp_async_wait_all();   // the path's cached projections, asked for one unit ahead
-    }
     tc_fence_after();
     __syncthreads();
     warm_l2_state(0);
-    // Form of the commit (unit-uniform; the path's scalars were written behind the last barrier of the unit before
-    // and are readable from here on): from the cache unless the path decays below 2^-80 (1 / A_t could overflow).
-    bool cached_commit = false;
-    if constexpr (FUSED && CACHED)
-        cached_commit = use_cache && path_len >= p.cached_min_len && path_len > 0 && ab_path[path_len - 1].x > 8.3e-25f;
     if (*flag == 0) {
-        if constexpr (FUSED && CACHED) {
-            // N = (I + M)^-1, M_tj = beta_t (k_t . k_j): lane j of warp 4 builds column j (u_m = N_{j+m,j})
-            if (cached_commit && warp == 4 && lane < path_len) {
-                const float *gm = reinterpret_cast<const float *>(smem + SM_GM);
-                float *nm = reinterpret_cast<float *>(smem + SM_NM);
-                const int j = lane;
-                nm[j * (j + 1) / 2 + j] = 1.f;
-                auto column = [&](auto lb) {   // unrolled for paths of at most LB nodes
-                    constexpr int LB = decltype(lb)::value;
-                    float u[LB];
-                    u[0] = 1.f;
-#pragma unroll
-                    for (int m = 1; m < LB; ++m) {
-                        const int t = j + m;
-                        float acc = 0.f;
-                        if (t < path_len) {
-#pragma unroll
-                            for (int n = 0; n < m; ++n) acc = fmaf(gm[t * (t - 1) / 2 + j + n], u[n], acc);
-                            acc *= -ab_path[t].y;
-                            nm[t * (t + 1) / 2 + j] = acc;
-                        }
-                        u[m] = acc;
-                    }
-                };
-                if (path_len <= 8) column(std::integral_constant<int, 8>{});
-                else column(std::integral_constant<int, 16>{});
-            }
-        }
         // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
         {
             const int row = (warp & 3) * 32 + lane;
@@ -1256,43 +1174,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 xs[idx] = onx[u] ? bi[u] * dec * gk[u] : 0.f;
             }
         }
-        if constexpr (FUSED && CACHED) {
-            // w = N r for value component c = tid / 2, r_j = beta_j (v_j[c] / A_j - p_j[c]); the two threads of a
-            // component take the even and the odd steps, and w replaces p in place (every r is in registers before
-            // either of them stores: __syncwarp)
-            if (cached_commit) {
-                const float *nm = reinterpret_cast<const float *>(smem + SM_NM);
-                float *pc = reinterpret_cast<float *>(smem + SM_PC);
-                const uint16_t *pv = reinterpret_cast<const uint16_t *>(smem + SM_PV);
-                const int c = tid >> 1, hf = tid & 1;
-                auto coefficients = [&](auto lb) {   // unrolled for paths of at most LB nodes
-                    constexpr int LB = decltype(lb)::value;
-                    float r[LB];
-#pragma unroll
-                    for (int j = 0; j < LB; ++j) {
-                        r[j] = 0.f;
-                        if (j < path_len) {
-                            const float4 ab = ab_path[j];
-                            r[j] = ab.y * fmaf(__uint_as_float((uint32_t)pv[j * FV_D + c] << 16), ab.w, -pc[j * FV_D + c]);
-                        }
-                    }
-                    __syncwarp();
-#pragma unroll
-                    for (int tt = 0; tt < LB / 2; ++tt) {
-                        const int t = 2 * tt + hf;
-                        if (2 * tt < path_len) {   // warp-uniform
-                            float acc = 0.f;
-#pragma unroll
-                            for (int j = 0; j <= 2 * tt + 1; ++j)
-                                if (j <= t) acc = fmaf(nm[t * (t + 1) / 2 + j], r[j], acc);
-                            if (t < path_len) pc[t * FV_D + c] = acc;
-                        }
-                    }
-                };
-                if (path_len <= 8) coefficients(std::integral_constant<int, 8>{});
-                else coefficients(std::integral_constant<int, 16>{});
-            }
-        }
     }
     cp_async_wait_all();
     __syncthreads();   // X and Y complete; the Gram copy is dead and its area can take the state operand
@@ -1304,40 +1185,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     const bool healthy = *flag == 0;   // uniform: every write of the flag so far lies before the barrier above
     if constexpr (FUSED) {
         if (!healthy) path_len = 0;    // a wait expired: this state is left as it was
-        if (cached_commit && healthy) {
-            // S_new = A_L (S0 + sum_t w_t k_t^T): rank-L update of the registers
-            const float *wcol = reinterpret_cast<const float *>(smem + SM_PC) + warp * 16 + r4;
-            const uint16_t *pks = reinterpret_cast<const uint16_t *>(smem + SM_PK);
-#pragma unroll 1
-            for (int t = 0; t < path_len; ++t) {
-                float2 kf2[8];
-#pragma unroll
-                for (int kh = 0; kh < 2; ++kh) {
-                    const uint4 kw = *reinterpret_cast<const uint4 *>(pks + t * FV_D + kh * 64 + l8 * 8);
-                    const uint32_t w4[4] = {kw.x, kw.y, kw.z, kw.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        kf2[kh * 4 + e] = make_float2(__uint_as_float(w4[e] << 16), __uint_as_float(w4[e] & 0xFFFF0000u));
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float wv = wcol[t * FV_D + i * 4];
-                    const float2 w2 = make_float2(wv, wv);
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, make_float2(x[i][q4].x, x[i][q4].y));
-                        const float2 hi = __ffma2_rn(kf2[q4 * 2 + 1], w2, make_float2(x[i][q4].z, x[i][q4].w));
-                        x[i][q4] = make_float4(lo.x, lo.y, hi.x, hi.y);
-                    }
-                }
-            }
-            const float aL = ab_path[path_len - 1].x;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4)
-                    x[i][q4] = make_float4(aL * x[i][q4].x, aL * x[i][q4].y, aL * x[i][q4].z, aL * x[i][q4].w);
-        } else if (path_len > 0) {
+        if (path_len > 0) {
             replay_path_on_tile(x, path_len, reinterpret_cast<const uint16_t *>(smem + SM_PK),
                                 reinterpret_cast<const uint16_t *>(smem + SM_PV), ab_path, warp, r4, l8);
         }
@@ -1391,22 +1239,32 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     int t_par = -1;
     bool t_bad = false;
     unsigned short t_g = 0, t_be = 0;
-    int q_pp0 = 0, q_len = 0, q_pb = 0, q_pT = 0, q_n = -1, q_par = -2;
+    int q_pp0 = 0, q_len = 0, q_pb = 0, q_pT = 0, q_ppar = 0, q_n = -1, q_par = -2;
     unsigned short q_g = 0, q_be = 0;
     bool q_shape_ok = false, q_mine = false;
     if (next_ok) {
         if (tbl_thread && tnode < nT) {
             const int n = nbase + tnode;
-            t_par = __ldg(p.parent + n);
+            t_par = __ldg(p.parent + npar0 + tnode);
             t_g = __ldg(reinterpret_cast<const unsigned short *>(p.g) + (size_t)n * p.h_v + nh);
             t_be = __ldg(reinterpret_cast<const unsigned short *>(p.beta) + (size_t)n * p.h_v + nh);
         }
         if constexpr (FUSED) {
             if (warp == 4) {
-                q_pp0 = p.path_offsets[nb];
-                q_len = p.path_offsets[nb + 1];
-                q_pb = p.pnode_offsets[nb];
-                q_pT = p.pnode_offsets[nb + 1];
+                if (PADDED && p.t_pad) {   // (stage 2 takes differences: hand it begin / end pairs)
+                    const int tree = nb % p.n_trees;
+                    q_pp0 = tree * p.path_stride;
+                    q_len = q_pp0 + p.path_len[tree];
+                    q_pb = nb * p.pt_pad;
+                    q_pT = q_pb + min(p.pn_nodes[tree], p.pt_pad);
+                    q_ppar = tree * p.pt_pad;
+                } else {
+                    q_pp0 = p.path_offsets[nb];
+                    q_len = p.path_offsets[nb + 1];
+                    q_pb = p.pnode_offsets[nb];
+                    q_pT = p.pnode_offsets[nb + 1];
+                    q_ppar = q_pb;
+                }
             }
         }
     }
@@ -1491,7 +1349,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                         slot[17] = q_pb;
                         slot[18] = q_shape_ok && all_in ? q_len : 0;
                     }
-                    if (in_range && p.pparent) q_par = p.pparent[q_pb + q_n];
+                    if (in_range && p.pparent) q_par = p.pparent[q_ppar + q_n];
                 }
             }
         }
@@ -1551,13 +1409,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                     bj[jj] = gj.z;
                 }
                 tmem_wait_ld();
-                // the projections S^T k_j go to the cache that a later commit of a path of this tree reads
-                if (CACHED && p.pcache_out) {
-                    float *dst = p.pcache_out + ((size_t)(base + j0) * p.h_v + h) * FV_D + c;
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj)
-                        if (j0 + jj < T) dst[(size_t)jj * p.h_v * FV_D] = __uint_as_float(rr[jj]);
-                }
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -1623,7 +1474,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
 
-        if (use_cache && next_ok) fetch_path_kv(nh, nhk, (iter + 1) & 1);   // into an area that is free from now on
         // stage 5, while the tensor core works: the next unit's tables (depth, root paths) from the staged parent[]
         if (next_ok) walk_tables(nT, (iter + 1) & 1, t_g, t_be, t_bad);
         if (!mbar_wait_bounded(mbar_d, par)) *flag = 1;
@@ -1656,17 +1506,14 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 }
             }
         }
-        if (use_cache) cp_async_wait_all();   // the path's k and v rows, needed for their Gram block below
         __syncthreads();
-        // stage 6: the next unit's decay tables; the cached projections of its path (whose final length was
-        // published behind the barrier before this one) are asked for, and the Gram block of the path's keys is formed
+        // stage 6: the next unit's decay tables, and its path rows (published above, behind a barrier now; the area
+        // they land in is free)
         if (next_ok) path_decay((iter + 1) & 1);
-        if (!use_cache && next_ok) fetch_path_kv(nh, nhk, (iter + 1) & 1);
-        if (next_ok) fetch_path_pc(nh, (iter + 1) & 1);
-        if (next_ok) path_gram((iter + 1) & 1);
+        if (next_ok) fetch_path_kv(nh, nhk, (iter + 1) & 1);
         if constexpr (FUSED) {   // ... and the scalars of that path (asked for a phase ago)
             if (next_ok && warp == 4) {   // lane t: decay of the path up to and including step t by a prefix sum
-                const float gt = lane < q_len ? __uint_as_float((uint32_t)q_g << 16) : 0.f;
+                const float gt = lane < q_len ? gate_log_decay(q_g, PADDED && p.raw_gates) : 0.f;
                 float gsum = gt;
 #pragma unroll
                 for (int off = 1; off < FV_MD; off <<= 1) {
@@ -1676,7 +1523,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 if (lane < q_len) {
                     const float A = expf(gsum);
                     reinterpret_cast<float4 *>(smem + SM_PATH + ((iter + 1) & 1) * SM_PATH_SLOT + 128)[lane] =
-                        make_float4(A, __uint_as_float((uint32_t)q_be << 16), expf(gt), 1.f / A);
+                        make_float4(A, gate_beta(q_be, PADDED && p.raw_gates), expf(gt), 1.f / A);
                 }
             }
         }
@@ -1753,14 +1600,12 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
             return cudaErrorNotSupported;
         const bool small = s.max_tree_nodes <= 32;
         // the instantiation with the projection cache (read and/or written) exists for the fused form only
-        const bool cached = FUSED && (p.pcache_out || p.pcache_prev);
+        const bool padded = p.t_pad != 0;   // the padded layout and the on-chip gate activations share an instantiation
         auto kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true, false>
                             : verify_sm100_persistent_kernel<TOut, FUSED, false, false>;
-        if constexpr (FUSED) {
-            if (cached)
-                kernel = small ? verify_sm100_persistent_kernel<TOut, true, true, true>
-                               : verify_sm100_persistent_kernel<TOut, true, false, true>;
-        }
+        if (padded)
+            kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true, true>
+                           : verify_sm100_persistent_kernel<TOut, FUSED, false, true>;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
         if (e != cudaSuccess) return e;
         const int grid = p.n_units < p.prefetch_dist ? p.n_units : p.prefetch_dist;
@@ -1794,7 +1639,6 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     p.node_offsets = node_offsets; p.o = o;
     p.n_seq = s.n_seq; p.total_nodes = s.total_nodes; p.max_tree_nodes = s.max_tree_nodes; p.max_depth = s.max_depth;
     p.tree_ok = plan.tree_ok; p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
-    p.cache_tag_out = plan.cache_tag;   // the projection cache is written on request only (the tag says so)
     p.groups_per_tree = (s.max_tree_nodes + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;   // upper bound; a CTA
                                                                                             // without a group leaves at once
     p.anc_stride = s.max_depth;
@@ -1804,6 +1648,42 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
 }
 
 }  // namespace
+
+// Padded layout (trees of at most 64 nodes; see VerifyFastParams): the persistent kernel with FUSED = false / true.
+cudaError_t launch_verify_sm100_padded(const gdn_shape_t &s, int n_trees, bool raw_gates, const float *S0,
+                                       const void *q, const void *k, const void *v, const void *g, const void *beta,
+                                       const int32_t *parent, const int32_t *n_nodes, void *o, int32_t *status_dev,
+                                       cudaStream_t stream)
+{
+    if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
+    VerifyFastParams p = make_params(s, S0, q, k, v, g, beta, nullptr, o, PlanPtrs{}, status_dev);
+    p.parent = parent;
+    p.t_pad = s.max_tree_nodes; p.n_trees = n_trees; p.n_nodes = n_nodes; p.raw_gates = raw_gates ? 1 : 0;
+    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false, false>(s, p, stream);
+    return launch_fast_typed<float, false, false>(s, p, stream);
+}
+
+cudaError_t launch_commit_verify_sm100_padded(const gdn_shape_t &s, int n_trees, bool raw_gates, float *S,
+                                              int prev_t_pad, const void *k_prev, const void *v_prev,
+                                              const void *g_prev, const void *beta_prev, const int32_t *parent_prev,
+                                              const int32_t *n_nodes_prev, const int32_t *path,
+                                              const int32_t *path_len, const void *q, const void *k, const void *v,
+                                              const void *g, const void *beta, const int32_t *parent,
+                                              const int32_t *n_nodes, void *o, int32_t *status_dev,
+                                              cudaStream_t stream)
+{
+    if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
+    VerifyFastParams p = make_params(s, S, q, k, v, g, beta, nullptr, o, PlanPtrs{}, status_dev);
+    p.parent = parent;
+    p.t_pad = s.max_tree_nodes; p.n_trees = n_trees; p.n_nodes = n_nodes; p.raw_gates = raw_gates ? 1 : 0;
+    p.S_rw = S;
+    p.pk = static_cast<const __nv_bfloat16 *>(k_prev); p.pv = static_cast<const __nv_bfloat16 *>(v_prev);
+    p.pg = static_cast<const __nv_bfloat16 *>(g_prev); p.pbeta = static_cast<const __nv_bfloat16 *>(beta_prev);
+    p.pparent = parent_prev; p.path = path;
+    p.pt_pad = prev_t_pad; p.pn_nodes = n_nodes_prev; p.path_len = path_len; p.path_stride = s.max_depth;
+    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, true, false>(s, p, stream);
+    return launch_fast_typed<float, true, false>(s, p, stream);
+}
 
 bool verify_sm100_supported(const gdn_shape_t &s)
 {
@@ -1834,20 +1714,12 @@ cudaError_t launch_commit_verify_sm100(const gdn_shape_t &s, float *S, const voi
                                        const int32_t *node_offsets_prev, const int32_t *path,
                                        const int32_t *path_offsets, const void *q, const void *k, const void *v,
                                        const void *g, const void *beta, const int32_t *parent,
-                                       const int32_t *node_offsets, void *o, const PlanPtrs &plan,
-                                       const float *pcache_prev, const int32_t *cache_tag_prev, int prev_total_nodes,
-                                       bool write_cache, int32_t *status_dev, cudaStream_t stream)
+                                       const int32_t *node_offsets, void *o, int32_t *status_dev,
+                                       cudaStream_t stream)
 {
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
-    VerifyFastParams p = make_params(s, S, q, k, v, g, beta, node_offsets, o, plan, status_dev);
+    VerifyFastParams p = make_params(s, S, q, k, v, g, beta, node_offsets, o, PlanPtrs{}, status_dev);
     p.parent = parent;
-    p.pcache_prev = pcache_prev; p.cache_tag_prev = cache_tag_prev; p.prev_total_nodes = prev_total_nodes;
-    if (write_cache) p.pcache_out = plan.pcache;
-    // Paths shorter than this are replayed even when the cache is there: inside this instantiation the cached form
-    // is the faster one from two nodes on (measured on B200; GDN_CACHED_MIN_LEN overrides the threshold, e.g. to
-    // time either form at every length).
-    p.cached_min_len = 2;
-    if (const char *e = getenv("GDN_CACHED_MIN_LEN")) p.cached_min_len = atoi(e);
     p.S_rw = S;
     p.pk = static_cast<const __nv_bfloat16 *>(k_prev); p.pv = static_cast<const __nv_bfloat16 *>(v_prev);
     p.pg = static_cast<const __nv_bfloat16 *>(g_prev); p.pbeta = static_cast<const __nv_bfloat16 *>(beta_prev);

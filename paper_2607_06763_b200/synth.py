@@ -338,6 +338,72 @@ def deep_stack(path_len: int, n_layers: int = 48, rep: int = 0, out_dtype: str =
                          out_dtype, rng, {"layers": n_layers})
 
 
+@dataclass
+class PaddedWorkload:
+    """A batch in the padded layout of Section 3.4.2: ``n_slots`` slots of ``t_pad`` rows, slot ``s`` carrying tree
+    ``s % n_trees``; node tensors ``[n_slots, t_pad, heads, d]`` (bf16 bit patterns), ``g_in / beta_in`` either finished
+    gates or raw gate inputs; one accepted path per tree, padded to ``MAX_DEPTH`` entries."""
+    n_slots: int
+    n_trees: int
+    t_pad: int
+    h_qk: int
+    h_v: int
+    d: int
+    raw_gates: bool
+    out_dtype: str
+    scale: float
+    S0: np.ndarray
+    q: np.ndarray
+    k: np.ndarray
+    v: np.ndarray
+    g_in: np.ndarray
+    beta_in: np.ndarray
+    parent: np.ndarray
+    n_nodes: np.ndarray
+    path: np.ndarray
+    path_len: np.ndarray
+
+    def f64(self, name: str) -> np.ndarray:
+        a = getattr(self, name)
+        return a.astype(np.float64) if a.dtype != np.uint16 else bf16_bits_to_f32(a).astype(np.float64)
+
+
+def padded_case(seed: int, trees, n_layers: int, t_pad: int, raw_gates: bool, h_qk: int = 2, h_v: int = 4,
+                out_dtype: str = BF16, paths=None, poison_padding: bool = True) -> PaddedWorkload:
+    """Seeded padded batch: ``len(trees)`` trees shared by ``n_layers`` slots each (slot order: layer-major, so slot
+    ``s`` carries tree ``s % len(trees)``), every slot with its own state and node tensors.  Rows beyond a tree's node
+    count hold NaN in q, k, v, g, beta when ``poison_padding`` (nothing may depend on them) and parent entries there
+    are out of range.  Accepted path per tree: ``paths[i]`` or the longest root path."""
+    rng = np.random.Generator(np.random.PCG64(SEED_BASE + 7919 * seed))
+    n_trees, d = len(trees), 128
+    B = n_trees * n_layers
+    S0, q, k, v, g, beta = random_tensors(rng, B, B * t_pad, h_qk, h_v, d, d, BF16)
+    if raw_gates:   # the layer's gate inputs themselves, N(0,1), in the storage type
+        g = store(rng.standard_normal((B * t_pad, h_v), dtype=np.float32), BF16)
+        beta = store(rng.standard_normal((B * t_pad, h_v), dtype=np.float32), BF16)
+    shape4 = lambda x: x.reshape((B, t_pad) + x.shape[1:])
+    q, k, v, g, beta = (shape4(x).copy() for x in (q, k, v, g, beta))
+    parent = np.full((n_trees, t_pad), 12345, np.int32)
+    n_nodes = np.zeros(n_trees, np.int32)
+    path = np.zeros((n_trees, MAX_DEPTH), np.int32)
+    path_len = np.zeros(n_trees, np.int32)
+    for i, t in enumerate(trees):
+        assert len(t) <= t_pad
+        parent[i, : len(t)] = t
+        n_nodes[i] = len(t)
+        pth = longest_path(t) if paths is None else np.asarray(paths[i], np.int32)
+        path[i, : len(pth)] = pth
+        path_len[i] = len(pth)
+    if poison_padding:
+        nan_bits = np.uint16(0x7FC0)
+        for s_ in range(B):
+            n = int(n_nodes[s_ % n_trees])
+            for x in (q, k, v, g, beta):
+                x[s_, n:] = nan_bits
+    return PaddedWorkload(B, n_trees, t_pad, h_qk, h_v, d, raw_gates, out_dtype, 1.0 / np.sqrt(d), S0, q, k, v, g, beta,
+                          parent, n_nodes, path, path_len)
+
+
 def random_case(seed: int, trees, h_qk, h_v, d_k, d_v, in_dtype=F32, out_dtype=F32, paths=None, name="case"):
     """A free-form case for tests: given trees, random accepted root paths unless ``paths`` is given."""
     rng = np.random.Generator(np.random.PCG64(seed))

@@ -1,0 +1,194 @@
+"""Padded, shape-static entry points (Section 3.4.2: dense [N, T, H, d] inputs, the tree shared by every layer slot,
+gate activations inside the call) against the oracle's padded front end, through the C ABI."""
+import numpy as np
+import pytest
+
+from paper_2607_06763_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+class PaddedDevice:
+    def __init__(self, w, max_depth=16):
+        import torch
+        import paper_2607_06763_b200 as gdn
+        from paper_2607_06763_b200.binding import to_device
+        self.w = w
+        self.shape = gdn.GdnShape(w.n_slots, w.h_qk, w.h_v, w.d, w.d, 1, 1 if w.out_dtype == synth.BF16 else 0, max_depth,
+                                  w.n_slots * w.t_pad, w.t_pad, w.scale)
+        for n in ("S0", "q", "k", "v", "g_in", "beta_in", "parent", "n_nodes", "path", "path_len"):
+            setattr(self, n, to_device(getattr(w, n)))
+        odt = torch.bfloat16 if w.out_dtype == synth.BF16 else torch.float32
+        self.o = torch.full((w.n_slots, w.t_pad, w.h_v, w.d), 7.0, dtype=odt, device="cuda")
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def status_value(self):
+        import torch
+        torch.cuda.synchronize()
+        return int(self.status.item())
+
+    def o_host(self):
+        return self.o.float().cpu().numpy().astype(np.float64)
+
+
+def _oracle_verify(w, S0=None):
+    from oracle import gdn_oracle as orc
+    return orc.verify_padded(w.S0.astype(np.float64) if S0 is None else S0, w.f64("q"), w.f64("k"), w.f64("v"),
+                             w.f64("g_in"), w.f64("beta_in"), w.parent, w.n_nodes, w.scale, w.raw_gates)
+
+
+def _oracle_commit(w, S0):
+    from oracle import gdn_oracle as orc
+    return orc.commit_padded(S0, w.f64("k"), w.f64("v"), w.f64("g_in"), w.f64("beta_in"), w.parent, w.n_nodes, w.path,
+                             w.path_len, w.raw_gates)
+
+
+def _assert_outputs(tl, d, o_ref, what):
+    """rows of each slot's tree against the oracle; rows beyond the node count must still hold the fill value"""
+    w = d.w
+    o = d.o_host()
+    for s in range(w.n_slots):
+        n = int(w.n_nodes[s % w.n_trees])
+        tl.assert_close_per_head(o[s, :n], o_ref[s, :n], np.array([0, n]), f"{what} slot {s}",
+                                 bf16_out=w.out_dtype == synth.BF16)
+        assert np.all(o[s, n:] == 7.0), f"{what}: rows beyond the tree of slot {s} were written"
+
+
+@pytest.fixture(scope="module")
+def tl(cuda_device):
+    from tests import gdn_testlib
+    return gdn_testlib
+
+
+def _trees(rng, sizes):
+    return [synth.tree_geo(rng, T) if T > 1 else np.array([-1], np.int32) for T in sizes]
+
+
+@pytest.mark.parametrize("raw_gates", [False, True])
+@pytest.mark.parametrize("t_pad,sizes,out_dtype", [(64, (64, 37, 64), synth.BF16), (64, (1, 50), synth.F32),
+                                                   (32, (32, 9), synth.BF16), (48, (48, 40, 3), synth.F32)])
+def test_verify_padded(tl, t_pad, sizes, out_dtype, raw_gates):
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(sum(sizes) + t_pad)
+    w = synth.padded_case(700 + t_pad + len(sizes), _trees(rng, sizes), 3, t_pad, raw_gates, out_dtype=out_dtype)
+    d = PaddedDevice(w)
+    S_before = d.S0.clone()
+    rc = gdn.gdn_tree_verify_padded(d.shape, w.n_trees, raw_gates, d.S0, d.q, d.k, d.v, d.g_in, d.beta_in, d.parent,
+                                    d.n_nodes, d.o, d.status)
+    assert rc == 0, gdn.gdn_status_string(rc)
+    assert d.status_value() == 0
+    assert bool((d.S0 == S_before).all())
+    _assert_outputs(tl, d, _oracle_verify(w), f"verify_padded T{t_pad} raw={raw_gates}")
+
+
+@pytest.mark.parametrize("raw_gates", [False, True])
+def test_commit_verify_padded(tl, raw_gates):
+    """Previous step padded to 48 rows, new step to 64; one tree commits nothing (path_len 0)."""
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(801)
+    prev_trees = _trees(rng, (48, 20, 33))
+    paths = [synth.longest_path(prev_trees[0]), np.zeros(0, np.int32), synth.root_path(prev_trees[2], 17)]
+    prev = synth.padded_case(810, prev_trees, 4, 48, raw_gates, paths=paths)
+    new = synth.padded_case(811, _trees(rng, (64, 64, 11)), 4, 64, raw_gates)
+    dp, dn = PaddedDevice(prev), PaddedDevice(new)
+    S = dp.S0.clone()
+    rc = gdn.gdn_tree_commit_verify_padded(dn.shape, new.n_trees, raw_gates, S, prev.t_pad, dp.k, dp.v, dp.g_in,
+                                           dp.beta_in, dp.parent, dp.n_nodes, dp.path, dp.path_len, dn.q, dn.k, dn.v,
+                                           dn.g_in, dn.beta_in, dn.parent, dn.n_nodes, dn.o, dn.status)
+    assert rc == 0, gdn.gdn_status_string(rc)
+    assert dn.status_value() == 0
+    S_ref = _oracle_commit(prev, prev.S0.astype(np.float64))
+    tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what="commit_verify_padded state")
+    for s in range(prev.n_slots):
+        if prev.path_len[s % prev.n_trees] == 0:
+            assert bool((S[s] == dp.S0[s]).all())
+    _assert_outputs(tl, dn, _oracle_verify(new, S_ref), f"commit_verify_padded raw={raw_gates}")
+
+
+def test_commit_verify_padded_with_nothing_to_commit(tl):
+    """All path lengths zero: a plain verification, every state untouched."""
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(803)
+    prev = synth.padded_case(820, _trees(rng, (64, 30)), 5, 64, True, paths=[np.zeros(0, np.int32)] * 2)
+    new = synth.padded_case(821, _trees(rng, (64, 41)), 5, 64, True)
+    dp, dn = PaddedDevice(prev), PaddedDevice(new)
+    S = dp.S0.clone()
+    rc = gdn.gdn_tree_commit_verify_padded(dn.shape, new.n_trees, True, S, prev.t_pad, dp.k, dp.v, dp.g_in, dp.beta_in,
+                                           dp.parent, dp.n_nodes, dp.path, dp.path_len, dn.q, dn.k, dn.v, dn.g_in,
+                                           dn.beta_in, dn.parent, dn.n_nodes, dn.o, dn.status)
+    assert rc == 0 and dn.status_value() == 0
+    assert bool((S == dp.S0).all())
+    _assert_outputs(tl, dn, _oracle_verify(new, prev.S0.astype(np.float64)), "padded, nothing to commit")
+
+
+def test_padded_call_captured_once_replayed_with_another_tree(tl):
+    """Shapes do not depend on the tree: capture the fused padded call in a CUDA graph, then overwrite the device
+    arrays (tree, node counts, accepted path, node tensors, state) in place and replay."""
+    import torch
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(901)
+    steps = []
+    for i, (ps, ns) in enumerate((((64,), (64,)), ((31,), (50,)), ((64,), (7,)))):
+        prev = synth.padded_case(910 + i, _trees(rng, ps), 6, 64, True)
+        new = synth.padded_case(920 + i, _trees(rng, ns), 6, 64, True)
+        steps.append((prev, new))
+    dp, dn = PaddedDevice(steps[0][0]), PaddedDevice(steps[0][1])
+    S = dp.S0.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+
+    def call(stream):
+        rc = gdn.gdn_tree_commit_verify_padded(dn.shape, 1, True, S, 64, dp.k, dp.v, dp.g_in, dp.beta_in, dp.parent,
+                                               dp.n_nodes, dp.path, dp.path_len, dn.q, dn.k, dn.v, dn.g_in, dn.beta_in,
+                                               dn.parent, dn.n_nodes, dn.o, dn.status, stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+
+    call(None)                      # warm-up outside the capture (kernel attributes, tensor-map entry point)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        call(torch.cuda.current_stream())
+    from paper_2607_06763_b200.binding import to_device
+    for prev, new in steps:
+        for dev, w in ((dp, prev), (dn, new)):
+            for n in ("q", "k", "v", "g_in", "beta_in", "parent", "n_nodes", "path", "path_len"):
+                getattr(dev, n).copy_(to_device(getattr(w, n)))
+            dev.w = w
+        S.copy_(to_device(prev.S0))
+        dn.o.fill_(7.0)
+        graph.replay()
+        assert dn.status_value() == 0
+        S_ref = _oracle_commit(prev, prev.S0.astype(np.float64))
+        tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what="graph replay state")
+        _assert_outputs(tl, dn, _oracle_verify(new, S_ref), "graph replay")
+
+
+def test_padded_rejections(tl):
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(5)
+    w = synth.padded_case(950, _trees(rng, (20, 30)), 2, 32, True)
+    d = PaddedDevice(w)
+    args = (d.S0, d.q, d.k, d.v, d.g_in, d.beta_in, d.parent, d.n_nodes, d.o, d.status)
+    assert gdn.gdn_tree_verify_padded(d.shape, 3, True, *args) == -2              # 4 slots do not split over 3 trees
+    bad = gdn.GdnShape.from_buffer_copy(d.shape)
+    bad.total_nodes -= 1
+    assert gdn.gdn_tree_verify_padded(bad, 2, True, *args) == -2
+    big = gdn.GdnShape.from_buffer_copy(d.shape)
+    big.max_tree_nodes, big.total_nodes = 96, 4 * 96
+    assert gdn.gdn_tree_verify_padded(big, 2, True, *args) == -5                  # more than 64 rows per slot
+    assert gdn.gdn_tree_verify_padded(d.shape, 2, True, None, *args[1:]) == -1
+    assert d.status_value() == 0 and bool((d.o == 7.0).all())
+    # device-side: a node count beyond the padded size, a parent that points forward
+    d.n_nodes[0] = 33
+    assert gdn.gdn_tree_verify_padded(d.shape, 2, True, *args) == 0
+    assert d.status_value() == -7
+    d.status.zero_()
+    d.n_nodes[0] = 20
+    d.parent[1, 5] = 9
+    d.o.fill_(7.0)
+    assert gdn.gdn_tree_verify_padded(d.shape, 2, True, *args) == 0
+    assert d.status_value() == -7
+    o = d.o_host()
+    assert np.all(o[1] == 7.0) and np.all(o[3] == 7.0), "slots of the rejected tree must stay untouched"
+    ref = _oracle_verify(w)
+    for s in (0, 2):
+        tl.assert_close_per_head(o[s, :20], ref[s, :20], np.array([0, 20]), f"good tree, slot {s}", bf16_out=True)

@@ -274,6 +274,16 @@ def test_host_buffer_entry_points(tl):
                                            new.beta, new.parent, new.node_offsets, o2, arena2, fb - 4096) == -10   # GDN_ERR_WORKSPACE
 
 
+def _oracle_step(S_ref, prev, new):
+    """oracle: commit prev's accepted paths on S_ref, then verify `new` on the result"""
+    from oracle import gdn_oracle as orc
+    S_new = orc.commit(S_ref, prev.f64("k"), prev.f64("v"), prev.f64("g"), prev.f64("beta"), prev.parent,
+                       prev.node_offsets, prev.path, prev.path_offsets)
+    o = orc.verify(S_new, new.f64("q"), new.f64("k"), new.f64("v"), new.f64("g"), new.f64("beta"), new.parent,
+                   new.node_offsets, new.scale)
+    return S_new, o
+
+
 def test_host_buffer_fused_call_pipelined_over_sequence_groups(tl):
     """More sequences than one: the host-buffer fused call cuts the batch into groups and overlaps copies and kernels
     on helper streams (node and path offsets rebased per group).  13 ragged sequences, empty paths and a rejected one
@@ -380,6 +390,30 @@ def test_fused_commit_verify_general_shapes_and_rejected_path(tl):
     o_ref = orc.verify(S_ref, new2.f64("q"), new2.f64("k"), new2.f64("v"), new2.f64("g"), new2.f64("beta"),
                        new2.parent, new2.node_offsets, new2.scale)
     tl.assert_close_per_head(dn.o_host(), o_ref, new2.node_offsets, "fused, rejected path o")
+
+
+@pytest.mark.parametrize("out_dtype", [synth.BF16, synth.F32])
+def test_fused_call_with_nothing_to_commit(tl, out_dtype):
+    """Every accepted path empty (the first step of a decode loop, or a step whose drafts were all rejected): the
+    fused call is then a plain verification and must leave every state bit-identical; path offsets come from a tensor
+    made just before the call.  One unit per CTA and several units per CTA."""
+    import torch
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(77)
+    for trees, hk, hv in (([synth.tree_geo(rng, 64)], 2, 4),
+                          ([synth.tree_geo(rng, T) for T in (64, 16, 37, 9, 64)], 2, 4),
+                          ([synth.tree_geo(rng, 64) for _ in range(12)], 16, 32)):
+        w = synth.random_case(78 + len(trees), trees, hk, hv, 128, 128, synth.BF16, out_dtype)
+        d = tl.DeviceCase(w)
+        S = d.S0.clone()
+        no_paths = torch.zeros(w.n_seq + 1, dtype=torch.int32, device="cuda")
+        rc = gdn.gdn_tree_commit_verify(d.shape, S, d.k, d.v, d.g, d.beta, d.parent, d.node_offsets, d.path, no_paths,
+                                        d.q, d.k, d.v, d.g, d.beta, d.parent, d.node_offsets, d.o, d.ws, d.ws_bytes,
+                                        d.status)
+        assert rc == 0 and d.device_status() == 0
+        assert bool((S == d.S0).all())
+        tl.assert_close_per_head(d.o_host(), tl.oracle_verify(w), w.node_offsets, f"nothing to commit, {len(trees)} trees",
+                                 bf16_out=tl.is_bf16_out(w))
 
 
 def test_refused_fused_call_launches_nothing(tl):
@@ -778,162 +812,3 @@ def test_recurrent_comparator_rejects_a_broken_branch(tl):
     assert gdn.gdn_tree_verify_recurrent(dc.shape, dc.S0, dc.q, dc.k, dc.v, dc.g, dc.beta, dc.parent, dc.node_offsets,
                                          dc.o, dc.status) == 0
     assert dc.device_status() == -8 and bool((dc.o == 7.0).all())
-
-
-# ------------------------------------------------------------------ fused step with the commit from the projection cache
-def _oracle_step(S_ref, prev, new):
-    """oracle: commit prev's accepted paths on S_ref, then verify `new` on the result"""
-    from oracle import gdn_oracle as orc
-    S_new = orc.commit(S_ref, prev.f64("k"), prev.f64("v"), prev.f64("g"), prev.f64("beta"), prev.parent,
-                       prev.node_offsets, prev.path, prev.path_offsets)
-    o = orc.verify(S_new, new.f64("q"), new.f64("k"), new.f64("v"), new.f64("g"), new.f64("beta"), new.parent,
-                   new.node_offsets, new.scale)
-    return S_new, o
-
-
-def _cached_chain(tl, steps, what, expect_status=0):
-    """steps[0] is verified by a gdn_tree_commit_verify_cached call that has nothing to commit (empty paths, no
-    previous workspace), which leaves the first projection cache; every later step goes through the same entry point
-    with the workspace of the call before it.  State and outputs are checked against the oracle after every call."""
-    import torch
-    import paper_2607_06763_b200 as gdn
-    cases = [tl.DeviceCase(w) for w in steps]
-    S = cases[0].S0.clone()
-    S_ref = steps[0].S0.astype(np.float64)
-    d0 = cases[0]
-    no_paths = torch.zeros(steps[0].n_seq + 1, dtype=torch.int32, device="cuda")
-    assert gdn.gdn_tree_commit_verify_cached(d0.shape, S, d0.k, d0.v, d0.g, d0.beta, d0.parent, d0.node_offsets,
-                                             d0.path, no_paths, None, 0, d0.q, d0.k, d0.v, d0.g, d0.beta, d0.parent,
-                                             d0.node_offsets, d0.o, d0.ws, d0.ws_bytes, d0.status) == 0
-    assert d0.device_status() == 0
-    assert bool((S == d0.S0).all())
-    tl.assert_close_per_head(d0.o_host(), tl.oracle_verify(steps[0]), steps[0].node_offsets, f"{what}: o of step 0",
-                             bf16_out=tl.is_bf16_out(steps[0]))
-    for i in range(1, len(steps)):
-        dp, dn = cases[i - 1], cases[i]
-        rc = gdn.gdn_tree_commit_verify_cached(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets,
-                                               dp.path, dp.path_offsets, dp.ws, steps[i - 1].total_nodes, dn.q, dn.k,
-                                               dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets, dn.o, dn.ws,
-                                               dn.ws_bytes, dn.status)
-        assert rc == 0, gdn.gdn_status_string(rc)
-        assert dn.device_status() == expect_status
-        S_ref, o_ref = _oracle_step(S_ref, steps[i - 1], steps[i])
-        tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what=f"{what}: state after step {i}")
-        tl.assert_close_per_head(dn.o_host(), o_ref, steps[i].node_offsets, f"{what}: o of step {i}",
-                                 bf16_out=tl.is_bf16_out(steps[i]))
-    return S
-
-
-@pytest.fixture(params=["1", None], ids=["every_length_from_cache", "default_dispatch"])
-def cached_min_len(request, monkeypatch):
-    """The library replays paths shorter than a measured crossover even when the cache is there; GDN_CACHED_MIN_LEN=1
-    sends every path through the cache, so that both forms are compared with the oracle."""
-    if request.param is None:
-        monkeypatch.delenv("GDN_CACHED_MIN_LEN", raising=False)
-    else:
-        monkeypatch.setenv("GDN_CACHED_MIN_LEN", request.param)
-    return request.param
-
-
-@pytest.mark.parametrize("out_dtype", [synth.BF16, synth.F32])
-def test_cached_commit_over_a_chain_of_decode_steps(tl, out_dtype, cached_min_len):
-    rng = np.random.default_rng(301)
-    steps = []
-    for i in range(4):
-        trees = [synth.tree_geo(rng, 64), synth.tree_chain(16), synth.tree_geo(rng, 37), synth.tree_star(9),
-                 synth.tree_bestfirst(rng, 64, width=2)]
-        paths = [synth.longest_path(trees[0]), np.arange(16 if i % 2 else 5, dtype=np.int32),
-                 np.zeros(0, np.int32), np.array([0, 5], np.int32), synth.longest_path(trees[4])]
-        steps.append(synth.random_case(310 + i, trees, 2, 4, 128, 128, synth.BF16, out_dtype, paths=paths,
-                                       name=f"chain{i}"))
-    _cached_chain(tl, steps, f"cached chain {out_dtype}")
-
-
-def test_cached_commit_full_layer_matches_replay_and_oracle(tl, cached_min_len):
-    """configuration 1 (one layer, 16/32 heads): three steps; the cached commit and the replayed commit of the same
-    step agree with the oracle and with each other."""
-    import paper_2607_06763_b200 as gdn
-    steps = [synth.config(1, rep) for rep in range(3)]
-    S_cached = _cached_chain(tl, steps, "cached cfg1")
-    cases = [tl.DeviceCase(w) for w in steps]
-    S = cases[0].S0.clone()
-    for i in range(1, 3):
-        dp, dn = cases[i - 1], cases[i]
-        assert gdn.gdn_tree_commit_verify(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path,
-                                          dp.path_offsets, dn.q, dn.k, dn.v, dn.g, dn.beta, dn.parent, dn.node_offsets,
-                                          dn.o, dn.ws, dn.ws_bytes, dn.status) == 0
-        assert dn.device_status() == 0
-    ref = S.cpu().numpy().astype(np.float64)
-    tl.assert_state_close(S_cached.cpu().numpy().astype(np.float64), ref, what="cached vs replayed commit")
-
-
-def test_cached_commit_falls_back_when_the_cache_is_not_there(tl, cached_min_len):
-    """No previous workspace, a workspace nothing has written (tag missing), one written by a call of another shape,
-    and one written by the general kernel: each time the commit is replayed and the results still hold."""
-    import torch
-    import paper_2607_06763_b200 as gdn
-    rng = np.random.default_rng(302)
-    prev = synth.random_case(320, [synth.tree_geo(rng, 40), synth.tree_chain(9)], 2, 4, 128, 128, synth.BF16, synth.F32,
-                             paths=None)
-    new = synth.random_case(321, [synth.tree_geo(rng, 64), synth.tree_geo(rng, 21)], 2, 4, 128, 128, synth.BF16, synth.F32)
-    other = synth.random_case(322, [synth.tree_geo(rng, 12), synth.tree_chain(3)], 2, 4, 128, 128, synth.BF16, synth.F32)
-    S_ref, o_ref = _oracle_step(prev.S0.astype(np.float64), prev, new)
-    dp, dn, do = tl.DeviceCase(prev), tl.DeviceCase(new), tl.DeviceCase(other)
-    no_paths = torch.zeros(other.n_seq + 1, dtype=torch.int32, device="cuda")
-    assert gdn.gdn_tree_commit_verify_cached(do.shape, do.S0.clone(), do.k, do.v, do.g, do.beta, do.parent,
-                                             do.node_offsets, do.path, no_paths, None, 0, do.q, do.k, do.v, do.g,
-                                             do.beta, do.parent, do.node_offsets, do.o, do.ws, do.ws_bytes,
-                                             do.status) == 0
-    assert do.device_status() == 0                                  # `other`'s workspace now carries a cache tag
-    blank = torch.zeros_like(dp.ws)
-    for label, prev_ws, prev_n in (("none", None, 0), ("blank", blank, prev.total_nodes),
-                                   ("other shape", do.ws, prev.total_nodes)):
-        S = dp.S0.clone()
-        dn.o.zero_()
-        rc = gdn.gdn_tree_commit_verify_cached(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets,
-                                               dp.path, dp.path_offsets, prev_ws, prev_n, dn.q, dn.k, dn.v, dn.g,
-                                               dn.beta, dn.parent, dn.node_offsets, dn.o, dn.ws, dn.ws_bytes, dn.status)
-        assert rc == 0 and dn.device_status() == 0, label
-        tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what=f"fallback ({label}) state")
-        tl.assert_close_per_head(dn.o_host(), o_ref, new.node_offsets, f"fallback ({label}) o")
-    # the same buffer as cache and as new workspace is refused before anything is launched
-    S = dp.S0.clone()
-    assert gdn.gdn_tree_commit_verify_cached(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path,
-                                             dp.path_offsets, dn.ws, prev.total_nodes, dn.q, dn.k, dn.v, dn.g, dn.beta,
-                                             dn.parent, dn.node_offsets, dn.o, dn.ws, dn.ws_bytes, dn.status) == -10
-    assert bool((S == dp.S0).all())
-
-
-def test_cached_commit_rejected_path_and_extreme_decay(tl, cached_min_len):
-    """A path that is not a chain leaves its state alone (GDN_ERR_PATH) while the other tree of the batch commits from
-    the cache; a path whose decay underflows the scaled form is replayed."""
-    import paper_2607_06763_b200 as gdn
-    prev_trees = [synth.tree_chain(6), synth.tree_chain(6)]
-    bad = synth.random_case(330, prev_trees, 1, 2, 128, 128, synth.BF16, synth.F32,
-                            paths=[np.array([0, 2], np.int32), np.array([0, 1, 2], np.int32)])
-    good = synth.random_case(330, prev_trees, 1, 2, 128, 128, synth.BF16, synth.F32,
-                             paths=[np.zeros(0, np.int32), np.array([0, 1, 2], np.int32)])
-    new = synth.random_case(331, [synth.tree_star(8), synth.tree_star(8)], 1, 2, 128, 128, synth.BF16, synth.F32)
-    dp, dn = tl.DeviceCase(bad), tl.DeviceCase(new)
-    S = dp.S0.clone()
-    import torch
-    no_paths = torch.zeros(bad.n_seq + 1, dtype=torch.int32, device="cuda")
-    assert gdn.gdn_tree_commit_verify_cached(dp.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets,
-                                             dp.path, no_paths, None, 0, dp.q, dp.k, dp.v, dp.g, dp.beta, dp.parent,
-                                             dp.node_offsets, dp.o, dp.ws, dp.ws_bytes, dp.status) == 0
-    assert dp.device_status() == 0
-    rc = gdn.gdn_tree_commit_verify_cached(dn.shape, S, dp.k, dp.v, dp.g, dp.beta, dp.parent, dp.node_offsets, dp.path,
-                                           dp.path_offsets, dp.ws, bad.total_nodes, dn.q, dn.k, dn.v, dn.g, dn.beta,
-                                           dn.parent, dn.node_offsets, dn.o, dn.ws, dn.ws_bytes, dn.status)
-    assert rc == 0 and dn.device_status() == -9
-    assert bool((S[0] == dp.S0[0]).all()), "a rejected path must leave its state untouched"
-    S_ref, o_ref = _oracle_step(good.S0.astype(np.float64), good, new)
-    tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what="cached, rejected path")
-    tl.assert_close_per_head(dn.o_host(), o_ref, new.node_offsets, "cached, rejected path o")
-    # extreme decay: g = -9 per step over 8 steps, A_L = e^-72
-    import dataclasses
-    deep = synth.random_case(332, [synth.tree_chain(8)], 1, 2, 128, 128, synth.BF16, synth.F32,
-                             paths=[np.arange(8, dtype=np.int32)])
-    deep = dataclasses.replace(deep, g=synth.store(np.full(deep.g.shape, -9.0, np.float32), synth.BF16))
-    new2 = synth.random_case(333, [synth.tree_geo(np.random.default_rng(5), 20)], 1, 2, 128, 128, synth.BF16, synth.F32)
-    _cached_chain(tl, [deep, new2], "cached, extreme decay")
