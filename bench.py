@@ -36,7 +36,7 @@ METRIC = "verified tree-nodes/sec per GDN layer"
 UNIT = "nodes/s"
 CONFIG_WORKLOADS = {"stack48_T64": 5, "layer_T64": 1, "stack48_T256": 2, "ragged32": 3, "chains64x16": 4}
 SWEEP_T = (32, 64, 128, 256, 512)
-WORKLOADS = sorted(CONFIG_WORKLOADS) + [f"sweep_T{t}" for t in SWEEP_T] + ["stack48_T64_deep"]
+WORKLOADS = sorted(CONFIG_WORKLOADS) + [f"sweep_T{t}" for t in SWEEP_T] + ["stack48_T64_deep", "stack48_T64_bestfirst"]
 DTYPE = "bf16 inputs/outputs, fp32 state; contractions as bf16 hi+lo splits on tcgen05 with fp32 accumulation"
 
 
@@ -45,6 +45,8 @@ def make_workload(args) -> synth.Workload:
         return synth.config(CONFIG_WORKLOADS[args.workload], 0, n_layers=args.layers)
     if args.workload == "stack48_T64_deep":
         return synth.deep_stack(args.path_len, n_layers=args.layers)
+    if args.workload == "stack48_T64_bestfirst":
+        return synth.bestfirst_stack(n_layers=args.layers)
     return synth.layer_sweep(int(args.workload.split("_T")[1]))
 
 

@@ -324,21 +324,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hk = h / (p.h_v / p.h_qk);
     uint16_t *vnode_s = reinterpret_cast<uint16_t *>(smem + SM_VNODE);
-    if constexpr (GROUPED) {
-        if (tid < FV_T) {
-            int node = tid;
-            if (!ident && tid < T) {
-                if (tid < n_prefix) {
-                    const int first = p.dfs_node[base + g0];
-                    node = p.anc16[(size_t)(base + first) * p.anc_stride + tid];
-                } else {
-                    node = p.dfs_node[base + g0 + tid - n_prefix];
-                }
-            }
-            vnode_s[tid] = (uint16_t)node;
-        }
-        __syncthreads();
-    }
     auto node_of = [&](int u) -> int { return GROUPED ? (int)vnode_s[u] : u; };
 
     // L2 warming for the unit that a CTA will pick up about one wave from now, issued in slices at
@@ -378,6 +363,22 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const Verif
 #pragma unroll
             for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
         }
+    }
+    // the node table of the group is looked up under the latency of the state loads
+    if constexpr (GROUPED) {
+        if (tid < FV_T) {
+            int node = tid;
+            if (!ident && tid < T) {
+                if (tid < n_prefix) {
+                    const int first = p.dfs_node[base + g0];
+                    node = p.anc16[(size_t)(base + first) * p.anc_stride + tid];
+                } else {
+                    node = p.dfs_node[base + g0 + tid - n_prefix];
+                }
+            }
+            vnode_s[tid] = (uint16_t)node;
+        }
+        __syncthreads();
     }
     // (2) k and q rows -> B operand tile (rows beyond T are zero-filled)
 #pragma unroll
@@ -793,6 +794,20 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // The first unit's state tile is an input of the call, not of that kernel: L2 is asked for it meanwhile.
     if (tid < 4 && (int)blockIdx.x < p.n_units)
         prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
+    // ... and for the rows of the first unit's tree.  Their place may depend on node_offsets[], which the kernel in
+    // front may still be writing: the value read here only steers prefetches (clamped to the tensors), it is read
+    // again behind the dependency wait before anything is computed from it.
+    if ((int)blockIdx.x < p.n_units && tid >= 128 && tid < 128 + FV_T) {
+        const int ub = (int)blockIdx.x / p.h_v, uh = (int)blockIdx.x % p.h_v, uhk = uh / (p.h_v / p.h_qk);
+        const int row = ((PADDED && p.t_pad) ? ub * p.t_pad : __ldg(p.node_offsets + ub)) + tid - 128;
+        if (row >= 0 && row < p.total_nodes) {
+            prefetch_l2_bulk(p.v + ((size_t)row * p.h_v + uh) * FV_D, 256);
+            prefetch_l2_bulk(p.k + ((size_t)row * p.h_qk + uhk) * FV_D, 256);
+            prefetch_l2_bulk(p.q + ((size_t)row * p.h_qk + uhk) * FV_D, 256);
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.g + (size_t)row * p.h_v + uh));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.beta + (size_t)row * p.h_v + uh));
+        }
+    }
     signed char *par_s = reinterpret_cast<signed char *>(smem + SM_PAR);
     volatile int *bad_s = reinterpret_cast<volatile int *>(smem + SM_BAD);
 

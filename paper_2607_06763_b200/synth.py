@@ -148,11 +148,11 @@ def tree_geo(rng: np.random.Generator, T: int, max_depth: int = MAX_DEPTH, fanou
 
 
 def tree_bestfirst(rng: np.random.Generator, T: int, width: int = 4, fanout: int = FANOUT,
-                   max_depth: int = MAX_DEPTH) -> np.ndarray:
+                   max_depth: int = MAX_DEPTH, concentration: float = 0.25) -> np.ndarray:
     """Shape of a width-``width`` best-first expansion (Algorithm 1) driven by seeded synthetic child probabilities.
 
     Only the shape is used: every node added to the tree proposes ``fanout`` children whose probabilities are a
-    Dirichlet draw sharpened towards one dominant child; a candidate's score is the product along its path, and
+    Dirichlet draw sharpened towards one dominant child (the smaller ``concentration``, the sharper, the deeper the tree); a candidate's score is the product along its path, and
     each round moves the ``width`` best candidates into the tree.
     """
     parent_of = [-1]
@@ -163,7 +163,7 @@ def tree_bestfirst(rng: np.random.Generator, T: int, width: int = 4, fanout: int
     while len(parent_of) < T:
         for n in batch:
             if dep[n] < max_depth:
-                pr = rng.dirichlet(np.full(fanout, 0.25))
+                pr = rng.dirichlet(np.full(fanout, concentration))
                 frontier.extend((score[n] * float(pc), n) for pc in pr)
         if not frontier:
             raise ValueError("frontier exhausted")
@@ -335,6 +335,17 @@ def deep_stack(path_len: int, n_layers: int = 48, rep: int = 0, out_dtype: str =
     t = bfs_renumber(np.asarray([i - 1 for i in range(16)] + [i % 15 for i in range(48)], np.int32))
     p = longest_path(t)[:path_len]
     return make_workload(f"stack{n_layers}_T64_deep_L{path_len}", [t] * n_layers, [p] * n_layers, 16, 32, 128, 128, BF16,
+                         out_dtype, rng, {"layers": n_layers})
+
+
+def bestfirst_stack(n_layers: int = 48, rep: int = 0, out_dtype: str = BF16, T: int = 64) -> Workload:
+    """Configuration "1x48" with the tree shape of Algorithm 1 (width-4 best-first expansion, fan-out 8, depth cap
+    16, seeded synthetic child probabilities) instead of the geometric one: deeper root paths, the report-only
+    second shape of the headline workload.  Accepted path = longest root path."""
+    rng = np.random.Generator(np.random.PCG64(SEED_BASE + 101 * 8 + rep))
+    t = tree_bestfirst(rng, T, concentration=0.1)   # accepted lengths of 12-14, as the paper reports for 64-node trees
+    p = longest_path(t)
+    return make_workload(f"stack{n_layers}_T{T}_bestfirst", [t] * n_layers, [p] * n_layers, 16, 32, 128, 128, BF16,
                          out_dtype, rng, {"layers": n_layers})
 
 
