@@ -167,6 +167,41 @@ int gdn_tree_commit_verify_padded(const gdn_shape_t *shape, int32_t n_trees, int
                                   const int32_t *n_nodes, void *o, int32_t *status_dev, void *cuda_stream);
 
 /*
+ * Padded layout for trees of any padded size up to 1024 rows, with the tree metadata as an object of its own
+ * (Section 3.4.2: the proposal tree is shared by every GDN layer, "so its verification metadata is computed
+ * once per decode step"): gdn_tree_plan builds the plan of the n_trees trees once; gdn_tree_verify_planned
+ * verifies any number of slots (layers) against it, in one call or in several; gdn_tree_commit_padded is the
+ * delayed commit (Section 3.4) in the same layout.  Shapes, layouts, raw_gates and errors as for
+ * gdn_tree_verify_padded, except that shape->max_tree_nodes = T may be anything up to 1024 (trees of more
+ * than 64 nodes are verified in ancestor-closed groups of a depth-first numbering, which the plan holds).
+ *   plan         : [device] >= gdn_tree_plan_bytes(shape, n_trees) bytes, 256-byte aligned; written by
+ *                  gdn_tree_plan, read-only for gdn_tree_verify_planned; depends on shape->max_tree_nodes,
+ *                  shape->max_depth and n_trees only (not on n_seq or the head counts), and must have been
+ *                  built with the same three values
+ *   gdn_tree_plan reports a bad tree (GDN_ERR_TREE, GDN_ERR_DEPTH) through *status_dev; the slots of such a
+ *   tree are skipped by gdn_tree_verify_planned (nothing of them is written).
+ *   gdn_tree_commit_padded: k, v, g, beta, parent [n_trees][T] (may be NULL), n_nodes, path
+ *   [n_trees][max_depth], path_len [n_trees] describe the tree whose accepted path is committed; d_k = d_v =
+ *   128, bf16 inputs, max_depth <= 16, else GDN_ERR_UNSUPPORTED.  A rejected path (GDN_ERR_PATH) leaves the
+ *   states of that tree's slots untouched.
+ * All three are shape-static and allocate nothing: plan + commit + verify can be captured in one CUDA graph.
+ */
+size_t gdn_tree_plan_bytes(const gdn_shape_t *shape, int32_t n_trees);
+
+int gdn_tree_plan(const gdn_shape_t *shape, int32_t n_trees, const int32_t *parent, const int32_t *n_nodes,
+                  void *plan, size_t plan_bytes, int32_t *status_dev, void *cuda_stream);
+
+int gdn_tree_verify_planned(const gdn_shape_t *shape, int32_t n_trees, int32_t raw_gates, const float *S0,
+                            const void *q, const void *k, const void *v, const void *g, const void *beta,
+                            const void *plan, size_t plan_bytes, void *o, int32_t *status_dev, void *cuda_stream);
+
+int gdn_tree_commit_padded(const gdn_shape_t *shape, int32_t n_trees, int32_t raw_gates, float *S, const void *k,
+                           const void *v, const void *g, const void *beta, const int32_t *parent,
+                           const int32_t *n_nodes, const int32_t *path, const int32_t *path_len,
+                           int32_t *status_dev, void *cuda_stream);
+
+
+/*
  * Per-branch recurrent verification: the baseline that Section 3.4 describes as "sequential scans
  * along tree branches" and that Section 5.2 / Figure 5 times against the fused kernel.  For every
  * leaf of every tree the state is copied and Eq. 7 is run token by token down the leaf's root path,

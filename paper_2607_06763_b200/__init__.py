@@ -10,15 +10,19 @@ from .binding import (  # noqa: F401
     gdn_status_string,
     gdn_tree_commit,
     gdn_tree_commit_host,
+    gdn_tree_commit_padded,
     gdn_tree_commit_verify,
     gdn_tree_commit_verify_padded,
     gdn_tree_commit_verify_host,
     gdn_tree_commit_verify_host_arena_bytes,
     gdn_tree_host_arena_bytes,
+    gdn_tree_plan,
+    gdn_tree_plan_bytes,
     gdn_tree_validate_host,
     gdn_tree_verify,
     gdn_tree_verify_host,
     gdn_tree_verify_padded,
+    gdn_tree_verify_planned,
     gdn_tree_verify_recurrent,
     gdn_tree_verify_static,
     gdn_tree_workspace_bytes,

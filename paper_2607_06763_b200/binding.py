@@ -33,6 +33,10 @@ EXPORTS = (
     "gdn_tree_verify_recurrent",
     "gdn_tree_verify_padded",
     "gdn_tree_commit_verify_padded",
+    "gdn_tree_plan_bytes",
+    "gdn_tree_plan",
+    "gdn_tree_verify_planned",
+    "gdn_tree_commit_padded",
 )
 
 GDN_STATIC_SCRATCH_BYTES = 4 << 20
@@ -107,6 +111,15 @@ def load_library():
         lib.gdn_tree_commit_verify_padded.restype = ctypes.c_int
         lib.gdn_tree_commit_verify_padded.argtypes = ([sp, ctypes.c_int32, ctypes.c_int32, vp, ctypes.c_int32] +
                                                       [vp] * 18)
+        lib.gdn_tree_plan_bytes.restype = ctypes.c_size_t
+        lib.gdn_tree_plan_bytes.argtypes = [sp, ctypes.c_int32]
+        lib.gdn_tree_plan.restype = ctypes.c_int
+        lib.gdn_tree_plan.argtypes = [sp, ctypes.c_int32, vp, vp, vp, ctypes.c_size_t, vp, vp]
+        lib.gdn_tree_verify_planned.restype = ctypes.c_int
+        lib.gdn_tree_verify_planned.argtypes = ([sp, ctypes.c_int32, ctypes.c_int32] + [vp] * 7 +
+                                                [ctypes.c_size_t, vp, vp, vp])
+        lib.gdn_tree_commit_padded.restype = ctypes.c_int
+        lib.gdn_tree_commit_padded.argtypes = [sp, ctypes.c_int32, ctypes.c_int32] + [vp] * 11
         lib.gdn_tree_verify_static.restype = ctypes.c_int
         lib.gdn_tree_verify_static.argtypes = [sp] + [vp] * 11
         lib.gdn_tree_verify_recurrent.restype = ctypes.c_int
@@ -223,6 +236,32 @@ def gdn_tree_commit_verify_padded(shape, n_trees, raw_gates, S, prev_t_pad, k_pr
         _ptr(g_prev), _ptr(beta_prev), _ptr(parent_prev), _ptr(n_nodes_prev), _ptr(path), _ptr(path_len), _ptr(q),
         _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(parent), _ptr(n_nodes), _ptr(o), _ptr(status_dev),
         _stream(stream)))
+
+
+def gdn_tree_plan_bytes(shape, n_trees) -> int:
+    """``gdn_tree_plan_bytes``: size of the shared-tree plan of the padded layout."""
+    return int(load_library().gdn_tree_plan_bytes(ctypes.byref(shape), int(n_trees)))
+
+
+def gdn_tree_plan(shape, n_trees, parent, n_nodes, plan, status_dev, stream=None) -> int:
+    """``gdn_tree_plan``: build the plan of the ``n_trees`` shared trees (once per decode step)."""
+    return int(load_library().gdn_tree_plan(ctypes.byref(shape), int(n_trees), _ptr(parent), _ptr(n_nodes), _ptr(plan),
+                                            int(plan.numel() * plan.element_size()), _ptr(status_dev), _stream(stream)))
+
+
+def gdn_tree_verify_planned(shape, n_trees, raw_gates, S0, q, k, v, g, beta, plan, o, status_dev, stream=None) -> int:
+    """``gdn_tree_verify_planned``: verification in the padded layout against a plan built by ``gdn_tree_plan``."""
+    return int(load_library().gdn_tree_verify_planned(
+        ctypes.byref(shape), int(n_trees), int(bool(raw_gates)), _ptr(S0), _ptr(q), _ptr(k), _ptr(v), _ptr(g),
+        _ptr(beta), _ptr(plan), int(plan.numel() * plan.element_size()), _ptr(o), _ptr(status_dev), _stream(stream)))
+
+
+def gdn_tree_commit_padded(shape, n_trees, raw_gates, S, k, v, g, beta, parent, n_nodes, path, path_len, status_dev,
+                           stream=None) -> int:
+    """``gdn_tree_commit_padded``: the delayed commit in the padded layout (one accepted path per tree)."""
+    return int(load_library().gdn_tree_commit_padded(
+        ctypes.byref(shape), int(n_trees), int(bool(raw_gates)), _ptr(S), _ptr(k), _ptr(v), _ptr(g), _ptr(beta),
+        _ptr(parent), _ptr(n_nodes), _ptr(path), _ptr(path_len), _ptr(status_dev), _stream(stream)))
 
 
 def gdn_tree_verify_recurrent(shape, S0, q, k, v, g, beta, parent, node_offsets, o, status_dev, stream=None) -> int:

@@ -182,7 +182,7 @@ extern "C" int gdn_tree_verify(const gdn_shape_t *shape, const float *S0, const 
     const PlanPtrs plan = plan_ptrs(workspace, lay);
     // trees of at most 64 nodes on the tensor-core path: that kernel builds the tree metadata itself
     if (!verify_sm100_single_group(s) &&
-        launch_plan(s, parent, node_offsets, plan, status_dev, stream) != cudaSuccess)
+        launch_plan(s, parent, node_offsets, nullptr, plan, status_dev, stream) != cudaSuccess)
         return GDN_ERR_CUDA;
     const cudaError_t e = verify_sm100_supported(s)
                               ? launch_verify_sm100(s, S0, q, k, v, g, beta, parent, node_offsets, o, plan, status_dev, stream)
@@ -255,6 +255,107 @@ extern "C" int gdn_tree_commit_verify_padded(const gdn_shape_t *shape, int32_t n
     if (launch_commit_verify_sm100_padded(s, n_trees, raw_gates != 0, S, prev_t_pad, k_prev, v_prev, g_prev, beta_prev,
                                           parent_prev, n_nodes_prev, path, path_len, q, k, v, g, beta, parent, n_nodes,
                                           o, status_dev, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
+namespace {
+
+// The shared-tree plan of the padded layout: the tree-metadata part of the verify workspace for n_trees trees of
+// shape.max_tree_nodes rows each (no u~ buffer).
+gdn_shape_t plan_shape(const gdn_shape_t &s, int32_t n_trees)
+{
+    gdn_shape_t ps = s;
+    ps.n_seq = n_trees;
+    ps.total_nodes = n_trees * s.max_tree_nodes;
+    ps.h_v = 0;   // sizes the u~ buffer of the general verify kernel, which the plan does not have
+    return ps;
+}
+
+int check_planned_shape(const gdn_shape_t &s, int32_t n_trees)
+{
+    if (n_trees < 1 || s.n_seq % n_trees != 0) return GDN_ERR_SHAPE;
+    if ((long long)s.n_seq * s.max_tree_nodes != s.total_nodes) return GDN_ERR_SHAPE;
+    if (!verify_sm100_supported(s)) return GDN_ERR_UNSUPPORTED;
+    return GDN_OK;
+}
+
+}  // namespace
+
+extern "C" size_t gdn_tree_plan_bytes(const gdn_shape_t *shape, int32_t n_trees)
+{
+    if (check_shape(shape) != GDN_OK || n_trees < 1) return 0;
+    return workspace_layout(plan_shape(*shape, n_trees)).total;
+}
+
+extern "C" int gdn_tree_plan(const gdn_shape_t *shape, int32_t n_trees, const int32_t *parent, const int32_t *n_nodes,
+                             void *plan, size_t plan_bytes, int32_t *status_dev, void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
+    rc = check_planned_shape(s, n_trees);
+    if (rc != GDN_OK) return rc;
+    if (!parent || !n_nodes || !status_dev) return GDN_ERR_NULL;
+    if (!plan) return GDN_ERR_WORKSPACE;
+    if (!aligned256(plan) || (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(n_nodes) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    const gdn_shape_t ps = plan_shape(s, n_trees);
+    const WorkspaceLayout lay = workspace_layout(ps);
+    if (plan_bytes < lay.total) return GDN_ERR_WORKSPACE;
+    if (launch_plan(ps, parent, nullptr, n_nodes, plan_ptrs(plan, lay), status_dev,
+                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
+extern "C" int gdn_tree_verify_planned(const gdn_shape_t *shape, int32_t n_trees, int32_t raw_gates, const float *S0,
+                                       const void *q, const void *k, const void *v, const void *g, const void *beta,
+                                       const void *plan, size_t plan_bytes, void *o, int32_t *status_dev,
+                                       void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
+    rc = check_planned_shape(s, n_trees);
+    if (rc != GDN_OK) return rc;
+    if (!S0 || !q || !k || !v || !g || !beta || !o || !status_dev) return GDN_ERR_NULL;
+    if (!plan) return GDN_ERR_WORKSPACE;
+    if (!aligned16(S0) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        !aligned16(o) || !aligned256(plan) || (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    const WorkspaceLayout lay = workspace_layout(plan_shape(s, n_trees));
+    if (plan_bytes < lay.total) return GDN_ERR_WORKSPACE;
+    if (launch_verify_sm100_planned(s, n_trees, raw_gates != 0, S0, q, k, v, g, beta,
+                                    plan_ptrs(const_cast<void *>(plan), lay), o, status_dev,
+                                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    return GDN_OK;
+}
+
+extern "C" int gdn_tree_commit_padded(const gdn_shape_t *shape, int32_t n_trees, int32_t raw_gates, float *S,
+                                      const void *k, const void *v, const void *g, const void *beta,
+                                      const int32_t *parent, const int32_t *n_nodes, const int32_t *path,
+                                      const int32_t *path_len, int32_t *status_dev, void *cuda_stream)
+{
+    int rc = check_shape(shape);
+    if (rc != GDN_OK) return rc;
+    const gdn_shape_t &s = *shape;
+    if (s.n_seq == 0 || s.total_nodes == 0) return GDN_OK;
+    if (n_trees < 1 || s.n_seq % n_trees != 0) return GDN_ERR_SHAPE;
+    if ((long long)s.n_seq * s.max_tree_nodes != s.total_nodes) return GDN_ERR_SHAPE;
+    if (!commit_padded_supported(s)) return GDN_ERR_UNSUPPORTED;
+    if (!S || !k || !v || !g || !beta || !n_nodes || !path || !path_len || !status_dev) return GDN_ERR_NULL;
+    if (!aligned16(S) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        (reinterpret_cast<uintptr_t>(parent) & 3u) || (reinterpret_cast<uintptr_t>(n_nodes) & 3u) ||
+        (reinterpret_cast<uintptr_t>(path) & 3u) || (reinterpret_cast<uintptr_t>(path_len) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return GDN_ERR_ALIGN;
+    if (launch_commit_padded(s, n_trees, raw_gates != 0, S, k, v, g, beta, parent, n_nodes, path, path_len, status_dev,
+                             static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return GDN_ERR_CUDA;
     return GDN_OK;
 }

@@ -29,6 +29,10 @@ struct CommitParams {
     const void *k, *v, *g, *beta;
     const int32_t *parent, *node_offsets, *path, *path_offsets;
     int32_t *status_dev;
+    // padded layout (tile kernel only; t_pad = 0: ragged packing): slot b keeps its rows at b * t_pad and carries
+    // tree b % n_trees, whose parent[] row, node count and accepted path are shared by its slots
+    int t_pad, n_trees, path_stride, raw_gates;
+    const int32_t *n_nodes, *path_len;
 };
 
 template <typename TIn>
@@ -165,8 +169,9 @@ __global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const Com
     const int hk = h / (p.h_v / p.h_qk);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r4 = lane >> 3, l8 = lane & 7;
-    const int pp0 = p.path_offsets[b];
-    int len = p.path_offsets[b + 1] - pp0;
+    const int tree = p.t_pad ? b % p.n_trees : b;
+    const int pp0 = p.t_pad ? tree * p.path_stride : p.path_offsets[b];
+    int len = p.t_pad ? p.path_len[tree] : p.path_offsets[b + 1] - pp0;
     if (len == 0) return;   // nothing accepted from this tree: state untouched
 
     // the state tile first: its latency covers the path fetch below
@@ -179,8 +184,9 @@ __global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const Com
         for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
     }
 
-    const int pb = p.node_offsets[b];
-    const int pT = p.node_offsets[b + 1] - pb;
+    const int pb = p.t_pad ? b * p.t_pad : p.node_offsets[b];
+    const int pT = p.t_pad ? min(p.n_nodes[tree], p.t_pad) : p.node_offsets[b + 1] - pb;
+    const int ppar = p.t_pad ? tree * p.t_pad : pb;   // first entry of the tree in parent[]
     const __nv_bfloat16 *k = static_cast<const __nv_bfloat16 *>(p.k), *v = static_cast<const __nv_bfloat16 *>(p.v);
     const __nv_bfloat16 *g = static_cast<const __nv_bfloat16 *>(p.g), *beta = static_cast<const __nv_bfloat16 *>(p.beta);
     const bool shape_ok = len > 0 && len <= CF_MD && len <= p.max_depth && pT > 0 && pp0 >= 0;
@@ -206,7 +212,7 @@ __global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const Com
         int n = -1, parent_n = -2;
         if (mine) {
             n = p.path[pp0 + lane];
-            if (p.parent && n >= 0 && n < pT) parent_n = p.parent[pb + n];
+            if (p.parent && n >= 0 && n < pT) parent_n = p.parent[ppar + n];
         }
         const int n_up = __shfl_up_sync(0xffffffffu, n, 1);
         bool bad = false;
@@ -222,8 +228,10 @@ __global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const Com
         // per-step scalars: decay of the path up to and including step t by a prefix sum over the lanes
         float gt = 0.f, be = 0.f;
         if (lane < len) {
-            gt = __bfloat162float(g[((size_t)pb + n) * p.h_v + h]);
-            be = __bfloat162float(beta[((size_t)pb + n) * p.h_v + h]);
+            const unsigned short *g16 = reinterpret_cast<const unsigned short *>(g);
+            const unsigned short *b16 = reinterpret_cast<const unsigned short *>(beta);
+            gt = gate_log_decay(g16[((size_t)pb + n) * p.h_v + h], p.raw_gates != 0);
+            be = gate_beta(b16[((size_t)pb + n) * p.h_v + h], p.raw_gates != 0);
         }
         float gsum = gt;
 #pragma unroll
@@ -262,7 +270,7 @@ cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k,
     const int grid = s.n_seq * s.h_v;
     if (grid == 0) return cudaSuccess;
     CommitParams p{s.h_qk, s.h_v, s.d_k, s.d_v, s.max_depth, S, k, v, g, beta,
-                   parent, node_offsets, path, path_offsets, status_dev};
+                   parent, node_offsets, path, path_offsets, status_dev, 0, 0, 0, 0, nullptr, nullptr};
     if (s.d_k == GDN_TILE_D && s.d_v == GDN_TILE_D && s.in_dtype == GDN_BF16 && s.max_depth <= CF_MD) {
         commit_tile128_kernel<<<grid, CF_THREADS, 0, stream>>>(p);
         return cudaGetLastError();
@@ -280,6 +288,24 @@ cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k,
         if (e != cudaSuccess) return e;
         commit_generic_kernel<float><<<grid, CM_THREADS, smem, stream>>>(p);
     }
+    return cudaGetLastError();
+}
+
+bool commit_padded_supported(const gdn_shape_t &s)
+{
+    return s.d_k == GDN_TILE_D && s.d_v == GDN_TILE_D && s.in_dtype == GDN_BF16 && s.max_depth <= CF_MD;
+}
+
+cudaError_t launch_commit_padded(const gdn_shape_t &s, int n_trees, bool raw_gates, float *S, const void *k,
+                                 const void *v, const void *g, const void *beta, const int32_t *parent,
+                                 const int32_t *n_nodes, const int32_t *path, const int32_t *path_len,
+                                 int32_t *status_dev, cudaStream_t stream)
+{
+    const int grid = s.n_seq * s.h_v;
+    if (grid == 0) return cudaSuccess;
+    CommitParams p{s.h_qk, s.h_v, s.d_k, s.d_v, s.max_depth, S, k, v, g, beta, parent, nullptr, path, nullptr,
+                   status_dev, s.max_tree_nodes, n_trees, s.max_depth, raw_gates ? 1 : 0, n_nodes, path_len};
+    commit_tile128_kernel<<<grid, CF_THREADS, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

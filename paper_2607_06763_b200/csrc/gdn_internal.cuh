@@ -25,12 +25,16 @@ namespace gdn {
 // (64 - n_prefix, i.e. at least GDN_GROUP_MIN_NODES).
 //   group_start uint16[n_seq][GDN_MAX_GROUPS + 1]  first position of group k of tree b; entries behind the
 //                                          last group hold the tree's size
+//   group_info uint16[n_seq][GDN_MAX_GROUPS][4]    per group (first position, own nodes, n_prefix, node id at the
+//                                          first position); own nodes = 0 behind the last group.  A tree of at
+//                                          most 64 nodes is its own single group (0, T, 0xFFFF, 0): identity
+//                                          numbering, tables in depth / anc8
 //   dfs_node  uint16[N]                    node id at position r
 //   dfs_depth uint8 [N]                    depth of that node
 //   dfs_anc8  uint8 [N][16]                its root path in virtual indices of its group (0xFF = unused)
 //   utilde   float [N][h_v][d_v]           solve result u~ (Eq. 10 with the W S0 term folded in; general kernel)
 struct WorkspaceLayout {
-    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, group_start, utilde, total;
+    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, group_start, group_info, utilde, total;
 };
 
 constexpr int GDN_GROUP_TILE = 64;            // nodes of a group and its prefix together
@@ -53,6 +57,7 @@ inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
     w.dfs_depth = off; off = align256(off + N);
     w.dfs_anc8 = off; off = align256(off + 16 * N);
     w.group_start = off; off = align256(off + sizeof(uint16_t) * (size_t)s.n_seq * (GDN_MAX_GROUPS + 1));
+    w.group_info = off; off = align256(off + sizeof(uint16_t) * 4 * (size_t)s.n_seq * GDN_MAX_GROUPS);
     w.utilde = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
     w.total = off;
     return w;
@@ -65,7 +70,7 @@ struct PlanPtrs {
     uint8_t *anc8;
     uint16_t *dfs_node;
     uint8_t *dfs_depth, *dfs_anc8;
-    uint16_t *group_start;
+    uint16_t *group_start, *group_info;
     float *utilde;
 };
 
@@ -76,12 +81,14 @@ inline PlanPtrs plan_ptrs(void *workspace, const WorkspaceLayout &w)
             reinterpret_cast<uint16_t *>(b + w.anc), reinterpret_cast<uint8_t *>(b + w.anc8),
             reinterpret_cast<uint16_t *>(b + w.dfs_node), reinterpret_cast<uint8_t *>(b + w.dfs_depth),
             reinterpret_cast<uint8_t *>(b + w.dfs_anc8), reinterpret_cast<uint16_t *>(b + w.group_start),
-            reinterpret_cast<float *>(b + w.utilde)};
+            reinterpret_cast<uint16_t *>(b + w.group_info), reinterpret_cast<float *>(b + w.utilde)};
 }
 
 // Host launchers (each returns the cudaError_t of its launch).
+// node_offsets == nullptr: padded layout, s.n_seq trees of s.max_tree_nodes rows each (parent [n_seq][rows], the node
+// counts in n_nodes [n_seq]); otherwise ragged packing and n_nodes is not read.
 cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32_t *node_offsets,
-                        const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream);
+                        const int32_t *n_nodes, const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream);
 
 cudaError_t launch_verify_generic(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
                                   const void *v, const void *g, const void *beta,
@@ -126,6 +133,12 @@ cudaError_t launch_commit_verify_sm100_padded(const gdn_shape_t &s, int n_trees,
                                               const int32_t *n_nodes, void *o, int32_t *status_dev,
                                               cudaStream_t stream);
 
+// Padded layout, any padded tree size up to GDN_GROUPED_MAX_NODES: the plan of the n_trees shared trees (built by
+// launch_plan with node_offsets == nullptr on a shape of n_trees trees) serves every slot; s.n_seq slots.
+cudaError_t launch_verify_sm100_planned(const gdn_shape_t &s, int n_trees, bool raw_gates, const float *S0,
+                                        const void *q, const void *k, const void *v, const void *g, const void *beta,
+                                        const PlanPtrs &plan, void *o, int32_t *status_dev, cudaStream_t stream);
+
 // Per-branch recurrent verification (the baseline of Section 5.2 / Figure 5): no workspace, no tree plan.
 cudaError_t launch_verify_recurrent(const gdn_shape_t &s, const float *S0, const void *q, const void *k,
                                     const void *v, const void *g, const void *beta, const int32_t *parent,
@@ -135,12 +148,37 @@ cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k,
                                   const void *g, const void *beta, const int32_t *parent,
                                   const int32_t *node_offsets, const int32_t *path,
                                   const int32_t *path_offsets, int32_t *status_dev, cudaStream_t stream);
+// Commit in the padded layout (d_k = d_v = 128, bf16, root paths of at most 16 nodes): slot b keeps its rows at
+// b * s.max_tree_nodes and carries tree b % n_trees; parent [n_trees][rows] (may be null), n_nodes [n_trees],
+// path [n_trees][s.max_depth], path_len [n_trees].
+bool commit_padded_supported(const gdn_shape_t &s);
+cudaError_t launch_commit_padded(const gdn_shape_t &s, int n_trees, bool raw_gates, float *S, const void *k,
+                                 const void *v, const void *g, const void *beta, const int32_t *parent,
+                                 const int32_t *n_nodes, const int32_t *path, const int32_t *path_len,
+                                 int32_t *status_dev, cudaStream_t stream);
 
 #ifdef __CUDACC__
 // First error wins; later ones are dropped.
 __device__ __forceinline__ void report_status(int32_t *status_dev, int code)
 {
     if (status_dev) atomicCAS(status_dev, 0, code);
+}
+
+// Gate activations of the "scalars" stage (Section 3.4.2; Table 1 row "scalars"): the kernel takes either the
+// finished log-decay g and write strength beta, or the layer's raw gate inputs a, b, for which
+// g = -softplus(a) = -log(1 + e^a) and beta = sigmoid(b) are formed here (fp32, never rounded to the input type).
+__device__ __forceinline__ float gate_log_decay(uint32_t bf16_bits, bool raw)
+{
+    const float x = __uint_as_float(bf16_bits << 16);
+    if (!raw) return x;
+    return x > 0.f ? -(x + log1pf(expf(-x))) : -log1pf(expf(x));
+}
+__device__ __forceinline__ float gate_beta(uint32_t bf16_bits, bool raw)
+{
+    const float x = __uint_as_float(bf16_bits << 16);
+    if (!raw) return x;
+    const float e = expf(-fabsf(x));
+    return x >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
 }
 
 template <typename T> __device__ __forceinline__ float load_as_float(const T *p);

@@ -16,9 +16,10 @@ constexpr int PLAN_THREADS = 128;
 __global__ void __launch_bounds__(PLAN_THREADS)
 plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
             const int32_t *__restrict__ parent, const int32_t *__restrict__ node_offsets,
-            int32_t *__restrict__ tree_ok, uint8_t *__restrict__ depth, uint16_t *__restrict__ anc,
+            const int32_t *__restrict__ n_nodes, int32_t *__restrict__ tree_ok, uint8_t *__restrict__ depth, uint16_t *__restrict__ anc,
             uint8_t *__restrict__ anc8, uint16_t *__restrict__ dfs_node, uint8_t *__restrict__ dfs_depth,
-            uint8_t *__restrict__ dfs_anc8, uint16_t *__restrict__ group_start, int32_t *status_dev)
+            uint8_t *__restrict__ dfs_anc8, uint16_t *__restrict__ group_start, uint16_t *__restrict__ group_info,
+            int32_t *status_dev)
 {
     __shared__ int size_s[GDN_GROUPED_MAX_NODES];        // subtree sizes
     __shared__ uint16_t left_s[GDN_GROUPED_MAX_NODES];   // nodes in the subtrees of earlier siblings
@@ -33,16 +34,20 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
     const int b = blockIdx.x;
-    const int lo = node_offsets[b], hi = node_offsets[b + 1];
+    // ragged packing: the tree's rows by node_offsets[]; padded layout: max_tree_nodes rows per tree, n_nodes[b] used
+    const int lo = node_offsets ? node_offsets[b] : b * max_tree_nodes;
+    const int hi = node_offsets ? node_offsets[b + 1] : lo + n_nodes[b];
     const int T = hi - lo;
     bool offsets_ok = lo >= 0 && T >= 0 && T <= max_tree_nodes && hi <= total_nodes;
-    if (b == 0) offsets_ok = offsets_ok && lo == 0;
-    if (b == n_seq - 1) offsets_ok = offsets_ok && hi == total_nodes;
+    if (node_offsets && b == 0) offsets_ok = offsets_ok && lo == 0;
+    if (node_offsets && b == n_seq - 1) offsets_ok = offsets_ok && hi == total_nodes;
     if (!offsets_ok) {
         if (threadIdx.x == 0) {
             report_status(status_dev, GDN_ERR_TREE);
             tree_ok[b] = 0;
         }
+        for (int k = threadIdx.x; k < GDN_MAX_GROUPS; k += PLAN_THREADS)
+            *reinterpret_cast<uint2 *>(group_info + ((size_t)b * GDN_MAX_GROUPS + k) * 4) = make_uint2(0u, 0u);
         return;
     }
     const bool grouped = max_depth <= 16 && T > 64 && T <= GDN_GROUPED_MAX_NODES;
@@ -84,7 +89,14 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     const int any_err = __syncthreads_or(err != 0);
     if (err) report_status(status_dev, err);
     if (threadIdx.x == 0) tree_ok[b] = any_err ? 0 : 1;
-    if (any_err || !grouped) return;
+    if (any_err || !grouped) {
+        // a tree that fits one tile is its own single group with the identity numbering, marked by n_prefix =
+        // 0xFFFF (no group at all if the tree was rejected)
+        for (int k = threadIdx.x; k < GDN_MAX_GROUPS; k += PLAN_THREADS)
+            *reinterpret_cast<uint2 *>(group_info + ((size_t)b * GDN_MAX_GROUPS + k) * 4) =
+                make_uint2(k == 0 && !any_err && T <= GDN_GROUP_TILE ? (uint32_t)T << 16 : 0u, 0xFFFFu);
+        return;
+    }
 
     // Pre-order position = (#proper ancestors) + sum over the root path of the sizes of the subtrees
     // hanging off earlier siblings (roots count as siblings of one another; siblings by increasing id).
@@ -119,6 +131,15 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     __syncthreads();
     for (int k = threadIdx.x; k <= GDN_MAX_GROUPS; k += PLAN_THREADS)
         group_start[(size_t)b * (GDN_MAX_GROUPS + 1) + k] = gstart_s[k];
+    for (int k = threadIdx.x; k < GDN_MAX_GROUPS; k += PLAN_THREADS) {
+        const int g0 = gstart_s[k], own = gstart_s[k + 1] - g0;
+        uint32_t w0 = 0, w1 = 0;   // (first position, own nodes), (n_prefix, node at the first position)
+        if (own > 0) {
+            w0 = (uint32_t)g0 | ((uint32_t)own << 16);
+            w1 = (uint32_t)(depth_at_s[g0] - 1) | ((uint32_t)dfs_node[lo + g0] << 16);
+        }
+        *reinterpret_cast<uint2 *>(group_info + ((size_t)b * GDN_MAX_GROUPS + k) * 4) = make_uint2(w0, w1);
+    }
     // Root path of every node in the virtual indices of its group: an ancestor before the group's first
     // position is an ancestor of the group's first node and gets index depth-1; one inside the group gets
     // n_prefix + its offset in the group, n_prefix = depth(first node) - 1.
@@ -143,7 +164,7 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
 }  // namespace
 
 cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32_t *node_offsets,
-                        const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream)
+                        const int32_t *n_nodes, const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream)
 {
     if (s.n_seq == 0) return cudaSuccess;
     cudaLaunchConfig_t cfg{};
@@ -157,8 +178,8 @@ cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, plan_kernel, s.n_seq, s.total_nodes, s.max_tree_nodes, s.max_depth, parent,
-                              node_offsets, plan.tree_ok, plan.depth, plan.anc, plan.anc8, plan.dfs_node,
-                              plan.dfs_depth, plan.dfs_anc8, plan.group_start, status_dev);
+                              node_offsets, n_nodes, plan.tree_ok, plan.depth, plan.anc, plan.anc8, plan.dfs_node,
+                              plan.dfs_depth, plan.dfs_anc8, plan.group_start, plan.group_info, status_dev);
 }
 
 }  // namespace gdn

@@ -1,5 +1,5 @@
-// Tree-verify fast path for sm_100a: d_k = d_v = 128, bf16 inputs, root paths of at most 16 nodes, trees of at
-// most 64 nodes per CTA (larger trees are cut into ancestor-closed groups, one CTA each).  It evaluates the
+// Tree-verify fast path for sm_100a: d_k = d_v = 128, bf16 inputs, root paths of at most 16 nodes, at most 64 nodes
+// per unit of work (larger trees are cut into ancestor-closed groups, each a unit of its own).  It evaluates the
 // triangular form of Section 3.4.1 (Eq. 9-11) restricted to real ancestors, with the W S0 term folded into the
 // right-hand side as in Section 3.4.2, and turns all of the per-component work into dense contractions on the
 // 5th-generation tensor cores (tcgen05.mma, bf16 operands, fp32 accumulators in tensor memory):
@@ -19,9 +19,9 @@
 //
 // Operand orientation: d_v on the TMEM lanes, nodes on the TMEM columns, so every thread of a warp owns one value
 // component.  256 threads, about 112 KB of shared memory and 256 TMEM columns per CTA, so two CTAs share an SM.
-// Two kernels: a persistent one for trees that fit one CTA (TMA tiles on mbarriers, a software pipeline across
-// the units of a CTA, optionally the commit of the previous step fused in front), and a one-shot one for the
-// groups of larger trees (row gathers through a node table).
+// One persistent kernel: a software pipeline across the units of a CTA, TMA tiles on mbarriers for trees that fit
+// one unit (optionally with the commit of the previous step fused in front), row gathers through the plan's node
+// table for the groups of larger trees.
 #include <cuda.h>   // CUtensorMap and the cuTensorMapEncodeTiled prototype (resolved at run time, no libcuda link)
 
 #include "gdn_internal.cuh"
@@ -35,21 +35,18 @@ constexpr int FV_THREADS = 256;
 constexpr int FV_D = 128;           // d_k = d_v
 constexpr int FV_T = 64;            // max nodes per tree
 constexpr int FV_MD = 16;           // max nodes on a root path
-constexpr int FV_TMEM_COLS = 256;   // P: columns [0,128); D (one-shot kernel: first the Gram block): [128,192);
-                                    // persistent kernel: Gram block of the unit to come in [192,256)
+constexpr int FV_TMEM_COLS = 256;   // P: columns [0,128); D: [128,192); Gram block of the unit to come: [192,256)
 
 // shared memory map (bytes from a 1024-byte aligned base)
 constexpr int SM_A_HI = 0;                       // S0 hi: [2][128 rows][128 B], 128B-swizzled, K-major
 constexpr int SM_A_LO = 32768;                   // S0 lo
-constexpr int SM_B_KQ = 65536;                   // k and q rows, same layout (one-shot kernel: row 2i = k_i, 2i+1 = q_i;
-                                                 // persistent kernel: rows 0..63 = k, 64..127 = q)
+constexpr int SM_B_KQ = 65536;                   // k and q rows, same layout: rows 0..63 = k, 64..127 = q
 // after the first MMA group the operand tiles are dead and are reused:
 constexpr int SM_GRAM = 0;                       // fp32 [128][64]: four-column piece c of row r at position c ^ (r & 15)
 constexpr int SM_RT_HI = 0;                      // then R^T hi: [128 rows = components][64 nodes] bf16, swizzled
 constexpr int SM_RT_LO = 16384;                  //      R^T lo
-constexpr int SM_V = 32768;                      // v rows of the tree, bf16 [64][128]
-constexpr int SM_VE = 40960;                     // persistent kernel: the v rows land here at the top of a unit (free until
-                                                 // the state operand is written) and move into registers before that
+constexpr int SM_VE = 40960;                     // v rows of the tree, bf16 [64][128]: they land here at the top of a unit (free
+                                                 // until the state operand is written) and move into registers before that
 constexpr int SM_Z_HI = 49152;                   // Z hi: [64 rows = nodes i][64 nodes j] bf16, swizzled
 constexpr int SM_Z_LO = 57344;                   // Z lo
 constexpr int SM_X = 98304;                      // fp32 [64][16]  X(i, t-th path node)
@@ -63,39 +60,38 @@ constexpr int SM_PATH = SM_DEPTH + FV_T;         // fused commit, two slots of 3
 constexpr int SM_PATH_SLOT = 384;
 constexpr int SM_PK = 32768;                     // fused commit: k rows of the accepted path, bf16 [16][128], parked in the
 constexpr int SM_PV = 36864;                     // state-operand area until the replay is over; v rows likewise
-constexpr int SM_VNODE = SM_PATH + 2 * SM_PATH_SLOT;          // grouped mode: u16 [64] node id of virtual index u
-constexpr int SM_TABLE2 = SM_VNODE + 128;        // persistent kernel: second copy of ANC / GAB / DEPTH (2112 B)
+constexpr int SM_TABLE2 = SM_PATH + 2 * SM_PATH_SLOT;   // second copy of ANC / GAB / DEPTH (2112 B)
 constexpr int SM_TABLE_STRIDE = SM_TABLE2 - SM_ANC;   // table buffer tb lives SM_TABLE_STRIDE * tb further on
 constexpr int SM_MBAR = SM_TABLE2 + 2176;        // 5 x u64: Gram done, P done, D done, k/q tile landed, v tile landed
 constexpr int SM_TMEM = SM_MBAR + 40;            // u32
 constexpr int SM_FLAG = SM_TMEM + 4;             // u32 (timeout flag)
-constexpr int SM_PAR = SM_FLAG + 4;              // persistent kernel: s8 [64] parent[] of the tree whose tables are being built
-constexpr int SM_BAD = SM_PAR + FV_T;            // persistent kernel: int [2], tree of table buffer tb was rejected
-constexpr int SM_BYTES = SM_BAD + 8;
+constexpr int SM_PAR = SM_FLAG + 4;              // s8 [64] parent[] of the tree whose tables are being built
+constexpr int SM_BAD = SM_PAR + FV_T;            // int [2], tree of table buffer tb was rejected
+constexpr int SM_VN2 = SM_BAD + 8;               // grouped mode: u16 [2][64] node id of virtual index u (per table buffer)
+constexpr int SM_BYTES = SM_VN2 + 2 * 2 * FV_T;
 constexpr int SM_ALLOC = SM_BYTES + 1024;        // slack for the 1024-byte alignment of the base
 
 struct VerifyFastParams {
-    // TMA descriptors of the packed k, q, v tensors viewed as [N][heads][128] bf16 (persistent kernel only)
+    // TMA descriptors of the packed k, q, v tensors viewed as [N][heads][128] bf16 (not used by the grouped mode)
     alignas(64) CUtensorMap tm_k;
     alignas(64) CUtensorMap tm_q;
     alignas(64) CUtensorMap tm_v;
     int h_qk, h_v;
-    int n_units;        // n_seq * h_v
+    int n_units;        // n_seq * h_v (grouped mode: times groups_per_tree)
     int prefetch_dist;  // a CTA warms L2 for unit blockIdx.x + prefetch_dist (about one wave ahead)
     float scale;
     const float *S0;
     const __nv_bfloat16 *q, *k, *v, *g, *beta;
     const int32_t *node_offsets;
-    const int32_t *parent;                             // persistent kernel: it builds the tree metadata itself
+    const int32_t *parent;                             // trees of at most 64 nodes: the kernel builds the metadata itself
     int n_seq, total_nodes, max_tree_nodes, max_depth;
     void *o;
-    const int32_t *tree_ok;
     const uint8_t *depth;
     const uint8_t *anc8;
     int32_t *status_dev;
     // grouped verification of trees with more than 64 nodes (only read by the GROUPED instantiation)
-    int groups_per_tree, anc_stride;                   // CTAs per (tree, head); entries per row of anc16
-    const uint16_t *anc16, *dfs_node, *group_start;
+    int groups_per_tree, anc_stride;                   // units per (tree, head); entries per row of anc16
+    const uint16_t *anc16, *dfs_node, *group_info;
     const uint8_t *dfs_depth, *dfs_anc8;
     // fused commit of the previous step's accepted paths (only read by the FUSED instantiation)
     float *S_rw;                                       // same tensor as S0, written in place
@@ -135,6 +131,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
                  ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar)
                  : "memory");
+}
+// The mbarrier receives one arrival from this thread once all cp.async it has issued so far have landed (the
+// barrier's expected count has to include that arrival).
+__device__ __forceinline__ void cp_async_arrive_on(uint32_t bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all()
 {
@@ -279,472 +281,8 @@ __device__ __forceinline__ void split_bf16(float x, float &hi, float &lo)
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <typename TOut, bool GROUPED>
-__global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_kernel(const VerifyFastParams p)
-{
-    extern __shared__ uint8_t fv_smem_raw[];
-    // GROUPED: the CTA takes group `grp` of tree b (see gdn_internal.cuh): T is then the size of the
-    // virtual tree (n_prefix ancestors of the group's first node + the group's own nodes), and virtual
-    // index u maps to node vnode[u].  Trees of at most 64 nodes are their own single group, identity map.
-    const int h = blockIdx.x % p.h_v;
-    const int b = GROUPED ? (blockIdx.x / p.h_v) / p.groups_per_tree : blockIdx.x / p.h_v;
-    const int grp = GROUPED ? (blockIdx.x / p.h_v) % p.groups_per_tree : 0;
-    if (!p.tree_ok[b]) return;
-    const int base = p.node_offsets[b];
-    const int T_tree = p.node_offsets[b + 1] - base;
-    if (T_tree <= 0) return;
-    if (!GROUPED && T_tree > FV_T) return;   // larger trees never reach that instantiation (host-side dispatch)
-    const bool ident = !GROUPED || T_tree <= FV_T;
-    int g0 = 0, n_own = T_tree;
-    if (GROUPED && !ident) {
-        const uint16_t *gs = p.group_start + (size_t)b * (GDN_MAX_GROUPS + 1);
-        g0 = grp <= GDN_MAX_GROUPS - 1 ? gs[grp] : T_tree;
-        n_own = (grp <= GDN_MAX_GROUPS - 1 ? gs[grp + 1] : T_tree) - g0;
-    }
-    if (GROUPED && (ident ? grp > 0 : n_own <= 0)) return;   // no such group in this tree
-    int n_prefix = 0, T = T_tree;
-    if (GROUPED && !ident) {
-        n_prefix = p.dfs_depth[base + g0] - 1;
-        T = n_prefix + n_own;
-    }
-
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fv_smem_raw) + 1023) & ~uintptr_t(1023));
-    const uint32_t sbase = smem_u32(smem);
-    float *xs = reinterpret_cast<float *>(smem + SM_X);
-    float *ys = reinterpret_cast<float *>(smem + SM_Y);
-    float4 *gab = reinterpret_cast<float4 *>(smem + SM_GAB);
-    uint8_t *anc_s = smem + SM_ANC;
-    uint8_t *depth_s = smem + SM_DEPTH;
-    float *gram = reinterpret_cast<float *>(smem + SM_GRAM);
-    const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(smem + SM_V);
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM_TMEM);
-    volatile uint32_t *flag = reinterpret_cast<volatile uint32_t *>(smem + SM_FLAG);
-    const uint32_t mbar_g = sbase + SM_MBAR, mbar_p = mbar_g + 8, mbar_d = mbar_g + 16;
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int hk = h / (p.h_v / p.h_qk);
-    uint16_t *vnode_s = reinterpret_cast<uint16_t *>(smem + SM_VNODE);
-    auto node_of = [&](int u) -> int { return GROUPED ? (int)vnode_s[u] : u; };
-
-    // L2 warming for the unit that a CTA will pick up about one wave from now, issued in slices at
-    // phase boundaries (one thread, a few instructions each) so that HBM keeps streaming while the resident
-    // CTAs compute, instead of all demand loads of a wave hitting it at once.
-    const int u_next = blockIdx.x + p.prefetch_dist;
-    auto warm_l2_state = [&](int slice) {   // slice 0..3 of the next unit's 64 KB state tile
-        if (!GROUPED && tid == 96 && u_next < p.n_units)
-            prefetch_l2_bulk(p.S0 + (size_t)u_next * FV_D * FV_D + (size_t)slice * 4096, 16384);
-    };
-    auto warm_l2_rows = [&]() {             // the next unit's q/k/v rows
-        if (!GROUPED && u_next < p.n_units && tid >= 128 && tid < 128 + FV_T) {
-            const int b2 = u_next / p.h_v, h2 = u_next % p.h_v;
-            const int base2 = p.node_offsets[b2];
-            const int T2 = min(p.node_offsets[b2 + 1] - base2, FV_T);
-            const int i = tid - 128;
-            if (i < T2) {
-                const int hk2 = h2 / (p.h_v / p.h_qk);
-                prefetch_l2_bulk(p.v + ((size_t)(base2 + i) * p.h_v + h2) * FV_D, 256);
-                if (h2 % (p.h_v / p.h_qk) == 0) {   // one value head per key head fetches q and k
-                    prefetch_l2_bulk(p.k + ((size_t)(base2 + i) * p.h_qk + hk2) * FV_D, 256);
-                    prefetch_l2_bulk(p.q + ((size_t)(base2 + i) * p.h_qk + hk2) * FV_D, 256);
-                }
-            }
-        }
-    };
-
-    // (1) state tile loads first (the longest latency of the prologue): a warp instruction covers
-    // four rows; the eight lanes of a row each own one 16-byte bf16 piece of either K half.
-    const int r4 = lane >> 3, l8 = lane & 7;
-    float4 x[4][4];   // [row i][kh*2 + half]
-    {
-        const float *S = p.S0 + (size_t)(b * p.h_v + h) * FV_D * FV_D;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float *src = S + (size_t)(warp * 16 + i * 4 + r4) * FV_D + l8 * 8;
-#pragma unroll
-            for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
-        }
-    }
-    // the node table of the group is looked up under the latency of the state loads
-    if constexpr (GROUPED) {
-        if (tid < FV_T) {
-            int node = tid;
-            if (!ident && tid < T) {
-                if (tid < n_prefix) {
-                    const int first = p.dfs_node[base + g0];
-                    node = p.anc16[(size_t)(base + first) * p.anc_stride + tid];
-                } else {
-                    node = p.dfs_node[base + g0 + tid - n_prefix];
-                }
-            }
-            vnode_s[tid] = (uint16_t)node;
-        }
-        __syncthreads();
-    }
-    // (2) k and q rows -> B operand tile (rows beyond T are zero-filled)
-#pragma unroll
-    for (int it = 0; it < (128 * 16) / FV_THREADS; ++it) {
-        const int idx = it * FV_THREADS + tid;
-        const int r = idx >> 4, c16 = idx & 15;
-        const int node = r >> 1;
-        const bool valid = node < T;
-        const __nv_bfloat16 *src = ((r & 1) ? p.q : p.k) + ((size_t)(base + (valid ? node_of(node) : 0)) * p.h_qk + hk) * FV_D + c16 * 8;
-        cp_async_16(sbase + SM_B_KQ + sw128_offset(r, c16), src, valid);
-    }
-    if (warp == 0) tmem_alloc(sbase + SM_TMEM, FV_TMEM_COLS);
-    if (tid == 32) {
-        mbar_init(mbar_g, 1);
-        mbar_init(mbar_p, 1);
-        mbar_init(mbar_d, 1);
-        *flag = 0;
-    }
-    // this tree's v rows are needed only after the first MMA group: pull them into L2 meanwhile
-    if (tid >= 192 && tid - 192 < T) prefetch_l2_bulk(p.v + ((size_t)(base + tid - 192) * p.h_v + h) * FV_D, 256);
-    // (3) per-node tables: depth, root-path ids, g, beta (zeros beyond T)
-    if (tid < FV_T) {
-        int d = 0;
-        uint4 row = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
-        float gi = 0.f, be = 0.f;
-        if (tid < T) {
-            const int n = base + node_of(tid);
-            if (ident) {
-                d = p.depth[n];
-                row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)n * 16));
-            } else if (tid < n_prefix) {   // an ancestor of the group's first node: its path is 0..tid
-                d = tid + 1;
-                const uint32_t all[4] = {0x03020100u, 0x07060504u, 0x0B0A0908u, 0x0F0E0D0Cu};
-                uint32_t w[4];
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int keep = d - 4 * q4;   // bytes of this word that are on the path
-                    w[q4] = keep >= 4 ? all[q4] : keep <= 0 ? 0xFFFFFFFFu : (all[q4] | (0xFFFFFFFFu << (8 * keep)));
-                }
-                row = make_uint4(w[0], w[1], w[2], w[3]);
-            } else {
-                const int r = base + g0 + tid - n_prefix;
-                d = p.dfs_depth[r];
-                row = __ldg(reinterpret_cast<const uint4 *>(p.dfs_anc8 + (size_t)r * 16));
-            }
-            gi = __bfloat162float(p.g[(size_t)n * p.h_v + h]);
-            be = __bfloat162float(p.beta[(size_t)n * p.h_v + h]);
-        }
-        depth_s[tid] = (uint8_t)d;
-        *reinterpret_cast<uint4 *>(anc_s + tid * 16) = row;
-        gab[tid] = make_float4(0.f, 0.f, be, gi);
-    }
-
-    cp_async_wait_all();
-    fence_proxy_async();   // the k/q tile (cp.async) becomes visible to the tensor core
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // warp-uniform by construction
-
-    // (4) Everything that depends only on q, k, g, beta runs now, under the latency of the state loads:
-    // Gram = [k;q].[k;q]^T on the tensor core, G_i / a_i tables, then X and Y of Eq. 9.
-    if (warp == 0 && elect_one()) {
-        const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
-        constexpr uint32_t id = idesc_bf16(128, 128);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-            umma_bf16(tmem + 128, b_kq + adv, b_kq + adv, id, ks > 0);
-        }
-        umma_commit(mbar_g);
-    }
-    // G_i = sum of g along the root path (root first), a_i = exp(G_i)
-    if (tid >= 64 && tid < 64 + FV_T) {
-        const int i = tid - 64;
-        const int d = depth_s[i];
-        float G = 0.f;
-        for (int t = 0; t < d; ++t) G += gab[anc_s[i * FV_MD + t]].w;
-        gab[i].x = G;
-        gab[i].y = d ? expf(G) : 0.f;
-    }
-    // one thread polls the mbarrier (bounded: on expiry it flags the error and everybody falls through to
-    // the clean-up), the others sleep in the CTA barrier
-    if (tid == 0 && !mbar_wait_bounded(mbar_g, 0)) *flag = 1;
-    __syncthreads();
-    tc_fence_after();
-    warm_l2_state(0);
-    if (*flag == 0) {
-        // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
-        {
-            const int row = (warp & 3) * 32 + lane;
-            const int half = warp >> 2;   // TMEM columns 128 + 64*half .. : k_j for j = 32*half ..
-            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 128 + half * 64;
-#pragma unroll 1
-            for (int part = 0; part < 2; ++part) {
-                uint32_t ra[32];
-                GDN_TMEM_LD32(taddr + part * 32, ra);
-                tmem_wait_ld();
-                // four-column piece c of row r goes to position c ^ (r & 15): 16-byte stores, conflict-free
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4)
-                    *reinterpret_cast<uint4 *>(gram + row * 64 + (((half * 8 + part * 4 + c4) ^ (row & 15)) << 2)) =
-                        make_uint4(ra[8 * c4], ra[8 * c4 + 2], ra[8 * c4 + 4], ra[8 * c4 + 6]);
-            }
-        }
-        tc_fence_before();
-        __syncthreads();
-        warm_l2_state(1);
-        // X and Y for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
-        {
-            float gdiff[4], gk[4], gq[4], bi[4];
-            bool on[4], onx[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int idx = u * FV_THREADS + tid;
-                const int i = idx >> 4, t = idx & 15;
-                const int d = depth_s[i];
-                on[u] = t < d;
-                onx[u] = t < d - 1;
-                const int j = on[u] ? anc_s[idx] : 0;
-                const float4 gi = gab[i];
-                gdiff[u] = gi.x - gab[j].x;
-                bi[u] = gi.z;
-                gq[u] = gram[(2 * i + 1) * 64 + ((((j >> 2) ^ ((2 * i + 1) & 15)) << 2) | (j & 3))];
-                gk[u] = gram[(2 * i) * 64 + ((((j >> 2) ^ ((2 * i) & 15)) << 2) | (j & 3))];
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int idx = u * FV_THREADS + tid;
-                const float dec = expf(gdiff[u]);
-                ys[idx] = on[u] ? dec * gq[u] : 0.f;
-                xs[idx] = onx[u] ? bi[u] * dec * gk[u] : 0.f;
-            }
-        }
-    }
-    cp_async_wait_all();
-    __syncthreads();   // X and Y complete; the Gram copy is dead and its area can take the state operand
-
-
-    // (4) fp32 -> bf16 hi + lo, written as the A operand
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int row = warp * 16 + i * 4 + r4;
-#pragma unroll
-        for (int kh = 0; kh < 2; ++kh) {
-            const float4 u = x[i][kh * 2 + 0], w = x[i][kh * 2 + 1];
-            const float f[8] = {u.x, u.y, u.z, u.w, w.x, w.y, w.z, w.w};
-            uint32_t hi[4], lo[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) split_pack_bf16(f[2 * e], f[2 * e + 1], hi[e], lo[e]);
-            const uint32_t off = sw128_offset(row, kh * 8 + l8);
-            *reinterpret_cast<uint4 *>(smem + SM_A_HI + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4 *>(smem + SM_A_LO + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        }
-    }
-    fence_proxy_async();   // generic-proxy writes of the operand become visible to the tensor core
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    warm_l2_state(2);
-
-    // (5) P = S0.[k;q]^T (hi then lo) on the tensor core; meanwhile the back-substitution below
-    if (warp == 0 && elect_one()) {
-        const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
-        const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
-        constexpr uint32_t id = idesc_bf16(128, 128);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-            umma_bf16(tmem, a_hi + adv, b_kq + adv, id, ks > 0);
-        }
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-            umma_bf16(tmem, a_lo + adv, b_kq + adv, id, 1);
-        }
-        umma_commit(mbar_p);
-    }
-    // (6) z^T = y^T (I + X_path)^-1 by back-substitution over the root path (column-oriented: once z_l is
-    // final, subtract z_l X(n_l, n_t) from every z_t, t < l).  Four threads per node, thread sq of the quad
-    // owning path positions 4 sq .. 4 sq + 3; z stays in registers until the k/q tile can be overwritten.
-    const int zi = tid >> 2, sq = tid & 3;
-        const int d = depth_s[zi];
-        const int dmax = __reduce_max_sync(0xffffffffu, d);
-        const uint4 row = *reinterpret_cast<const uint4 *>(anc_s + zi * 16);
-        const uint32_t idw[4] = {row.x, row.y, row.z, row.w};
-        const float4 y4 = *reinterpret_cast<const float4 *>(ys + zi * FV_MD + sq * 4);
-        float z[4] = {y4.x, y4.y, y4.z, y4.w};
-#pragma unroll
-        for (int l = FV_MD - 1; l >= 1; --l) {
-            if (l < dmax) {   // warp-uniform
-                const float zl = __shfl_sync(0xffffffffu, z[l & 3], (lane & ~3) | (l >> 2));
-                if (l < d && sq * 4 < l) {
-                    const int nl = (int)((idw[l >> 2] >> ((l & 3) * 8)) & 0xFFu);
-                    const float4 x4 = *reinterpret_cast<const float4 *>(xs + nl * FV_MD + sq * 4);
-                    const float xv[4] = {x4.x, x4.y, x4.z, x4.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (sq * 4 + e < l) z[e] = fmaf(-zl, xv[e], z[e]);
-                }
-            }
-        }
-    if (tid == 0 && !mbar_wait_bounded(mbar_p, 0)) *flag = 1;
-    __syncthreads();
-    tc_fence_after();
-    bool ok = *flag == 0;
-    warm_l2_state(3);
-
-    if (ok) {
-        // (7) both operand tiles are dead now: the tree's v rows go over the state operand, and z is
-        // scattered into the dense bf16 hi/lo tiles Z[i][j] (zero off the root path) over the k/q tile
-#pragma unroll
-        for (int it = 0; it < (FV_T * 16) / FV_THREADS; ++it) {
-            const int idx = it * FV_THREADS + tid;
-            const int i = idx >> 4, c16 = idx & 15;
-            const bool valid = i < T;
-            cp_async_16(sbase + SM_V + i * 256 + c16 * 16,
-                        p.v + ((size_t)(base + (valid ? node_of(i) : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
-        }
-        {
-            const int i = zi;
-            const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, 2 * sq)) = zero4;
-            *reinterpret_cast<uint4 *>(smem + SM_Z_HI + sw128_row_offset(i, 2 * sq + 1)) = zero4;
-            *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, 2 * sq)) = zero4;
-            *reinterpret_cast<uint4 *>(smem + SM_Z_LO + sw128_row_offset(i, 2 * sq + 1)) = zero4;
-            __syncwarp();   // the quad's zero fill precedes the scattered stores below
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int t = sq * 4 + e;
-                if (t < d) {
-                    const int j = (int)((idw[sq] >> (e * 8)) & 0xFFu);
-                    float hi, lo;
-                    split_bf16(z[e], hi, lo);
-                    const uint32_t off = sw128_row_offset(i, j >> 3) + (j & 7) * 2;
-                    *reinterpret_cast<__nv_bfloat16 *>(smem + SM_Z_HI + off) = __float2bfloat16_rn(hi);
-                    *reinterpret_cast<__nv_bfloat16 *>(smem + SM_Z_LO + off) = __float2bfloat16_rn(lo);
-                }
-            }
-        }
-        cp_async_wait_all();
-        __syncthreads();
-
-        // (8) all warps: r_j[c] = beta_j (v_j[c] - a_j p^k_j[c]) for component c = TMEM lane and 32 nodes,
-        // split into bf16 hi/lo and stored as the K-major A operand R^T[c][j]
-        {
-            const int c = (warp & 3) * 32 + lane;
-            const int half = warp >> 2;
-            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
-#pragma unroll 1
-            for (int part = 0; part < 2; ++part) {
-                const int j0 = half * 32 + part * 16;
-                uint32_t rr[32];
-                GDN_TMEM_LD32(taddr + part * 32, rr);   // columns 2j, 2j+1 for 16 nodes: p^k_j, p^q_j
-                float vv[16], aj[16], bj[16];
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) {
-                    vv[jj] = __bfloat162float(vs[(j0 + jj) * FV_D + c]);
-                    const float4 gj = gab[j0 + jj];
-                    aj[jj] = gj.y;
-                    bj[jj] = gj.z;
-                }
-                tmem_wait_ld();
-                uint32_t hi[8], lo[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float r0 = bj[2 * e] * (vv[2 * e] - aj[2 * e] * __uint_as_float(rr[4 * e]));
-                    const float r1 = bj[2 * e + 1] * (vv[2 * e + 1] - aj[2 * e + 1] * __uint_as_float(rr[4 * e + 2]));
-                    split_pack_bf16(r0, r1, hi[e], lo[e]);
-                }
-#pragma unroll
-                for (int oct = 0; oct < 2; ++oct) {
-                    const uint32_t off = sw128_row_offset(c, half * 4 + part * 2 + oct);
-                    *reinterpret_cast<uint4 *>(smem + SM_RT_HI + off) = make_uint4(hi[4 * oct], hi[4 * oct + 1], hi[4 * oct + 2], hi[4 * oct + 3]);
-                    *reinterpret_cast<uint4 *>(smem + SM_RT_LO + off) = make_uint4(lo[4 * oct], lo[4 * oct + 1], lo[4 * oct + 2], lo[4 * oct + 3]);
-                }
-            }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        warm_l2_rows();
-
-        // (9) second MMA group: D[c][i] = sum_j R^T[c][j] Z[i][j] with the hi/lo cross terms
-        if (warp == 0 && elect_one()) {
-            constexpr uint32_t id2 = idesc_bf16(128, 64);
-            const uint64_t a2[2] = {smem_desc_sw128(sbase + SM_RT_HI), smem_desc_sw128(sbase + SM_RT_LO)};
-            const uint64_t b2[2] = {smem_desc_sw128(sbase + SM_Z_HI), smem_desc_sw128(sbase + SM_Z_LO)};
-#pragma unroll
-            for (int combo = 0; combo < 3; ++combo) {   // hi.hi, lo.hi, hi.lo; lo.lo is below 2^-18 of the result
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_bf16(tmem + 128, a2[combo & 1] + (uint64_t)(ks * 2), b2[combo >> 1] + (uint64_t)(ks * 2), id2,
-                              (combo | ks) != 0);
-            }
-            umma_commit(mbar_d);
-        }
-        if (tid == 0 && !mbar_wait_bounded(mbar_d, 0)) *flag = 1;
-        __syncthreads();
-        tc_fence_after();
-        ok = *flag == 0;
-
-        // (10) outputs: o_i[c] = scale (a_i p^q_i[c] + D[c][i]), staged through shared memory (over the
-        // dead R^T tiles) so that global memory sees 16-byte stores of whole rows
-        if (ok) {
-            const int c = (warp & 3) * 32 + lane;
-            const int half = warp >> 2;
-            const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-            TOut *o_s = reinterpret_cast<TOut *>(smem + SM_RT_HI);   // [64][128] TOut: 16 or 32 KB
-#pragma unroll 1
-            for (int part = 0; part < 2; ++part) {
-                const int i0 = half * 32 + part * 16;
-                uint32_t pp[32], dd[16];
-                GDN_TMEM_LD32(trow + 2 * i0, pp);
-                GDN_TMEM_LD16(trow + 128 + i0, dd);
-                float ai[16];
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) ai[jj] = gab[i0 + jj].y;
-                tmem_wait_ld();
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) {
-                    const float out = p.scale * fmaf(ai[jj], __uint_as_float(pp[2 * jj + 1]), __uint_as_float(dd[jj]));
-                    store_from_float(o_s + (i0 + jj) * FV_D + c, out);
-                }
-            }
-        }
-        __syncthreads();
-        if (*flag == 0) {
-            constexpr int ROW_CHUNKS = FV_D * (int)sizeof(TOut) / 16;   // 16-byte pieces per output row
-            uint8_t *o = static_cast<uint8_t *>(p.o);
-            for (int idx = tid; idx < T * ROW_CHUNKS; idx += FV_THREADS) {
-                const int i = idx / ROW_CHUNKS, ck = idx % ROW_CHUNKS;
-                const uint4 val = *reinterpret_cast<const uint4 *>(smem + SM_RT_HI + (size_t)i * FV_D * sizeof(TOut) + ck * 16);
-                if (i >= n_prefix)   // the ancestors in front of a group belong to other groups' outputs
-                    *reinterpret_cast<uint4 *>(o + (((size_t)(base + node_of(i)) * p.h_v + h) * FV_D) * sizeof(TOut) + ck * 16) = val;
-            }
-        }
-    }
-    if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
-
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, FV_TMEM_COLS);
-}
-
-// Gate activations of the "scalars" stage (Section 3.4.2; Table 1 row "scalars"): the kernel takes either the
-// finished log-decay g and write strength beta, or the layer's raw gate inputs a, b, for which
-// g = -softplus(a) = -log(1 + e^a) and beta = sigmoid(b) are formed here (fp32, never rounded to the input type).
-__device__ __forceinline__ float gate_log_decay(uint32_t bf16_bits, bool raw)
-{
-    const float x = __uint_as_float(bf16_bits << 16);
-    if (!raw) return x;
-    return x > 0.f ? -(x + log1pf(expf(-x))) : -log1pf(expf(x));
-}
-__device__ __forceinline__ float gate_beta(uint32_t bf16_bits, bool raw)
-{
-    const float x = __uint_as_float(bf16_bits << 16);
-    if (!raw) return x;
-    const float e = expf(-fabsf(x));
-    return x >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
-}
-
-// Persistent form of the kernel above for trees that fit one CTA, with the optional fused commit.  The k/q tile
-// holds the k rows first and the q rows second (rows i and 64 + i), so P has p^k in columns 0..63 and p^q in
-// columns 64..127, and the Gram block needs only N = 64.
+// The k/q tile holds the k rows first and the q rows second (rows i and 64 + i), so P has p^k in columns 0..63 and
+// p^q in columns 64..127, and the Gram block needs only N = 64.
 // FUSED: Eq. 7 is replayed along the previous step's accepted path on the state tile while it sits in registers
 // -- per row c, s_c <- alpha s_c + k beta (v_c - alpha k.s_c), the eight lanes that share a row reducing k.s_c with
 // three shuffles -- the tile is written back as the only state write of the step, and the new tree is verified
@@ -756,9 +294,16 @@ __device__ __forceinline__ float gate_beta(uint32_t bf16_bits, bool raw)
 // its value is used.  The state tile is asked for at the top of the unit and is needed only after the Gram /
 // coefficient phases; the v rows land by TMA in an area that is free until the state operand is written.
 // SMALL (every tree of the call has at most 32 nodes): the R and output phases skip the 16-node pieces beyond the tree.
-template <typename TOut, bool FUSED, bool SMALL, bool PADDED>
+// GROUPED (trees of more than 64 nodes, cut into ancestor-closed groups by the plan kernel): a unit is (tree, value
+// head, group); it is verified as a virtual tree of the <= 15 proper ancestors of the group's first node followed by
+// the group's own nodes.  The rows of a virtual tree are not contiguous, so its k/q/v rows are gathered with
+// cp.async (completing on the same mbarriers as the TMA tiles otherwise), its tables come from the plan, and
+// outputs are stored for the group's own nodes only.  The five or so groups of a (tree, head) run on neighbouring
+// CTAs at about the same time, so the state tile crosses HBM once.
+template <typename TOut, bool FUSED, bool SMALL, bool PADDED, bool GROUPED>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const __grid_constant__ VerifyFastParams p)
 {
+    static_assert(!GROUPED || (!FUSED && !SMALL), "the grouped mode is verification only");
     extern __shared__ uint8_t fv_smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fv_smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
@@ -775,14 +320,15 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // carries all of it: warp 0 the projection MMA group, warp 1 the D group, warp 2 the Gram block of the unit to
     // come, warp 3 the TMA loads.  Every issuer commits its own MMAs to an mbarrier.
     constexpr int W_MMA_P = 0, W_MMA_D = 1, W_MMA_G = 2, W_TMA = 3;
+    auto tbl_thread_g = [&]() -> bool { return tid >= FV_T && tid < 2 * FV_T; };   // thread FV_T + i keeps node i's tables
 
     if (warp == 0) tmem_alloc(sbase + SM_TMEM, FV_TMEM_COLS);
     if (tid == 32) {
         mbar_init(mbar_g, 1);
         mbar_init(mbar_p, 1);
         mbar_init(mbar_d, 1);
-        mbar_init(mbar_kq, 1);
-        mbar_init(mbar_v, 1);
+        mbar_init(mbar_kq, GROUPED ? FV_THREADS : 1);   // gathered rows: every thread arrives once its copies have landed
+        mbar_init(mbar_v, GROUPED ? FV_THREADS : 1);
         *flag = 0;
     }
     tc_fence_before();
@@ -792,12 +338,13 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // Launched with programmatic stream serialization: everything above overlaps the tail of the kernel
     // in front (the tree-metadata kernel); nothing below may run before that kernel's writes are visible.
     // The first unit's state tile is an input of the call, not of that kernel: L2 is asked for it meanwhile.
+    const int G = GROUPED ? p.groups_per_tree : 1;   // units per state tile
     if (tid < 4 && (int)blockIdx.x < p.n_units)
-        prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
+        prefetch_l2_bulk(p.S0 + (size_t)((int)blockIdx.x / G) * FV_D * FV_D + (size_t)tid * 4096, 16384);
     // ... and for the rows of the first unit's tree.  Their place may depend on node_offsets[], which the kernel in
     // front may still be writing: the value read here only steers prefetches (clamped to the tensors), it is read
     // again behind the dependency wait before anything is computed from it.
-    if ((int)blockIdx.x < p.n_units && tid >= 128 && tid < 128 + FV_T) {
+    if (!GROUPED && (int)blockIdx.x < p.n_units && tid >= 128 && tid < 128 + FV_T) {
         const int ub = (int)blockIdx.x / p.h_v, uh = (int)blockIdx.x % p.h_v, uhk = uh / (p.h_v / p.h_qk);
         const int row = ((PADDED && p.t_pad) ? ub * p.t_pad : __ldg(p.node_offsets + ub)) + tid - 128;
         if (row >= 0 && row < p.total_nodes) {
@@ -813,7 +360,28 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 
     // unit -> (tree, head, first node, size); a unit whose node_offsets[] are inconsistent (reported) or whose tree
     // is empty is skipped.  parent[] itself is checked when the unit's tables are built.
-    auto decode = [&](int u, int &ub, int &uh, int &uhk, int &ubase, int &uT, int &upar) -> bool {
+    // The loads a decode needs are issued by decode_load() and looked at by decode() / decode_g() later (the unit after
+    // next is asked for at the top of a unit and decoded in its middle), so that no thread waits for them.
+    struct DecodeRaw { int lo, hi; uint2 gi; };
+    auto decode_load = [&](int u) -> DecodeRaw {
+        DecodeRaw r{0, 0, make_uint2(0u, 0u)};
+        if (u >= p.n_units) return r;
+        const int ub = (u / G) / p.h_v;
+        const int tree = (PADDED && p.t_pad) ? ub % p.n_trees : ub;
+        if constexpr (GROUPED) {
+            const int grp = u % G;
+            if (grp < GDN_MAX_GROUPS)
+                r.gi = __ldg(reinterpret_cast<const uint2 *>(p.group_info + ((size_t)tree * GDN_MAX_GROUPS + grp) * 4));
+            if (!(PADDED && p.t_pad)) r.lo = p.node_offsets[ub];
+        } else if (PADDED && p.t_pad) {
+            r.lo = p.n_nodes[tree];
+        } else {
+            r.lo = p.node_offsets[ub];
+            r.hi = p.node_offsets[ub + 1];
+        }
+        return r;
+    };
+    auto decode = [&](int u, const DecodeRaw &raw, int &ub, int &uh, int &uhk, int &ubase, int &uT, int &upar) -> bool {
         if (u >= p.n_units) return false;
         ub = u / p.h_v;
         uh = u % p.h_v;
@@ -822,12 +390,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if (PADDED && p.t_pad) {   // padded layout: rows of the slot, node count and parent[] row of its tree
             const int tree = ub % p.n_trees;
             ubase = ub * p.t_pad;
-            uT = p.n_nodes[tree];
+            uT = raw.lo;
             upar = tree * p.t_pad;
             off_ok = uT >= 0 && uT <= FV_T && uT <= p.t_pad;
         } else {
-            ubase = p.node_offsets[ub];
-            const int uend = p.node_offsets[ub + 1];
+            ubase = raw.lo;
+            const int uend = raw.hi;
             uT = uend - ubase;
             upar = ubase;
             off_ok = ubase >= 0 && uT >= 0 && uT <= FV_T && uT <= p.max_tree_nodes && uend <= p.total_nodes;
@@ -845,6 +413,95 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             return true;
         }
         return tree_good;
+    };
+    // GROUPED: unit -> (tree, head, group).  pb = first row of the tree in the plan's tables, g0 = first depth-first
+    // position of the group, n_prefix = proper ancestors of its first node (virtual indices 0 .. n_prefix - 1),
+    // first = node at position g0; ident: a tree of at most 64 nodes inside a grouped call (identity numbering).
+    struct GroupX { int pb, g0, n_prefix, first; bool ident; };
+    auto decode_g = [&](int u, const DecodeRaw &raw, int &ub, int &uh, int &uhk, int &ubase, int &uT, GroupX &gx) -> bool {
+        if (u >= p.n_units) return false;
+        const int tile = u / G;
+        ub = tile / p.h_v;
+        uh = tile % p.h_v;
+        uhk = uh / (p.h_v / p.h_qk);
+        if (PADDED && p.t_pad) {
+            ubase = ub * p.t_pad;
+            gx.pb = (ub % p.n_trees) * p.t_pad;
+        } else {
+            ubase = raw.lo;   // checked by the plan kernel (a tree with bad offsets has no groups)
+            gx.pb = ubase;
+        }
+        const uint2 gi = raw.gi;
+        const int own = (int)(gi.x >> 16);
+        if (own == 0) return false;   // no such group (or the plan rejected the tree, which it has reported)
+        gx.g0 = (int)(gi.x & 0xFFFFu);
+        gx.ident = (gi.y & 0xFFFFu) == 0xFFFFu;
+        gx.n_prefix = gx.ident ? 0 : (int)(gi.y & 0xFFFFu);
+        gx.first = (int)(gi.y >> 16);
+        uT = gx.n_prefix + own;
+        return true;
+    };
+    // node id of virtual index u (< T) of a group, from the plan
+    auto vnode_global = [&](const GroupX &gx, int u) -> int {
+        if (gx.ident) return u;
+        if (u < gx.n_prefix) return (int)__ldg(p.anc16 + (size_t)(gx.pb + gx.first) * p.anc_stride + u);
+        return (int)__ldg(p.dfs_node + gx.pb + gx.g0 + u - gx.n_prefix);
+    };
+    // table entries of virtual index tnode: node id, depth, root path in virtual indices
+    auto lookup_tables_g = [&](const GroupX &gx, int uT, int &node, int &d, uint4 &row) {
+        node = 0;
+        d = 0;
+        row = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+        if (tbl_thread_g() && tid - FV_T < uT) {
+            const int t = tid - FV_T;
+            if (gx.ident) {
+                node = t;
+                d = p.depth[gx.pb + t];
+                row = __ldg(reinterpret_cast<const uint4 *>(p.anc8 + (size_t)(gx.pb + t) * 16));
+            } else if (t < gx.n_prefix) {   // an ancestor of the group's first node: its path is 0..t
+                node = vnode_global(gx, t);
+                d = t + 1;
+                const uint32_t all[4] = {0x03020100u, 0x07060504u, 0x0B0A0908u, 0x0F0E0D0Cu};
+                uint32_t w[4];
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int keep = d - 4 * q4;   // bytes of this word that are on the path
+                    w[q4] = keep >= 4 ? all[q4] : keep <= 0 ? 0xFFFFFFFFu : (all[q4] | (0xFFFFFFFFu << (8 * keep)));
+                }
+                row = make_uint4(w[0], w[1], w[2], w[3]);
+            } else {
+                const int r = gx.pb + gx.g0 + t - gx.n_prefix;
+                node = (int)__ldg(p.dfs_node + r);
+                d = p.dfs_depth[r];
+                row = __ldg(reinterpret_cast<const uint4 *>(p.dfs_anc8 + (size_t)r * 16));
+            }
+        }
+    };
+    auto put_tables_g = [&](int uT, int tb, int node, int d, uint4 row, uint32_t g_bits, uint32_t be_bits) {
+        if (tbl_thread_g()) {
+            const int t = tid - FV_T;
+            const bool on = t < uT;
+            (smem + SM_DEPTH + tb * SM_TABLE_STRIDE)[t] = (uint8_t)(on ? d : 0);
+            *reinterpret_cast<uint4 *>(smem + SM_ANC + tb * SM_TABLE_STRIDE + t * 16) = row;
+            reinterpret_cast<float4 *>(smem + SM_GAB + tb * SM_TABLE_STRIDE)[t] =
+                make_float4(0.f, 0.f, on ? gate_beta(be_bits, PADDED && p.raw_gates) : 0.f,
+                            on ? gate_log_decay(g_bits, PADDED && p.raw_gates) : 0.f);
+            reinterpret_cast<uint16_t *>(smem + SM_VN2)[tb * FV_T + t] = (uint16_t)(on ? node : 0);
+        }
+    };
+    // k and q rows of a virtual tree -> B operand tile (rows beyond the tree zero-filled): thread (r16, c16) fetches
+    // 16-byte piece c16 of the rows r16, r16 + 16, r16 + 32, r16 + 48, whose node ids it is handed
+    auto gather_kq = [&](int uhk, int ubase, int uT, const int (&nid)[4]) {
+        const int r16 = tid >> 4, c16 = tid & 15;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int u = r16 + 16 * j;
+            const bool valid = u < uT;
+            const size_t off = ((size_t)(ubase + (valid ? nid[j] : 0)) * p.h_qk + uhk) * FV_D + c16 * 8;
+            cp_async_16(sbase + SM_B_KQ + sw128_offset(u, c16), p.k + off, valid);
+            cp_async_16(sbase + SM_B_KQ + sw128_offset(FV_T + u, c16), p.q + off, valid);
+        }
+        cp_async_arrive_on(mbar_kq);
     };
     // k and q rows -> B operand tile by TMA: four 64-row x 64-column boxes (k and q, either K half), 128-byte
     // swizzled, completing on mbar_kq.  A box always spans 64 nodes: rows beyond the tree belong to the next tree
@@ -1035,6 +692,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     auto issue_gram = [&](uint32_t kq_parity) {
         if (warp == W_MMA_G && elect_one()) {
             if (!mbar_wait_bounded(mbar_kq, kq_parity)) *flag = 1;
+            if constexpr (GROUPED) fence_proxy_async();   // rows written by cp.async become visible to the tensor core
             tc_fence_after();
             const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
             constexpr uint32_t id = idesc_bf16(128, 64);   // B = the 64 k rows
@@ -1052,62 +710,104 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // ... and whatever is launched behind this grid with the same attribute (the next call's tree-metadata kernel,
     // which itself waits for this grid to complete before it reads or writes anything) may be made resident now.
     asm volatile("griddepcontrol.launch_dependents;");
-    bool cur_ok = decode(blockIdx.x, b, h, hk, base, T, par0);
-    bool par_bad = false;
-    if (cur_ok) {
-        issue_kq(b, hk, base, T);
-        fetch_path(b, 0);
-        par_bad = load_parent(par0, T, 0);
-    }
-    __syncthreads();
-    if (cur_ok) load_tables(h, base, T, 0, par_bad);
-    __syncthreads();
-    if (cur_ok) {
-        path_decay(0);
-        fetch_path_kv(h, hk, 0);
-        path_scalars_direct(h, 0);
-        issue_gram(0);
+    GroupX gx{0, 0, 0, 0, true}, ngx{0, 0, 0, 0, true};
+    int unit0 = blockIdx.x;
+    bool cur_ok;
+    if constexpr (GROUPED) {
+        // units without a group (the grid is sized for the largest tree) are stepped over here and at the top of
+        // every unit, so that the loop below only ever sees real ones
+        cur_ok = decode_g(unit0, decode_load(unit0), b, h, hk, base, T, gx);
+        while (!cur_ok && (unit0 += gridDim.x) < p.n_units) cur_ok = decode_g(unit0, decode_load(unit0), b, h, hk, base, T, gx);
+        int t_node, t_d;
+        uint4 t_row;
+        lookup_tables_g(gx, T, t_node, t_d, t_row);
+        uint32_t gb = 0, bb = 0;
+        if (cur_ok && tbl_thread_g() && tid - FV_T < T) {
+            const size_t n = (size_t)(base + t_node);
+            gb = __ldg(reinterpret_cast<const unsigned short *>(p.g) + n * p.h_v + h);
+            bb = __ldg(reinterpret_cast<const unsigned short *>(p.beta) + n * p.h_v + h);
+        }
+        if (cur_ok) put_tables_g(T, 0, t_node, t_d, t_row, gb, bb);
+        __syncthreads();
+        if (cur_ok) {
+            path_decay(0);
+            const uint16_t *vn = reinterpret_cast<const uint16_t *>(smem + SM_VN2);
+            const int nid[4] = {vn[tid >> 4], vn[(tid >> 4) + 16], vn[(tid >> 4) + 32], vn[(tid >> 4) + 48]};
+            gather_kq(hk, base, T, nid);
+            issue_gram(0);
+        }
+    } else {
+        cur_ok = decode(blockIdx.x, decode_load(blockIdx.x), b, h, hk, base, T, par0);
+        bool par_bad = false;
+        if (cur_ok) {
+            issue_kq(b, hk, base, T);
+            fetch_path(b, 0);
+            par_bad = load_parent(par0, T, 0);
+        }
+        __syncthreads();
+        if (cur_ok) load_tables(h, base, T, 0, par_bad);
+        __syncthreads();
+        if (cur_ok) {
+            path_decay(0);
+            fetch_path_kv(h, hk, 0);
+            path_scalars_direct(h, 0);
+            issue_gram(0);
+        }
     }
     int done_units = 0;
 #pragma unroll 1
-    for (int unit = blockIdx.x, iter = 0; unit < p.n_units; unit += gridDim.x, ++iter) {
+    for (int unit = unit0, iter = 0; unit < p.n_units; ++iter) {
     const bool unit_ok = cur_ok;
     const uint32_t par = (uint32_t)(done_units & 1);   // every barrier completes once per processed unit
     int nb = 0, nh = 0, nhk = 0, nbase = 0, nT = 0, npar0 = 0;
-    const bool next_ok = decode(unit + gridDim.x, nb, nh, nhk, nbase, nT, npar0);
+    int next_unit = unit + gridDim.x;
+    bool next_ok = false;
+    const DecodeRaw next_raw = decode_load(next_unit);   // looked at in the middle of the unit (stage 1)
+    auto decode_next = [&]() {
+        if constexpr (GROUPED) {
+            next_ok = decode_g(next_unit, next_raw, nb, nh, nhk, nbase, nT, ngx);
+            while (!next_ok && (next_unit += gridDim.x) < p.n_units)   // a unit without a group: look further on
+                next_ok = decode_g(next_unit, decode_load(next_unit), nb, nh, nhk, nbase, nT, ngx);
+        } else {
+            next_ok = decode(next_unit, next_raw, nb, nh, nhk, nbase, nT, npar0);
+        }
+    };
     float4 *gab = reinterpret_cast<float4 *>(smem + SM_GAB + (iter & 1) * SM_TABLE_STRIDE);
     uint8_t *anc_s = smem + SM_ANC + (iter & 1) * SM_TABLE_STRIDE;
     uint8_t *depth_s = smem + SM_DEPTH + (iter & 1) * SM_TABLE_STRIDE;
-    if (!unit_ok) {   // nothing to compute here: only keep the pipeline fed
-        __syncthreads();
-        bool nbad = false;
-        if (next_ok) {
-            issue_kq(nb, nhk, nbase, nT);
-            nbad = load_parent(npar0, nT, (iter + 1) & 1);
-            fetch_path(nb, (iter + 1) & 1);
-        }
-        __syncthreads();
-        if (next_ok) load_tables(nh, nbase, nT, (iter + 1) & 1, nbad);
-        __syncthreads();
-        if (next_ok) {
-            path_decay((iter + 1) & 1);
-            fetch_path_kv(nh, nhk, (iter + 1) & 1);
-            path_scalars_direct(nh, (iter + 1) & 1);
-            issue_gram(par);   // no unit was processed in between: the tile's barrier phase is this one
+    if (!unit_ok) {   // nothing to compute here: only keep the pipeline fed (never taken in the grouped mode)
+        decode_next();
+        if constexpr (!GROUPED) {
+            __syncthreads();
+            bool nbad = false;
+            if (next_ok) {
+                issue_kq(nb, nhk, nbase, nT);
+                nbad = load_parent(npar0, nT, (iter + 1) & 1);
+                fetch_path(nb, (iter + 1) & 1);
+            }
+            __syncthreads();
+            if (next_ok) load_tables(nh, nbase, nT, (iter + 1) & 1, nbad);
+            __syncthreads();
+            if (next_ok) {
+                path_decay((iter + 1) & 1);
+                fetch_path_kv(nh, nhk, (iter + 1) & 1);
+                path_scalars_direct(nh, (iter + 1) & 1);
+                issue_gram(par);   // no unit was processed in between: the tile's barrier phase is this one
+            }
         }
         b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
+        unit = next_unit;
         continue;
     }
     // L2 warming for this CTA's next unit, in slices at phase boundaries
-    const int u_next = unit + gridDim.x;
     auto warm_l2_state = [&](int slice) {
-        if (tid == 96 && u_next < p.n_units)
-            prefetch_l2_bulk(p.S0 + (size_t)u_next * FV_D * FV_D + (size_t)slice * 4096, 16384);
+        if (tid == 96 && next_unit < p.n_units)
+            prefetch_l2_bulk(p.S0 + (size_t)(next_unit / G) * FV_D * FV_D + (size_t)slice * 4096, 16384);
     };
 
     // a tree whose parent[] was rejected while its tables were built runs as a tree of no nodes: nothing of it
     // is stored (fused form: its accepted path of the previous step is committed all the same)
-    if (bad_s[iter & 1]) {
+    if (!GROUPED && bad_s[iter & 1]) {
         T = 0;
         if (tid < FV_T) depth_s[tid] = 0;
     }
@@ -1123,8 +823,19 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
         }
     }
+    const uint16_t *vnode_s = reinterpret_cast<const uint16_t *>(smem + SM_VN2) + (iter & 1) * FV_T;
     // this tree's v rows: one TMA box into an area that stays free until the state operand is written
-    if (warp == W_TMA && elect_one()) {
+    if constexpr (GROUPED) {   // ... gathered row by row (rows beyond the virtual tree zero-filled)
+        const int r16 = tid >> 4, c16 = tid & 15;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int u = r16 + 16 * j;
+            const bool valid = u < T;
+            cp_async_16(sbase + SM_VE + u * 256 + c16 * 16,
+                        p.v + ((size_t)(base + (valid ? (int)vnode_s[u] : 0)) * p.h_v + h) * FV_D + c16 * 8, valid);
+        }
+        cp_async_arrive_on(mbar_v);
+    } else if (warp == W_TMA && elect_one()) {
         mbar_expect_tx(mbar_v, FV_T * FV_D * 2);
         tma_load_3d(sbase + SM_VE, &p.tm_v, 0, h, base, mbar_v);
     }
@@ -1257,7 +968,21 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     int q_pp0 = 0, q_len = 0, q_pb = 0, q_pT = 0, q_ppar = 0, q_n = -1, q_par = -2;
     unsigned short q_g = 0, q_be = 0;
     bool q_shape_ok = false, q_mine = false;
-    if (next_ok) {
+    decode_next();
+    int t_node = 0, t_d = 0;                 // grouped mode: table entries of virtual index tnode, and the
+    uint4 t_row = make_uint4(0u, 0u, 0u, 0u);   // node ids of the four rows this thread gathers
+    int nid[4] = {0, 0, 0, 0};
+    if constexpr (GROUPED) {
+        if (next_ok) {
+            lookup_tables_g(ngx, nT, t_node, t_d, t_row);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int u = (tid >> 4) + 16 * j;
+                nid[j] = u < nT ? vnode_global(ngx, u) : 0;
+            }
+        }
+    }
+    if (!GROUPED && next_ok) {
         if (tbl_thread && tnode < nT) {
             const int n = nbase + tnode;
             t_par = __ldg(p.parent + npar0 + tnode);
@@ -1347,7 +1072,17 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         // the root path) over the state operand
         // the k/q tile is dead: start on the next unit of this CTA (its k/q tile, its tables), to be
         // consumed after the loop comes round
-        if (next_ok) {
+        if constexpr (GROUPED) {
+            if (next_ok) {
+                gather_kq(nhk, nbase, nT, nid);
+                if (tbl_thread && tnode < nT) {   // stage 3: the gates of the node found in stage 1
+                    const size_t n = (size_t)(nbase + t_node);
+                    t_g = __ldg(reinterpret_cast<const unsigned short *>(p.g) + n * p.h_v + nh);
+                    t_be = __ldg(reinterpret_cast<const unsigned short *>(p.beta) + n * p.h_v + nh);
+                }
+            }
+        }
+        if (!GROUPED && next_ok) {
             issue_kq(nb, nhk, nbase, nT);
             // stage 3: parent[] of the next tree is staged for the walk behind the next CTA barrier; the parents of
             // the path entries are asked for
@@ -1490,7 +1225,11 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
 
         // stage 5, while the tensor core works: the next unit's tables (depth, root paths) from the staged parent[]
-        if (next_ok) walk_tables(nT, (iter + 1) & 1, t_g, t_be, t_bad);
+        if constexpr (GROUPED) {
+            if (next_ok) put_tables_g(nT, (iter + 1) & 1, t_node, t_d, t_row, t_g, t_be);
+        } else {
+            if (next_ok) walk_tables(nT, (iter + 1) & 1, t_g, t_be, t_bad);
+        }
         if (!mbar_wait_bounded(mbar_d, par)) *flag = 1;
         tc_fence_after();
 
@@ -1549,7 +1288,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             for (int idx = tid; idx < T * ROW_CHUNKS; idx += FV_THREADS) {
                 const int i = idx / ROW_CHUNKS, ck = idx % ROW_CHUNKS;
                 const uint4 val = *reinterpret_cast<const uint4 *>(smem + SM_RT_HI + (size_t)i * FV_D * sizeof(TOut) + ck * 16);
-                *reinterpret_cast<uint4 *>(o + (((size_t)(base + i) * p.h_v + h) * FV_D) * sizeof(TOut) + ck * 16) = val;
+                if constexpr (GROUPED) {   // the ancestors in front of a group belong to other groups' outputs
+                    if (i >= gx.n_prefix)
+                        *reinterpret_cast<uint4 *>(o + (((size_t)(base + vnode_s[i]) * p.h_v + h) * FV_D) * sizeof(TOut) + ck * 16) = val;
+                } else {
+                    *reinterpret_cast<uint4 *>(o + (((size_t)(base + i) * p.h_v + h) * FV_D) * sizeof(TOut) + ck * 16) = val;
+                }
             }
         }
     }
@@ -1557,6 +1301,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (!unit_done_ok) break;   // a bounded wait expired: stop, report, release
     if (next_ok) issue_gram((uint32_t)(done_units & 1));   // the next unit's Gram block, as soon as its tile is there
     b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
+    gx = ngx;
+    unit = next_unit;
     }   // unit loop
 
     if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
@@ -1600,43 +1346,49 @@ bool make_row_tensor_map(CUtensorMap *tm, const void *ptr, int n_rows, int heads
 template <typename TOut, bool FUSED, bool GROUPED>
 cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, cudaStream_t stream)
 {
+    // persistent CTAs, two per SM, pipelined across units
+    VerifyFastParams pt = p;
+    const bool padded = p.t_pad != 0;   // the padded layout and the on-chip gate activations share an instantiation
+    void (*kernel)(const VerifyFastParams);
     if constexpr (GROUPED) {
-        cudaError_t e = cudaFuncSetAttribute(verify_sm100_kernel<TOut, GROUPED>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
-        if (e != cudaSuccess) return e;
-        const int grid = s.n_seq * s.h_v * p.groups_per_tree;
-        verify_sm100_kernel<TOut, GROUPED><<<grid, FV_THREADS, SM_ALLOC, stream>>>(p);
+        // trees of more than 64 nodes: a unit is one ancestor-closed group of a (tree, head); rows are gathered
+        pt.n_units = p.n_units * p.groups_per_tree;
+        kernel = padded ? verify_sm100_persistent_kernel<TOut, false, false, true, true>
+                        : verify_sm100_persistent_kernel<TOut, false, false, false, true>;
     } else {
-        // trees that fit one CTA: persistent CTAs, two per SM, pipelined across units
-        VerifyFastParams pt = p;
+        // trees that fit one CTA: TMA tiles of the packed row tensors
         if (!make_row_tensor_map(&pt.tm_k, p.k, s.total_nodes, s.h_qk, 64, true) ||
             !make_row_tensor_map(&pt.tm_q, p.q, s.total_nodes, s.h_qk, 64, true) ||
             !make_row_tensor_map(&pt.tm_v, p.v, s.total_nodes, s.h_v, FV_D, false))
             return cudaErrorNotSupported;
         const bool small = s.max_tree_nodes <= 32;
-        // the instantiation with the projection cache (read and/or written) exists for the fused form only
-        const bool padded = p.t_pad != 0;   // the padded layout and the on-chip gate activations share an instantiation
-        auto kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true, false>
-                            : verify_sm100_persistent_kernel<TOut, FUSED, false, false>;
+        kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true, false, false>
+                       : verify_sm100_persistent_kernel<TOut, FUSED, false, false, false>;
         if (padded)
-            kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true, true>
-                           : verify_sm100_persistent_kernel<TOut, FUSED, false, true>;
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
-        if (e != cudaSuccess) return e;
-        const int grid = p.n_units < p.prefetch_dist ? p.n_units : p.prefetch_dist;
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3((unsigned)grid);
-        cfg.blockDim = dim3(FV_THREADS);
-        cfg.dynamicSmemBytes = SM_ALLOC;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kernel, pt);
+            kernel = small ? verify_sm100_persistent_kernel<TOut, FUSED, true, true, false>
+                           : verify_sm100_persistent_kernel<TOut, FUSED, false, true, false>;
     }
-    return cudaGetLastError();
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
+    if (e != cudaSuccess) return e;
+    int grid = pt.n_units < p.prefetch_dist ? pt.n_units : p.prefetch_dist;
+    if constexpr (GROUPED) {
+        // A CTA walks the units blockIdx.x, blockIdx.x + grid, ...; the group index is the unit index modulo the groups
+        // per tree, and the last groups of a tree may not exist.  With a grid size coprime to the groups per tree every
+        // CTA meets every group index equally often, so the missing groups are spread evenly over the CTAs.
+        auto gcd = [](int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; };
+        while (grid > 1 && gcd(grid, p.groups_per_tree) != 1) --grid;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(FV_THREADS);
+    cfg.dynamicSmemBytes = SM_ALLOC;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, pt);
 }
 
 VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *q, const void *k, const void *v,
@@ -1653,12 +1405,12 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     p.beta = static_cast<const __nv_bfloat16 *>(beta);
     p.node_offsets = node_offsets; p.o = o;
     p.n_seq = s.n_seq; p.total_nodes = s.total_nodes; p.max_tree_nodes = s.max_tree_nodes; p.max_depth = s.max_depth;
-    p.tree_ok = plan.tree_ok; p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
-    p.groups_per_tree = (s.max_tree_nodes + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;   // upper bound; a CTA
-                                                                                            // without a group leaves at once
+    p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
+    // upper bound of the groups of a tree; a unit without a group is stepped over
+    p.groups_per_tree = s.max_tree_nodes <= FV_T ? 1 : (s.max_tree_nodes + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;
     p.anc_stride = s.max_depth;
     p.anc16 = plan.anc; p.dfs_node = plan.dfs_node; p.dfs_depth = plan.dfs_depth; p.dfs_anc8 = plan.dfs_anc8;
-    p.group_start = plan.group_start;
+    p.group_info = plan.group_info;
     return p;
 }
 
@@ -1700,6 +1452,17 @@ cudaError_t launch_commit_verify_sm100_padded(const gdn_shape_t &s, int n_trees,
     return launch_fast_typed<float, true, false>(s, p, stream);
 }
 
+cudaError_t launch_verify_sm100_planned(const gdn_shape_t &s, int n_trees, bool raw_gates, const float *S0,
+                                        const void *q, const void *k, const void *v, const void *g, const void *beta,
+                                        const PlanPtrs &plan, void *o, int32_t *status_dev, cudaStream_t stream)
+{
+    if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
+    VerifyFastParams p = make_params(s, S0, q, k, v, g, beta, nullptr, o, plan, status_dev);
+    p.t_pad = s.max_tree_nodes; p.n_trees = n_trees; p.raw_gates = raw_gates ? 1 : 0;
+    if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false, true>(s, p, stream);
+    return launch_fast_typed<float, false, true>(s, p, stream);
+}
+
 bool verify_sm100_supported(const gdn_shape_t &s)
 {
     return s.d_k == FV_D && s.d_v == FV_D && s.in_dtype == GDN_BF16 && s.max_tree_nodes <= GDN_GROUPED_MAX_NODES &&
@@ -1716,7 +1479,7 @@ cudaError_t launch_verify_sm100(const gdn_shape_t &s, const float *S0, const voi
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
     VerifyFastParams p = make_params(s, S0, q, k, v, g, beta, node_offsets, o, plan, status_dev);
     p.parent = parent;
-    if (s.max_tree_nodes > FV_T) {
+    if (!verify_sm100_single_group(s)) {
         if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false, true>(s, p, stream);
         return launch_fast_typed<float, false, true>(s, p, stream);
     }

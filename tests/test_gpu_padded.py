@@ -192,3 +192,144 @@ def test_padded_rejections(tl):
     ref = _oracle_verify(w)
     for s in (0, 2):
         tl.assert_close_per_head(o[s, :20], ref[s, :20], np.array([0, 20]), f"good tree, slot {s}", bf16_out=True)
+
+
+# ----------------------------------------------------------------------------- plan as an object of its own (any T)
+def _plan(d, w):
+    import torch
+    import paper_2607_06763_b200 as gdn
+    nbytes = gdn.gdn_tree_plan_bytes(d.shape, w.n_trees)
+    assert nbytes > 0
+    plan = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    rc = gdn.gdn_tree_plan(d.shape, w.n_trees, d.parent, d.n_nodes, plan, d.status)
+    assert rc == 0, gdn.gdn_status_string(rc)
+    return plan
+
+
+@pytest.mark.parametrize("raw_gates", [False, True])
+@pytest.mark.parametrize("t_pad,sizes,n_layers,out_dtype", [(64, (64, 37), 3, synth.BF16), (128, (128, 70, 5), 2, synth.F32),
+                                                            (256, (256, 131), 2, synth.BF16), (200, (66,), 3, synth.F32),
+                                                            (512, (512,), 1, synth.BF16)])
+def test_verify_planned(tl, t_pad, sizes, n_layers, out_dtype, raw_gates):
+    """Trees of up to 512 rows per slot, several slots per tree, rows beyond the node count poisoned; one plan serves
+    two verification calls (the plan is read-only for them)."""
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(sum(sizes) + t_pad)
+    w = synth.padded_case(1200 + t_pad + len(sizes), _trees(rng, sizes), n_layers, t_pad, raw_gates, out_dtype=out_dtype)
+    d = PaddedDevice(w)
+    plan = _plan(d, w)
+    S_before = d.S0.clone()
+    ref = _oracle_verify(w)
+    for rep in range(2):
+        d.o.fill_(7.0)
+        rc = gdn.gdn_tree_verify_planned(d.shape, w.n_trees, raw_gates, d.S0, d.q, d.k, d.v, d.g_in, d.beta_in, plan, d.o,
+                                         d.status)
+        assert rc == 0, gdn.gdn_status_string(rc)
+        assert d.status_value() == 0
+        assert bool((d.S0 == S_before).all())
+        _assert_outputs(tl, d, ref, f"verify_planned T{t_pad} raw={raw_gates} call {rep}")
+
+
+@pytest.mark.parametrize("raw_gates", [False, True])
+def test_commit_padded_then_verify_planned(tl, raw_gates):
+    """A decode step on 256-row slots: the accepted paths of the previous trees are committed, then the new trees
+    are verified against the advanced states; one tree commits nothing."""
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(1301)
+    prev_trees = _trees(rng, (256, 90))
+    paths = [synth.longest_path(prev_trees[0]), np.zeros(0, np.int32)]
+    prev = synth.padded_case(1310, prev_trees, 2, 256, raw_gates, paths=paths)
+    new = synth.padded_case(1311, _trees(rng, (200, 256)), 2, 256, raw_gates)
+    dp, dn = PaddedDevice(prev), PaddedDevice(new)
+    S = dp.S0.clone()
+    rc = gdn.gdn_tree_commit_padded(dp.shape, prev.n_trees, raw_gates, S, dp.k, dp.v, dp.g_in, dp.beta_in, dp.parent,
+                                    dp.n_nodes, dp.path, dp.path_len, dn.status)
+    assert rc == 0, gdn.gdn_status_string(rc)
+    plan = _plan(dn, new)
+    rc = gdn.gdn_tree_verify_planned(dn.shape, new.n_trees, raw_gates, S, dn.q, dn.k, dn.v, dn.g_in, dn.beta_in, plan,
+                                     dn.o, dn.status)
+    assert rc == 0, gdn.gdn_status_string(rc)
+    assert dn.status_value() == 0
+    S_ref = _oracle_commit(prev, prev.S0.astype(np.float64))
+    tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what="commit_padded state")
+    for s in range(prev.n_slots):
+        if prev.path_len[s % prev.n_trees] == 0:
+            assert bool((S[s] == dp.S0[s]).all())
+    _assert_outputs(tl, dn, _oracle_verify(new, S_ref), f"commit_padded + verify_planned raw={raw_gates}")
+
+
+def test_planned_step_captured_once_replayed_with_another_tree(tl):
+    """plan + commit + verify of 128-row slots in one CUDA graph; trees, node counts, paths and tensors are then
+    overwritten in place and the graph replayed."""
+    import torch
+    import paper_2607_06763_b200 as gdn
+    from paper_2607_06763_b200.binding import to_device
+    rng = np.random.default_rng(1401)
+    steps = []
+    for i, (ps, ns) in enumerate((((128,), (128,)), ((40,), (99,)), ((128,), (65,)))):
+        prev = synth.padded_case(1410 + i, _trees(rng, ps), 3, 128, True)
+        new = synth.padded_case(1420 + i, _trees(rng, ns), 3, 128, True)
+        steps.append((prev, new))
+    dp, dn = PaddedDevice(steps[0][0]), PaddedDevice(steps[0][1])
+    S = dp.S0.clone()
+    plan = torch.empty(gdn.gdn_tree_plan_bytes(dn.shape, 1), dtype=torch.uint8, device="cuda")
+
+    def call(stream):
+        assert gdn.gdn_tree_plan(dn.shape, 1, dn.parent, dn.n_nodes, plan, dn.status, stream) == 0
+        assert gdn.gdn_tree_commit_padded(dp.shape, 1, True, S, dp.k, dp.v, dp.g_in, dp.beta_in, dp.parent, dp.n_nodes,
+                                          dp.path, dp.path_len, dn.status, stream) == 0
+        assert gdn.gdn_tree_verify_planned(dn.shape, 1, True, S, dn.q, dn.k, dn.v, dn.g_in, dn.beta_in, plan, dn.o,
+                                           dn.status, stream) == 0
+
+    call(None)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        call(torch.cuda.current_stream())
+    for prev, new in steps:
+        for dev, w in ((dp, prev), (dn, new)):
+            for n in ("q", "k", "v", "g_in", "beta_in", "parent", "n_nodes", "path", "path_len"):
+                getattr(dev, n).copy_(to_device(getattr(w, n)))
+            dev.w = w
+        S.copy_(to_device(prev.S0))
+        dn.o.fill_(7.0)
+        graph.replay()
+        assert dn.status_value() == 0
+        S_ref = _oracle_commit(prev, prev.S0.astype(np.float64))
+        tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what="planned graph replay state")
+        _assert_outputs(tl, dn, _oracle_verify(new, S_ref), "planned graph replay")
+
+
+def test_planned_rejections(tl):
+    import torch
+    import paper_2607_06763_b200 as gdn
+    rng = np.random.default_rng(15)
+    w = synth.padded_case(1500, _trees(rng, (100, 128)), 2, 128, False)
+    d = PaddedDevice(w)
+    plan = torch.empty(gdn.gdn_tree_plan_bytes(d.shape, 2), dtype=torch.uint8, device="cuda")
+    assert gdn.gdn_tree_plan(d.shape, 3, d.parent, d.n_nodes, plan, d.status) == -2       # 4 slots, 3 trees
+    assert gdn.gdn_tree_plan(d.shape, 2, d.parent, d.n_nodes, plan[:1024], d.status) == -10   # plan too small
+    assert gdn.gdn_tree_plan(d.shape, 2, None, d.n_nodes, plan, d.status) == -1
+    # device-side: a parent that points forward in tree 1 -> its slots are skipped, tree 0 is verified
+    d.parent[1, 70] = 90
+    assert gdn.gdn_tree_plan(d.shape, 2, d.parent, d.n_nodes, plan, d.status) == 0
+    assert d.status_value() == -7
+    d.status.zero_()
+    rc = gdn.gdn_tree_verify_planned(d.shape, 2, False, d.S0, d.q, d.k, d.v, d.g_in, d.beta_in, plan, d.o, d.status)
+    assert rc == 0 and d.status_value() == 0
+    o = d.o_host()
+    assert np.all(o[1] == 7.0) and np.all(o[3] == 7.0), "slots of the rejected tree must stay untouched"
+    ref = _oracle_verify(w)
+    for s in (0, 2):
+        tl.assert_close_per_head(o[s, :100], ref[s, :100], np.array([0, 100]), f"good tree, slot {s}", bf16_out=True)
+    # a path that does not start at a root: the commit reports it and leaves the states of that tree's slots alone
+    S = d.S0.clone()
+    d.path[0, :2] = torch.tensor([5, 0], dtype=torch.int32)
+    d.path_len[0] = 2
+    rc = gdn.gdn_tree_commit_padded(d.shape, 2, False, S, d.k, d.v, d.g_in, d.beta_in, d.parent, d.n_nodes, d.path,
+                                    d.path_len, d.status)
+    assert rc == 0
+    assert d.status_value() == -9
+    assert bool((S[0] == d.S0[0]).all()) and bool((S[2] == d.S0[2]).all())
+    assert not bool((S[1] == d.S0[1]).all()), "the other tree's path is committed all the same"
