@@ -206,7 +206,7 @@ def run_reference(args, w: synth.Workload):
 
 def workload_config(w: synth.Workload, args):
     sizes = np.diff(w.node_offsets)
-    return {"workload": args.workload, "mode": getattr(args, "mode", "fused"),
+    return {"workload": args.workload, "mode": getattr(args, "mode", "fused"), "layout": getattr(args, "layout", "ragged"),
             "launch": "cuda graph replay" if getattr(args, "graph", False) else "api call per step", "name": w.name,
             "n_seq_or_layer_slots": w.n_seq, "h_qk": w.h_qk, "h_v": w.h_v,
             "d_k": w.d_k, "d_v": w.d_v, "tree_nodes": int(sizes.max()), "total_nodes": w.total_nodes,
@@ -223,20 +223,26 @@ def report(args):
                                                           if wl.startswith("sweep_")]
     runs += [(wl, "verify", "recurrent") for wl in WORKLOADS if wl.startswith("sweep_")]
     runs += [("stack48_T64", "separate", "ours")]
-    for wl, mode, impl in runs:
+    runs = [r + ("ragged",) for r in runs]
+    # the shape-static entry points on the padded layout (slots sharing one full-size tree)
+    runs += [(wl, "fused", "ours", "padded") for wl in ("stack48_T64", "stack48_T256", "layer_T64")]
+    runs += [(wl, "verify", "ours", "padded") for wl in WORKLOADS if wl.startswith("sweep_")]
+    for wl, mode, impl, layout in runs:
         cmd = [sys.executable, os.path.abspath(__file__), "--workload", wl, "--mode", mode, "--impl", impl, "--steps",
                str(args.steps), "--warmup", str(args.warmup), "--min-time", str(args.min_time), "--no-e2e"]
+        if layout != "ragged":
+            cmd += ["--layout", layout]
         if wl != "stack48_T64" or mode != "fused":
             cmd += ["--oracle-slots", "4"]
         res = subprocess.run(cmd, capture_output=True, text=True)
         line = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
         if res.returncode != 0 or not line:
-            rows.append(f"| {wl} | {mode} | {impl} | failed (rc {res.returncode}) | | | | | |")
+            rows.append(f"| {wl} | {mode} | {impl}{'' if layout == 'ragged' else ', ' + layout} | failed (rc {res.returncode}) | | | | | |")
             continue
         d = json.loads(line[-1])
         cpu = d.get("cpu_baseline", {})
         rows.append("| {} | {} | {} | {:.1f} | {:.1f} | {:.0f} | {:.3f} | {:.3g} | {} |".format(
-            wl, mode, impl, d["ms_per_step"] * 1e3, d["timing"]["ms_per_step_fastest_region"] * 1e3,
+            wl, mode, impl if layout == "ragged" else impl + ", " + layout, d["ms_per_step"] * 1e3, d["timing"]["ms_per_step_fastest_region"] * 1e3,
             d["step_roofline"]["achieved_gbs"], d["step_roofline"]["frac_of_" + src], d["value"],
             "{:.3g} ({} cores)".format(cpu["value"], cpu["cores"]) if cpu else ""))
     print(f"| workload | mode | impl | us/step (median region) | us/step (fastest) | GB/s | fraction of {src} "
@@ -262,6 +268,10 @@ def main():
     ap.add_argument("--mode", default="fused", choices=["fused", "separate", "verify"],
                     help="fused: one gdn_tree_commit_verify call per step; separate: gdn_tree_verify + gdn_tree_commit; "
                          "verify: gdn_tree_verify alone (no commit; for kernel comparisons)")
+    ap.add_argument("--layout", default="ragged", choices=["ragged", "padded"],
+                    help="padded: the shape-static entry points on the dense [slots, T, heads, d] layout with the tree given "
+                         "once for all layer slots (workloads whose slots share one full-size tree); trees of more than 64 "
+                         "nodes then run as gdn_tree_plan once per step + gdn_tree_commit_padded + gdn_tree_verify_planned")
     ap.add_argument("--path-len", type=int, default=16,
                     help="workload stack48_T64_deep: nodes on the accepted path (0..16)")
     ap.add_argument("--graph", action="store_true",
@@ -317,6 +327,50 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
 
+    padded = args.layout == "padded"
+    if padded:
+        # every slot carries the same full-size tree, so the ragged packing of the workload already is the padded
+        # layout [slots, T, heads, d]; the tree, its node count and its accepted path are given once
+        T = int(w.node_offsets[1])
+        same = all(np.array_equal(w.parent[b * T:(b + 1) * T], w.parent[:T]) for b in range(w.n_seq))
+        assert same and w.total_nodes == w.n_seq * T and args.impl == "ours", "--layout padded: one shared full-size tree"
+        plen = int(w.path_offsets[1])
+        path1 = np.zeros((1, shape.max_depth), np.int32)
+        path1[0, :plen] = w.path[:plen]
+        p_parent, p_nodes = to_dev(w.parent[:T].reshape(1, T).copy()), to_dev(np.array([T], np.int32))
+        p_path, p_len = to_dev(path1), to_dev(np.array([plen], np.int32))
+        plan_bytes = gdn.gdn_tree_plan_bytes(shape, 1)
+        plan = torch.empty(max(plan_bytes, 256), dtype=torch.uint8, device="cuda")
+        small = T <= 64
+
+    def step_verify_padded(d, stream=stream):
+        if small:
+            rc = gdn.gdn_tree_verify_padded(shape, 1, False, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], p_parent,
+                                            p_nodes, d["o"], status, stream)
+        else:
+            rc = gdn.gdn_tree_plan(shape, 1, p_parent, p_nodes, plan, status, stream)
+            assert rc == 0, gdn.gdn_status_string(rc)
+            rc = gdn.gdn_tree_verify_planned(shape, 1, False, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], plan,
+                                             d["o"], status, stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+
+    def step_fused_padded(d, stream=stream):
+        if small:
+            rc = gdn.gdn_tree_commit_verify_padded(shape, 1, False, d["S0"], T, d["k"], d["v"], d["g"], d["beta"],
+                                                   p_parent, p_nodes, p_path, p_len, d["q"], d["k"], d["v"], d["g"],
+                                                   d["beta"], p_parent, p_nodes, d["o"], status, stream)
+            assert rc == 0, gdn.gdn_status_string(rc)
+            return
+        # the decode step of a larger tree: metadata once, commit of the previous path, verification
+        rc = gdn.gdn_tree_plan(shape, 1, p_parent, p_nodes, plan, status, stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+        rc = gdn.gdn_tree_commit_padded(shape, 1, False, d["S0"], d["k"], d["v"], d["g"], d["beta"], p_parent, p_nodes,
+                                        p_path, p_len, status, stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+        rc = gdn.gdn_tree_verify_planned(shape, 1, False, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], plan,
+                                         d["o"], status, stream)
+        assert rc == 0, gdn.gdn_status_string(rc)
+
     def step_verify(d, stream=stream):
         if args.impl == "recurrent":
             rc = gdn.gdn_tree_verify_recurrent(shape, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], d["parent"],
@@ -342,6 +396,9 @@ def main():
         assert rc == 0, gdn.gdn_status_string(rc)
 
     step = {"fused": step_fused, "separate": step_separate, "verify": step_verify}[args.mode]
+    if padded:
+        assert args.mode in ("fused", "verify"), "--layout padded: modes fused and verify"
+        step = step_fused_padded if args.mode == "fused" else step_verify_padded
 
     def barrier():
         if world > 1:
@@ -352,7 +409,17 @@ def main():
         step(sets[i % n_sets])
     barrier()
     graphs = None
-    if args.graph and args.mode == "fused":
+    if args.graph and args.mode == "fused" and padded:
+        graphs, side = [], torch.cuda.Stream()
+        for d in sets:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                step_fused_padded(d, torch.cuda.current_stream())
+            graphs.append(g)
+        for i in range(args.warmup):
+            graphs[i % n_sets].replay()
+        barrier()
+    elif args.graph and args.mode == "fused":
         # one captured step per buffer set (the launches of a call, dependent-launch edge included)
         graphs, side = [], torch.cuda.Stream()
         for d in sets:
@@ -490,7 +557,7 @@ def main():
             dom_bytes = sbytes if fused else vbytes
             dom_ms = ms_per_step if args.mode != "separate" else split[0]
         else:   # larger trees: tree plan + grouped verify kernel; the fused call runs commit and verify back to back
-            kernel_name = "verify_sm100_kernel<grouped>"
+            kernel_name = "verify_sm100_persistent_kernel<grouped>"
             launches_per_step = {"fused": 3, "separate": 3, "verify": 2}[args.mode]
             dom_bytes = vbytes
             dom_ms = None if args.mode == "fused" else (ms_per_step if args.mode == "verify" else split[0])

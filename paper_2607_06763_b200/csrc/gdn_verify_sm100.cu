@@ -959,6 +959,24 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     __syncthreads();
     tc_fence_after();
     warm_l2_state(2);
+    // (5) P = S0.[k;q]^T (hi then lo) on the tensor core, issued before anything else; meanwhile the loads of stage 1
+    // and the back-substitution below
+    if (warp == W_MMA_P && elect_one()) {
+        const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
+        const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
+        constexpr uint32_t id = idesc_bf16(128, 128);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+            umma_bf16(tmem, a_hi + adv, b_kq + adv, id, ks > 0);
+        }
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+            umma_bf16(tmem, a_lo + adv, b_kq + adv, id, 1);
+        }
+        umma_commit(mbar_p);
+    }
     // The next unit's tables and accepted path are fetched in stages, each load issued one phase before its
     // value is used, so that no global-memory latency is paid in front of a barrier.
     // stage 1: table entries of node `tid` and the path bounds (registers only)
@@ -1009,23 +1027,6 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
     }
 
-    // (5) P = S0.[k;q]^T (hi then lo) on the tensor core; meanwhile the back-substitution below
-    if (warp == W_MMA_P && elect_one()) {
-        const uint64_t a_hi = smem_desc_sw128(sbase + SM_A_HI), a_lo = smem_desc_sw128(sbase + SM_A_LO);
-        const uint64_t b_kq = smem_desc_sw128(sbase + SM_B_KQ);
-        constexpr uint32_t id = idesc_bf16(128, 128);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-            umma_bf16(tmem, a_hi + adv, b_kq + adv, id, ks > 0);
-        }
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t adv = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-            umma_bf16(tmem, a_lo + adv, b_kq + adv, id, 1);
-        }
-        umma_commit(mbar_p);
-    }
     // (6) z^T = y^T (I + X_path)^-1 by back-substitution over the root path (column-oriented: once z_l is
     // final, subtract z_l X(n_l, n_t) from every z_t, t < l).  Four threads per node, thread sq of the quad
     // owning path positions 4 sq .. 4 sq + 3; z stays in registers until the k/q tile can be overwritten.
@@ -1376,7 +1377,7 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
         // per tree, and the last groups of a tree may not exist.  With a grid size coprime to the groups per tree every
         // CTA meets every group index equally often, so the missing groups are spread evenly over the CTAs.
         auto gcd = [](int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; };
-        while (grid > 1 && gcd(grid, p.groups_per_tree) != 1) --grid;
+        while (grid < pt.n_units && grid > 1 && gcd(grid, p.groups_per_tree) != 1) --grid;   // (one unit per CTA: no walk)
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
