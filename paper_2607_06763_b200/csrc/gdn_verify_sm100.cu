@@ -814,15 +814,20 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // (1) state tile loads: a warp instruction covers four rows; the eight lanes of a row each own one
     // 16-byte bf16 piece of either K half.  Needed only after the Gram / coefficient phases.
     float4 x[4][4];   // [row i][kh*2 + half]
-    {
+    // The load/store unit takes a while to accept 64 KB of requests: the tile is asked for in pieces -- a half at the
+    // top and a half behind the Gram copy when the commit needs the tile right after the coefficients; a quarter at
+    // the top, a quarter behind the Gram wait and a half behind the Gram copy otherwise -- so that the threads are
+    // not held at the top of the unit for all of it.
+    auto load_state_rows = [&](int i0, int i1) {
         const float *S = p.S0 + (size_t)(b * p.h_v + h) * FV_D * FV_D;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = i0; i < i1; ++i) {
             const float *src = S + (size_t)(warp * 16 + i * 4 + r4) * FV_D + l8 * 8;
 #pragma unroll
             for (int kh = 0; kh < 2; ++kh) ldg_v8(src + kh * 64, x[i][kh * 2 + 0], x[i][kh * 2 + 1]);
         }
-    }
+    };
+    load_state_rows(0, FUSED ? 2 : 1);
     const uint16_t *vnode_s = reinterpret_cast<const uint16_t *>(smem + SM_VN2) + (iter & 1) * FV_T;
     // this tree's v rows: one TMA box into an area that stays free until the state operand is written
     if constexpr (GROUPED) {   // ... gathered row by row (rows beyond the virtual tree zero-filled)
@@ -850,6 +855,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (!mbar_wait_bounded(mbar_g, par)) *flag = 1;
     tc_fence_after();
     __syncthreads();
+    if constexpr (!FUSED) load_state_rows(1, 2);
     warm_l2_state(0);
     if (*flag == 0) {
         // k-columns of the Gram block out of tensor memory, into the (still unused) state-operand area
@@ -870,6 +876,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                         make_uint4(ra[4 * c4], ra[4 * c4 + 1], ra[4 * c4 + 2], ra[4 * c4 + 3]);
             }
         }
+        load_state_rows(2, 4);
         tc_fence_before();
         __syncthreads();
         warm_l2_state(1);
