@@ -29,7 +29,7 @@ __device__ __forceinline__ void stg_v8(float *p, const float4 &a, const float4 &
 
 // Eq. 7 replayed along an accepted path of L >= 1 nodes on the tile x (Section 3.4: the delayed commit is a short
 // recurrence).  Per row c: s_c <- alpha s_c + k beta (v_c - alpha k.s_c); the eight lanes that share a row reduce
-// k.s_c with three shuffles, the four rows of a thread advance together.
+// k.s_c by shuffles (the four rows of a thread folded into one butterfly), the four rows of a thread advance together.
 //   pks, pvs : the path's k and v rows in shared memory, bf16 [L][128]
 //   ab_path  : per step (A_t = decay of the path up to and including step t, beta_t, alpha_t, 1 / A_t)
 __device__ __forceinline__ void replay_path_on_tile(float4 (&x)[4][4], int L, const uint16_t *pks, const uint16_t *pvs,
@@ -70,18 +70,35 @@ __device__ __forceinline__ void replay_path_on_tile(float4 (&x)[4][4], int L, co
             }
             dot[i] = acc.x + acc.y;
         }
-#pragma unroll
-        for (int m = 1; m < 8; m <<= 1)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) dot[i] += __shfl_xor_sync(0xffffffffu, dot[i], m);
+        // Reduction over the eight lanes of a row group with the four rows folded as it goes: after the exchange
+        // with lane ^ 1 a lane keeps two rows, after lane ^ 2 one, after lane ^ 4 it holds the complete k.s of row
+        // my_i (4 shuffles instead of 12); it forms w of that row alone and the four w come back by shuffles.
+        const bool b0 = (l8 & 1) != 0, b1 = (l8 & 2) != 0;
+        const int my_i = (b0 ? 2 : 0) + (b1 ? 1 : 0);
+        float a0, a1;
+        {
+            const float s0 = b0 ? dot[0] : dot[2], s1 = b0 ? dot[1] : dot[3];
+            const float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
+            a0 = (b0 ? dot[2] : dot[0]) + r0;
+            a1 = (b0 ? dot[3] : dot[1]) + r1;
+        }
+        float d1 = (b1 ? a1 : a0) + __shfl_xor_sync(0xffffffffu, b1 ? a0 : a1, 2);
+        d1 += __shfl_xor_sync(0xffffffffu, d1, 4);
+        const int my_row = warp * 16 + my_i * 4 + r4;
+        const float vc = __uint_as_float((uint32_t)pvs[t * GDN_TILE_D + my_row] << 16);
+        // scaled form: x holds s / A_t and w = beta_t (v / A_t - k.s~); plain form: w = beta_t (v - alpha_t k.s)
+        const float w_mine = scaled ? ab.y * fmaf(vc, ab.w, -d1) : ab.y * (vc - ab.z * d1);
+        const int g8 = (r4 << 3);   // first lane of this row group
+        float wv[4];
+        wv[0] = __shfl_sync(0xffffffffu, w_mine, g8 | 0);
+        wv[1] = __shfl_sync(0xffffffffu, w_mine, g8 | 2);
+        wv[2] = __shfl_sync(0xffffffffu, w_mine, g8 | 1);
+        wv[3] = __shfl_sync(0xffffffffu, w_mine, g8 | 3);
         if (scaled) {
-            // x holds s / A_t: s~ += k beta_t (v / A_t - k.s~), one packed FMA per pair
+            // s~ += k w, one packed FMA per pair
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int row = warp * 16 + i * 4 + r4;
-                const float vc = __uint_as_float((uint32_t)pvs[t * GDN_TILE_D + row] << 16);
-                const float w = ab.y * fmaf(vc, ab.w, -dot[i]);
-                const float2 w2 = make_float2(w, w);
+                const float2 w2 = make_float2(wv[i], wv[i]);
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
                     const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, make_float2(x[i][q4].x, x[i][q4].y));
@@ -92,10 +109,7 @@ __device__ __forceinline__ void replay_path_on_tile(float4 (&x)[4][4], int L, co
         } else {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int row = warp * 16 + i * 4 + r4;
-                const float vc = __uint_as_float((uint32_t)pvs[t * GDN_TILE_D + row] << 16);
-                const float w = ab.y * (vc - ab.z * dot[i]);
-                const float2 w2 = make_float2(w, w), a2 = make_float2(ab.z, ab.z);
+                const float2 w2 = make_float2(wv[i], wv[i]), a2 = make_float2(ab.z, ab.z);
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
                     const float2 lo = __ffma2_rn(kf2[q4 * 2 + 0], w2, __fmul2_rn(a2, make_float2(x[i][q4].x, x[i][q4].y)));
