@@ -335,9 +335,9 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // warp-uniform by construction
-    // Launched with programmatic stream serialization: everything above overlaps the tail of the kernel
-    // in front (the tree-metadata kernel); nothing below may run before that kernel's writes are visible.
-    // The first unit's state tile is an input of the call, not of that kernel: L2 is asked for it meanwhile.
+    // Launched with programmatic stream serialization: everything above overlaps the tail of the kernel in front
+    // (the previous call, or the plan kernel); nothing that is computed from memory may run before that kernel's
+    // writes are visible.  L2 can be asked for the first unit's state tile meanwhile (a prefetch consumes nothing).
     const int G = GROUPED ? p.groups_per_tree : 1;   // units per state tile
     if (tid < 4 && (int)blockIdx.x < p.n_units)
         prefetch_l2_bulk(p.S0 + (size_t)((int)blockIdx.x / G) * FV_D * FV_D + (size_t)tid * 4096, 16384);
@@ -707,8 +707,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 
     int b = 0, h = 0, hk = 0, base = 0, T = 0, par0 = 0;
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // ... and whatever is launched behind this grid with the same attribute (the next call's tree-metadata kernel,
-    // which itself waits for this grid to complete before it reads or writes anything) may be made resident now.
+    // ... and whatever is launched behind this grid with the same attribute (the next call's kernel, which itself
+    // waits for this grid to complete before it reads or writes anything) may be made resident now.
     asm volatile("griddepcontrol.launch_dependents;");
     GroupX gx{0, 0, 0, 0, true}, ngx{0, 0, 0, 0, true};
     int unit0 = blockIdx.x;

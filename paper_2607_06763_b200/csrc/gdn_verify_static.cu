@@ -1,6 +1,6 @@
 // gdn_tree_verify_static: tree verification for callers that must not allocate device memory.
 //
-// gdn_tree_verify needs device scratch (per-node tree metadata and the cached solve result) and
+// gdn_tree_verify needs device scratch (per-node tree metadata and the solve result of the general kernel) and
 // asks its caller to provide it.  Some callers of this library have no way to get such a buffer:
 // a serving process that handed all free device memory to its own pool at start-up and would see
 // cudaMalloc fail, a decode loop in which cudaMalloc's implicit device-wide synchronisation would
