@@ -685,6 +685,18 @@ extern "C" int gdn_tree_commit_verify_host(const gdn_shape_t *shape, float *S_h,
         const size_t row_o = (size_t)s.h_v * s.d_v * osz, slot_state = (size_t)s.h_v * s.d_v * s.d_k * sizeof(float);
         auto at = [](const void *base, size_t off) { return static_cast<const char *>(base) + off; };
         auto atw = [](void *base, size_t off) { return static_cast<char *>(base) + off; };
+        // the small tensors (gates, trees, paths: a percent of the bytes) go up whole in front of the first group: a
+        // copy costs a few microseconds whatever its size, and per group only the large slices are left
+        {
+            cudaStream_t si = pipe->s_in;
+            GDN_CUDA_TRY(cudaMemcpyAsync(g, g_h, t.gb, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(beta, beta_h, t.gb, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(parent, parent_h, t.parent, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(gp, g_prev_h, tp.gb, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(bp, beta_prev_h, tp.gb, cudaMemcpyHostToDevice, si));
+            if (parent_p) GDN_CUDA_TRY(cudaMemcpyAsync(parent_p, parent_prev_h, tp.parent, cudaMemcpyHostToDevice, si));
+            GDN_CUDA_TRY(cudaMemcpyAsync(path, path_h, path_bytes, cudaMemcpyHostToDevice, si));
+        }
         for (int i = 0; i < G; ++i) {
             const int b0 = first[i], nb = first[i + 1] - b0;
             const size_t n0 = (size_t)node_offsets_h[b0], nn = (size_t)node_offsets_h[b0 + nb] - n0;
@@ -695,15 +707,8 @@ extern "C" int gdn_tree_commit_verify_host(const gdn_shape_t *shape, float *S_h,
             GDN_CUDA_TRY(cudaMemcpyAsync(atw(q, n0 * row_qk), at(q_h, n0 * row_qk), nn * row_qk, cudaMemcpyHostToDevice, si));
             GDN_CUDA_TRY(cudaMemcpyAsync(atw(k, n0 * row_qk), at(k_h, n0 * row_qk), nn * row_qk, cudaMemcpyHostToDevice, si));
             GDN_CUDA_TRY(cudaMemcpyAsync(atw(v, n0 * row_v), at(v_h, n0 * row_v), nn * row_v, cudaMemcpyHostToDevice, si));
-            GDN_CUDA_TRY(cudaMemcpyAsync(atw(g, n0 * row_gb), at(g_h, n0 * row_gb), nn * row_gb, cudaMemcpyHostToDevice, si));
-            GDN_CUDA_TRY(cudaMemcpyAsync(atw(beta, n0 * row_gb), at(beta_h, n0 * row_gb), nn * row_gb, cudaMemcpyHostToDevice, si));
-            GDN_CUDA_TRY(cudaMemcpyAsync(parent + n0, parent_h + n0, nn * sizeof(int32_t), cudaMemcpyHostToDevice, si));
             GDN_CUDA_TRY(cudaMemcpyAsync(atw(kp, m0 * row_qk), at(k_prev_h, m0 * row_qk), mm * row_qk, cudaMemcpyHostToDevice, si));
             GDN_CUDA_TRY(cudaMemcpyAsync(atw(vp, m0 * row_v), at(v_prev_h, m0 * row_v), mm * row_v, cudaMemcpyHostToDevice, si));
-            GDN_CUDA_TRY(cudaMemcpyAsync(atw(gp, m0 * row_gb), at(g_prev_h, m0 * row_gb), mm * row_gb, cudaMemcpyHostToDevice, si));
-            GDN_CUDA_TRY(cudaMemcpyAsync(atw(bp, m0 * row_gb), at(beta_prev_h, m0 * row_gb), mm * row_gb, cudaMemcpyHostToDevice, si));
-            if (parent_p) GDN_CUDA_TRY(cudaMemcpyAsync(parent_p + m0, parent_prev_h + m0, mm * sizeof(int32_t), cudaMemcpyHostToDevice, si));
-            if (pl) GDN_CUDA_TRY(cudaMemcpyAsync(path + p0, path_h + p0, pl * sizeof(int32_t), cudaMemcpyHostToDevice, si));
             GDN_CUDA_TRY(cudaEventRecord(pipe->in[i], si));
             GDN_CUDA_TRY(cudaStreamWaitEvent(stream, pipe->in[i], 0));
             gdn_shape_t gs = s;
