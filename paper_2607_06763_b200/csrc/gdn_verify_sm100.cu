@@ -360,16 +360,45 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 
     // unit -> (tree, head, first node, size); a unit whose node_offsets[] are inconsistent (reported) or whose tree
     // is empty is skipped.  parent[] itself is checked when the unit's tables are built.
+    // A CTA walks the units blockIdx.x, blockIdx.x + gridDim.x, ...: (tile, slot, head, group) of a unit follow from
+    // those of the unit before by additions and carries, so that the integer divisions by the head and group counts
+    // (a few dozen instructions each, for every thread) are paid once per CTA and not once per unit.
+    struct Cursor { int u, b, h, grp; };
+    const int ratio = p.h_v / p.h_qk;
+    const int ratio_shift = (ratio & (ratio - 1)) == 0 ? 31 - __clz(ratio) : -1;
+    auto hk_of = [&](int h_) -> int { return ratio_shift >= 0 ? h_ >> ratio_shift : h_ / ratio; };
+    auto tree_of = [&](int b_) -> int { return p.n_trees == 1 ? 0 : b_ % p.n_trees; };   // padded layout only
+    const int step_grp = (int)gridDim.x % G, step_tile = (int)gridDim.x / G;
+    const int step_h = step_tile % p.h_v, step_b = step_tile / p.h_v;
+    auto cursor_at = [&](int u) -> Cursor {
+        Cursor c;
+        c.u = u;
+        const int tile = u / G;
+        c.grp = u % G;
+        c.b = tile / p.h_v;
+        c.h = tile % p.h_v;
+        return c;
+    };
+    auto advance = [&](Cursor &c) {
+        c.u += (int)gridDim.x;
+        c.grp += step_grp;
+        const int carry = c.grp >= G ? 1 : 0;
+        c.grp -= carry ? G : 0;
+        c.h += step_h + carry;
+        const int carry_h = c.h >= p.h_v ? 1 : 0;
+        c.h -= carry_h ? p.h_v : 0;
+        c.b += step_b + carry_h;
+    };
     // The loads a decode needs are issued by decode_load() and looked at by decode() / decode_g() later (the unit after
     // next is asked for at the top of a unit and decoded in its middle), so that no thread waits for them.
     struct DecodeRaw { int lo, hi; uint2 gi; };
-    auto decode_load = [&](int u) -> DecodeRaw {
+    auto decode_load = [&](const Cursor &c) -> DecodeRaw {
         DecodeRaw r{0, 0, make_uint2(0u, 0u)};
-        if (u >= p.n_units) return r;
-        const int ub = (u / G) / p.h_v;
-        const int tree = (PADDED && p.t_pad) ? ub % p.n_trees : ub;
+        if (c.u >= p.n_units) return r;
+        const int ub = c.b;
+        const int tree = (PADDED && p.t_pad) ? tree_of(ub) : ub;
         if constexpr (GROUPED) {
-            const int grp = u % G;
+            const int grp = c.grp;
             if (grp < GDN_MAX_GROUPS)
                 r.gi = __ldg(reinterpret_cast<const uint2 *>(p.group_info + ((size_t)tree * GDN_MAX_GROUPS + grp) * 4));
             if (!(PADDED && p.t_pad)) r.lo = p.node_offsets[ub];
@@ -381,14 +410,14 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         }
         return r;
     };
-    auto decode = [&](int u, const DecodeRaw &raw, int &ub, int &uh, int &uhk, int &ubase, int &uT, int &upar) -> bool {
-        if (u >= p.n_units) return false;
-        ub = u / p.h_v;
-        uh = u % p.h_v;
-        uhk = uh / (p.h_v / p.h_qk);
+    auto decode = [&](const Cursor &c, const DecodeRaw &raw, int &ub, int &uh, int &uhk, int &ubase, int &uT, int &upar) -> bool {
+        if (c.u >= p.n_units) return false;
+        ub = c.b;
+        uh = c.h;
+        uhk = hk_of(uh);
         bool off_ok;
         if (PADDED && p.t_pad) {   // padded layout: rows of the slot, node count and parent[] row of its tree
-            const int tree = ub % p.n_trees;
+            const int tree = tree_of(ub);
             ubase = ub * p.t_pad;
             uT = raw.lo;
             upar = tree * p.t_pad;
@@ -418,15 +447,14 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // position of the group, n_prefix = proper ancestors of its first node (virtual indices 0 .. n_prefix - 1),
     // first = node at position g0; ident: a tree of at most 64 nodes inside a grouped call (identity numbering).
     struct GroupX { int pb, g0, n_prefix, first; bool ident; };
-    auto decode_g = [&](int u, const DecodeRaw &raw, int &ub, int &uh, int &uhk, int &ubase, int &uT, GroupX &gx) -> bool {
-        if (u >= p.n_units) return false;
-        const int tile = u / G;
-        ub = tile / p.h_v;
-        uh = tile % p.h_v;
-        uhk = uh / (p.h_v / p.h_qk);
+    auto decode_g = [&](const Cursor &c, const DecodeRaw &raw, int &ub, int &uh, int &uhk, int &ubase, int &uT, GroupX &gx) -> bool {
+        if (c.u >= p.n_units) return false;
+        ub = c.b;
+        uh = c.h;
+        uhk = hk_of(uh);
         if (PADDED && p.t_pad) {
             ubase = ub * p.t_pad;
-            gx.pb = (ub % p.n_trees) * p.t_pad;
+            gx.pb = tree_of(ub) * p.t_pad;
         } else {
             ubase = raw.lo;   // checked by the plan kernel (a tree with bad offsets has no groups)
             gx.pb = ubase;
@@ -589,7 +617,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 int *slot = reinterpret_cast<int *>(smem + SM_PATH + ps * SM_PATH_SLOT);
                 int pp0, len, pb = 0, pT = 0, ppar = 0;   // len 0 leaves the state alone
                 if (PADDED && p.t_pad) {
-                    const int tree = ub % p.n_trees;
+                    const int tree = tree_of(ub);
                     pp0 = tree * p.path_stride;
                     len = p.path_len[tree];
                     pb = ub * p.pt_pad;
@@ -711,13 +739,13 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // waits for this grid to complete before it reads or writes anything) may be made resident now.
     asm volatile("griddepcontrol.launch_dependents;");
     GroupX gx{0, 0, 0, 0, true}, ngx{0, 0, 0, 0, true};
-    int unit0 = blockIdx.x;
+    Cursor ucur = cursor_at((int)blockIdx.x);
     bool cur_ok;
     if constexpr (GROUPED) {
         // units without a group (the grid is sized for the largest tree) are stepped over here and at the top of
         // every unit, so that the loop below only ever sees real ones
-        cur_ok = decode_g(unit0, decode_load(unit0), b, h, hk, base, T, gx);
-        while (!cur_ok && (unit0 += gridDim.x) < p.n_units) cur_ok = decode_g(unit0, decode_load(unit0), b, h, hk, base, T, gx);
+        cur_ok = decode_g(ucur, decode_load(ucur), b, h, hk, base, T, gx);
+        while (!cur_ok && (advance(ucur), ucur.u < p.n_units)) cur_ok = decode_g(ucur, decode_load(ucur), b, h, hk, base, T, gx);
         int t_node, t_d;
         uint4 t_row;
         lookup_tables_g(gx, T, t_node, t_d, t_row);
@@ -737,7 +765,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             issue_gram(0);
         }
     } else {
-        cur_ok = decode(blockIdx.x, decode_load(blockIdx.x), b, h, hk, base, T, par0);
+        cur_ok = decode(ucur, decode_load(ucur), b, h, hk, base, T, par0);
         bool par_bad = false;
         if (cur_ok) {
             issue_kq(b, hk, base, T);
@@ -756,20 +784,21 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     }
     int done_units = 0;
 #pragma unroll 1
-    for (int unit = unit0, iter = 0; unit < p.n_units; ++iter) {
+    for (int iter = 0; ucur.u < p.n_units; ++iter) {
     const bool unit_ok = cur_ok;
     const uint32_t par = (uint32_t)(done_units & 1);   // every barrier completes once per processed unit
     int nb = 0, nh = 0, nhk = 0, nbase = 0, nT = 0, npar0 = 0;
-    int next_unit = unit + gridDim.x;
+    Cursor ncur = ucur;
+    advance(ncur);
     bool next_ok = false;
-    const DecodeRaw next_raw = decode_load(next_unit);   // looked at in the middle of the unit (stage 1)
+    const DecodeRaw next_raw = decode_load(ncur);   // looked at in the middle of the unit (stage 1)
     auto decode_next = [&]() {
         if constexpr (GROUPED) {
-            next_ok = decode_g(next_unit, next_raw, nb, nh, nhk, nbase, nT, ngx);
-            while (!next_ok && (next_unit += gridDim.x) < p.n_units)   // a unit without a group: look further on
-                next_ok = decode_g(next_unit, decode_load(next_unit), nb, nh, nhk, nbase, nT, ngx);
+            next_ok = decode_g(ncur, next_raw, nb, nh, nhk, nbase, nT, ngx);
+            while (!next_ok && (advance(ncur), ncur.u < p.n_units))   // a unit without a group: look further on
+                next_ok = decode_g(ncur, decode_load(ncur), nb, nh, nhk, nbase, nT, ngx);
         } else {
-            next_ok = decode(next_unit, next_raw, nb, nh, nhk, nbase, nT, npar0);
+            next_ok = decode(ncur, next_raw, nb, nh, nhk, nbase, nT, npar0);
         }
     };
     float4 *gab = reinterpret_cast<float4 *>(smem + SM_GAB + (iter & 1) * SM_TABLE_STRIDE);
@@ -796,13 +825,13 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
             }
         }
         b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
-        unit = next_unit;
+        ucur = ncur;
         continue;
     }
     // L2 warming for this CTA's next unit, in slices at phase boundaries
     auto warm_l2_state = [&](int slice) {
-        if (tid == 96 && next_unit < p.n_units)
-            prefetch_l2_bulk(p.S0 + (size_t)(next_unit / G) * FV_D * FV_D + (size_t)slice * 4096, 16384);
+        if (tid == 96 && ncur.u < p.n_units)
+            prefetch_l2_bulk(p.S0 + (size_t)(ncur.b * p.h_v + ncur.h) * FV_D * FV_D + (size_t)slice * 4096, 16384);
     };
 
     // a tree whose parent[] was rejected while its tables were built runs as a tree of no nodes: nothing of it
@@ -1017,7 +1046,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         if constexpr (FUSED) {
             if (warp == 4) {
                 if (PADDED && p.t_pad) {   // (stage 2 takes differences: hand it begin / end pairs)
-                    const int tree = nb % p.n_trees;
+                    const int tree = tree_of(nb);
                     q_pp0 = tree * p.path_stride;
                     q_len = q_pp0 + p.path_len[tree];
                     q_pb = nb * p.pt_pad;
@@ -1310,7 +1339,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if (next_ok) issue_gram((uint32_t)(done_units & 1));   // the next unit's Gram block, as soon as its tile is there
     b = nb; h = nh; hk = nhk; base = nbase; T = nT; cur_ok = next_ok;
     gx = ngx;
-    unit = next_unit;
+    ucur = ncur;
     }   // unit loop
 
     if (*flag != 0 && tid == 0) report_status(p.status_dev, GDN_ERR_TIMEOUT);
