@@ -333,3 +333,50 @@ def test_planned_rejections(tl):
     assert d.status_value() == -9
     assert bool((S[0] == d.S0[0]).all()) and bool((S[2] == d.S0[2]).all())
     assert not bool((S[1] == d.S0[1]).all()), "the other tree's path is committed all the same"
+
+
+# ----------------------------------------------------------------------------- full-size workloads in the padded layout
+@pytest.mark.parametrize("cfg", [5, 2])
+def test_full_size_stack_through_the_padded_entry_points(tl, cfg):
+    """The 48-slot stacks of the benchmark (64- and 256-node trees, every slot carrying the same full-size tree, so
+    that their ragged packing already is the padded layout) through the shape-static entry points in the launch
+    configuration bench.py --layout padded times: commit of the accepted path, then verification, whole workload
+    against the oracle."""
+    import torch
+    import paper_2607_06763_b200 as gdn
+    from paper_2607_06763_b200.binding import to_device
+    from oracle import gdn_oracle as orc
+    w = synth.config(cfg, 1)
+    T = int(w.node_offsets[1])
+    assert w.total_nodes == w.n_seq * T
+    shape = gdn.GdnShape.from_workload(w)
+    d = {n: to_device(getattr(w, n)) for n in ("S0", "q", "k", "v", "g", "beta")}
+    plen = int(w.path_offsets[1])
+    path1 = np.zeros((1, shape.max_depth), np.int32)
+    path1[0, :plen] = w.path[:plen]
+    parent1, nodes1 = to_device(w.parent[:T].reshape(1, T).copy()), to_device(np.array([T], np.int32))
+    path_d, len_d = to_device(path1), to_device(np.array([plen], np.int32))
+    o = torch.zeros((w.total_nodes, w.h_v, w.d_v), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    S = d["S0"].clone()
+    if T <= 64:
+        rc = gdn.gdn_tree_commit_verify_padded(shape, 1, False, S, T, d["k"], d["v"], d["g"], d["beta"], parent1, nodes1,
+                                               path_d, len_d, d["q"], d["k"], d["v"], d["g"], d["beta"], parent1, nodes1,
+                                               o, status)
+        assert rc == 0, gdn.gdn_status_string(rc)
+    else:
+        plan = torch.empty(gdn.gdn_tree_plan_bytes(shape, 1), dtype=torch.uint8, device="cuda")
+        assert gdn.gdn_tree_plan(shape, 1, parent1, nodes1, plan, status) == 0
+        assert gdn.gdn_tree_commit_padded(shape, 1, False, S, d["k"], d["v"], d["g"], d["beta"], parent1, nodes1, path_d,
+                                          len_d, status) == 0
+        assert gdn.gdn_tree_verify_planned(shape, 1, False, S, d["q"], d["k"], d["v"], d["g"], d["beta"], plan, o,
+                                           status) == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    S_ref = orc.commit(w.S0.astype(np.float64), w.f64("k"), w.f64("v"), w.f64("g"), w.f64("beta"), w.parent,
+                       w.node_offsets, w.path, w.path_offsets)
+    o_ref = orc.verify(S_ref, w.f64("q"), w.f64("k"), w.f64("v"), w.f64("g"), w.f64("beta"), w.parent, w.node_offsets,
+                       w.scale)
+    tl.assert_state_close(S.cpu().numpy().astype(np.float64), S_ref, what=f"padded full-size cfg{cfg} state")
+    tl.assert_close_per_head(o.float().cpu().numpy().astype(np.float64), o_ref, w.node_offsets,
+                             f"padded full-size cfg{cfg}", bf16_out=True)
