@@ -11,7 +11,7 @@ namespace gdn {
 
 namespace {
 
-constexpr int PLAN_THREADS = 128;
+constexpr int PLAN_THREADS = 256;
 
 __global__ void __launch_bounds__(PLAN_THREADS)
 plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
