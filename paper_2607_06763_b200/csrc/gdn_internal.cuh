@@ -25,16 +25,20 @@ namespace gdn {
 // (64 - n_prefix, i.e. at least GDN_GROUP_MIN_NODES).
 //   group_start uint16[n_seq][GDN_MAX_GROUPS + 1]  first position of group k of tree b; entries behind the
 //                                          last group hold the tree's size
-//   group_info uint16[n_seq][GDN_MAX_GROUPS][4]    per group (first position, own nodes, n_prefix, node id at the
-//                                          first position); own nodes = 0 behind the last group.  A tree of at
-//                                          most 64 nodes is its own single group (0, T, 0xFFFF, 0): identity
-//                                          numbering, tables in depth / anc8
+//   unit_count int32 [1]                   number of groups over all trees (zeroed in front of the plan kernel)
+//   unit_list uint32[..][4]                one record per group, the groups of a tree next to one another, the trees
+//                                          in the order in which their plan CTAs got there: (tree, first row of the
+//                                          tree, first position | own nodes << 16, n_prefix | node at the first
+//                                          position << 16).  A tree of at most 64 nodes is its own single group
+//                                          (., ., T << 16, 0xFFFF): identity numbering, tables in depth / anc8.  The
+//                                          tensor-core verify kernel walks this list, so that its units are real
+//                                          groups only and spread evenly over the CTAs whatever the tree sizes.
 //   dfs_node  uint16[N]                    node id at position r
 //   dfs_depth uint8 [N]                    depth of that node
 //   dfs_anc8  uint8 [N][16]                its root path in virtual indices of its group (0xFF = unused)
 //   utilde   float [N][h_v][d_v]           solve result u~ (Eq. 10 with the W S0 term folded in; general kernel)
 struct WorkspaceLayout {
-    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, group_start, group_info, utilde, total;
+    size_t tree_ok, depth, anc, anc8, dfs_node, dfs_depth, dfs_anc8, group_start, unit_count, unit_list, utilde, total;
 };
 
 constexpr int GDN_GROUP_TILE = 64;            // nodes of a group and its prefix together
@@ -57,7 +61,8 @@ inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
     w.dfs_depth = off; off = align256(off + N);
     w.dfs_anc8 = off; off = align256(off + 16 * N);
     w.group_start = off; off = align256(off + sizeof(uint16_t) * (size_t)s.n_seq * (GDN_MAX_GROUPS + 1));
-    w.group_info = off; off = align256(off + sizeof(uint16_t) * 4 * (size_t)s.n_seq * GDN_MAX_GROUPS);
+    w.unit_count = off; off = align256(off + sizeof(int32_t));
+    w.unit_list = off; off = align256(off + 16 * (N / GDN_GROUP_MIN_NODES + (size_t)s.n_seq + 1));
     w.utilde = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
     w.total = off;
     return w;
@@ -70,7 +75,9 @@ struct PlanPtrs {
     uint8_t *anc8;
     uint16_t *dfs_node;
     uint8_t *dfs_depth, *dfs_anc8;
-    uint16_t *group_start, *group_info;
+    uint16_t *group_start;
+    int32_t *unit_count;
+    uint4 *unit_list;
     float *utilde;
 };
 
@@ -81,7 +88,8 @@ inline PlanPtrs plan_ptrs(void *workspace, const WorkspaceLayout &w)
             reinterpret_cast<uint16_t *>(b + w.anc), reinterpret_cast<uint8_t *>(b + w.anc8),
             reinterpret_cast<uint16_t *>(b + w.dfs_node), reinterpret_cast<uint8_t *>(b + w.dfs_depth),
             reinterpret_cast<uint8_t *>(b + w.dfs_anc8), reinterpret_cast<uint16_t *>(b + w.group_start),
-            reinterpret_cast<uint16_t *>(b + w.group_info), reinterpret_cast<float *>(b + w.utilde)};
+            reinterpret_cast<int32_t *>(b + w.unit_count), reinterpret_cast<uint4 *>(b + w.unit_list),
+            reinterpret_cast<float *>(b + w.utilde)};
 }
 
 // Host launchers (each returns the cudaError_t of its launch).

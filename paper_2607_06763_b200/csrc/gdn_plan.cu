@@ -18,7 +18,8 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
             const int32_t *__restrict__ parent, const int32_t *__restrict__ node_offsets,
             const int32_t *__restrict__ n_nodes, int32_t *__restrict__ tree_ok, uint8_t *__restrict__ depth, uint16_t *__restrict__ anc,
             uint8_t *__restrict__ anc8, uint16_t *__restrict__ dfs_node, uint8_t *__restrict__ dfs_depth,
-            uint8_t *__restrict__ dfs_anc8, uint16_t *__restrict__ group_start, uint16_t *__restrict__ group_info,
+            uint8_t *__restrict__ dfs_anc8, uint16_t *__restrict__ group_start, int32_t *__restrict__ unit_count,
+            uint4 *__restrict__ unit_list,
             int32_t *status_dev)
 {
     __shared__ int size_s[GDN_GROUPED_MAX_NODES];        // subtree sizes
@@ -45,10 +46,9 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
         if (threadIdx.x == 0) {
             report_status(status_dev, GDN_ERR_TREE);
             tree_ok[b] = 0;
+            if (n_seq == 1) *unit_count = 0;
         }
-        for (int k = threadIdx.x; k < GDN_MAX_GROUPS; k += PLAN_THREADS)
-            *reinterpret_cast<uint2 *>(group_info + ((size_t)b * GDN_MAX_GROUPS + k) * 4) = make_uint2(0u, 0u);
-        return;
+        return;   // no record in the unit list: nothing of this tree is verified
     }
     const bool grouped = max_depth <= 16 && T > 64 && T <= GDN_GROUPED_MAX_NODES;
     for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
@@ -91,10 +91,13 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     if (threadIdx.x == 0) tree_ok[b] = any_err ? 0 : 1;
     if (any_err || !grouped) {
         // a tree that fits one tile is its own single group with the identity numbering, marked by n_prefix =
-        // 0xFFFF (no group at all if the tree was rejected)
-        for (int k = threadIdx.x; k < GDN_MAX_GROUPS; k += PLAN_THREADS)
-            *reinterpret_cast<uint2 *>(group_info + ((size_t)b * GDN_MAX_GROUPS + k) * 4) =
-                make_uint2(k == 0 && !any_err && T <= GDN_GROUP_TILE ? (uint32_t)T << 16 : 0u, 0xFFFFu);
+        // 0xFFFF (no group at all if the tree was rejected or is empty)
+        // (a call with a single tree keeps the count itself; otherwise the counter was zeroed in front of this grid)
+        const bool one = !any_err && T > 0 && T <= GDN_GROUP_TILE;
+        if (threadIdx.x == 0 && n_seq == 1) *unit_count = one ? 1 : 0;
+        if (threadIdx.x == 0 && one)
+            unit_list[n_seq == 1 ? 0 : atomicAdd(unit_count, 1)] =
+                make_uint4((uint32_t)b, (uint32_t)lo, (uint32_t)T << 16, 0xFFFFu);
         return;
     }
 
@@ -131,14 +134,24 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     __syncthreads();
     for (int k = threadIdx.x; k <= GDN_MAX_GROUPS; k += PLAN_THREADS)
         group_start[(size_t)b * (GDN_MAX_GROUPS + 1) + k] = gstart_s[k];
+    // one record per group in the unit list, the groups of this tree next to one another
+    __shared__ int list_base_s;
+    if (threadIdx.x == 0) {
+        int n_groups = 0;
+        while (n_groups < GDN_MAX_GROUPS && gstart_s[n_groups] < T) ++n_groups;
+        if (n_seq == 1) {
+            *unit_count = n_groups;
+            list_base_s = 0;
+        } else {
+            list_base_s = atomicAdd(unit_count, n_groups);
+        }
+    }
+    __syncthreads();
     for (int k = threadIdx.x; k < GDN_MAX_GROUPS; k += PLAN_THREADS) {
         const int g0 = gstart_s[k], own = gstart_s[k + 1] - g0;
-        uint32_t w0 = 0, w1 = 0;   // (first position, own nodes), (n_prefix, node at the first position)
-        if (own > 0) {
-            w0 = (uint32_t)g0 | ((uint32_t)own << 16);
-            w1 = (uint32_t)(depth_at_s[g0] - 1) | ((uint32_t)dfs_node[lo + g0] << 16);
-        }
-        *reinterpret_cast<uint2 *>(group_info + ((size_t)b * GDN_MAX_GROUPS + k) * 4) = make_uint2(w0, w1);
+        if (own > 0)   // (first position, own nodes), (n_prefix, node at the first position)
+            unit_list[list_base_s + k] = make_uint4((uint32_t)b, (uint32_t)lo, (uint32_t)g0 | ((uint32_t)own << 16),
+                                                    (uint32_t)(depth_at_s[g0] - 1) | ((uint32_t)dfs_node[lo + g0] << 16));
     }
     // Root path of every node in the virtual indices of its group: an ancestor before the group's first
     // position is an ancestor of the group's first node and gets index depth-1; one inside the group gets
@@ -167,6 +180,10 @@ cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32
                         const int32_t *n_nodes, const PlanPtrs &plan, int32_t *status_dev, cudaStream_t stream)
 {
     if (s.n_seq == 0) return cudaSuccess;
+    if (s.n_seq > 1) {   // the trees' CTAs claim their places in the unit list from a counter
+        cudaError_t e0 = cudaMemsetAsync(plan.unit_count, 0, sizeof(int32_t), stream);
+        if (e0 != cudaSuccess) return e0;
+    }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)s.n_seq);
     cfg.blockDim = dim3(PLAN_THREADS);
@@ -179,7 +196,7 @@ cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, plan_kernel, s.n_seq, s.total_nodes, s.max_tree_nodes, s.max_depth, parent,
                               node_offsets, n_nodes, plan.tree_ok, plan.depth, plan.anc, plan.anc8, plan.dfs_node,
-                              plan.dfs_depth, plan.dfs_anc8, plan.group_start, plan.group_info, status_dev);
+                              plan.dfs_depth, plan.dfs_anc8, plan.group_start, plan.unit_count, plan.unit_list, status_dev);
 }
 
 }  // namespace gdn

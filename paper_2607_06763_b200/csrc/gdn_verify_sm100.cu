@@ -77,7 +77,7 @@ struct VerifyFastParams {
     alignas(64) CUtensorMap tm_q;
     alignas(64) CUtensorMap tm_v;
     int h_qk, h_v;
-    int n_units;        // n_seq * h_v (grouped mode: times groups_per_tree)
+    int n_units;        // n_seq * h_v (grouped mode: an upper bound that only sizes the grid)
     int prefetch_dist;  // a CTA warms L2 for unit blockIdx.x + prefetch_dist (about one wave ahead)
     float scale;
     const float *S0;
@@ -91,7 +91,9 @@ struct VerifyFastParams {
     int32_t *status_dev;
     // grouped verification of trees with more than 64 nodes (only read by the GROUPED instantiation)
     int groups_per_tree, anc_stride;                   // units per (tree, head); entries per row of anc16
-    const uint16_t *anc16, *dfs_node, *group_info;
+    const uint16_t *anc16, *dfs_node;
+    const uint4 *unit_list;                            // one record per group (see the workspace layout)
+    const int32_t *unit_count;
     const uint8_t *dfs_depth, *dfs_anc8;
     // fused commit of the previous step's accepted paths (only read by the FUSED instantiation)
     float *S_rw;                                       // same tensor as S0, written in place
@@ -338,9 +340,8 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // Launched with programmatic stream serialization: everything above overlaps the tail of the kernel in front
     // (the previous call, or the plan kernel); nothing that is computed from memory may run before that kernel's
     // writes are visible.  L2 can be asked for the first unit's state tile meanwhile (a prefetch consumes nothing).
-    const int G = GROUPED ? p.groups_per_tree : 1;   // units per state tile
-    if (tid < 4 && (int)blockIdx.x < p.n_units)
-        prefetch_l2_bulk(p.S0 + (size_t)((int)blockIdx.x / G) * FV_D * FV_D + (size_t)tid * 4096, 16384);
+    if (!GROUPED && tid < 4 && (int)blockIdx.x < p.n_units)
+        prefetch_l2_bulk(p.S0 + (size_t)blockIdx.x * FV_D * FV_D + (size_t)tid * 4096, 16384);
     // ... and for the rows of the first unit's tree.  Their place may depend on node_offsets[], which the kernel in
     // front may still be writing: the value read here only steers prefetches (clamped to the tensors), it is read
     // again behind the dependency wait before anything is computed from it.
@@ -360,50 +361,57 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
 
     // unit -> (tree, head, first node, size); a unit whose node_offsets[] are inconsistent (reported) or whose tree
     // is empty is skipped.  parent[] itself is checked when the unit's tables are built.
-    // A CTA walks the units blockIdx.x, blockIdx.x + gridDim.x, ...: (tile, slot, head, group) of a unit follow from
-    // those of the unit before by additions and carries, so that the integer divisions by the head and group counts
-    // (a few dozen instructions each, for every thread) are paid once per CTA and not once per unit.
+    // A CTA walks the units blockIdx.x, blockIdx.x + gridDim.x, ...: the indices of a unit follow from those of the
+    // unit before by additions and carries, so that the integer divisions by the head and group counts (a few dozen
+    // instructions each, for every thread) are paid once per CTA and not once per unit.
+    // Trees of at most 64 nodes: unit = slot b * h_v + head h.  GROUPED: unit = (layer b * E + record grp) * h_v + h,
+    // where E is the number of records in the plan's unit list (one per group; known behind the dependency wait) and
+    // `layer` counts the repetitions of the n_trees shared trees in the padded layout (always 0 otherwise).
     struct Cursor { int u, b, h, grp; };
+    int n_units = GROUPED ? 0 : p.n_units;
+    int n_records = 1, gstep_h = 0, gstep_e = 0, gstep_l = 0;   // GROUPED, set behind the dependency wait
     const int ratio = p.h_v / p.h_qk;
     const int ratio_shift = (ratio & (ratio - 1)) == 0 ? 31 - __clz(ratio) : -1;
     auto hk_of = [&](int h_) -> int { return ratio_shift >= 0 ? h_ >> ratio_shift : h_ / ratio; };
     auto tree_of = [&](int b_) -> int { return p.n_trees == 1 ? 0 : b_ % p.n_trees; };   // padded layout only
-    const int step_grp = (int)gridDim.x % G, step_tile = (int)gridDim.x / G;
-    const int step_h = step_tile % p.h_v, step_b = step_tile / p.h_v;
+    const int step_h = (int)gridDim.x % p.h_v, step_b = (int)gridDim.x / p.h_v;
     auto cursor_at = [&](int u) -> Cursor {
         Cursor c;
         c.u = u;
-        const int tile = u / G;
-        c.grp = u % G;
-        c.b = tile / p.h_v;
-        c.h = tile % p.h_v;
+        c.h = u % p.h_v;
+        const int t = u / p.h_v;
+        c.grp = GROUPED ? t % n_records : 0;
+        c.b = GROUPED ? t / n_records : t;
         return c;
     };
     auto advance = [&](Cursor &c) {
         c.u += (int)gridDim.x;
-        c.grp += step_grp;
-        const int carry = c.grp >= G ? 1 : 0;
-        c.grp -= carry ? G : 0;
-        c.h += step_h + carry;
-        const int carry_h = c.h >= p.h_v ? 1 : 0;
-        c.h -= carry_h ? p.h_v : 0;
-        c.b += step_b + carry_h;
+        if constexpr (GROUPED) {
+            c.h += gstep_h;
+            const int carry_h = c.h >= p.h_v ? 1 : 0;
+            c.h -= carry_h ? p.h_v : 0;
+            c.grp += gstep_e + carry_h;
+            const int carry_e = c.grp >= n_records ? 1 : 0;
+            c.grp -= carry_e ? n_records : 0;
+            c.b += gstep_l + carry_e;
+        } else {
+            c.h += step_h;
+            const int carry_h = c.h >= p.h_v ? 1 : 0;
+            c.h -= carry_h ? p.h_v : 0;
+            c.b += step_b + carry_h;
+        }
     };
     // The loads a decode needs are issued by decode_load() and looked at by decode() / decode_g() later (the unit after
     // next is asked for at the top of a unit and decoded in its middle), so that no thread waits for them.
-    struct DecodeRaw { int lo, hi; uint2 gi; };
+    struct DecodeRaw { int lo, hi; uint4 rec; };
     auto decode_load = [&](const Cursor &c) -> DecodeRaw {
-        DecodeRaw r{0, 0, make_uint2(0u, 0u)};
-        if (c.u >= p.n_units) return r;
+        DecodeRaw r{0, 0, make_uint4(0u, 0u, 0u, 0u)};
+        if (c.u >= n_units) return r;
         const int ub = c.b;
-        const int tree = (PADDED && p.t_pad) ? tree_of(ub) : ub;
         if constexpr (GROUPED) {
-            const int grp = c.grp;
-            if (grp < GDN_MAX_GROUPS)
-                r.gi = __ldg(reinterpret_cast<const uint2 *>(p.group_info + ((size_t)tree * GDN_MAX_GROUPS + grp) * 4));
-            if (!(PADDED && p.t_pad)) r.lo = p.node_offsets[ub];
+            r.rec = p.unit_list[c.grp];   // written by the plan kernel in front of this grid: no read-only path
         } else if (PADDED && p.t_pad) {
-            r.lo = p.n_nodes[tree];
+            r.lo = p.n_nodes[tree_of(ub)];
         } else {
             r.lo = p.node_offsets[ub];
             r.hi = p.node_offsets[ub + 1];
@@ -411,7 +419,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         return r;
     };
     auto decode = [&](const Cursor &c, const DecodeRaw &raw, int &ub, int &uh, int &uhk, int &ubase, int &uT, int &upar) -> bool {
-        if (c.u >= p.n_units) return false;
+        if (c.u >= n_units) return false;
         ub = c.b;
         uh = c.h;
         uhk = hk_of(uh);
@@ -448,18 +456,20 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // first = node at position g0; ident: a tree of at most 64 nodes inside a grouped call (identity numbering).
     struct GroupX { int pb, g0, n_prefix, first; bool ident; };
     auto decode_g = [&](const Cursor &c, const DecodeRaw &raw, int &ub, int &uh, int &uhk, int &ubase, int &uT, GroupX &gx) -> bool {
-        if (c.u >= p.n_units) return false;
-        ub = c.b;
+        if (c.u >= n_units) return false;
+        const int tree = (int)raw.rec.x;
         uh = c.h;
         uhk = hk_of(uh);
-        if (PADDED && p.t_pad) {
+        if (PADDED && p.t_pad) {   // slot = layer * n_trees + tree
+            ub = c.b * p.n_trees + tree;
             ubase = ub * p.t_pad;
-            gx.pb = tree_of(ub) * p.t_pad;
+            gx.pb = tree * p.t_pad;
         } else {
-            ubase = raw.lo;   // checked by the plan kernel (a tree with bad offsets has no groups)
+            ub = tree;
+            ubase = (int)raw.rec.y;   // checked by the plan kernel (a tree with bad offsets has no record)
             gx.pb = ubase;
         }
-        const uint2 gi = raw.gi;
+        const uint2 gi = make_uint2(raw.rec.z, raw.rec.w);
         const int own = (int)(gi.x >> 16);
         if (own == 0) return false;   // no such group (or the plan rejected the tree, which it has reported)
         gx.g0 = (int)(gi.x & 0xFFFFu);
@@ -739,13 +749,23 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     // waits for this grid to complete before it reads or writes anything) may be made resident now.
     asm volatile("griddepcontrol.launch_dependents;");
     GroupX gx{0, 0, 0, 0, true}, ngx{0, 0, 0, 0, true};
+    if constexpr (GROUPED) {
+        // the plan kernel has counted the groups of all trees: that many records, times the heads, times the layers
+        // that share the trees in the padded layout, are the units of this grid
+        const int n_rec = *reinterpret_cast<const volatile int32_t *>(p.unit_count);
+        const int n_layers = (PADDED && p.t_pad) ? p.n_seq / p.n_trees : 1;
+        n_records = n_rec > 0 ? n_rec : 1;
+        n_units = n_rec > 0 ? n_rec * p.h_v * n_layers : 0;
+        gstep_h = (int)gridDim.x % p.h_v;
+        const int t = (int)gridDim.x / p.h_v;
+        gstep_e = t % n_records;
+        gstep_l = t / n_records;
+    }
     Cursor ucur = cursor_at((int)blockIdx.x);
     bool cur_ok;
     if constexpr (GROUPED) {
-        // units without a group (the grid is sized for the largest tree) are stepped over here and at the top of
-        // every unit, so that the loop below only ever sees real ones
         cur_ok = decode_g(ucur, decode_load(ucur), b, h, hk, base, T, gx);
-        while (!cur_ok && (advance(ucur), ucur.u < p.n_units)) cur_ok = decode_g(ucur, decode_load(ucur), b, h, hk, base, T, gx);
+        while (!cur_ok && (advance(ucur), ucur.u < n_units)) cur_ok = decode_g(ucur, decode_load(ucur), b, h, hk, base, T, gx);
         int t_node, t_d;
         uint4 t_row;
         lookup_tables_g(gx, T, t_node, t_d, t_row);
@@ -784,7 +804,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     }
     int done_units = 0;
 #pragma unroll 1
-    for (int iter = 0; ucur.u < p.n_units; ++iter) {
+    for (int iter = 0; ucur.u < n_units; ++iter) {
     const bool unit_ok = cur_ok;
     const uint32_t par = (uint32_t)(done_units & 1);   // every barrier completes once per processed unit
     int nb = 0, nh = 0, nhk = 0, nbase = 0, nT = 0, npar0 = 0;
@@ -795,7 +815,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     auto decode_next = [&]() {
         if constexpr (GROUPED) {
             next_ok = decode_g(ncur, next_raw, nb, nh, nhk, nbase, nT, ngx);
-            while (!next_ok && (advance(ncur), ncur.u < p.n_units))   // a unit without a group: look further on
+            while (!next_ok && (advance(ncur), ncur.u < n_units))   // (every record is a real group: not taken)
                 next_ok = decode_g(ncur, decode_load(ncur), nb, nh, nhk, nbase, nT, ngx);
         } else {
             next_ok = decode(ncur, next_raw, nb, nh, nhk, nbase, nT, npar0);
@@ -830,8 +850,18 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     }
     // L2 warming for this CTA's next unit, in slices at phase boundaries
     auto warm_l2_state = [&](int slice) {
-        if (tid == 96 && ncur.u < p.n_units)
-            prefetch_l2_bulk(p.S0 + (size_t)(ncur.b * p.h_v + ncur.h) * FV_D * FV_D + (size_t)slice * 4096, 16384);
+        if constexpr (GROUPED) {
+            // the next unit's slot is known once its record has been looked at (stage 1): both halves of the tile are
+            // asked for behind that; the groups of a (tree, head) are neighbours, so most of the time L2 has it already
+            if (tid == 96 && slice >= 2 && next_ok) {
+                const float *S = p.S0 + (size_t)(nb * p.h_v + nh) * FV_D * FV_D + (size_t)(slice - 2) * 8192;
+                prefetch_l2_bulk(S, 16384);
+                prefetch_l2_bulk(S + 4096, 16384);
+            }
+        } else {
+            if (tid == 96 && ncur.u < n_units)
+                prefetch_l2_bulk(p.S0 + (size_t)(ncur.b * p.h_v + ncur.h) * FV_D * FV_D + (size_t)slice * 4096, 16384);
+        }
     };
 
     // a tree whose parent[] was rejected while its tables were built runs as a tree of no nodes: nothing of it
@@ -1388,7 +1418,8 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
     const bool padded = p.t_pad != 0;   // the padded layout and the on-chip gate activations share an instantiation
     void (*kernel)(const VerifyFastParams);
     if constexpr (GROUPED) {
-        // trees of more than 64 nodes: a unit is one ancestor-closed group of a (tree, head); rows are gathered
+        // trees of more than 64 nodes: a unit is one ancestor-closed group of a (tree, head), taken from the plan's
+        // unit list (its length is read on the device; this bound only sizes the grid); rows are gathered
         pt.n_units = p.n_units * p.groups_per_tree;
         kernel = padded ? verify_sm100_persistent_kernel<TOut, false, false, true, true>
                         : verify_sm100_persistent_kernel<TOut, false, false, false, true>;
@@ -1407,14 +1438,7 @@ cudaError_t launch_fast_typed(const gdn_shape_t &s, const VerifyFastParams &p, c
     }
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
     if (e != cudaSuccess) return e;
-    int grid = pt.n_units < p.prefetch_dist ? pt.n_units : p.prefetch_dist;
-    if constexpr (GROUPED) {
-        // A CTA walks the units blockIdx.x, blockIdx.x + grid, ...; the group index is the unit index modulo the groups
-        // per tree, and the last groups of a tree may not exist.  With a grid size coprime to the groups per tree every
-        // CTA meets every group index equally often, so the missing groups are spread evenly over the CTAs.
-        auto gcd = [](int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; };
-        while (grid < pt.n_units && grid > 1 && gcd(grid, p.groups_per_tree) != 1) --grid;   // (one unit per CTA: no walk)
-    }
+    const int grid = pt.n_units < p.prefetch_dist ? pt.n_units : p.prefetch_dist;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(FV_THREADS);
@@ -1447,7 +1471,8 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     p.groups_per_tree = s.max_tree_nodes <= FV_T ? 1 : (s.max_tree_nodes + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;
     p.anc_stride = s.max_depth;
     p.anc16 = plan.anc; p.dfs_node = plan.dfs_node; p.dfs_depth = plan.dfs_depth; p.dfs_anc8 = plan.dfs_anc8;
-    p.group_info = plan.group_info;
+    p.unit_list = plan.unit_list;
+    p.unit_count = plan.unit_count;
     return p;
 }
 
