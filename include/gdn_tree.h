@@ -177,7 +177,8 @@ int gdn_tree_commit_verify_padded(const gdn_shape_t *shape, int32_t n_trees, int
  *   plan         : [device] >= gdn_tree_plan_bytes(shape, n_trees) bytes, 256-byte aligned; written by
  *                  gdn_tree_plan, read-only for gdn_tree_verify_planned; depends on shape->max_tree_nodes,
  *                  shape->max_depth and n_trees only (not on n_seq or the head counts), and must have been
- *                  built with the same three values
+ *                  built with the same three values: a buffer no plan was built in, or a plan built for other
+ *                  values, is refused on the device (GDN_ERR_WORKSPACE in *status_dev, nothing is written)
  *   gdn_tree_plan reports a bad tree (GDN_ERR_TREE, GDN_ERR_DEPTH) through *status_dev; the slots of such a
  *   tree are skipped by gdn_tree_verify_planned (nothing of them is written).
  *   gdn_tree_commit_padded: k, v, g, beta, parent [n_trees][T] (may be NULL), n_nodes, path

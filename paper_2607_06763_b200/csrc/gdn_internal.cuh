@@ -25,7 +25,8 @@ namespace gdn {
 // (64 - n_prefix, i.e. at least GDN_GROUP_MIN_NODES).
 //   group_start uint16[n_seq][GDN_MAX_GROUPS + 1]  first position of group k of tree b; entries behind the
 //                                          last group hold the tree's size
-//   unit_count int32 [1]                   number of groups over all trees (zeroed in front of the plan kernel)
+//   unit_count int32 [2]                   number of groups over all trees (zeroed in front of the plan kernel), and
+//                                          a word that says for which shape the plan was built (plan_magic)
 //   unit_list uint32[..][4]                one record per group, the groups of a tree next to one another, the trees
 //                                          in the order in which their plan CTAs got there: (tree, first row of the
 //                                          tree, first position | own nodes << 16, n_prefix | node at the first
@@ -48,6 +49,17 @@ constexpr int GDN_MAX_GROUPS = (GDN_GROUPED_MAX_NODES + GDN_GROUP_MIN_NODES - 1)
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
+// Written next to the unit count by the plan kernel and checked by the grouped verify kernel: a plan that was never
+// built, or was built for another padded size, depth bound or number of trees, is refused instead of followed.
+__host__ __device__ inline int32_t plan_magic(int n_trees, int max_tree_nodes, int max_depth)
+{
+    return (int32_t)(0x504C4E31u ^ ((uint32_t)n_trees * 2654435761u) ^ ((uint32_t)max_tree_nodes << 8) ^ (uint32_t)max_depth);
+}
+inline size_t unit_list_capacity(const gdn_shape_t &s)
+{
+    return (size_t)s.total_nodes / 49 + (size_t)s.n_seq + 1;
+}
+
 inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
 {
     WorkspaceLayout w;
@@ -61,8 +73,8 @@ inline WorkspaceLayout workspace_layout(const gdn_shape_t &s)
     w.dfs_depth = off; off = align256(off + N);
     w.dfs_anc8 = off; off = align256(off + 16 * N);
     w.group_start = off; off = align256(off + sizeof(uint16_t) * (size_t)s.n_seq * (GDN_MAX_GROUPS + 1));
-    w.unit_count = off; off = align256(off + sizeof(int32_t));
-    w.unit_list = off; off = align256(off + 16 * (N / GDN_GROUP_MIN_NODES + (size_t)s.n_seq + 1));
+    w.unit_count = off; off = align256(off + 2 * sizeof(int32_t));
+    w.unit_list = off; off = align256(off + 16 * unit_list_capacity(s));
     w.utilde = off;   off = align256(off + sizeof(float) * N * (size_t)s.h_v * (size_t)s.d_v);
     w.total = off;
     return w;

@@ -35,6 +35,7 @@ plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
     const int b = blockIdx.x;
+    if (b == 0 && threadIdx.x == 0) unit_count[1] = plan_magic(n_seq, max_tree_nodes, max_depth);
     // ragged packing: the tree's rows by node_offsets[]; padded layout: max_tree_nodes rows per tree, n_nodes[b] used
     const int lo = node_offsets ? node_offsets[b] : b * max_tree_nodes;
     const int hi = node_offsets ? node_offsets[b + 1] : lo + n_nodes[b];

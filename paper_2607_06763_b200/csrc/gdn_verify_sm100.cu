@@ -93,7 +93,8 @@ struct VerifyFastParams {
     int groups_per_tree, anc_stride;                   // units per (tree, head); entries per row of anc16
     const uint16_t *anc16, *dfs_node;
     const uint4 *unit_list;                            // one record per group (see the workspace layout)
-    const int32_t *unit_count;
+    const int32_t *unit_count;                         // [0] records in the list, [1] plan_magic of the plan's shape
+    int unit_capacity, plan_magic;                     // what the list can hold; what [1] has to read
     const uint8_t *dfs_depth, *dfs_anc8;
     // fused commit of the previous step's accepted paths (only read by the FUSED instantiation)
     float *S_rw;                                       // same tensor as S0, written in place
@@ -752,7 +753,12 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
     if constexpr (GROUPED) {
         // the plan kernel has counted the groups of all trees: that many records, times the heads, times the layers
         // that share the trees in the padded layout, are the units of this grid
-        const int n_rec = *reinterpret_cast<const volatile int32_t *>(p.unit_count);
+        int n_rec = reinterpret_cast<const volatile int32_t *>(p.unit_count)[0];
+        if (reinterpret_cast<const volatile int32_t *>(p.unit_count)[1] != p.plan_magic || n_rec < 0 ||
+            n_rec > p.unit_capacity) {   // not a plan of this shape (never built, or built for other sizes)
+            if (tid == 0) report_status(p.status_dev, GDN_ERR_WORKSPACE);
+            n_rec = 0;
+        }
         const int n_layers = (PADDED && p.t_pad) ? p.n_seq / p.n_trees : 1;
         n_records = n_rec > 0 ? n_rec : 1;
         n_units = n_rec > 0 ? n_rec * p.h_v * n_layers : 0;
@@ -1473,6 +1479,8 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     p.anc16 = plan.anc; p.dfs_node = plan.dfs_node; p.dfs_depth = plan.dfs_depth; p.dfs_anc8 = plan.dfs_anc8;
     p.unit_list = plan.unit_list;
     p.unit_count = plan.unit_count;
+    p.unit_capacity = (int)unit_list_capacity(s);
+    p.plan_magic = plan_magic(s.n_seq, s.max_tree_nodes, s.max_depth);
     return p;
 }
 
@@ -1521,6 +1529,11 @@ cudaError_t launch_verify_sm100_planned(const gdn_shape_t &s, int n_trees, bool 
     if (s.n_seq == 0 || s.total_nodes == 0) return cudaSuccess;
     VerifyFastParams p = make_params(s, S0, q, k, v, g, beta, nullptr, o, plan, status_dev);
     p.t_pad = s.max_tree_nodes; p.n_trees = n_trees; p.raw_gates = raw_gates ? 1 : 0;
+    gdn_shape_t ps = s;   // the shape the plan was built for: n_trees trees of t_pad rows
+    ps.n_seq = n_trees;
+    ps.total_nodes = n_trees * s.max_tree_nodes;
+    p.unit_capacity = (int)unit_list_capacity(ps);
+    p.plan_magic = plan_magic(n_trees, s.max_tree_nodes, s.max_depth);
     if (s.out_dtype == GDN_BF16) return launch_fast_typed<__nv_bfloat16, false, true>(s, p, stream);
     return launch_fast_typed<float, false, true>(s, p, stream);
 }

@@ -311,6 +311,22 @@ def test_planned_rejections(tl):
     assert gdn.gdn_tree_plan(d.shape, 3, d.parent, d.n_nodes, plan, d.status) == -2       # 4 slots, 3 trees
     assert gdn.gdn_tree_plan(d.shape, 2, d.parent, d.n_nodes, plan[:1024], d.status) == -10   # plan too small
     assert gdn.gdn_tree_plan(d.shape, 2, None, d.n_nodes, plan, d.status) == -1
+    # a plan buffer that no plan was built in, and a plan built for another depth bound: refused on the device
+    # (GDN_ERR_WORKSPACE in *status_dev), nothing is written
+    blank = torch.zeros_like(plan)
+    assert gdn.gdn_tree_verify_planned(d.shape, 2, False, d.S0, d.q, d.k, d.v, d.g_in, d.beta_in, blank, d.o, d.status) == 0
+    assert d.status_value() == -10 and bool((d.o == 7.0).all())
+    d.status.zero_()
+    shallow = gdn.GdnShape.from_buffer_copy(d.shape)
+    shallow.max_depth = 12
+    plan12 = torch.empty(gdn.gdn_tree_plan_bytes(shallow, 2), dtype=torch.uint8, device="cuda")
+    assert gdn.gdn_tree_plan(shallow, 2, d.parent, d.n_nodes, plan12, d.status) == 0
+    assert d.status_value() == 0
+    if plan12.numel() >= plan.numel():
+        assert gdn.gdn_tree_verify_planned(d.shape, 2, False, d.S0, d.q, d.k, d.v, d.g_in, d.beta_in, plan12, d.o,
+                                           d.status) == 0
+        assert d.status_value() == -10 and bool((d.o == 7.0).all())
+        d.status.zero_()
     # device-side: a parent that points forward in tree 1 -> its slots are skipped, tree 0 is verified
     d.parent[1, 70] = 90
     assert gdn.gdn_tree_plan(d.shape, 2, d.parent, d.n_nodes, plan, d.status) == 0
