@@ -292,7 +292,7 @@ int gdn_tree_commit_host(const gdn_shape_t *shape, float *S_h, const void *k_h, 
  * gdn_tree_commit_verify_host_arena_bytes(shape, prev_total_nodes, total_path_len) bytes.
  * S_h is written back only if total_path_len > 0 (otherwise no state changes); o_h receives the
  * outputs of the new trees.  Returns the host-side status, or the device-side status if non-zero.
- * With two or more sequences the call is pipelined: the batch is cut into up to eight groups of
+ * With two or more sequences the call is pipelined: the batch is cut into up to six groups of
  * sequences, and the copies up of one group, the kernels of the group before it and the copies down
  * of the group before that run at the same time (both directions of the host link busy).  The
  * copies run on two helper streams that the library creates on first use for each device and keeps

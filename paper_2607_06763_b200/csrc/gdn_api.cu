@@ -561,7 +561,7 @@ namespace {
 
 // Helper streams and events of the pipelined host-buffer call, created on first use for each device and kept for
 // the life of the process (the one piece of state the library keeps besides the static scratch array).
-constexpr int HOST_PIPE_GROUPS = 8;
+constexpr int HOST_PIPE_GROUPS = 6;
 struct HostPipe {
     bool ready = false;
     cudaStream_t s_in = nullptr, s_out = nullptr;
