@@ -90,7 +90,8 @@ struct VerifyFastParams {
     const uint8_t *anc8;
     int32_t *status_dev;
     // grouped verification of trees with more than 64 nodes (only read by the GROUPED instantiation)
-    int groups_per_tree, anc_stride;                   // units per (tree, head); entries per row of anc16
+    int groups_per_tree, anc_stride;                   // upper bound of the groups of a tree (sizes the grid); entries
+                                                       // per row of anc16
     const uint16_t *anc16, *dfs_node;
     const uint4 *unit_list;                            // one record per group (see the workspace layout)
     const int32_t *unit_count;                         // [0] records in the list, [1] plan_magic of the plan's shape
@@ -301,8 +302,10 @@ __device__ __forceinline__ void split_bf16(float x, float &hi, float &lo)
 // head, group); it is verified as a virtual tree of the <= 15 proper ancestors of the group's first node followed by
 // the group's own nodes.  The rows of a virtual tree are not contiguous, so its k/q/v rows are gathered with
 // cp.async (completing on the same mbarriers as the TMA tiles otherwise), its tables come from the plan, and
-// outputs are stored for the group's own nodes only.  The five or so groups of a (tree, head) run on neighbouring
-// CTAs at about the same time, so the state tile crosses HBM once.
+// outputs are stored for the group's own nodes only.  The units are the records of the plan's unit list (one per
+// real group, the groups of a tree next to one another) times the heads: the five or so groups of a (tree, head) run
+// on neighbouring CTAs at about the same time, so the state tile crosses HBM once, and the work spreads evenly over
+// the CTAs whatever the tree sizes.
 template <typename TOut, bool FUSED, bool SMALL, bool PADDED, bool GROUPED>
 __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(const __grid_constant__ VerifyFastParams p)
 {
@@ -1473,7 +1476,7 @@ VerifyFastParams make_params(const gdn_shape_t &s, const float *S0, const void *
     p.node_offsets = node_offsets; p.o = o;
     p.n_seq = s.n_seq; p.total_nodes = s.total_nodes; p.max_tree_nodes = s.max_tree_nodes; p.max_depth = s.max_depth;
     p.depth = plan.depth; p.anc8 = plan.anc8; p.status_dev = status_dev;
-    // upper bound of the groups of a tree; a unit without a group is stepped over
+    // upper bound of the groups of a tree (the real ones are in the plan's unit list)
     p.groups_per_tree = s.max_tree_nodes <= FV_T ? 1 : (s.max_tree_nodes + GDN_GROUP_MIN_NODES - 1) / GDN_GROUP_MIN_NODES;
     p.anc_stride = s.max_depth;
     p.anc16 = plan.anc; p.dfs_node = plan.dfs_node; p.dfs_depth = plan.dfs_depth; p.dfs_anc8 = plan.dfs_anc8;
