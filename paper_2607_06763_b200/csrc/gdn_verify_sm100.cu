@@ -949,11 +949,13 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
         __syncthreads();
         warm_l2_state(1);
         // X and Y for real ancestors only; the decay ratio a_i / a_j is exp(G_i - G_j)
+        // (SMALL: nodes 32.. do not exist; their rows of X and Y are never looked at)
         {
+            constexpr int NU = SMALL ? 2 : 4;
             float gdiff[4], gk[4], gq[4], bi[4];
             bool on[4], onx[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < NU; ++u) {
                 const int idx = u * FV_THREADS + tid;
                 const int i = idx >> 4, t = idx & 15;
                 const int d = depth_s[i];
@@ -968,7 +970,7 @@ __global__ void __launch_bounds__(FV_THREADS, 2) verify_sm100_persistent_kernel(
                 gk[u] = gram[i * 64 + jpos];          // row i: k_i
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < NU; ++u) {
                 const int idx = u * FV_THREADS + tid;
                 const float dec = __expf(gdiff[u]);
                 ys[idx] = on[u] ? dec * gq[u] : 0.f;
