@@ -70,6 +70,48 @@ def test_workspace_bytes(lib):
     assert gdn.gdn_tree_host_arena_bytes(s, 3) > n
 
 
+def test_plan_bytes_and_padded_entry_points_on_the_host(lib):
+    """Size of the shared-tree plan and the host-side refusals of the padded entry points (no CUDA call is made)."""
+    def shape(n_seq, t_pad, h_v=32, max_depth=16):
+        return gdn.GdnShape(n_seq, 16, h_v, 128, 128, 1, 1, max_depth, n_seq * t_pad, t_pad, 0.0883883)
+    base = gdn.gdn_tree_plan_bytes(shape(48, 256), 1)
+    assert base > 0 and base % 256 == 0
+    # the plan depends on the padded size, the depth bound and the number of trees -- not on slots or heads
+    assert gdn.gdn_tree_plan_bytes(shape(96, 256), 1) == base
+    assert gdn.gdn_tree_plan_bytes(shape(48, 256, h_v=16), 1) == base
+    assert gdn.gdn_tree_plan_bytes(shape(48, 512), 1) > base
+    assert gdn.gdn_tree_plan_bytes(shape(48, 256), 2) > base
+    assert gdn.gdn_tree_plan_bytes(shape(48, 256, max_depth=8), 1) < base
+    assert gdn.gdn_tree_plan_bytes(shape(48, 256), 0) == 0
+    s = shape(4, 128)
+    assert gdn.gdn_tree_plan(s, 3, 16, 16, _FakeBuf(1 << 20), 16) == -2               # 4 slots, 3 trees
+    assert gdn.gdn_tree_plan(s, 2, None, 16, _FakeBuf(1 << 20), 16) == -1
+    assert gdn.gdn_tree_plan(s, 2, 16, 16, _FakeBuf(256), 16) == -10                  # plan buffer too small
+    assert gdn.gdn_tree_verify_planned(s, 2, 0, 16, 16, 16, 16, 16, 16, _FakeBuf(256), 16, 16) == -10
+    assert gdn.gdn_tree_verify_planned(s, 2, 0, None, 16, 16, 16, 16, 16, _FakeBuf(1 << 20), 16, 16) == -1
+    far = gdn.GdnShape(4, 16, 32, 128, 128, 1, 1, 16, 4 * 2048, 2048, 0.0883883)
+    assert gdn.gdn_tree_verify_planned(far, 2, 0, 16, 16, 16, 16, 16, 16, _FakeBuf(1 << 24), 16, 16) in (-2, -5)
+    f32 = gdn.GdnShape(4, 16, 32, 128, 128, 0, 0, 16, 4 * 128, 128, 0.0883883)        # fp32 inputs: general path only
+    assert gdn.gdn_tree_commit_padded(f32, 2, 0, 16, 16, 16, 16, 16, 16, 16, 16, 16, 16) == -5
+    assert gdn.gdn_tree_commit_padded(s, 2, 0, 16, 16, 16, 16, 16, 16, None, 16, 16, 16) == -1   # n_nodes missing
+
+
+class _FakeBuf:
+    """Stands in for a device buffer in calls that are refused before any CUDA work: an aligned fake address and a
+    size, with the two methods the binding asks of a tensor."""
+    def __init__(self, nbytes):
+        self._n = nbytes
+
+    def data_ptr(self):
+        return 1 << 20
+
+    def numel(self):
+        return self._n
+
+    def element_size(self):
+        return 1
+
+
 def test_validate_host(lib):
     rng = np.random.default_rng(0)
     trees = [synth.tree_geo(rng, 20), synth.tree_chain(16), synth.tree_star(9)]
