@@ -556,9 +556,10 @@ def main():
             launches_per_step = {"fused": 1, "separate": 2, "verify": 1}[args.mode]
             dom_bytes = sbytes if fused else vbytes
             dom_ms = ms_per_step if args.mode != "separate" else split[0]
-        else:   # larger trees: tree plan + grouped verify kernel; the fused call runs commit and verify back to back
+        else:   # larger trees: tree plan + the verify kernel in its grouped mode; the fused call builds the plan in
+                # extra CTAs of the commit kernel's grid (two launches), the padded layout plans in a call of its own
             kernel_name = "verify_sm100_persistent_kernel<grouped>"
-            launches_per_step = {"fused": 3, "separate": 3, "verify": 2}[args.mode]
+            launches_per_step = {"fused": 3 if args.layout == "padded" else 2, "separate": 3, "verify": 2}[args.mode]
             dom_bytes = vbytes
             dom_ms = None if args.mode == "fused" else (ms_per_step if args.mode == "verify" else split[0])
         step_bytes = sbytes if args.mode != "verify" else vbytes
@@ -586,7 +587,7 @@ def main():
                          "avg_launch_us": (dom_ms if dom_ms else ms_per_step) * 1e3,
                          "note": ("launch time = timed region / steps (one kernel per call)" if dom_ms == ms_per_step
                                   else "launch time from events around the verify call" if dom_ms
-                                  else "whole step (commit kernel + plan + grouped verify kernel) over the step's bytes")},
+                                  else "whole step (commit + plan kernel, grouped verify kernel) over the step's bytes")},
             "gpu_launches": launches_per_step * args.steps * len(region_ms),
             "gpu_launches_per_step": launches_per_step,
             "clocks": clocks, "buffer_sets": n_sets,

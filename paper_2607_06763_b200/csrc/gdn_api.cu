@@ -423,6 +423,20 @@ extern "C" int gdn_tree_commit_verify(const gdn_shape_t *shape, float *S, const 
                                    status_dev);
             if (rc != GDN_OK) return rc;
         }
+        if (s.total_nodes > 0 && verify_sm100_supported(s) && commit_tile128_supported(s)) {
+            // trees of more than 64 nodes on the tensor-core path: the plan of the new trees does not depend on the
+            // commit, so it is built by extra CTAs of the commit grid; then the verify kernel in its grouped mode
+            const WorkspaceLayout lay = workspace_layout(s);
+            const PlanPtrs plan = plan_ptrs(workspace, lay);
+            cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+            if (launch_commit_plan(s, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
+                                   path_offsets, parent, node_offsets, plan, status_dev, stream) != cudaSuccess)
+                return GDN_ERR_CUDA;
+            if (launch_verify_sm100(s, S, q, k, v, g, beta, parent, node_offsets, o, plan, status_dev, stream) !=
+                cudaSuccess)
+                return GDN_ERR_CUDA;
+            return GDN_OK;
+        }
         rc = gdn_tree_commit(shape, S, k_prev, v_prev, g_prev, beta_prev, parent_prev, node_offsets_prev, path,
                              path_offsets, status_dev, cuda_stream);
         if (rc != GDN_OK) return rc;

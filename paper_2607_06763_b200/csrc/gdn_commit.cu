@@ -12,6 +12,7 @@
 // are issued before anything else so that the path checks and the k-row staging run under their
 // latency, and the kernel keeps to 64 registers so that two CTAs (32 warps) share an SM.
 #include "gdn_internal.cuh"
+#include "gdn_plan.cuh"
 #include "gdn_replay.cuh"
 
 namespace gdn {
@@ -158,14 +159,14 @@ __device__ __forceinline__ void cf_cp_async_16(uint32_t dst, const void *src)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 
-__global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const CommitParams p)
+__device__ __forceinline__ void commit_tile128_unit(const CommitParams &p, const int unit)
 {
     __shared__ __align__(16) uint16_t pk_s[CF_MD * GDN_TILE_D];
     __shared__ __align__(16) uint16_t pv_s[CF_MD * GDN_TILE_D];
     __shared__ __align__(16) float4 ab_s[CF_MD];
     __shared__ int len_s;
 
-    const int b = blockIdx.x / p.h_v, h = blockIdx.x % p.h_v;
+    const int b = unit / p.h_v, h = unit % p.h_v;
     const int hk = h / (p.h_v / p.h_qk);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r4 = lane >> 3, l8 = lane & 7;
@@ -260,6 +261,23 @@ __global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const Com
     }
 }
 
+__global__ void __launch_bounds__(CF_THREADS, 2) commit_tile128_kernel(const CommitParams p)
+{
+    commit_tile128_unit(p, (int)blockIdx.x);
+}
+
+// The fused call on trees of more than 64 nodes: the plans of the NEW trees do not depend on the commit of the previous
+// step's paths, so they are built by the first n_seq CTAs of the same grid instead of by a launch of their own in
+// between (one launch and one dependency hop less in front of the verify kernel).
+static_assert(PLAN_THREADS == CF_THREADS, "the plan CTAs and the commit CTAs share a block size");
+__global__ void __launch_bounds__(CF_THREADS, 2) commit_plan_kernel(const CommitParams p, const PlanArgs a)
+{
+    if ((int)blockIdx.x < a.n_seq)
+        plan_tree(a, (int)blockIdx.x);
+    else
+        commit_tile128_unit(p, (int)blockIdx.x - a.n_seq);
+}
+
 }  // namespace
 
 cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k, const void *v,
@@ -288,6 +306,27 @@ cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k,
         if (e != cudaSuccess) return e;
         commit_generic_kernel<float><<<grid, CM_THREADS, smem, stream>>>(p);
     }
+    return cudaGetLastError();
+}
+
+bool commit_tile128_supported(const gdn_shape_t &s) { return commit_padded_supported(s); }
+
+// Commit of the previous step's paths (ragged packing, tile kernel) and the plan of the new trees in one grid.
+cudaError_t launch_commit_plan(const gdn_shape_t &s, float *S, const void *k, const void *v, const void *g,
+                               const void *beta, const int32_t *parent_prev, const int32_t *node_offsets_prev,
+                               const int32_t *path, const int32_t *path_offsets, const int32_t *parent,
+                               const int32_t *node_offsets, const PlanPtrs &plan, int32_t *status_dev,
+                               cudaStream_t stream)
+{
+    if (s.n_seq == 0) return cudaSuccess;
+    if (s.n_seq > 1) {   // the trees' CTAs claim their places in the unit list from a counter
+        cudaError_t e0 = cudaMemsetAsync(plan.unit_count, 0, sizeof(int32_t), stream);
+        if (e0 != cudaSuccess) return e0;
+    }
+    CommitParams p{s.h_qk, s.h_v, s.d_k, s.d_v, s.max_depth, S, k, v, g, beta, parent_prev, node_offsets_prev, path,
+                   path_offsets, status_dev, 0, 0, 0, 0, nullptr, nullptr};
+    const int grid = s.n_seq + s.n_seq * s.h_v;
+    commit_plan_kernel<<<grid, CF_THREADS, 0, stream>>>(p, plan_args(s, parent, node_offsets, nullptr, plan, status_dev));
     return cudaGetLastError();
 }
 

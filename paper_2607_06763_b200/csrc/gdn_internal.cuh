@@ -168,6 +168,16 @@ cudaError_t launch_commit_generic(const gdn_shape_t &s, float *S, const void *k,
                                   const void *g, const void *beta, const int32_t *parent,
                                   const int32_t *node_offsets, const int32_t *path,
                                   const int32_t *path_offsets, int32_t *status_dev, cudaStream_t stream);
+// d_k = d_v = 128, bf16 inputs, root paths of at most 16 nodes: the tile kernel's shapes.
+bool commit_tile128_supported(const gdn_shape_t &s);
+// The commit of the previous step's accepted paths (tile kernel, ragged packing) and the plan of the new trees in one
+// grid: the fused call on trees of more than 64 nodes.  The new trees' shape is `s`; the commit reads only head counts
+// and the depth bound from it.
+cudaError_t launch_commit_plan(const gdn_shape_t &s, float *S, const void *k, const void *v, const void *g,
+                               const void *beta, const int32_t *parent_prev, const int32_t *node_offsets_prev,
+                               const int32_t *path, const int32_t *path_offsets, const int32_t *parent,
+                               const int32_t *node_offsets, const PlanPtrs &plan, int32_t *status_dev,
+                               cudaStream_t stream);
 // Commit in the padded layout (d_k = d_v = 128, bf16, root paths of at most 16 nodes): slot b keeps its rows at
 // b * s.max_tree_nodes and carries tree b % n_trees; parent [n_trees][rows] (may be null), n_nodes [n_trees],
 // path [n_trees][s.max_depth], path_len [n_trees].

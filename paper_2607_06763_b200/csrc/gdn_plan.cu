@@ -5,174 +5,20 @@
 // Trees of more than 64 nodes additionally get a depth-first numbering cut into groups that are
 // closed under "ancestor of" once the first node's root path is added (see gdn_internal.cuh); the
 // tensor-core verify kernel takes one such group at a time.
-#include "gdn_internal.cuh"
+#include "gdn_plan.cuh"
 
 namespace gdn {
 
 namespace {
 
-constexpr int PLAN_THREADS = 256;
-
-__global__ void __launch_bounds__(PLAN_THREADS)
-plan_kernel(int n_seq, int total_nodes, int max_tree_nodes, int max_depth,
-            const int32_t *__restrict__ parent, const int32_t *__restrict__ node_offsets,
-            const int32_t *__restrict__ n_nodes, int32_t *__restrict__ tree_ok, uint8_t *__restrict__ depth, uint16_t *__restrict__ anc,
-            uint8_t *__restrict__ anc8, uint16_t *__restrict__ dfs_node, uint8_t *__restrict__ dfs_depth,
-            uint8_t *__restrict__ dfs_anc8, uint16_t *__restrict__ group_start, int32_t *__restrict__ unit_count,
-            uint4 *__restrict__ unit_list,
-            int32_t *status_dev)
+__global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const PlanArgs a)
 {
-    __shared__ int size_s[GDN_GROUPED_MAX_NODES];        // subtree sizes
-    __shared__ uint16_t left_s[GDN_GROUPED_MAX_NODES];   // nodes in the subtrees of earlier siblings
-    __shared__ uint16_t pos_s[GDN_GROUPED_MAX_NODES];    // pre-order position of node i
-    __shared__ uint8_t depth_at_s[GDN_GROUPED_MAX_NODES];   // depth of the node at pre-order position r
-    __shared__ uint16_t gstart_s[GDN_MAX_GROUPS + 1];        // first position of each group (then the tree's size)
-    // parent[] of this tree, staged once so that the root-path walks below run out of shared memory
-    __shared__ int32_t par_s[GDN_MAX_TREE_NODES];
     // Programmatic stream serialization on both sides: this grid may have been launched under the tail of the
     // kernel in front of it (nothing is read before that kernel has completed), and the kernel behind this one
     // may be launched early in turn; it waits for this grid to finish before it reads anything written here.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
-    const int b = blockIdx.x;
-    if (b == 0 && threadIdx.x == 0) unit_count[1] = plan_magic(n_seq, max_tree_nodes, max_depth);
-    // ragged packing: the tree's rows by node_offsets[]; padded layout: max_tree_nodes rows per tree, n_nodes[b] used
-    const int lo = node_offsets ? node_offsets[b] : b * max_tree_nodes;
-    const int hi = node_offsets ? node_offsets[b + 1] : lo + n_nodes[b];
-    const int T = hi - lo;
-    bool offsets_ok = lo >= 0 && T >= 0 && T <= max_tree_nodes && hi <= total_nodes;
-    if (node_offsets && b == 0) offsets_ok = offsets_ok && lo == 0;
-    if (node_offsets && b == n_seq - 1) offsets_ok = offsets_ok && hi == total_nodes;
-    if (!offsets_ok) {
-        if (threadIdx.x == 0) {
-            report_status(status_dev, GDN_ERR_TREE);
-            tree_ok[b] = 0;
-            if (n_seq == 1) *unit_count = 0;
-        }
-        return;   // no record in the unit list: nothing of this tree is verified
-    }
-    const bool grouped = max_depth <= 16 && T > 64 && T <= GDN_GROUPED_MAX_NODES;
-    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
-        par_s[i] = parent[lo + i];
-        if (grouped) size_s[i] = 1;
-    }
-    __syncthreads();
-    int err = 0;
-    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
-        // first walk: count the nodes on the root path, checking parent[] as we go
-        int d = 0, cur = i;
-        while (cur >= 0) {
-            if (++d > max_depth) { err = GDN_ERR_DEPTH; break; }
-            const int p = par_s[cur];
-            if (p < -1 || p >= cur) { err = GDN_ERR_TREE; break; }
-            cur = p;
-        }
-        if (err) break;
-        depth[lo + i] = (uint8_t)d;
-        // second walk: fill the list root first, the node itself last
-        uint16_t *row = anc + (size_t)(lo + i) * max_depth;
-        cur = i;
-        uint32_t w0 = 0xFFFFFFFFu, w1 = 0xFFFFFFFFu, w2 = 0xFFFFFFFFu, w3 = 0xFFFFFFFFu;
-        for (int t = d - 1; t >= 0; --t) {
-            row[t] = (uint16_t)cur;
-            // the same list as bytes, one 16-byte row per node (used when max_depth <= 16, T <= 256)
-            const uint32_t keep = ~(0xFFu << ((t & 3) * 8)), put = ((uint32_t)cur & 0xFFu) << ((t & 3) * 8);
-            if ((t >> 2) == 0) w0 = (w0 & keep) | put;
-            else if ((t >> 2) == 1) w1 = (w1 & keep) | put;
-            else if ((t >> 2) == 2) w2 = (w2 & keep) | put;
-            else if ((t >> 2) == 3) w3 = (w3 & keep) | put;
-            cur = par_s[cur];
-            if (grouped && cur >= 0) atomicAdd(&size_s[cur], 1);   // node i lies in the subtree of each proper ancestor
-        }
-        if (max_depth <= 16 && T <= 256)
-            *reinterpret_cast<uint4 *>(anc8 + (size_t)(lo + i) * 16) = make_uint4(w0, w1, w2, w3);
-    }
-    const int any_err = __syncthreads_or(err != 0);
-    if (err) report_status(status_dev, err);
-    if (threadIdx.x == 0) tree_ok[b] = any_err ? 0 : 1;
-    if (any_err || !grouped) {
-        // a tree that fits one tile is its own single group with the identity numbering, marked by n_prefix =
-        // 0xFFFF (no group at all if the tree was rejected or is empty)
-        // (a call with a single tree keeps the count itself; otherwise the counter was zeroed in front of this grid)
-        const bool one = !any_err && T > 0 && T <= GDN_GROUP_TILE;
-        if (threadIdx.x == 0 && n_seq == 1) *unit_count = one ? 1 : 0;
-        if (threadIdx.x == 0 && one)
-            unit_list[n_seq == 1 ? 0 : atomicAdd(unit_count, 1)] =
-                make_uint4((uint32_t)b, (uint32_t)lo, (uint32_t)T << 16, 0xFFFFu);
-        return;
-    }
-
-    // Pre-order position = (#proper ancestors) + sum over the root path of the sizes of the subtrees
-    // hanging off earlier siblings (roots count as siblings of one another; siblings by increasing id).
-    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
-        const int p = par_s[i];
-        int acc = 0;
-        for (int j = p + 1; j < i; ++j)
-            if (par_s[j] == p) acc += size_s[j];
-        left_s[i] = (uint16_t)acc;
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
-        const uint16_t *row = anc + (size_t)(lo + i) * max_depth;
-        const int d = depth[lo + i];
-        int pos = d - 1;
-        for (int t = 0; t < d; ++t) pos += left_s[row[t]];
-        pos_s[i] = (uint16_t)pos;
-        dfs_node[lo + pos] = (uint16_t)i;
-        dfs_depth[lo + pos] = (uint8_t)d;
-        depth_at_s[pos] = (uint8_t)d;
-    }
-    __syncthreads();
-    // Groups: each takes as many positions as the tile leaves after the proper ancestors of its first node
-    if (threadIdx.x == 0) {
-        int start = 0, k = 0;
-        while (start < T && k < GDN_MAX_GROUPS) {
-            gstart_s[k++] = (uint16_t)start;
-            start += GDN_GROUP_TILE - (depth_at_s[start] - 1);
-        }
-        for (; k <= GDN_MAX_GROUPS; ++k) gstart_s[k] = (uint16_t)T;
-    }
-    __syncthreads();
-    for (int k = threadIdx.x; k <= GDN_MAX_GROUPS; k += PLAN_THREADS)
-        group_start[(size_t)b * (GDN_MAX_GROUPS + 1) + k] = gstart_s[k];
-    // one record per group in the unit list, the groups of this tree next to one another
-    __shared__ int list_base_s;
-    if (threadIdx.x == 0) {
-        int n_groups = 0;
-        while (n_groups < GDN_MAX_GROUPS && gstart_s[n_groups] < T) ++n_groups;
-        if (n_seq == 1) {
-            *unit_count = n_groups;
-            list_base_s = 0;
-        } else {
-            list_base_s = atomicAdd(unit_count, n_groups);
-        }
-    }
-    __syncthreads();
-    for (int k = threadIdx.x; k < GDN_MAX_GROUPS; k += PLAN_THREADS) {
-        const int g0 = gstart_s[k], own = gstart_s[k + 1] - g0;
-        if (own > 0)   // (first position, own nodes), (n_prefix, node at the first position)
-            unit_list[list_base_s + k] = make_uint4((uint32_t)b, (uint32_t)lo, (uint32_t)g0 | ((uint32_t)own << 16),
-                                                    (uint32_t)(depth_at_s[g0] - 1) | ((uint32_t)dfs_node[lo + g0] << 16));
-    }
-    // Root path of every node in the virtual indices of its group: an ancestor before the group's first
-    // position is an ancestor of the group's first node and gets index depth-1; one inside the group gets
-    // n_prefix + its offset in the group, n_prefix = depth(first node) - 1.
-    for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
-        const uint16_t *row = anc + (size_t)(lo + i) * max_depth;
-        const int d = depth[lo + i];
-        const int pos = pos_s[i];
-        int k = 0;
-        while (gstart_s[k + 1] <= pos) ++k;   // the group of this position (at most GDN_MAX_GROUPS steps)
-        const int g0 = gstart_s[k];
-        const int n_prefix = depth_at_s[g0] - 1;
-        uint32_t w[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
-        for (int t = 0; t < d; ++t) {
-            const int pa = pos_s[row[t]];
-            const uint32_t v = pa < g0 ? (uint32_t)t : (uint32_t)(n_prefix + pa - g0);
-            w[t >> 2] = (w[t >> 2] & ~(0xFFu << ((t & 3) * 8))) | (v << ((t & 3) * 8));
-        }
-        *reinterpret_cast<uint4 *>(dfs_anc8 + (size_t)(lo + pos) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
+    plan_tree(a, (int)blockIdx.x);
 }
 
 }  // namespace
@@ -195,9 +41,7 @@ cudaError_t launch_plan(const gdn_shape_t &s, const int32_t *parent, const int32
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, plan_kernel, s.n_seq, s.total_nodes, s.max_tree_nodes, s.max_depth, parent,
-                              node_offsets, n_nodes, plan.tree_ok, plan.depth, plan.anc, plan.anc8, plan.dfs_node,
-                              plan.dfs_depth, plan.dfs_anc8, plan.group_start, plan.unit_count, plan.unit_list, status_dev);
+    return cudaLaunchKernelEx(&cfg, plan_kernel, plan_args(s, parent, node_offsets, n_nodes, plan, status_dev));
 }
 
 }  // namespace gdn
