@@ -130,11 +130,20 @@ __device__ __forceinline__ void plan_tree(const PlanArgs &a, const int b)
 
     // Pre-order position = (#proper ancestors) + sum over the root path of the sizes of the subtrees
     // hanging off earlier siblings (roots count as siblings of one another; siblings by increasing id).
+    // With a breadth-first numbering (parent[] non-decreasing, what tree builders emit) the siblings of a node are
+    // its neighbours: the earlier ones are the run in front of it; any other topological numbering is searched.
+    bool sorted_here = true;
+    for (int i = threadIdx.x + 1; i < T; i += PLAN_THREADS) sorted_here = sorted_here && par_s[i] >= par_s[i - 1];
+    const bool sorted = __syncthreads_and(sorted_here);
     for (int i = threadIdx.x; i < T; i += PLAN_THREADS) {
         const int p = par_s[i];
         int acc = 0;
-        for (int j = p + 1; j < i; ++j)
-            if (par_s[j] == p) acc += size_s[j];
+        if (sorted) {
+            for (int j = i - 1; j > p && par_s[j] == p; --j) acc += size_s[j];
+        } else {
+            for (int j = p + 1; j < i; ++j)
+                if (par_s[j] == p) acc += size_s[j];
+        }
         left_s[i] = (uint16_t)acc;
     }
     __syncthreads();
