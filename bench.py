@@ -212,6 +212,7 @@ def workload_config(w: synth.Workload, args):
             "d_k": w.d_k, "d_v": w.d_v, "tree_nodes": int(sizes.max()), "total_nodes": w.total_nodes,
             "in_dtype": w.in_dtype, "state_dtype": "f32", "out_dtype": w.out_dtype,
             "accepted_path_len_mean": float(np.diff(w.path_offsets).mean()),
+            "tree_plan": "built once in front of the timed region" if getattr(args, "plan_once", False) else "per step",
             "l2_policy": "inputs rotate over buffer sets larger than L2 in total"}
 
 
@@ -227,11 +228,13 @@ def report(args):
     # the shape-static entry points on the padded layout (slots sharing one full-size tree)
     runs += [(wl, "fused", "ours", "padded") for wl in ("stack48_T64", "stack48_T256", "layer_T64")]
     runs += [(wl, "verify", "ours", "padded") for wl in WORKLOADS if wl.startswith("sweep_")]
+    # ... with the plan of the shared tree built once for all layers (a layer's call is then the verify kernel alone)
+    runs += [(wl, "verify", "ours", "padded, plan once") for wl in ("sweep_T128", "sweep_T256", "sweep_T512")]
     for wl, mode, impl, layout in runs:
         cmd = [sys.executable, os.path.abspath(__file__), "--workload", wl, "--mode", mode, "--impl", impl, "--steps",
                str(args.steps), "--warmup", str(args.warmup), "--min-time", str(args.min_time), "--no-e2e"]
         if layout != "ragged":
-            cmd += ["--layout", layout]
+            cmd += ["--layout", "padded"] + (["--plan-once"] if "plan once" in layout else [])
         if wl != "stack48_T64" or mode != "fused":
             cmd += ["--oracle-slots", "4"]
         res = subprocess.run(cmd, capture_output=True, text=True)
@@ -272,6 +275,9 @@ def main():
                     help="padded: the shape-static entry points on the dense [slots, T, heads, d] layout with the tree given "
                          "once for all layer slots (workloads whose slots share one full-size tree); trees of more than 64 "
                          "nodes then run as gdn_tree_plan once per step + gdn_tree_commit_padded + gdn_tree_verify_planned")
+    ap.add_argument("--plan-once", action="store_true",
+                    help="--layout padded, trees of more than 64 nodes: build the tree plan once in front of the timed "
+                         "region instead of in every step (a stack of layers calling one after the other shares it)")
     ap.add_argument("--path-len", type=int, default=16,
                     help="workload stack48_T64_deep: nodes on the accepted path (0..16)")
     ap.add_argument("--graph", action="store_true",
@@ -342,14 +348,17 @@ def main():
         plan_bytes = gdn.gdn_tree_plan_bytes(shape, 1)
         plan = torch.empty(max(plan_bytes, 256), dtype=torch.uint8, device="cuda")
         small = T <= 64
+        if args.plan_once and not small:
+            assert gdn.gdn_tree_plan(shape, 1, p_parent, p_nodes, plan, status, stream) == 0
 
     def step_verify_padded(d, stream=stream):
         if small:
             rc = gdn.gdn_tree_verify_padded(shape, 1, False, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], p_parent,
                                             p_nodes, d["o"], status, stream)
         else:
-            rc = gdn.gdn_tree_plan(shape, 1, p_parent, p_nodes, plan, status, stream)
-            assert rc == 0, gdn.gdn_status_string(rc)
+            if not args.plan_once:
+                rc = gdn.gdn_tree_plan(shape, 1, p_parent, p_nodes, plan, status, stream)
+                assert rc == 0, gdn.gdn_status_string(rc)
             rc = gdn.gdn_tree_verify_planned(shape, 1, False, d["S0"], d["q"], d["k"], d["v"], d["g"], d["beta"], plan,
                                              d["o"], status, stream)
         assert rc == 0, gdn.gdn_status_string(rc)
@@ -362,8 +371,9 @@ def main():
             assert rc == 0, gdn.gdn_status_string(rc)
             return
         # the decode step of a larger tree: metadata once, commit of the previous path, verification
-        rc = gdn.gdn_tree_plan(shape, 1, p_parent, p_nodes, plan, status, stream)
-        assert rc == 0, gdn.gdn_status_string(rc)
+        if not args.plan_once:
+            rc = gdn.gdn_tree_plan(shape, 1, p_parent, p_nodes, plan, status, stream)
+            assert rc == 0, gdn.gdn_status_string(rc)
         rc = gdn.gdn_tree_commit_padded(shape, 1, False, d["S0"], d["k"], d["v"], d["g"], d["beta"], p_parent, p_nodes,
                                         p_path, p_len, status, stream)
         assert rc == 0, gdn.gdn_status_string(rc)
